@@ -1,0 +1,327 @@
+"""Benchmark of the GP-EI candidate-scoring hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--impl ours|reference]
+
+One step = one pass of the whole hot path over one pool: r3_gp_score_topk (cross-covariance, mean,
+variance contraction, EI, top-k) on a fitted handle.  The default workload is the largest one:
+a single GP with d=64, n=4096 observations and m=1,048,576 candidates (top-128).  Metric:
+candidates scored per second, whole job.  The fit (once per BO round) is timed separately and
+reported in ``fit_ms``.  Prints ONE JSON line.
+
+N > 1 (launched with torch.distributed.run): every rank scores its own pool of m candidates of the
+same GP (weak scaling) and the ranks' top-k lists are merged with one all-gather per step.
+``--impl reference`` times the FP64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+NOMINAL_TF32_OVER_BF16 = 1.1 / 2.25   # nominal dense peaks: 1.1 PF tf32 vs 2.25 PF bf16
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            return json.load(fh), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._pump, daemon=True)
+        self.thread.start()
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                smax.append(float(parts[2]))
+                power.append(float(parts[3]))
+            except ValueError:
+                continue
+            for name, v in zip(names, parts[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(smax)), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": float(max(power))}
+
+
+def oracle_rate(c, g, budget_s: float):
+    """Times the oracle as it stands on a bounded sample: returns (cand/s, threads, description, fit_s)."""
+    from oracle import gp_oracle as o
+    t0 = time.perf_counter()
+    fits = [o.fit(g["X"][q], g["y"][q], g["ell"][q], g["sf2"][q], g["sn2"][q]) for q in range(min(c.batch, 1))]
+    fit_s = time.perf_counter() - t0
+    chunk = 256 if c.n >= 2048 else 2048
+    done, t0 = 0, time.perf_counter()
+    while True:
+        lo = done % max(c.m - chunk, 1)
+        o.score(fits[0], g["Xcand"][0][lo:lo + chunk])
+        done += min(chunk, c.m - lo)
+        el = time.perf_counter() - t0
+        if el >= budget_s or done >= c.m:
+            break
+    return done / el, o.threads(), f"{done} candidates of GP 0 of {c.name} in {el:.1f} s (fit {fit_s:.1f} s excluded)", fit_s
+
+
+def run_reference(args, c):
+    """The CPU oracle as the reference arm: rank 0 only."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from paper_2604_11109_b200 import workloads as w
+    from oracle import gp_oracle as o
+    small = w.get_config(c.cfg, m=min(c.m, 65536), batch=1)
+    g = w.generate(small)
+    f = o.fit(g["X"][0], g["y"][0], g["ell"][0], g["sf2"][0], g["sn2"][0])
+    per_step = 512 if c.n >= 2048 else (2048 if c.n >= 512 else 16384)
+    per_step = min(per_step, small.m)
+
+    def step(i):
+        lo = (i * per_step) % max(small.m - per_step + 1, 1)
+        mu, sd, ei = o.score(f, g["Xcand"][0][lo:lo + per_step])
+        o.topk(ei, min(c.k, per_step))
+
+    for i in range(args.warmup):
+        step(i)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        step(args.warmup + i)
+    el = time.perf_counter() - t0
+    value = per_step * args.steps / el
+    sample = f"{per_step} candidates per step of {c.name} (n={c.n}, d={c.d}), fit excluded"
+    print(json.dumps({
+        "impl": "reference", "metric": "gp_ei_candidates_scored_per_sec", "value": value, "unit": "candidates/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * el / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": c.name, "n": c.n, "d": c.d, "m": c.m, "k": c.k, "batch": c.batch},
+        "cpu_baseline": {"value": value, "unit": "candidates/s", "cores": o.threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "candidates/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=5, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--engine", default="auto", choices=["auto", "simt", "tensor"])
+    ap.add_argument("--m", type=int, default=None, help="override the pool size (profiling of small cases)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" and args.m is None else args.warmup
+
+    from paper_2604_11109_b200 import workloads as w
+    c = w.get_config(args.config, m=args.m)
+    if args.impl == "reference":
+        run_reference(args, c)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2604_11109_b200 import binding as b
+    from paper_2604_11109_b200.sharding import merge_topk
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    # every rank: the same GP history, its own pool (weak scaling): pool r is drawn with seed offset r
+    g = w.generate(c)
+    if rank > 0 and c.batch == 1:
+        g["Xcand"] = w.generate_gp(c, rank)["Xcand"][None]   # another seeded pool from the same grid
+    X, y = torch.from_numpy(g["X"]).cuda(), torch.from_numpy(g["y"]).cuda()
+    xc = torch.from_numpy(g["Xcand"]).cuda()
+    B, m, k, n, d = c.batch, c.m, c.k, c.n, c.d
+
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    ev[0].record()
+    gp = b.r3_gp_fit(X, y, g["ell"], g["sf2"], g["sn2"])
+    ev[1].record()
+    torch.cuda.synchronize()
+    fit_ms = ev[0].elapsed_time(ev[1])
+    if args.engine != "auto":
+        b.r3_gp_set_engine(gp, {"simt": b.ENGINE_SIMT, "tensor": b.ENGINE_TENSOR}[args.engine])
+    engine = {b.ENGINE_SIMT: "simt", b.ENGINE_TENSOR: "tensor"}[b.r3_gp_engine(gp)]
+
+    out = (torch.empty((B, m), device="cuda"), torch.empty((B, m), device="cuda"), torch.empty((B, m), device="cuda"),
+           torch.empty((B, k), dtype=torch.int32, device="cuda"), torch.empty((B, k), device="cuda"))
+
+    def step():
+        b.r3_gp_score_topk(gp, xc, k, out)
+        if world > 1 and B == 1:
+            merge_topk(out[4][0], out[3][0], k, rank * m, topk_fn=lambda v, kk: b.r3_topk(v, kk)[0])
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    b.r3_gp_check(gp)
+
+    # ---- device-resident timing ---------------------------------------------------------------
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    b.r3_gp_profile(gp, True)
+    b.r3_launch_count_reset()
+    barrier()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(args.steps):
+        step()
+    stop.record()
+    barrier()
+    launches = b.r3_launch_count()
+    ms_total = start.elapsed_time(stop)
+    kernel_ms, kernel_launches = b.r3_gp_profile_read(gp)
+    b.r3_gp_profile(gp, False)
+    clocks = sampler.stop() if rank == 0 else None
+    b.r3_gp_check(gp)
+    if world > 1:
+        t = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    value = world * B * m / (ms_per_step * 1e-3)
+
+    # ---- end to end through the host-buffer entry point ------------------------------------------
+    xh = torch.from_numpy(g["Xcand"]).pin_memory()
+    oh = (torch.empty((B, m)).pin_memory(), torch.empty((B, m)).pin_memory(), torch.empty((B, m)).pin_memory(),
+          torch.empty((B, k), dtype=torch.int32).pin_memory(), torch.empty((B, k)).pin_memory())
+    e2e_steps = max(2, min(args.steps, 5))
+    b.r3_gp_score_topk_host(gp, xh, k, oh)
+    barrier()
+    start.record()
+    for _ in range(e2e_steps):
+        b.r3_gp_score_topk_host(gp, xh, k, oh)
+    stop.record()
+    barrier()
+    e2e_ms = start.elapsed_time(stop) / e2e_steps
+    if world > 1:
+        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    same = all(torch.equal(a.cpu(), h) for a, h in zip(out[:3], oh[:3]))
+
+    if rank != 0:
+        gp.close()
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (the variance contraction) -----------------------------
+    peaks, peak_kind = load_peaks()
+    per_launch_ms = kernel_ms / max(kernel_launches, 1)
+    cands_per_launch = B * m * args.steps / max(kernel_launches, 1)
+    npad = (n + 31) // 32 * 32
+    if engine == "tensor":
+        # algorithmic flops per candidate of S4 (n^2, lower triangle, 2 flops per MAC on n^2/2 MACs); the kernel
+        # issues 3 TF32 MMAs per product, so issued = 3x that
+        alg_flops = float(npad) * npad
+        issued = 3.0 * alg_flops
+        achieved = issued * cands_per_launch / (per_launch_ms * 1e-3) / 1e12
+        peak = peaks["bf16_tflops_sustained" if per_launch_ms > 50 else "bf16_tflops"] * NOMINAL_TF32_OVER_BF16
+        roofline = {"bound": "tensor", "kernel": "score_tc_kernel", "achieved": achieved, "peak": peak,
+                    "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                    "note": f"issued 3xTF32 flops; algorithmic = achieved/3; peak = {peak_kind} bf16 x 1.1/2.25",
+                    "algorithmic_tflops": achieved / 3.0}
+    else:
+        alg_flops = float(npad) * npad
+        achieved = alg_flops * cands_per_launch / (per_launch_ms * 1e-3) / 1e12
+        sm_mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
+        peak = 148 * 128 * 2 * sm_mhz * 1e6 / 1e12
+        roofline = {"bound": "alu", "kernel": "trigemm_sq_kernel", "achieved": achieved, "peak": peak,
+                    "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                    "note": "FP32 FMA path; peak = 148 SMs x 128 lanes x 2 flop x max SM clock"}
+    roofline["kernel_ms_per_launch"] = per_launch_ms
+    roofline["kernel_launches"] = kernel_launches
+    roofline["kernel_share_of_step"] = kernel_ms / ms_total if ms_total > 0 else None
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        v, threads, sample, ofit = oracle_rate(c, g, 12.0)
+        cpu = {"value": v, "unit": "candidates/s", "cores": threads, "kind": "oracle", "sample": sample,
+               "fit_s": ofit}
+
+    h2d = int(xh.numel() * 4)
+    d2h = int(sum(t.numel() * 4 for t in oh))
+    print(json.dumps({
+        "metric": "gp_ei_candidates_scored_per_sec", "value": value, "unit": "candidates/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32" if engine == "simt" else "tf32x3", "data": "synthetic",
+        "config": {"workload": c.name, "batch": B, "n": n, "d": d, "m": m, "k": k, "engine": engine,
+                   "l2": "pool (%.0f MB) and outputs exceed the 126 MB L2" % (xc.numel() * 4 / 1e6)
+                   if xc.numel() * 4 > 126e6 else "pool smaller than L2; not flushed"},
+        "fit_ms": fit_ms, "clocks": clocks,
+        "e2e": {"value": world * B * m / (e2e_ms * 1e-3), "unit": "candidates/s", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "matches_device_run": bool(same)},
+        "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu, "peaks": peak_kind,
+    }))
+    gp.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

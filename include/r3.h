@@ -1,0 +1,179 @@
+/*
+ * r3.h -- C ABI of libr3gp: Gaussian-process candidate scoring for the inner
+ * Bayesian-optimisation loop of R^3 on one NVIDIA B200 (sm_100a).
+ *
+ * Where this sits in the paper.  Section IV: for every source candidate the
+ * replay server runs a parallel Bayesian-optimisation search over compiler pass
+ * configurations and launch parameters and keeps the best runtime.  Section
+ * V-B: a sampled point is one replay experiment (pipeline + launch configuration
+ * -> runtime), and the mechanism is agnostic to the search strategy.  The paper
+ * prints no formula for the surrogate; this library implements the "propose the
+ * next points" step with a zero-mean Gaussian process (ARD Matern-5/2
+ * covariance), Expected Improvement for minimisation, and top-k selection:
+ *
+ *   history (X, y)  --r3_gp_fit-->  factor handle
+ *   handle, pool    --r3_gp_score-> mu, sigma, EI per candidate
+ *   EI              --r3_topk-->    the k pool members to replay next
+ *
+ * Conventions
+ *   - Smaller y is better (y = log-runtime).  A maximiser negates y.
+ *   - All matrices are row-major and dense.  "device" pointers are CUDA global
+ *     memory of the current device; "host" pointers are ordinary memory.
+ *   - The caller owns every array it passes; the library only reads or writes
+ *     through the pointer during the call (asynchronously on `cuda_stream` where
+ *     stated) and never frees it.  The library owns a handle until r3_gp_free.
+ *   - `cuda_stream` is a cudaStream_t cast to void* (NULL = the default stream).
+ *   - Every call returns a status and never aborts, throws or prints.  On error
+ *     the outputs are unspecified, `*out` (if any) is NULL and r3_last_error()
+ *     describes the failure (thread-local text).
+ *   - There is no CPU fallback: without a CUDA device every compute entry point
+ *     returns R3_ERR_CUDA.
+ */
+#ifndef R3_H
+#define R3_H
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct r3_gp r3_gp_t; /* opaque; owns device memory */
+
+typedef enum {
+    R3_OK = 0,
+    R3_ERR_INVALID_ARG = 1,    /* NULL pointer, size out of range, non-positive hyper-parameter */
+    R3_ERR_NONFINITE = 2,      /* X, y or Xcand contains NaN/Inf (detected on the device) */
+    R3_ERR_NOT_PD = 3,         /* a Cholesky pivot of K(X,X)+noise*I was not positive */
+    R3_ERR_ALLOC = 4,          /* device or host allocation failed */
+    R3_ERR_CUDA = 5,           /* a CUDA runtime call failed (no device, launch error, ...) */
+    R3_ERR_DEVICE_TIMEOUT = 6, /* a bounded device-side wait ran out; results invalid */
+    R3_ERR_UNSUPPORTED = 7     /* valid request outside the implemented limits */
+} r3_status_t;
+
+/* Scoring engines, for r3_gp_set_engine. */
+typedef enum {
+    R3_ENGINE_AUTO = 0,   /* tensor-core path where it applies, else SIMT */
+    R3_ENGINE_SIMT = 1,   /* FP32 CUDA-core path (direct-difference distances) */
+    R3_ENGINE_TENSOR = 2  /* tcgen05 3xTF32 path (distance GEMM + triangular contraction) */
+} r3_engine_t;
+
+/*
+ * r3_gp_fit -- condition `batch` independent GPs on their histories.
+ *
+ * Computes, per GP and in FP64 on the device: K = k(X,X) + noise_var*I with
+ *   k(x,z) = signal_var * (1 + s + s^2/3) * exp(-s),  s = sqrt(5) * r,
+ *   r^2 = sum_j ((x_j - z_j)/lengthscale_j)^2            (ARD Matern-5/2),
+ * its lower Cholesky factor L, the weights alpha = K^-1 y, the inverse factor
+ * W = L^-1 used by the variance contraction, and best = min_i y_i.
+ * (Inner BO search of Section IV; surrogate as stated above.)
+ *
+ *   X            device [batch][n][d]   observed configurations (feature rows)
+ *   y            device [batch][n]      observed values
+ *   lengthscales host   [batch][d]      > 0
+ *   signal_var   host   [batch]         > 0
+ *   noise_var    host   [batch]         >= 0
+ *   batch >= 1, 1 <= n <= 8192, 1 <= d <= 256
+ *   out          receives the handle (NULL on error)
+ *
+ * Synchronises `cuda_stream` before returning, so that R3_ERR_NOT_PD and
+ * R3_ERR_NONFINITE are reported by this call.  No jitter is added: a
+ * non-positive-definite K is an error, never silently repaired.
+ */
+r3_status_t r3_gp_fit(const float* X, const float* y, const float* lengthscales,
+                      const float* signal_var, const float* noise_var, int batch, int n, int d,
+                      void* cuda_stream, r3_gp_t** out);
+
+/*
+ * r3_gp_score -- posterior mean, latent standard deviation and Expected
+ * Improvement of every candidate of every GP's pool.
+ *
+ *   k*_i  = k(x_i, x*),  mu = k* . alpha,
+ *   sigma = sqrt(max(signal_var - |W k*|^2, 0))       (observation noise NOT added),
+ *   z = (best - mu)/sigma,  EI = (best - mu)*Phi(z) + sigma*phi(z);
+ *   sigma == 0  ->  EI = max(best - mu, 0).
+ *
+ *   Xcand  device [batch][m][d]      candidate pool of each GP, 1 <= m < 2^31
+ *   mu, sigma, ei  device [batch][m] caller-allocated outputs (FP32)
+ *
+ * Asynchronous on `cuda_stream`; does not synchronise.  Device-side problems
+ * (non-finite candidate, a bounded wait that ran out) are latched in the handle
+ * and returned by r3_gp_check.  May grow the handle's private workspace (a
+ * synchronising allocation) the first time a larger m is seen.
+ */
+r3_status_t r3_gp_score(r3_gp_t* gp, const float* Xcand, long long m, float* mu, float* sigma,
+                        float* ei, void* cuda_stream);
+
+/*
+ * r3_topk -- indices of the k largest values of each row of `ei`.
+ *
+ *   ei   device [batch][m]
+ *   idx  device [batch][k]  int32, sorted by value descending, ties by index ascending
+ *   val  device [batch][k]  the selected values, or NULL
+ *   1 <= k <= min(m, 1024).  NaN ranks below every number.
+ *   scratch / scratch_bytes: device workspace of at least
+ *   r3_topk_scratch_bytes(batch, m, k) bytes, or NULL/0 to let the call allocate
+ *   and free one itself (which synchronises).
+ *
+ * Asynchronous on `cuda_stream` when a workspace is supplied.
+ */
+r3_status_t r3_topk(const float* ei, int batch, long long m, int k, int* idx, float* val,
+                    void* scratch, unsigned long long scratch_bytes, void* cuda_stream);
+unsigned long long r3_topk_scratch_bytes(int batch, long long m, int k);
+
+/*
+ * r3_gp_score_topk -- r3_gp_score followed by r3_topk on the EI it produced, with
+ * the handle's own workspace; asynchronous on `cuda_stream`.  This is the "one
+ * BO proposal round" call: idx [batch][k] are the pool members to replay next.
+ */
+r3_status_t r3_gp_score_topk(r3_gp_t* gp, const float* Xcand, long long m, int k, float* mu,
+                             float* sigma, float* ei, int* idx, float* val, void* cuda_stream);
+
+/*
+ * Host-buffer convenience form of r3_gp_score_topk: Xcand and all outputs are
+ * HOST arrays (pinned memory makes the copies asynchronous); the call stages
+ * them through the handle's workspace, and synchronises the stream before
+ * returning.  Any of mu, sigma, ei, val may be NULL to skip that copy.
+ */
+r3_status_t r3_gp_score_topk_host(r3_gp_t* gp, const float* Xcand_host, long long m, int k,
+                                  float* mu_host, float* sigma_host, float* ei_host, int* idx_host,
+                                  float* val_host, void* cuda_stream);
+
+/* Synchronise `cuda_stream` and return (then clear) the handle's latched device status. */
+r3_status_t r3_gp_check(r3_gp_t* gp, void* cuda_stream);
+
+/* Incumbent used by EI: defaults to min(y); may be overridden per GP.  host [batch]. */
+r3_status_t r3_gp_get_best(const r3_gp_t* gp, float* best);
+r3_status_t r3_gp_set_best(r3_gp_t* gp, const float* best);
+
+/* Select the scoring engine (default R3_ENGINE_AUTO).  R3_ERR_UNSUPPORTED if the
+ * requested engine cannot serve this handle's (n, d). */
+r3_status_t r3_gp_set_engine(r3_gp_t* gp, r3_engine_t engine);
+/* Engine that r3_gp_score will actually use for this handle. */
+r3_engine_t r3_gp_engine(const r3_gp_t* gp);
+
+/*
+ * Timing of the dominant scoring kernel (the variance contraction).  While enabled, every launch
+ * of that kernel is bracketed by a CUDA event pair on the launching stream.  r3_gp_profile_read
+ * waits for the recorded events, returns the summed kernel time in milliseconds and the number
+ * of launches it covers, and clears the record.  Off by default; costs two event records per launch.
+ */
+r3_status_t r3_gp_profile(r3_gp_t* gp, int enable);
+r3_status_t r3_gp_profile_read(r3_gp_t* gp, double* kernel_ms, long long* launches);
+
+/* Copy fit results to host arrays (diagnostics and tests): alpha [batch][n] FP64,
+ * L [batch][n][n] FP64 lower-triangular (upper part zero).  Either may be NULL. */
+r3_status_t r3_gp_get_factor(const r3_gp_t* gp, double* alpha, double* L);
+
+/* Kernels launched by this library on the calling thread since the last reset. */
+unsigned long long r3_launch_count(void);
+void r3_launch_count_reset(void);
+
+void r3_gp_free(r3_gp_t* gp);
+
+const char* r3_status_string(r3_status_t status);
+const char* r3_last_error(void);
+int r3_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* R3_H */

@@ -1,0 +1,279 @@
+"""Thin Python binding of ``libr3gp.so`` (the C ABI declared in ``include/r3.h``).
+
+Argument marshalling only: every step of the scoring path runs in the library's
+CUDA kernels.  PyTorch supplies device memory (``torch.Tensor.data_ptr``) and the
+current stream; there is no CPU fallback -- if the library or a CUDA device is
+missing, the calls raise.
+
+The functions carry the names of the C entry points.  Tensors passed in must be
+contiguous float32 on the current CUDA device (host arrays where the C ABI says
+"host").
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libr3gp.so")
+
+R3_OK = 0
+STATUS_NAMES = {
+    0: "R3_OK", 1: "R3_ERR_INVALID_ARG", 2: "R3_ERR_NONFINITE", 3: "R3_ERR_NOT_PD", 4: "R3_ERR_ALLOC",
+    5: "R3_ERR_CUDA", 6: "R3_ERR_DEVICE_TIMEOUT", 7: "R3_ERR_UNSUPPORTED",
+}
+ENGINE_AUTO, ENGINE_SIMT, ENGINE_TENSOR = 0, 1, 2
+
+_lib = None
+
+_vp, _i, _ll, _ull = ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong, ctypes.c_ulonglong
+_fp = ctypes.POINTER(ctypes.c_float)
+
+# name -> (restype, argtypes); every symbol include/r3.h declares
+SIGNATURES = {
+    "r3_gp_fit": (_i, [_vp, _vp, _fp, _fp, _fp, _i, _i, _i, _vp, ctypes.POINTER(_vp)]),
+    "r3_gp_score": (_i, [_vp, _vp, _ll, _vp, _vp, _vp, _vp]),
+    "r3_topk": (_i, [_vp, _i, _ll, _i, _vp, _vp, _vp, _ull, _vp]),
+    "r3_topk_scratch_bytes": (_ull, [_i, _ll, _i]),
+    "r3_gp_score_topk": (_i, [_vp, _vp, _ll, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "r3_gp_score_topk_host": (_i, [_vp, _vp, _ll, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "r3_gp_check": (_i, [_vp, _vp]),
+    "r3_gp_get_best": (_i, [_vp, _fp]),
+    "r3_gp_set_best": (_i, [_vp, _fp]),
+    "r3_gp_set_engine": (_i, [_vp, _i]),
+    "r3_gp_engine": (_i, [_vp]),
+    "r3_gp_get_factor": (_i, [_vp, _vp, _vp]),
+    "r3_gp_profile": (_i, [_vp, _i]),
+    "r3_gp_profile_read": (_i, [_vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_ll)]),
+    "r3_launch_count": (_ull, []),
+    "r3_launch_count_reset": (None, []),
+    "r3_gp_free": (None, [_vp]),
+    "r3_status_string": (ctypes.c_char_p, [_i]),
+    "r3_last_error": (ctypes.c_char_p, []),
+    "r3_version": (_i, []),
+}
+
+
+class R3Error(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{STATUS_NAMES.get(status, status)}: {message}")
+        self.status = status
+
+
+def load():
+    """Load ``libr3gp.so``; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2604_11109_b200.build`")
+    lib = ctypes.CDLL(LIB_PATH)
+    for name, (res, args) in SIGNATURES.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    _lib = lib
+    return lib
+
+
+def _check(status: int):
+    if status != R3_OK:
+        raise R3Error(status, load().r3_last_error().decode())
+
+
+def _stream():
+    import torch
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dev_f32(t, name):
+    import torch
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+        raise TypeError(f"{name} must be a contiguous float32 CUDA tensor")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _host_f32(a, shape, name):
+    a = np.ascontiguousarray(np.broadcast_to(np.asarray(a, dtype=np.float32), shape))
+    return a, a.ctypes.data_as(_fp)
+
+
+class GP:
+    """Owner of one ``r3_gp_t*``; freed on ``close()`` or garbage collection."""
+
+    def __init__(self, handle: int, batch: int, n: int, d: int):
+        self._h = ctypes.c_void_p(handle)
+        self.batch, self.n, self.d = batch, n, d
+
+    @property
+    def handle(self):
+        if not self._h:
+            raise ValueError("GP handle already freed")
+        return self._h
+
+    def close(self):
+        if self._h:
+            load().r3_gp_free(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def r3_gp_fit(X, y, lengthscales, signal_var, noise_var) -> GP:
+    """X [batch][n][d] (or [n][d]) and y [batch][n] CUDA float32; hyper-parameters host arrays."""
+    if X.dim() == 2:
+        X, y = X.unsqueeze(0), y.unsqueeze(0)
+    batch, n, d = X.shape
+    if tuple(y.shape) != (batch, n):
+        raise ValueError("y must be [batch][n]")
+    ell, ell_p = _host_f32(lengthscales, (batch, d), "lengthscales")
+    sf2, sf2_p = _host_f32(signal_var, (batch,), "signal_var")
+    sn2, sn2_p = _host_f32(noise_var, (batch,), "noise_var")
+    out = ctypes.c_void_p()
+    _check(load().r3_gp_fit(_dev_f32(X, "X"), _dev_f32(y, "y"), ell_p, sf2_p, sn2_p, batch, n, d, _stream(),
+                            ctypes.byref(out)))
+    return GP(out.value, batch, n, d)
+
+
+def _pool(gp: GP, Xcand):
+    if Xcand.dim() == 2:
+        Xcand = Xcand.unsqueeze(0)
+    if Xcand.shape[0] != gp.batch or Xcand.shape[2] != gp.d:
+        raise ValueError("Xcand must be [batch][m][d]")
+    return Xcand, int(Xcand.shape[1])
+
+
+def r3_gp_score(gp: GP, Xcand, out=None):
+    """Returns (mu, sigma, ei), each CUDA float32 [batch][m]; asynchronous on the current stream."""
+    import torch
+    Xcand, m = _pool(gp, Xcand)
+    mu, sigma, ei = out if out is not None else (
+        torch.empty((gp.batch, m), dtype=torch.float32, device=Xcand.device) for _ in range(3))
+    _check(load().r3_gp_score(gp.handle, _dev_f32(Xcand, "Xcand"), m, _dev_f32(mu, "mu"), _dev_f32(sigma, "sigma"),
+                              _dev_f32(ei, "ei"), _stream()))
+    return mu, sigma, ei
+
+
+def r3_topk(ei, k: int, scratch=None):
+    """ei CUDA float32 [batch][m] (or [m]) -> (idx int32 [batch][k], val float32 [batch][k])."""
+    import torch
+    squeeze = ei.dim() == 1
+    if squeeze:
+        ei = ei.unsqueeze(0)
+    batch, m = ei.shape
+    lib = load()
+    idx = torch.empty((batch, k), dtype=torch.int32, device=ei.device)
+    val = torch.empty((batch, k), dtype=torch.float32, device=ei.device)
+    if scratch is None:
+        nbytes = int(lib.r3_topk_scratch_bytes(batch, m, k))
+        scratch = torch.empty(max(nbytes, 1), dtype=torch.uint8, device=ei.device)
+    _check(lib.r3_topk(_dev_f32(ei, "ei"), batch, m, k, ctypes.c_void_p(idx.data_ptr()),
+                       ctypes.c_void_p(val.data_ptr()), ctypes.c_void_p(scratch.data_ptr()), scratch.numel(),
+                       _stream()))
+    return (idx[0], val[0]) if squeeze else (idx, val)
+
+
+def r3_topk_scratch_bytes(batch: int, m: int, k: int) -> int:
+    return int(load().r3_topk_scratch_bytes(int(batch), int(m), int(k)))
+
+
+def r3_gp_score_topk(gp: GP, Xcand, k: int, out=None):
+    """One proposal round on device buffers: returns (mu, sigma, ei, idx, val)."""
+    import torch
+    Xcand, m = _pool(gp, Xcand)
+    if out is None:
+        mu, sigma, ei = (torch.empty((gp.batch, m), dtype=torch.float32, device=Xcand.device) for _ in range(3))
+        idx = torch.empty((gp.batch, k), dtype=torch.int32, device=Xcand.device)
+        val = torch.empty((gp.batch, k), dtype=torch.float32, device=Xcand.device)
+    else:
+        mu, sigma, ei, idx, val = out
+    _check(load().r3_gp_score_topk(gp.handle, _dev_f32(Xcand, "Xcand"), m, k, _dev_f32(mu, "mu"),
+                                   _dev_f32(sigma, "sigma"), _dev_f32(ei, "ei"), ctypes.c_void_p(idx.data_ptr()),
+                                   _dev_f32(val, "val"), _stream()))
+    return mu, sigma, ei, idx, val
+
+
+def r3_gp_score_topk_host(gp: GP, Xcand_host, k: int, out):
+    """Host-buffer form: Xcand_host and the tensors of ``out`` = (mu, sigma, ei, idx, val) live in
+    (ideally pinned) host memory; any of mu/sigma/ei/val may be None.  Synchronises."""
+    m = int(Xcand_host.shape[-2])
+    mu, sigma, ei, idx, val = out
+
+    def hp(t):
+        return ctypes.c_void_p(t.data_ptr()) if t is not None else ctypes.c_void_p()
+
+    _check(load().r3_gp_score_topk_host(gp.handle, hp(Xcand_host), m, k, hp(mu), hp(sigma), hp(ei), hp(idx), hp(val),
+                                        _stream()))
+    return out
+
+
+def r3_gp_check(gp: GP):
+    _check(load().r3_gp_check(gp.handle, _stream()))
+
+
+def r3_gp_get_best(gp: GP) -> np.ndarray:
+    best = np.empty(gp.batch, dtype=np.float32)
+    _check(load().r3_gp_get_best(gp.handle, best.ctypes.data_as(_fp)))
+    return best
+
+
+def r3_gp_set_best(gp: GP, best):
+    b, p = _host_f32(best, (gp.batch,), "best")
+    _check(load().r3_gp_set_best(gp.handle, p))
+
+
+def r3_gp_set_engine(gp: GP, engine: int):
+    _check(load().r3_gp_set_engine(gp.handle, int(engine)))
+
+
+def r3_gp_engine(gp: GP) -> int:
+    return int(load().r3_gp_engine(gp.handle))
+
+
+def r3_gp_get_factor(gp: GP):
+    """(alpha [batch][n], L [batch][n][n]) as FP64 numpy arrays."""
+    alpha = np.empty((gp.batch, gp.n), dtype=np.float64)
+    L = np.empty((gp.batch, gp.n, gp.n), dtype=np.float64)
+    _check(load().r3_gp_get_factor(gp.handle, alpha.ctypes.data_as(_vp), L.ctypes.data_as(_vp)))
+    return alpha, L
+
+
+def r3_gp_profile(gp: GP, enable: bool):
+    _check(load().r3_gp_profile(gp.handle, 1 if enable else 0))
+
+
+def r3_gp_profile_read(gp: GP):
+    """(summed milliseconds of the dominant kernel, number of launches) since the last read."""
+    ms, cnt = ctypes.c_double(), _ll()
+    _check(load().r3_gp_profile_read(gp.handle, ctypes.byref(ms), ctypes.byref(cnt)))
+    return float(ms.value), int(cnt.value)
+
+
+def r3_launch_count() -> int:
+    return int(load().r3_launch_count())
+
+
+def r3_launch_count_reset():
+    load().r3_launch_count_reset()
+
+
+def r3_gp_free(gp: GP):
+    gp.close()
+
+
+def r3_version() -> int:
+    return int(load().r3_version())
+
+
+def r3_status_string(status: int) -> str:
+    return load().r3_status_string(int(status)).decode()
+
+
+def r3_last_error() -> str:
+    return load().r3_last_error().decode()

@@ -1,0 +1,486 @@
+// C ABI of libr3gp: argument validation, handle life cycle, engine dispatch.  See include/r3.h.
+#include <limits.h>
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+
+#include <new>
+
+#include "r3_internal.cuh"
+
+namespace r3 {
+
+static thread_local char g_error[512] = "";
+thread_local unsigned long long g_launches = 0;
+
+void set_error(const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_error, sizeof(g_error), fmt, ap);
+    va_end(ap);
+}
+
+r3_status_t ensure_workspace(r3_gp* gp, size_t bytes)
+{
+    if (bytes <= gp->ws_bytes) return R3_OK;
+    // growing synchronises the device: wait for work that may still use the old buffer
+    R3_CUDA_TRY(cudaDeviceSynchronize());
+    if (gp->ws) cudaFree(gp->ws);
+    gp->ws = nullptr;
+    gp->ws_bytes = 0;
+    const size_t want = (bytes + (1u << 20)) & ~((size_t)(1u << 20) - 1);
+    R3_CUDA_TRY(cudaMalloc(&gp->ws, want));
+    gp->ws_bytes = want;
+    return R3_OK;
+}
+
+void prof_begin(r3_gp* gp, cudaStream_t stream)
+{
+    if (!gp->profile) return;
+    if (gp->events_used + 2 > gp->events.size()) {
+        if (gp->events.size() >= 16384) return;  // cap: further launches go untimed
+        cudaEvent_t a, b;
+        if (cudaEventCreate(&a) != cudaSuccess) return;
+        if (cudaEventCreate(&b) != cudaSuccess) {
+            cudaEventDestroy(a);
+            return;
+        }
+        gp->events.push_back(a);
+        gp->events.push_back(b);
+    }
+    cudaEventRecord(gp->events[gp->events_used], stream);
+}
+
+void prof_end(r3_gp* gp, cudaStream_t stream)
+{
+    if (!gp->profile || gp->events_used + 2 > gp->events.size()) return;
+    cudaEventRecord(gp->events[gp->events_used + 1], stream);
+    gp->events_used += 2;
+}
+
+static r3_engine_t pick_engine(const r3_gp* gp)
+{
+    const bool tc_ok = gp->tc != nullptr;
+    switch (gp->engine_req) {
+        case R3_ENGINE_SIMT: return R3_ENGINE_SIMT;
+        case R3_ENGINE_TENSOR: return tc_ok ? R3_ENGINE_TENSOR : R3_ENGINE_SIMT;
+        default:
+            // small feature counts keep the direct-difference distances of the SIMT engine
+            return (tc_ok && gp->d > 16) ? R3_ENGINE_TENSOR : R3_ENGINE_SIMT;
+    }
+}
+
+static size_t score_workspace_bytes(const r3_gp* gp, long long m)
+{
+    return pick_engine(gp) == R3_ENGINE_TENSOR ? score_tc_workspace_bytes(gp, m)
+                                               : score_simt_workspace_bytes(gp, m);
+}
+
+static size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+static r3_status_t check_score_args(const r3_gp* gp, const void* Xcand, long long m, const void* mu,
+                                    const void* sigma, const void* ei)
+{
+    if (!gp || !Xcand || !mu || !sigma || !ei) {
+        set_error("r3_gp_score: NULL argument");
+        return R3_ERR_INVALID_ARG;
+    }
+    if (m < 1 || m >= (1ll << 31)) {
+        set_error("r3_gp_score: m=%lld out of range [1, 2^31)", m);
+        return R3_ERR_INVALID_ARG;
+    }
+    return R3_OK;
+}
+
+static r3_status_t run_score(r3_gp* gp, const float* Xcand, long long m, float* mu, float* sigma, float* ei,
+                             void* ws, size_t ws_bytes, cudaStream_t stream)
+{
+    if (pick_engine(gp) == R3_ENGINE_TENSOR) return score_tc(gp, Xcand, m, mu, sigma, ei, ws, ws_bytes, stream);
+    return score_simt(gp, Xcand, m, mu, sigma, ei, ws, ws_bytes, stream);
+}
+
+}  // namespace r3
+
+using namespace r3;
+
+extern "C" {
+
+int r3_version(void) { return 100; }
+
+const char* r3_last_error(void) { return g_error; }
+
+const char* r3_status_string(r3_status_t s)
+{
+    switch (s) {
+        case R3_OK: return "ok";
+        case R3_ERR_INVALID_ARG: return "invalid argument";
+        case R3_ERR_NONFINITE: return "non-finite input";
+        case R3_ERR_NOT_PD: return "covariance matrix is not positive definite";
+        case R3_ERR_ALLOC: return "allocation failed";
+        case R3_ERR_CUDA: return "CUDA error";
+        case R3_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+        case R3_ERR_UNSUPPORTED: return "unsupported";
+    }
+    return "unknown status";
+}
+
+unsigned long long r3_launch_count(void) { return g_launches; }
+void r3_launch_count_reset(void) { g_launches = 0; }
+
+void r3_gp_free(r3_gp_t* gp)
+{
+    if (!gp) return;
+    tc_release(gp);
+    cudaFree(gp->X);
+    cudaFree(gp->ell_d);
+    cudaFree(gp->inv_ell);
+    cudaFree(gp->sn2_d);
+    cudaFree(gp->sf2_d);
+    cudaFree(gp->best_d);
+    cudaFree(gp->L64);
+    cudaFree(gp->W64);
+    cudaFree(gp->W32);
+    cudaFree(gp->alpha64);
+    cudaFree(gp->alpha32);
+    cudaFree(gp->status_d);
+    if (gp->status_h) cudaFreeHost(gp->status_h);
+    for (cudaEvent_t e : gp->events) cudaEventDestroy(e);
+    cudaFree(gp->ws);
+    delete gp;
+}
+
+r3_status_t r3_gp_fit(const float* X, const float* y, const float* lengthscales, const float* signal_var,
+                      const float* noise_var, int batch, int n, int d, void* cuda_stream, r3_gp_t** out)
+{
+    if (out) *out = nullptr;
+    if (!X || !y || !lengthscales || !signal_var || !noise_var || !out) {
+        set_error("r3_gp_fit: NULL argument");
+        return R3_ERR_INVALID_ARG;
+    }
+    if (batch < 1 || batch > 4096 || n < 1 || n > kMaxN || d < 1 || d > kMaxD) {
+        set_error("r3_gp_fit: sizes out of range (batch=%d in [1,4096], n=%d in [1,%d], d=%d in [1,%d])", batch,
+                  n, kMaxN, d, kMaxD);
+        return R3_ERR_INVALID_ARG;
+    }
+    for (int g = 0; g < batch; ++g) {
+        if (!(signal_var[g] > 0.f) || !isfinite(signal_var[g]) || !(noise_var[g] >= 0.f) ||
+            !isfinite(noise_var[g])) {
+            set_error("r3_gp_fit: GP %d needs signal_var > 0 and noise_var >= 0", g);
+            return R3_ERR_INVALID_ARG;
+        }
+        for (int j = 0; j < d; ++j) {
+            const float l = lengthscales[(size_t)g * d + j];
+            if (!(l > 0.f) || !isfinite(l)) {
+                set_error("r3_gp_fit: GP %d lengthscale %d must be positive and finite", g, j);
+                return R3_ERR_INVALID_ARG;
+            }
+        }
+    }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    r3_gp* gp = new (std::nothrow) r3_gp;
+    if (!gp) {
+        set_error("r3_gp_fit: out of host memory");
+        return R3_ERR_ALLOC;
+    }
+    auto bail = [&](r3_status_t st) {
+        r3_gp_free(gp);
+        return st;
+    };
+#define TRY_BAIL(expr)                                                                             \
+    do {                                                                                           \
+        cudaError_t e__ = (expr);                                                                  \
+        if (e__ != cudaSuccess) {                                                                  \
+            set_error("%s failed: %s", #expr, cudaGetErrorString(e__));                            \
+            return bail(e__ == cudaErrorMemoryAllocation ? R3_ERR_ALLOC : R3_ERR_CUDA);            \
+        }                                                                                          \
+    } while (0)
+    TRY_BAIL(cudaGetDevice(&gp->device));
+    gp->batch = batch;
+    gp->n = n;
+    gp->d = d;
+    gp->npad = round_up(n, kFitBlock);
+    gp->ell.assign(lengthscales, lengthscales + (size_t)batch * d);
+    gp->sf2.assign(signal_var, signal_var + batch);
+    gp->sn2.assign(noise_var, noise_var + batch);
+    gp->best.assign(batch, 0.f);
+    std::vector<float> inv((size_t)batch * d);
+    for (size_t i = 0; i < inv.size(); ++i) inv[i] = (float)(1.0 / (double)gp->ell[i]);
+
+    const size_t mat = (size_t)gp->npad * gp->npad;
+    TRY_BAIL(cudaMalloc(&gp->X, sizeof(float) * batch * (size_t)n * d));
+    TRY_BAIL(cudaMalloc(&gp->ell_d, sizeof(float) * batch * d));
+    TRY_BAIL(cudaMalloc(&gp->inv_ell, sizeof(float) * batch * d));
+    TRY_BAIL(cudaMalloc(&gp->sn2_d, sizeof(float) * batch));
+    TRY_BAIL(cudaMalloc(&gp->sf2_d, sizeof(float) * batch));
+    TRY_BAIL(cudaMalloc(&gp->best_d, sizeof(float) * batch));
+    TRY_BAIL(cudaMalloc(&gp->L64, sizeof(double) * batch * mat));
+    TRY_BAIL(cudaMalloc(&gp->W64, sizeof(double) * batch * mat));
+    TRY_BAIL(cudaMalloc(&gp->W32, sizeof(float) * batch * mat));
+    TRY_BAIL(cudaMalloc(&gp->alpha64, sizeof(double) * batch * gp->npad));
+    TRY_BAIL(cudaMalloc(&gp->alpha32, sizeof(float) * batch * gp->npad));
+    TRY_BAIL(cudaMalloc(&gp->status_d, 2 * sizeof(int)));
+    TRY_BAIL(cudaMallocHost(&gp->status_h, 2 * sizeof(int)));
+    gp->status_h[0] = 0;
+    gp->status_h[1] = INT_MAX;
+    TRY_BAIL(cudaMemcpyAsync(gp->status_d, gp->status_h, 2 * sizeof(int), cudaMemcpyHostToDevice, stream));
+    TRY_BAIL(cudaMemcpyAsync(gp->X, X, sizeof(float) * batch * (size_t)n * d, cudaMemcpyDeviceToDevice, stream));
+    TRY_BAIL(cudaMemcpyAsync(gp->ell_d, gp->ell.data(), sizeof(float) * batch * d, cudaMemcpyHostToDevice, stream));
+    TRY_BAIL(cudaMemcpyAsync(gp->inv_ell, inv.data(), sizeof(float) * batch * d, cudaMemcpyHostToDevice, stream));
+    TRY_BAIL(cudaMemcpyAsync(gp->sn2_d, gp->sn2.data(), sizeof(float) * batch, cudaMemcpyHostToDevice, stream));
+    TRY_BAIL(cudaMemcpyAsync(gp->sf2_d, gp->sf2.data(), sizeof(float) * batch, cudaMemcpyHostToDevice, stream));
+    TRY_BAIL(cudaStreamSynchronize(stream));  // `inv` is a pageable temporary
+#undef TRY_BAIL
+
+    r3_status_t st = fit_device(gp, y, stream);  // synchronises, fills status_h
+    if (st != R3_OK) return bail(st);
+    if (gp->status_h[0] & DEV_NONFINITE) {
+        set_error("r3_gp_fit: X or y contains a non-finite value");
+        return bail(R3_ERR_NONFINITE);
+    }
+    if (gp->status_h[0] & DEV_NOT_PD) {
+        set_error("r3_gp_fit: pivot %d of K + noise*I is not positive (duplicate rows with zero noise?)",
+                  gp->status_h[1]);
+        return bail(R3_ERR_NOT_PD);
+    }
+    if (cudaMemcpy(gp->best.data(), gp->best_d, sizeof(float) * batch, cudaMemcpyDeviceToHost) != cudaSuccess) {
+        set_error("r3_gp_fit: reading back the incumbent failed");
+        return bail(R3_ERR_CUDA);
+    }
+    if (tc_supported(n, d)) {
+        st = tc_prepare(gp, stream);
+        if (st != R3_OK) return bail(st);
+    }
+    *out = gp;
+    return R3_OK;
+}
+
+r3_status_t r3_gp_score(r3_gp_t* gp, const float* Xcand, long long m, float* mu, float* sigma, float* ei,
+                        void* cuda_stream)
+{
+    r3_status_t st = check_score_args(gp, Xcand, m, mu, sigma, ei);
+    if (st != R3_OK) return st;
+    st = ensure_workspace(gp, score_workspace_bytes(gp, m));
+    if (st != R3_OK) return st;
+    return run_score(gp, Xcand, m, mu, sigma, ei, gp->ws, gp->ws_bytes, (cudaStream_t)cuda_stream);
+}
+
+unsigned long long r3_topk_scratch_bytes(int batch, long long m, int k)
+{
+    if (batch < 1 || m < 1 || k < 1) return 0;
+    return topk_workspace_bytes(batch, m, k);
+}
+
+static r3_status_t check_topk_args(const void* ei, int batch, long long m, int k, const void* idx)
+{
+    if (!ei || !idx) {
+        set_error("r3_topk: NULL argument");
+        return R3_ERR_INVALID_ARG;
+    }
+    if (batch < 1 || m < 1 || m >= (1ll << 31) || k < 1 || k > kMaxK || k > m) {
+        set_error("r3_topk: need batch >= 1, 1 <= m < 2^31, 1 <= k <= min(m, %d) (batch=%d m=%lld k=%d)", kMaxK,
+                  batch, m, k);
+        return R3_ERR_INVALID_ARG;
+    }
+    return R3_OK;
+}
+
+r3_status_t r3_topk(const float* ei, int batch, long long m, int k, int* idx, float* val, void* scratch,
+                    unsigned long long scratch_bytes, void* cuda_stream)
+{
+    r3_status_t st = check_topk_args(ei, batch, m, k, idx);
+    if (st != R3_OK) return st;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (scratch) return topk_device(ei, batch, m, k, idx, val, scratch, (size_t)scratch_bytes, stream);
+    void* ws = nullptr;
+    const size_t bytes = topk_workspace_bytes(batch, m, k);
+    R3_CUDA_TRY(cudaMalloc(&ws, bytes));
+    st = topk_device(ei, batch, m, k, idx, val, ws, bytes, stream);
+    cudaError_t e = cudaStreamSynchronize(stream);
+    cudaFree(ws);
+    if (st == R3_OK && e != cudaSuccess) {
+        set_error("r3_topk: %s", cudaGetErrorString(e));
+        st = R3_ERR_CUDA;
+    }
+    return st;
+}
+
+r3_status_t r3_gp_score_topk(r3_gp_t* gp, const float* Xcand, long long m, int k, float* mu, float* sigma,
+                             float* ei, int* idx, float* val, void* cuda_stream)
+{
+    r3_status_t st = check_score_args(gp, Xcand, m, mu, sigma, ei);
+    if (st != R3_OK) return st;
+    st = check_topk_args(ei, gp->batch, m, k, idx);
+    if (st != R3_OK) return st;
+    const size_t sb = align256(score_workspace_bytes(gp, m));
+    const size_t tb = topk_workspace_bytes(gp->batch, m, k);
+    st = ensure_workspace(gp, sb + tb);
+    if (st != R3_OK) return st;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    st = run_score(gp, Xcand, m, mu, sigma, ei, gp->ws, sb, stream);
+    if (st != R3_OK) return st;
+    return topk_device(ei, gp->batch, m, k, idx, val, (char*)gp->ws + sb, tb, stream);
+}
+
+r3_status_t r3_gp_score_topk_host(r3_gp_t* gp, const float* Xcand_host, long long m, int k, float* mu_host,
+                                  float* sigma_host, float* ei_host, int* idx_host, float* val_host,
+                                  void* cuda_stream)
+{
+    if (!gp || !Xcand_host || !idx_host) {
+        set_error("r3_gp_score_topk_host: NULL argument");
+        return R3_ERR_INVALID_ARG;
+    }
+    if (m < 1 || m >= (1ll << 31) || k < 1 || k > kMaxK || k > m) {
+        set_error("r3_gp_score_topk_host: m or k out of range");
+        return R3_ERR_INVALID_ARG;
+    }
+    const size_t B = gp->batch;
+    const size_t sb = align256(score_workspace_bytes(gp, m));
+    const size_t tb = align256(topk_workspace_bytes(gp->batch, m, k));
+    const size_t xb = align256(sizeof(float) * B * m * gp->d);
+    const size_t ob = align256(sizeof(float) * B * m);
+    const size_t kb = align256(sizeof(float) * B * k);
+    r3_status_t st = ensure_workspace(gp, sb + tb + xb + 3 * ob + 2 * kb);
+    if (st != R3_OK) return st;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    char* p = (char*)gp->ws + sb + tb;
+    float* xc = (float*)p;
+    p += xb;
+    float* mu = (float*)p;
+    p += ob;
+    float* sg = (float*)p;
+    p += ob;
+    float* e = (float*)p;
+    p += ob;
+    int* idx = (int*)p;
+    p += kb;
+    float* val = (float*)p;
+    R3_CUDA_TRY(cudaMemcpyAsync(xc, Xcand_host, sizeof(float) * B * m * gp->d, cudaMemcpyHostToDevice, stream));
+    st = run_score(gp, xc, m, mu, sg, e, gp->ws, sb, stream);
+    if (st != R3_OK) return st;
+    st = topk_device(e, gp->batch, m, k, idx, val, (char*)gp->ws + sb, tb, stream);
+    if (st != R3_OK) return st;
+    if (mu_host) R3_CUDA_TRY(cudaMemcpyAsync(mu_host, mu, sizeof(float) * B * m, cudaMemcpyDeviceToHost, stream));
+    if (sigma_host) R3_CUDA_TRY(cudaMemcpyAsync(sigma_host, sg, sizeof(float) * B * m, cudaMemcpyDeviceToHost, stream));
+    if (ei_host) R3_CUDA_TRY(cudaMemcpyAsync(ei_host, e, sizeof(float) * B * m, cudaMemcpyDeviceToHost, stream));
+    R3_CUDA_TRY(cudaMemcpyAsync(idx_host, idx, sizeof(int) * B * k, cudaMemcpyDeviceToHost, stream));
+    if (val_host) R3_CUDA_TRY(cudaMemcpyAsync(val_host, val, sizeof(float) * B * k, cudaMemcpyDeviceToHost, stream));
+    R3_CUDA_TRY(cudaStreamSynchronize(stream));
+    return R3_OK;
+}
+
+r3_status_t r3_gp_check(r3_gp_t* gp, void* cuda_stream)
+{
+    if (!gp) {
+        set_error("r3_gp_check: NULL handle");
+        return R3_ERR_INVALID_ARG;
+    }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    R3_CUDA_TRY(cudaMemcpyAsync(gp->status_h, gp->status_d, 2 * sizeof(int), cudaMemcpyDeviceToHost, stream));
+    R3_CUDA_TRY(cudaMemsetAsync(gp->status_d, 0, sizeof(int), stream));
+    R3_CUDA_TRY(cudaStreamSynchronize(stream));
+    const int bits = gp->status_h[0];
+    if (bits & DEV_TIMEOUT) {
+        set_error("a bounded device-side wait ran out; results are invalid");
+        return R3_ERR_DEVICE_TIMEOUT;
+    }
+    if (bits & DEV_NONFINITE) {
+        set_error("a candidate contains a non-finite value");
+        return R3_ERR_NONFINITE;
+    }
+    return R3_OK;
+}
+
+r3_status_t r3_gp_get_best(const r3_gp_t* gp, float* best)
+{
+    if (!gp || !best) {
+        set_error("r3_gp_get_best: NULL argument");
+        return R3_ERR_INVALID_ARG;
+    }
+    for (int g = 0; g < gp->batch; ++g) best[g] = gp->best[g];
+    return R3_OK;
+}
+
+r3_status_t r3_gp_set_best(r3_gp_t* gp, const float* best)
+{
+    if (!gp || !best) {
+        set_error("r3_gp_set_best: NULL argument");
+        return R3_ERR_INVALID_ARG;
+    }
+    for (int g = 0; g < gp->batch; ++g)
+        if (!isfinite(best[g])) {
+            set_error("r3_gp_set_best: non-finite incumbent for GP %d", g);
+            return R3_ERR_INVALID_ARG;
+        }
+    R3_CUDA_TRY(cudaDeviceSynchronize());
+    R3_CUDA_TRY(cudaMemcpy(gp->best_d, best, sizeof(float) * gp->batch, cudaMemcpyHostToDevice));
+    gp->best.assign(best, best + gp->batch);
+    return R3_OK;
+}
+
+r3_status_t r3_gp_set_engine(r3_gp_t* gp, r3_engine_t engine)
+{
+    if (!gp || (int)engine < 0 || (int)engine > 2) {
+        set_error("r3_gp_set_engine: invalid argument");
+        return R3_ERR_INVALID_ARG;
+    }
+    if (engine == R3_ENGINE_TENSOR && !gp->tc) {
+        set_error("r3_gp_set_engine: the tensor-core engine does not serve n=%d d=%d", gp->n, gp->d);
+        return R3_ERR_UNSUPPORTED;
+    }
+    gp->engine_req = engine;
+    return R3_OK;
+}
+
+r3_status_t r3_gp_profile(r3_gp_t* gp, int enable)
+{
+    if (!gp) {
+        set_error("r3_gp_profile: NULL handle");
+        return R3_ERR_INVALID_ARG;
+    }
+    gp->profile = enable != 0;
+    gp->events_used = 0;
+    return R3_OK;
+}
+
+r3_status_t r3_gp_profile_read(r3_gp_t* gp, double* kernel_ms, long long* launches)
+{
+    if (!gp || !kernel_ms || !launches) {
+        set_error("r3_gp_profile_read: NULL argument");
+        return R3_ERR_INVALID_ARG;
+    }
+    double total = 0.0;
+    for (size_t i = 0; i + 1 < gp->events_used; i += 2) {
+        R3_CUDA_TRY(cudaEventSynchronize(gp->events[i + 1]));
+        float ms = 0.f;
+        R3_CUDA_TRY(cudaEventElapsedTime(&ms, gp->events[i], gp->events[i + 1]));
+        total += ms;
+    }
+    *kernel_ms = total;
+    *launches = (long long)(gp->events_used / 2);
+    gp->events_used = 0;
+    return R3_OK;
+}
+
+r3_engine_t r3_gp_engine(const r3_gp_t* gp) { return gp ? pick_engine(gp) : R3_ENGINE_SIMT; }
+
+r3_status_t r3_gp_get_factor(const r3_gp_t* gp, double* alpha, double* L)
+{
+    if (!gp) {
+        set_error("r3_gp_get_factor: NULL handle");
+        return R3_ERR_INVALID_ARG;
+    }
+    R3_CUDA_TRY(cudaDeviceSynchronize());
+    const int n = gp->n, npad = gp->npad;
+    for (int g = 0; g < gp->batch; ++g) {
+        if (alpha)
+            R3_CUDA_TRY(cudaMemcpy(alpha + (size_t)g * n, gp->alpha64 + (size_t)g * npad, sizeof(double) * n,
+                                   cudaMemcpyDeviceToHost));
+        if (L)
+            R3_CUDA_TRY(cudaMemcpy2D(L + (size_t)g * n * n, sizeof(double) * n, gp->L64 + (size_t)g * npad * npad,
+                                     sizeof(double) * npad, sizeof(double) * n, n, cudaMemcpyDeviceToHost));
+    }
+    return R3_OK;
+}
+
+}  // extern "C"

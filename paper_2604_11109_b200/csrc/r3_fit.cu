@@ -1,0 +1,408 @@
+// r3_gp_fit on the device: FP64 Gram matrix, blocked batched Cholesky, inverse factor, weights.
+//
+// Everything here runs once per BO round, in FP64, and is rounded to FP32 once at the end:
+//   K = k(X,X) + noise*I           gram_kernel            (direct differences, like the definition)
+//   K = L L^T                      potrf_diag / panel / syrk kernels, right-looking, block 32
+//   W = L^-1                       diagonal-block inverses, then recursive doubling with two
+//                                  batched GEMMs per level:  W21 = -W22 (L21 W11)
+//   alpha = W^T (W y)              two triangular matrix-vector products
+// All kernels take the GP index from blockIdx.z (or .y), so `batch` GPs are factored together.
+// n is padded to a multiple of 32 with an identity block, which leaves L, W and alpha unchanged.
+#include "r3_internal.cuh"
+
+namespace r3 {
+
+namespace {
+
+constexpr int NB = kFitBlock;
+
+// ------------------------------------------------------------------------------------ checks
+__global__ void check_finite_kernel(const float* __restrict__ a, size_t count, int* status)
+{
+    bool bad = false;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < count;
+         i += (size_t)gridDim.x * blockDim.x)
+        bad |= !isfinite(a[i]);
+    if (__syncthreads_or(bad) && threadIdx.x == 0) atomicOr(status, DEV_NONFINITE);
+}
+
+__global__ void min_y_kernel(const float* __restrict__ y, int n, float* best)
+{
+    __shared__ float s[256];
+    const float* yg = y + (size_t)blockIdx.x * n;
+    float v = INFINITY;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) v = fminf(v, yg[i]);
+    s[threadIdx.x] = v;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) s[threadIdx.x] = fminf(s[threadIdx.x], s[threadIdx.x + o]);
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) best[blockIdx.x] = s[0];
+}
+
+// ------------------------------------------------------------------------------------ Gram
+// One 16x16 tile of the lower triangle per block; r^2 by direct differences in FP64 with a true
+// division by the lengthscale, the Matern-5/2 profile, noise on the diagonal.
+__global__ void gram_kernel(const float* __restrict__ X, const float* __restrict__ ell,
+                            const float* __restrict__ sf2, const float* __restrict__ sn2, int n, int d,
+                            int npad, double* __restrict__ K)
+{
+    const int g = blockIdx.z;
+    const int ti = blockIdx.y, tj = blockIdx.x;
+    const int tx = threadIdx.x, ty = threadIdx.y;
+    const int i = ti * 16 + ty, j = tj * 16 + tx;
+    double* Kg = K + (size_t)g * npad * npad;
+    if (tj > ti) {
+        Kg[(size_t)i * npad + j] = 0.0;
+        return;
+    }
+    __shared__ float sxi[16][33], sxj[16][33];
+    __shared__ float sl[32];
+    const float* Xg = X + (size_t)g * n * d;
+    double r2 = 0.0;
+    for (int c0 = 0; c0 < d; c0 += 32) {
+        const int t = ty * 16 + tx;  // 0..255
+        for (int e = t; e < 16 * 32; e += 256) {
+            int r = e / 32, c = e % 32;
+            int gi = ti * 16 + r, gj = tj * 16 + r;
+            sxi[r][c] = (gi < n && c0 + c < d) ? Xg[(size_t)gi * d + c0 + c] : 0.f;
+            sxj[r][c] = (gj < n && c0 + c < d) ? Xg[(size_t)gj * d + c0 + c] : 0.f;
+        }
+        if (t < 32) sl[t] = (c0 + t < d) ? ell[(size_t)g * d + c0 + t] : 1.f;
+        __syncthreads();
+        const int cmax = min(32, d - c0);
+        for (int c = 0; c < cmax; ++c) {
+            double diff = ((double)sxi[ty][c] - (double)sxj[tx][c]) / (double)sl[c];
+            r2 += diff * diff;
+        }
+        __syncthreads();
+    }
+    double v;
+    if (i < n && j < n) {
+        double s = sqrt(5.0) * sqrt(r2);
+        v = (double)sf2[g] * (1.0 + s + s * s / 3.0) * exp(-s);
+        if (i == j) v += (double)sn2[g];
+        if (j > i) v = 0.0;
+    } else {
+        v = (i == j) ? 1.0 : 0.0;
+    }
+    Kg[(size_t)i * npad + j] = v;
+}
+
+// ------------------------------------------------------------------------------------ Cholesky
+// Factor the 32x32 diagonal block at j0 in shared memory, write it back (upper part zeroed) and
+// store its inverse in Dinv[g][j0/32].
+__global__ void __launch_bounds__(1024) potrf_diag_kernel(double* __restrict__ A, int npad, int j0,
+                                                          double* __restrict__ Dinv, int* status)
+{
+    const int g = blockIdx.x;
+    const int tx = threadIdx.x, ty = threadIdx.y;
+    double* Ag = A + (size_t)g * npad * npad + (size_t)j0 * npad + j0;
+    __shared__ double a[NB][NB + 1];
+    __shared__ double inv[NB][NB + 1];
+    a[ty][tx] = Ag[(size_t)ty * npad + tx];
+    __syncthreads();
+    for (int k = 0; k < NB; ++k) {
+        if (tx == k && ty == k) {
+            double p = a[k][k];
+            if (!(p > 0.0) || !isfinite(p)) {
+                atomicOr(&status[0], DEV_NOT_PD);
+                atomicMin(&status[1], j0 + k);
+                p = 1.0;  // keep going without NaNs; the call reports the failure
+            }
+            a[k][k] = sqrt(p);
+        }
+        __syncthreads();
+        if (tx == k && ty > k) a[ty][k] /= a[k][k];
+        __syncthreads();
+        if (tx > k && ty >= tx) a[ty][tx] -= a[ty][k] * a[tx][k];
+        __syncthreads();
+    }
+    // inverse of the lower-triangular block, one column per thread of the first warp row
+    if (ty == 0) {
+        const int c = tx;
+        for (int i = 0; i < NB; ++i) {
+            double s = (i == c) ? 1.0 : 0.0;
+            if (i < c) {
+                inv[i][c] = 0.0;
+                continue;
+            }
+            for (int k = c; k < i; ++k) s -= a[i][k] * inv[k][c];
+            inv[i][c] = s / a[i][i];
+        }
+    }
+    __syncthreads();
+    Ag[(size_t)ty * npad + tx] = (tx <= ty) ? a[ty][tx] : 0.0;
+    Dinv[((size_t)g * (npad / NB) + j0 / NB) * NB * NB + ty * NB + tx] = inv[ty][tx];
+}
+
+// Panel below the diagonal block: L_panel = A_panel * inv(L_jj)^T, 64 rows per block.
+__global__ void __launch_bounds__(256) panel_kernel(double* __restrict__ A, int npad, int j0,
+                                                    const double* __restrict__ Dinv)
+{
+    const int g = blockIdx.y;
+    const int r0 = j0 + NB + blockIdx.x * 64;
+    double* Ag = A + (size_t)g * npad * npad;
+    const double* Dg = Dinv + ((size_t)g * (npad / NB) + j0 / NB) * NB * NB;
+    __shared__ double sd[NB][NB + 1];
+    __shared__ double sa[64][NB + 1];
+    const int t = threadIdx.x;
+    for (int e = t; e < NB * NB; e += 256) sd[e / NB][e % NB] = Dg[e];
+    for (int e = t; e < 64 * NB; e += 256) {
+        int r = e / NB, c = e % NB;
+        sa[r][c] = (r0 + r < npad) ? Ag[(size_t)(r0 + r) * npad + j0 + c] : 0.0;
+    }
+    __syncthreads();
+    const int r = t / 4, cb = (t % 4) * 8;
+    if (r0 + r < npad) {
+        for (int c = cb; c < cb + 8; ++c) {
+            double s = 0.0;
+            for (int k = 0; k <= c; ++k) s += sa[r][k] * sd[c][k];
+            Ag[(size_t)(r0 + r) * npad + j0 + c] = s;
+        }
+    }
+}
+
+// Trailing update: A[i][j] -= sum_k P[i][k] P[j][k] over the 32 panel columns, 64x64 tiles of the
+// lower triangle of the trailing matrix.
+__global__ void __launch_bounds__(256) syrk_kernel(double* __restrict__ A, int npad, int j0)
+{
+    const int ti = blockIdx.y, tj = blockIdx.x;
+    if (tj > ti) return;
+    const int g = blockIdx.z;
+    const int base = j0 + NB;
+    double* Ag = A + (size_t)g * npad * npad;
+    __shared__ double pi[64][NB + 1], pj[64][NB + 1];
+    const int t = threadIdx.x;
+    for (int e = t; e < 64 * NB; e += 256) {
+        int r = e / NB, c = e % NB;
+        int gi = base + ti * 64 + r, gj = base + tj * 64 + r;
+        pi[r][c] = (gi < npad) ? Ag[(size_t)gi * npad + j0 + c] : 0.0;
+        pj[r][c] = (gj < npad) ? Ag[(size_t)gj * npad + j0 + c] : 0.0;
+    }
+    __syncthreads();
+    const int ty = t / 16, tx = t % 16;
+    double acc[4][4] = {};
+#pragma unroll 8
+    for (int k = 0; k < NB; ++k) {
+        double a[4], b[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            a[u] = pi[ty + 16 * u][k];
+            b[u] = pj[tx + 16 * u][k];
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+#pragma unroll
+            for (int v = 0; v < 4; ++v) acc[u][v] += a[u] * b[v];
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            int gi = base + ti * 64 + ty + 16 * u, gj = base + tj * 64 + tx + 16 * v;
+            if (gi < npad && gj <= gi) Ag[(size_t)gi * npad + gj] -= acc[u][v];
+        }
+}
+
+// ------------------------------------------------------------------------------------ inverse
+__global__ void scatter_dinv_kernel(const double* __restrict__ Dinv, int npad, double* __restrict__ W)
+{
+    // W = block-diag(Dinv): one 32x32 block per blockIdx.x, GP per blockIdx.y; rest zero already
+    const int g = blockIdx.y, b = blockIdx.x;
+    const double* Dg = Dinv + ((size_t)g * (npad / NB) + b) * NB * NB;
+    double* Wg = W + (size_t)g * npad * npad + (size_t)(b * NB) * npad + b * NB;
+    Wg[(size_t)threadIdx.y * npad + threadIdx.x] = Dg[threadIdx.y * NB + threadIdx.x];
+}
+
+// Batched FP64 GEMM used by the recursive-doubling inverse.  For pair p (blockIdx.z % npairs) of
+// GP g (blockIdx.z / npairs), with block size s:  rows2 = [(2p+1)s, min((2p+2)s, npad)),
+// cols1 = [2p s, (2p+1)s).
+//   mode 0:  T[rows2][cols1]  =  L[rows2][cols1] * W[cols1][cols1]     (W11 lower: k >= j)
+//   mode 1:  W[rows2][cols1]  = -W[rows2][rows2] * T[rows2][cols1]     (W22 lower: k <= i)
+__global__ void __launch_bounds__(256) trtri_gemm_kernel(const double* __restrict__ Amat,
+                                                         const double* __restrict__ Bmat,
+                                                         double* __restrict__ Cmat, int npad, int s,
+                                                         int npairs, int mode)
+{
+    const int p = blockIdx.z % npairs, g = blockIdx.z / npairs;
+    const int row2 = (2 * p + 1) * s, col1 = 2 * p * s;
+    const int M = min(s, npad - row2);
+    const int N = s;
+    const int i0 = blockIdx.y * 64, j0 = blockIdx.x * 64;
+    if (i0 >= M || j0 >= N) return;
+    const size_t gs = (size_t)g * npad * npad;
+    const double* A;
+    const double* B;
+    double* C = Cmat + gs + (size_t)row2 * npad + col1;
+    int K, kbeg, kend;
+    if (mode == 0) {
+        A = Amat + gs + (size_t)row2 * npad + col1;
+        B = Bmat + gs + (size_t)col1 * npad + col1;
+        K = s;
+        kbeg = j0;  // W11[k][j] == 0 for k < j
+        kend = K;
+    } else {
+        A = Amat + gs + (size_t)row2 * npad + row2;
+        B = Bmat + gs + (size_t)row2 * npad + col1;
+        K = M;
+        kbeg = 0;
+        kend = min(K, i0 + 64);  // W22[i][k] == 0 for k > i
+    }
+    __shared__ double sa[64][17], sb[16][65];
+    const int t = threadIdx.x, ty = t / 16, tx = t % 16;
+    double acc[4][4] = {};
+    for (int k0 = kbeg; k0 < kend; k0 += 16) {
+        for (int e = t; e < 64 * 16; e += 256) {
+            int r = e / 16, c = e % 16;
+            sa[r][c] = (i0 + r < M && k0 + c < K) ? A[(size_t)(i0 + r) * npad + k0 + c] : 0.0;
+        }
+        for (int e = t; e < 16 * 64; e += 256) {
+            int r = e / 64, c = e % 64;
+            sb[r][c] = (k0 + r < K && j0 + c < N) ? B[(size_t)(k0 + r) * npad + j0 + c] : 0.0;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            double a[4], b[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                a[u] = sa[ty + 16 * u][k];
+                b[u] = sb[k][tx + 16 * u];
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int v = 0; v < 4; ++v) acc[u][v] += a[u] * b[v];
+        }
+        __syncthreads();
+    }
+    const double sign = mode == 0 ? 1.0 : -1.0;
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            int i = i0 + ty + 16 * u, j = j0 + tx + 16 * v;
+            if (i < M && j < N) C[(size_t)i * npad + j] = sign * acc[u][v];
+        }
+}
+
+// ------------------------------------------------------------------------------------ weights
+// u = W y (lower-triangular W, one warp per row); rows >= n give 0.
+__global__ void w_times_y_kernel(const double* __restrict__ W, const float* __restrict__ y, int n,
+                                 int npad, double* __restrict__ u)
+{
+    const int g = blockIdx.y;
+    const int row = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
+    const int lane = threadIdx.x % 32;
+    if (row >= npad) return;
+    const double* Wr = W + (size_t)g * npad * npad + (size_t)row * npad;
+    double s = 0.0;
+    if (row < n)
+        for (int k = lane; k <= row; k += 32) s += Wr[k] * (double)y[(size_t)g * n + k];
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) u[(size_t)g * npad + row] = s;
+}
+
+// alpha = W^T u (one thread per column, coalesced across columns); also the FP32 copy.
+__global__ void wt_times_u_kernel(const double* __restrict__ W, const double* __restrict__ u, int n,
+                                  int npad, double* __restrict__ alpha64, float* __restrict__ alpha32)
+{
+    const int g = blockIdx.y;
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= npad) return;
+    const double* Wg = W + (size_t)g * npad * npad;
+    double s = 0.0;
+    if (j < n)
+        for (int i = j; i < n; ++i) s += Wg[(size_t)i * npad + j] * u[(size_t)g * npad + i];
+    alpha64[(size_t)g * npad + j] = s;
+    alpha32[(size_t)g * npad + j] = (float)s;
+}
+
+__global__ void to_float_kernel(const double* __restrict__ a, float* __restrict__ b, size_t count)
+{
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < count;
+         i += (size_t)gridDim.x * blockDim.x)
+        b[i] = (float)a[i];
+}
+
+}  // namespace
+
+// Runs the whole fit on `stream`.  gp->X, ell (device copies) and the scalar arrays are already in
+// place; L64, W64, W32, alpha*, best_d are filled.  The caller synchronises and reads status_d.
+r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream)
+{
+    const int B = gp->batch, n = gp->n, d = gp->d, npad = gp->npad;
+    const size_t mat = (size_t)npad * npad;
+    double *Dinv = nullptr, *T = nullptr, *u = nullptr;
+    R3_CUDA_TRY(cudaMalloc(&Dinv, sizeof(double) * B * (size_t)(npad / NB) * NB * NB));
+    auto fail = [&](r3_status_t st) {
+        cudaFree(Dinv);
+        cudaFree(T);
+        cudaFree(u);
+        return st;
+    };
+#define TRY_OR_FAIL(expr)                                                                          \
+    do {                                                                                           \
+        cudaError_t e__ = (expr);                                                                  \
+        if (e__ != cudaSuccess) {                                                                  \
+            set_error("%s failed: %s", #expr, cudaGetErrorString(e__));                            \
+            return fail(e__ == cudaErrorMemoryAllocation ? R3_ERR_ALLOC : R3_ERR_CUDA);            \
+        }                                                                                          \
+    } while (0)
+#define LAUNCH_OR_FAIL(kernel, grid, block, ...)                                                   \
+    do {                                                                                           \
+        kernel<<<(grid), (block), 0, stream>>>(__VA_ARGS__);                                       \
+        ++g_launches;                                                                              \
+        cudaError_t e__ = cudaGetLastError();                                                      \
+        if (e__ != cudaSuccess) {                                                                  \
+            set_error("launch of %s failed: %s", #kernel, cudaGetErrorString(e__));                \
+            return fail(R3_ERR_CUDA);                                                              \
+        }                                                                                          \
+    } while (0)
+
+    TRY_OR_FAIL(cudaMalloc(&T, sizeof(double) * B * mat));
+    TRY_OR_FAIL(cudaMalloc(&u, sizeof(double) * B * npad));
+
+    LAUNCH_OR_FAIL(check_finite_kernel, 296, 256, gp->X, (size_t)B * n * d, gp->status_d);
+    LAUNCH_OR_FAIL(check_finite_kernel, 64, 256, y, (size_t)B * n, gp->status_d);
+    LAUNCH_OR_FAIL(min_y_kernel, B, 256, y, n, gp->best_d);
+
+    LAUNCH_OR_FAIL(gram_kernel, dim3(npad / 16, npad / 16, B), dim3(16, 16), gp->X, gp->ell_d, gp->sf2_d,
+                   gp->sn2_d, n, d, npad, gp->L64);
+
+    for (int j0 = 0; j0 < npad; j0 += NB) {
+        LAUNCH_OR_FAIL(potrf_diag_kernel, B, dim3(NB, NB), gp->L64, npad, j0, Dinv, gp->status_d);
+        const int rows = npad - j0 - NB;
+        if (rows > 0) {
+            const int tiles = (rows + 63) / 64;
+            LAUNCH_OR_FAIL(panel_kernel, dim3(tiles, B), 256, gp->L64, npad, j0, Dinv);
+            LAUNCH_OR_FAIL(syrk_kernel, dim3(tiles, tiles, B), 256, gp->L64, npad, j0);
+        }
+    }
+
+    TRY_OR_FAIL(cudaMemsetAsync(gp->W64, 0, sizeof(double) * B * mat, stream));
+    LAUNCH_OR_FAIL(scatter_dinv_kernel, dim3(npad / NB, B), dim3(NB, NB), Dinv, npad, gp->W64);
+    for (int s = NB; s < npad; s *= 2) {
+        const int npairs = (npad + 2 * s - 1) / (2 * s);   // a last lone block has M <= 0 and exits
+        const int tiles = (s + 63) / 64;
+        dim3 grid(tiles, tiles, npairs * B);
+        LAUNCH_OR_FAIL(trtri_gemm_kernel, grid, 256, gp->L64, gp->W64, T, npad, s, npairs, 0);
+        LAUNCH_OR_FAIL(trtri_gemm_kernel, grid, 256, gp->W64, T, gp->W64, npad, s, npairs, 1);
+    }
+
+    LAUNCH_OR_FAIL(w_times_y_kernel, dim3((npad + 7) / 8, B), 256, gp->W64, y, n, npad, u);
+    LAUNCH_OR_FAIL(wt_times_u_kernel, dim3((npad + 127) / 128, B), 128, gp->W64, u, n, npad,
+                   gp->alpha64, gp->alpha32);
+    LAUNCH_OR_FAIL(to_float_kernel, 1184, 256, gp->W64, gp->W32, (size_t)B * mat);
+
+    TRY_OR_FAIL(cudaMemcpyAsync(gp->status_h, gp->status_d, 2 * sizeof(int), cudaMemcpyDeviceToHost, stream));
+    TRY_OR_FAIL(cudaStreamSynchronize(stream));
+#undef TRY_OR_FAIL
+#undef LAUNCH_OR_FAIL
+    fail(R3_OK);  // frees the temporaries
+    return R3_OK;
+}
+
+}  // namespace r3

@@ -1,0 +1,132 @@
+// Internal declarations shared by the translation units of libr3gp (CUDA, sm_100a).
+// Nothing here is part of the public ABI; see include/r3.h for that.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "r3.h"
+
+namespace r3 {
+
+// ---------------------------------------------------------------------------------------------
+// error text (thread-local) and launch accounting
+void set_error(const char* fmt, ...);
+extern thread_local unsigned long long g_launches;
+
+#define R3_CUDA_TRY(expr)                                                                \
+    do {                                                                                 \
+        cudaError_t e__ = (expr);                                                        \
+        if (e__ != cudaSuccess) {                                                        \
+            r3::set_error("%s failed: %s (%s:%d)", #expr, cudaGetErrorString(e__),       \
+                          __FILE__, __LINE__);                                           \
+            return e__ == cudaErrorMemoryAllocation ? R3_ERR_ALLOC : R3_ERR_CUDA;        \
+        }                                                                                \
+    } while (0)
+
+// Launch a kernel, count it, and turn a launch error into a status.
+#define R3_LAUNCH(kernel, grid, block, smem, stream, ...)                                \
+    do {                                                                                 \
+        kernel<<<(grid), (block), (smem), (stream)>>>(__VA_ARGS__);                      \
+        ++r3::g_launches;                                                                \
+        cudaError_t e__ = cudaGetLastError();                                            \
+        if (e__ != cudaSuccess) {                                                        \
+            r3::set_error("launch of %s failed: %s (%s:%d)", #kernel,                    \
+                          cudaGetErrorString(e__), __FILE__, __LINE__);                  \
+            return R3_ERR_CUDA;                                                          \
+        }                                                                                \
+    } while (0)
+
+// Bits of the device status word (one int per handle, OR-ed by kernels).
+enum : int {
+    DEV_NONFINITE = 1,   // NaN/Inf met in an input
+    DEV_NOT_PD = 2,      // non-positive Cholesky pivot
+    DEV_TIMEOUT = 4,     // a bounded wait gave up
+};
+
+constexpr int kFitBlock = 32;   // Cholesky / inverse block size; n is padded to a multiple of it
+constexpr int kMaxN = 8192;
+constexpr int kMaxD = 256;
+constexpr int kMaxK = 1024;
+
+inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
+inline long long round_up_ll(long long a, long long b) { return (a + b - 1) / b * b; }
+
+}  // namespace r3
+
+// The handle.  Device arrays are allocated at fit time and freed by r3_gp_free.
+struct r3_gp {
+    int batch = 0, n = 0, d = 0;
+    int npad = 0;              // n rounded up to kFitBlock; padded rows/cols are identity / zero
+    int device = 0;
+    std::vector<float> ell, sf2, sn2, best;   // host copies [batch][d], [batch], [batch], [batch]
+
+    float* X = nullptr;        // [batch][n][d]   raw observations (FP32 as given)
+    float* ell_d = nullptr;    // [batch][d]      lengthscales as given
+    float* inv_ell = nullptr;  // [batch][d]      1/lengthscale
+    float* sn2_d = nullptr;    // [batch]
+    float* sf2_d = nullptr;    // [batch]
+    float* best_d = nullptr;   // [batch]
+    double* L64 = nullptr;     // [batch][npad][npad] lower Cholesky factor (upper part zero)
+    double* W64 = nullptr;     // [batch][npad][npad] W = L^-1, lower
+    float* W32 = nullptr;      // [batch][npad][npad] W rounded to FP32
+    double* alpha64 = nullptr; // [batch][npad]  (zero in the padding)
+    float* alpha32 = nullptr;  // [batch][npad]
+    int* status_d = nullptr;   // [2]: status bits, first bad pivot index
+    int* status_h = nullptr;   // pinned mirror of status_d
+
+    // tensor-core operands (built by fit when the tensor engine can serve (n, d))
+    void* tc = nullptr;        // r3::TensorOperands*, see r3_score_tc.cu
+
+    // grow-only private workspace used by scoring and top-k
+    void* ws = nullptr;
+    size_t ws_bytes = 0;
+
+    r3_engine_t engine_req = R3_ENGINE_AUTO;
+
+    // optional timing of the dominant scoring kernel: event pairs recorded around its launches
+    bool profile = false;
+    std::vector<cudaEvent_t> events;   // pairs (start, stop)
+    size_t events_used = 0;
+};
+
+namespace r3 {
+
+// fit (r3_fit.cu)
+r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream);
+
+// SIMT scoring (r3_score_simt.cu)
+size_t score_simt_workspace_bytes(const r3_gp* gp, long long m);
+r3_status_t score_simt(r3_gp* gp, const float* Xcand, long long m, float* mu, float* sigma, float* ei,
+                       void* ws, size_t ws_bytes, cudaStream_t stream);
+
+// FP64 rescue of the candidates whose variance is too small for FP32-level partial results
+// (r3_rescue.cu).  The engines append such candidates to a list while they write their own
+// FP32-level mu/sigma/EI; this pass recomputes those entries entirely in FP64 and overwrites them.
+//   list  [cap]  flat candidate ids g*m + j;  count[0] = entries appended (may exceed cap: clamped)
+r3_status_t rescue(r3_gp* gp, const float* Xcand, long long m, const int* count, const long long* list,
+                   long long cap, float* mu, float* sigma, float* ei, cudaStream_t stream);
+
+// tensor-core scoring (r3_score_tc.cu)
+bool tc_supported(int n, int d);
+r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream);
+void tc_release(r3_gp* gp);
+size_t score_tc_workspace_bytes(const r3_gp* gp, long long m);
+r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, float* sigma, float* ei,
+                     void* ws, size_t ws_bytes, cudaStream_t stream);
+
+// top-k (r3_topk.cu)
+size_t topk_workspace_bytes(int batch, long long m, int k);
+r3_status_t topk_device(const float* ei, int batch, long long m, int k, int* idx, float* val, void* ws,
+                        size_t ws_bytes, cudaStream_t stream);
+
+r3_status_t ensure_workspace(r3_gp* gp, size_t bytes);
+
+// Event pair around one launch of the dominant kernel (no-ops unless profiling is on).
+void prof_begin(r3_gp* gp, cudaStream_t stream);
+void prof_end(r3_gp* gp, cudaStream_t stream);
+
+}  // namespace r3

@@ -1,0 +1,284 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the FP64 CPU oracle.
+
+Small cases compare every output element; the five workloads run at their full sizes on the GPU and
+are compared on every candidate where the oracle finishes in seconds, else on a seeded sample of
+candidates, with top-k checked against the oracle's EI on the sample pool or a stored full-pool
+top list.  Tolerances are the ones in tests/parity.py.
+"""
+import json
+import os
+
+import numpy as np
+import pytest
+
+from oracle import gp_oracle as o
+from paper_2604_11109_b200 import binding as b
+from paper_2604_11109_b200 import workloads as w
+from tests.parity import check_scores, check_topk
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+ENGINES = [b.ENGINE_SIMT, b.ENGINE_TENSOR]
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def fit_gpu(g, engine=None):
+    gp = b.r3_gp_fit(dev(g["X"]), dev(g["y"]), g["ell"], g["sf2"], g["sn2"])
+    if engine is not None:
+        try:
+            b.r3_gp_set_engine(gp, engine)
+        except b.R3Error as e:
+            if e.status == 7:
+                gp.close()
+                pytest.skip("engine does not serve this shape")
+            raise
+    return gp
+
+
+def rand_problem(seed, batch, n, d, m, sn2=1e-3, sf2=1.0, spread=1.0):
+    rng = np.random.default_rng(seed)
+    return {
+        "X": rng.uniform(0, 1, (batch, n, d)).astype(np.float32),
+        "y": rng.normal(0, 1, (batch, n)).astype(np.float32),
+        "ell": (rng.uniform(0.3, 1.5, (batch, d)) * spread).astype(np.float32),
+        "sf2": np.full(batch, sf2, np.float32) * rng.uniform(0.5, 2.0, batch).astype(np.float32),
+        "sn2": np.full(batch, sn2, np.float32),
+        "Xcand": rng.uniform(-0.1, 1.1, (batch, m, d)).astype(np.float32),
+    }
+
+
+def oracle_all(g):
+    fits = o.fit_batch(g["X"], g["y"], g["ell"], g["sf2"], g["sn2"])
+    mu, sd, ei = o.score_batch(fits, g["Xcand"])
+    return fits, mu, sd, ei
+
+
+def compare_everything(g, gp, k, what):
+    fits, mu_r, sd_r, ei_r = oracle_all(g)
+    mu, sd, ei, idx, val = b.r3_gp_score_topk(gp, dev(g["Xcand"]), k)
+    b.r3_gp_check(gp)
+    mu, sd, ei, idx, val = (t.cpu().numpy() for t in (mu, sd, ei, idx, val))
+    for q in range(g["X"].shape[0]):
+        check_scores(mu[q], sd[q], ei[q], mu_r[q], sd_r[q], ei_r[q], float(np.abs(g["y"][q]).max()),
+                     float(g["sf2"][q]), what=f"{what} gp{q}")
+        ridx, rval = o.topk(ei_r[q], min(k + 1, ei_r[q].size))
+        nxt = rval[k] if rval.size > k else -np.inf
+        check_topk(idx[q], lambda i, q=q: ei_r[q][i], ridx[:k], rval[:k], nxt, ei_r[q].max(), what=f"{what} gp{q}")
+        # the returned values are the EI entries at the returned indices, in descending order
+        assert np.array_equal(val[q], ei[q][idx[q]])
+        assert np.all(np.diff(val[q]) <= 0)
+
+
+# ------------------------------------------------------------------------------------------ fit
+@pytest.mark.parametrize("batch,n,d", [(1, 1, 1), (1, 7, 2), (2, 33, 5), (1, 64, 6), (3, 100, 17), (1, 257, 40)])
+def test_fit_factor_and_weights_match_oracle(batch, n, d):
+    g = rand_problem(100 + n, batch, n, d, 4)
+    gp = fit_gpu(g)
+    alpha, L = b.r3_gp_get_factor(gp)
+    best = b.r3_gp_get_best(gp)
+    for q, f in enumerate(o.fit_batch(g["X"], g["y"], g["ell"], g["sf2"], g["sn2"])):
+        assert np.allclose(L[q], f.L, rtol=1e-9, atol=1e-11)
+        assert np.allclose(alpha[q], f.alpha, rtol=1e-7, atol=1e-9 * np.abs(f.alpha).max())
+        assert best[q] == np.float32(f.best)
+    gp.close()
+
+
+def test_fit_reports_not_positive_definite_and_non_finite():
+    X = np.array([[[0.1, 0.2], [0.1, 0.2], [0.7, 0.3]]], dtype=np.float32)
+    y = np.zeros((1, 3), np.float32)
+    with pytest.raises(b.R3Error) as e:
+        b.r3_gp_fit(dev(X), dev(y), np.ones((1, 2)), 1.0, 0.0)
+    assert e.value.status == 3
+    X[0, 1, 0] = np.nan
+    with pytest.raises(b.R3Error) as e:
+        b.r3_gp_fit(dev(X), dev(y), np.ones((1, 2)), 1.0, 0.1)
+    assert e.value.status == 2
+    # the context stays usable
+    g = rand_problem(1, 1, 8, 2, 4)
+    fit_gpu(g).close()
+
+
+# ------------------------------------------------------------------------------------------ small, element by element
+SMALL = [  # batch, n, d, m, k: several tiles and ragged tails in every dimension
+    (1, 1, 1, 1, 1),
+    (1, 5, 1, 3, 2),
+    (1, 50, 3, 333, 8),
+    (2, 64, 6, 1000, 16),
+    (1, 130, 33, 1500, 32),
+    (3, 200, 16, 777, 5),
+    (1, 300, 70, 2049, 64),
+    (1, 520, 128, 640, 128),
+]
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+@pytest.mark.parametrize("batch,n,d,m,k", SMALL)
+def test_small_cases_every_element(engine, batch, n, d, m, k):
+    g = rand_problem(7 * n + d, batch, n, d, m)
+    gp = fit_gpu(g, engine)
+    compare_everything(g, gp, k, f"small n{n} d{d} m{m}")
+    gp.close()
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+def test_candidates_on_and_near_observations_are_rescued(engine):
+    # sigma ~ sqrt(noise) at observed points: the regime where sf2 - q cancels
+    g = rand_problem(55, 1, 96, 6, 512, sn2=1e-4, spread=2.0)
+    g["Xcand"][0, :96] = g["X"][0]
+    g["Xcand"][0, 96:192] = g["X"][0] + np.float32(1e-3)
+    gp = fit_gpu(g, engine)
+    compare_everything(g, gp, 8, "near-observation")
+    gp.close()
+
+
+def test_incumbent_override_and_engine_query():
+    g = rand_problem(77, 2, 40, 4, 300)
+    gp = fit_gpu(g)
+    assert b.r3_gp_engine(gp) in (b.ENGINE_SIMT, b.ENGINE_TENSOR)
+    best = b.r3_gp_get_best(gp) - np.float32(0.5)
+    b.r3_gp_set_best(gp, best)
+    assert np.array_equal(b.r3_gp_get_best(gp), best)
+    mu, sd, ei = (t.cpu().numpy() for t in b.r3_gp_score(gp, dev(g["Xcand"])))
+    fits = o.fit_batch(g["X"], g["y"], g["ell"], g["sf2"], g["sn2"])
+    for q, f in enumerate(fits):
+        mu_r, sd_r, ei_r = o.score(f, g["Xcand"][q], best=float(best[q]))
+        check_scores(mu[q], sd[q], ei[q], mu_r, sd_r, ei_r, float(np.abs(g["y"][q]).max()), float(g["sf2"][q]))
+    gp.close()
+
+
+def test_non_finite_candidate_is_latched_not_fatal():
+    g = rand_problem(78, 1, 20, 3, 100)
+    gp = fit_gpu(g)
+    xc = g["Xcand"].copy()
+    xc[0, 17, 1] = np.inf
+    b.r3_gp_score(gp, dev(xc))
+    with pytest.raises(b.R3Error) as e:
+        b.r3_gp_check(gp)
+    assert e.value.status == 2
+    b.r3_gp_score(gp, dev(g["Xcand"]))
+    b.r3_gp_check(gp)  # cleared
+    gp.close()
+
+
+def test_host_buffer_form_equals_device_form():
+    g = rand_problem(79, 2, 70, 9, 1234)
+    gp = fit_gpu(g)
+    k = 10
+    mu, sd, ei, idx, val = (t.cpu() for t in b.r3_gp_score_topk(gp, dev(g["Xcand"]), k))
+    xh = torch.from_numpy(g["Xcand"]).pin_memory()
+    out = (torch.empty(2, 1234).pin_memory(), torch.empty(2, 1234).pin_memory(), torch.empty(2, 1234).pin_memory(),
+           torch.empty(2, k, dtype=torch.int32).pin_memory(), torch.empty(2, k).pin_memory())
+    b.r3_gp_score_topk_host(gp, xh, k, out)
+    for a, c in zip((mu, sd, ei, idx, val), out):
+        assert torch.equal(a, c)
+    gp.close()
+
+
+# ------------------------------------------------------------------------------------------ top-k alone (bit-exact)
+@pytest.mark.parametrize("batch,m,k", [(1, 1, 1), (1, 100, 100), (2, 4096, 7), (1, 4097, 1024), (3, 70001, 33),
+                                       (1, 1 << 20, 128), (64, 65536, 16)])
+def test_topk_matches_oracle_exactly(batch, m, k):
+    rng = np.random.default_rng(m + k)
+    e = rng.random((batch, m)).astype(np.float32)
+    if m > 50:
+        e[:, [3, m // 2, m - 1]] = 2.0                    # ties at the top: lower index first
+        e[:, 10:20] = e[:, 5:6]                           # a run of equal values
+    if m > 4200:
+        e[0, 4095] = e[0, 4096] = 3.0                     # a tie across a chunk boundary
+    idx, val = b.r3_topk(dev(e), k)
+    idx, val = idx.cpu().numpy(), val.cpu().numpy()
+    for q in range(batch):
+        ridx, rval = o.topk(e[q], k)
+        assert np.array_equal(idx[q], ridx)
+        assert np.array_equal(val[q], rval.astype(np.float32))
+
+
+def test_topk_special_values():
+    e = np.array([[0.0, -0.0, np.nan, -np.inf, 1.0, np.inf, -1.0, 0.0]], dtype=np.float32)
+    idx, val = b.r3_topk(dev(e), 8)
+    assert idx.cpu().numpy().tolist() == [[5, 4, 0, 1, 7, 6, 3, 2]]   # -0 ties with +0; NaN last
+    idx, _ = b.r3_topk(dev(e[0]), 3)
+    assert idx.cpu().numpy().tolist() == [5, 4, 0]
+
+
+# ------------------------------------------------------------------------------------------ the five workloads
+def _run_full(c, engine):
+    g = w.generate(c)
+    gp = fit_gpu(g, engine)
+    xc = dev(g["Xcand"])
+    out = b.r3_gp_score_topk(gp, xc, c.k)
+    b.r3_gp_check(gp)
+    out = tuple(t.cpu().numpy() for t in out)
+    gp.close()
+    del xc
+    torch.cuda.empty_cache()
+    return g, out
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+@pytest.mark.parametrize("cfg", [1, 2])
+def test_workload_full_pool_every_candidate(cfg, engine):
+    c = w.get_config(cfg)
+    g, (mu, sd, ei, idx, val) = _run_full(c, engine)
+    fits, mu_r, sd_r, ei_r = oracle_all(g)
+    check_scores(mu[0], sd[0], ei[0], mu_r[0], sd_r[0], ei_r[0], float(np.abs(g["y"]).max()), 1.0, what=c.name)
+    ridx, rval = o.topk(ei_r[0], c.k + 1)
+    check_topk(idx[0], lambda i: ei_r[0][i], ridx[:c.k], rval[:c.k], rval[c.k], ei_r[0].max(), what=c.name)
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+def test_workload_cfg1_stress_twin(engine):
+    c = w.get_config(1, stress=True)
+    g, (mu, sd, ei, idx, val) = _run_full(c, engine)
+    fits, mu_r, sd_r, ei_r = oracle_all(g)
+    check_scores(mu[0], sd[0], ei[0], mu_r[0], sd_r[0], ei_r[0], float(np.abs(g["y"]).max()), 1.0, what=c.name)
+
+
+def _sampled_check(c, g, out, per_gp):
+    mu, sd, ei, idx, val = out
+    sample = w.sample_indices(c, per_gp)
+    for q in range(c.batch):
+        f = o.fit(g["X"][q], g["y"][q], g["ell"][q], g["sf2"][q], g["sn2"][q])
+        # the sample, plus whatever the GPU chose, scored one by one by the oracle
+        pick = np.unique(np.concatenate([sample, idx[q].astype(np.int64)]))
+        mu_r, sd_r, ei_r = o.score(f, g["Xcand"][q][pick])
+        check_scores(mu[q][pick], sd[q][pick], ei[q][pick], mu_r, sd_r, ei_r, float(np.abs(g["y"][q]).max()),
+                     float(g["sf2"][q]), what=f"{c.name} gp{q}")
+        # the library's own top-k is exactly the top-k of the EI it wrote
+        order = np.lexsort((np.arange(c.m), -ei[q].astype(np.float64)))[:c.k]
+        assert np.array_equal(idx[q], order)
+        assert np.array_equal(val[q], ei[q][order])
+        yield q, f, pick, ei_r
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+def test_workload_cfg3_batched_full_size_sampled(engine):
+    c = w.get_config(3)
+    g, out = _run_full(c, engine)
+    for _ in _sampled_check(c, g, out, 256):
+        pass
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+@pytest.mark.parametrize("cfg", [4, 5])
+def test_workload_full_size_sampled_and_full_pool_topk(cfg, engine):
+    c = w.get_config(cfg)
+    g, out = _run_full(c, engine)
+    idx = out[3]
+    for q, f, pick, ei_r in _sampled_check(c, g, out, 8192):
+        path = os.path.join(GOLDEN, f"topk_{c.name}.json")
+        if not os.path.exists(path):
+            pytest.skip(f"{path} not generated")
+        gold = json.load(open(path))
+        assert gold["m"] == c.m and gold["n"] == c.n and gold["seed"] == c.seed
+        ref_idx = np.array(gold["idx"], dtype=np.int64)
+        ref_val = np.array([float(v) for v in gold["ei"]])
+        known = dict(zip(ref_idx.tolist(), ref_val.tolist()))
+        known.update(zip(pick.tolist(), ei_r.tolist()))
+        check_topk(idx[q], lambda i: known[i], ref_idx[:c.k], ref_val[:c.k], ref_val[c.k], float(gold["ei_max"]),
+                   what=c.name)
