@@ -151,6 +151,14 @@ r3_status_t r3_gp_set_engine(r3_gp_t* gp, r3_engine_t engine);
 r3_engine_t r3_gp_engine(const r3_gp_t* gp);
 
 /*
+ * Diagnostics: synchronises `cuda_stream` and returns how many candidates the last scoring call on
+ * this handle recomputed in FP64 (summed over the first 64 GPs of the batch).  The scoring engines
+ * work at FP32 level and hand to an FP64 pass every candidate whose estimated rounding error could
+ * exceed the accuracy contract (candidates on top of observations, ill-conditioned histories).
+ */
+r3_status_t r3_gp_last_rescued(r3_gp_t* gp, void* cuda_stream, long long* total);
+
+/*
  * Timing of the dominant scoring kernel (the variance contraction).  While enabled, every launch
  * of that kernel is bracketed by a CUDA event pair on the launching stream.  r3_gp_profile_read
  * waits for the recorded events, returns the summed kernel time in milliseconds and the number

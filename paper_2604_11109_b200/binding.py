@@ -45,6 +45,7 @@ SIGNATURES = {
     "r3_gp_set_engine": (_i, [_vp, _i]),
     "r3_gp_engine": (_i, [_vp]),
     "r3_gp_get_factor": (_i, [_vp, _vp, _vp]),
+    "r3_gp_last_rescued": (_i, [_vp, _vp, ctypes.POINTER(_ll)]),
     "r3_gp_profile": (_i, [_vp, _i]),
     "r3_gp_profile_read": (_i, [_vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_ll)]),
     "r3_launch_count": (_ull, []),
@@ -242,6 +243,13 @@ def r3_gp_get_factor(gp: GP):
     L = np.empty((gp.batch, gp.n, gp.n), dtype=np.float64)
     _check(load().r3_gp_get_factor(gp.handle, alpha.ctypes.data_as(_vp), L.ctypes.data_as(_vp)))
     return alpha, L
+
+
+def r3_gp_last_rescued(gp: GP) -> int:
+    """Candidates the last scoring call recomputed in FP64 (synchronises the current stream)."""
+    total = _ll()
+    _check(load().r3_gp_last_rescued(gp.handle, _stream(), ctypes.byref(total)))
+    return int(total.value)
 
 
 def r3_gp_profile(gp: GP, enable: bool):

@@ -138,6 +138,8 @@ void r3_gp_free(r3_gp_t* gp)
     cudaFree(gp->sn2_d);
     cudaFree(gp->sf2_d);
     cudaFree(gp->best_d);
+    cudaFree(gp->yabs_d);
+    cudaFree(gp->wnorm_d);
     cudaFree(gp->L64);
     cudaFree(gp->W64);
     cudaFree(gp->W32);
@@ -145,6 +147,7 @@ void r3_gp_free(r3_gp_t* gp)
     cudaFree(gp->alpha32);
     cudaFree(gp->status_d);
     if (gp->status_h) cudaFreeHost(gp->status_h);
+    if (gp->rescued_h) cudaFreeHost(gp->rescued_h);
     for (cudaEvent_t e : gp->events) cudaEventDestroy(e);
     cudaFree(gp->ws);
     delete gp;
@@ -214,6 +217,8 @@ r3_status_t r3_gp_fit(const float* X, const float* y, const float* lengthscales,
     TRY_BAIL(cudaMalloc(&gp->sn2_d, sizeof(float) * batch));
     TRY_BAIL(cudaMalloc(&gp->sf2_d, sizeof(float) * batch));
     TRY_BAIL(cudaMalloc(&gp->best_d, sizeof(float) * batch));
+    TRY_BAIL(cudaMalloc(&gp->yabs_d, sizeof(float) * batch));
+    TRY_BAIL(cudaMalloc(&gp->wnorm_d, sizeof(double) * batch));
     TRY_BAIL(cudaMalloc(&gp->L64, sizeof(double) * batch * mat));
     TRY_BAIL(cudaMalloc(&gp->W64, sizeof(double) * batch * mat));
     TRY_BAIL(cudaMalloc(&gp->W32, sizeof(float) * batch * mat));
@@ -221,6 +226,8 @@ r3_status_t r3_gp_fit(const float* X, const float* y, const float* lengthscales,
     TRY_BAIL(cudaMalloc(&gp->alpha32, sizeof(float) * batch * gp->npad));
     TRY_BAIL(cudaMalloc(&gp->status_d, 2 * sizeof(int)));
     TRY_BAIL(cudaMallocHost(&gp->status_h, 2 * sizeof(int)));
+    TRY_BAIL(cudaMallocHost(&gp->rescued_h, 64 * sizeof(int)));
+    for (int i = 0; i < 64; ++i) gp->rescued_h[i] = 0;
     gp->status_h[0] = 0;
     gp->status_h[1] = INT_MAX;
     TRY_BAIL(cudaMemcpyAsync(gp->status_d, gp->status_h, 2 * sizeof(int), cudaMemcpyHostToDevice, stream));
@@ -243,7 +250,11 @@ r3_status_t r3_gp_fit(const float* X, const float* y, const float* lengthscales,
                   gp->status_h[1]);
         return bail(R3_ERR_NOT_PD);
     }
-    if (cudaMemcpy(gp->best.data(), gp->best_d, sizeof(float) * batch, cudaMemcpyDeviceToHost) != cudaSuccess) {
+    gp->y_absmax.assign(batch, 0.f);
+    gp->wnorm.assign(batch, 0.0);
+    if (cudaMemcpy(gp->best.data(), gp->best_d, sizeof(float) * batch, cudaMemcpyDeviceToHost) != cudaSuccess ||
+        cudaMemcpy(gp->y_absmax.data(), gp->yabs_d, sizeof(float) * batch, cudaMemcpyDeviceToHost) != cudaSuccess ||
+        cudaMemcpy(gp->wnorm.data(), gp->wnorm_d, sizeof(double) * batch, cudaMemcpyDeviceToHost) != cudaSuccess) {
         set_error("r3_gp_fit: reading back the incumbent failed");
         return bail(R3_ERR_CUDA);
     }
@@ -429,6 +440,19 @@ r3_status_t r3_gp_set_engine(r3_gp_t* gp, r3_engine_t engine)
         return R3_ERR_UNSUPPORTED;
     }
     gp->engine_req = engine;
+    return R3_OK;
+}
+
+r3_status_t r3_gp_last_rescued(r3_gp_t* gp, void* cuda_stream, long long* total)
+{
+    if (!gp || !total) {
+        set_error("r3_gp_last_rescued: NULL argument");
+        return R3_ERR_INVALID_ARG;
+    }
+    R3_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)cuda_stream));
+    long long t = 0;
+    for (int g = 0; g < gp->batch && g < 64; ++g) t += gp->rescued_h[g];
+    *total = t;
     return R3_OK;
 }
 

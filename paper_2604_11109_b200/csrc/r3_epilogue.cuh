@@ -7,13 +7,8 @@
 
 namespace r3 {
 
-// A candidate whose variance is below this fraction of the signal variance is recomputed in FP64:
-// sf2 - q cancels there and FP32-level q cannot give sigma to 1e-4 relative.
-constexpr double kRescueFraction = 0.05;
-
 struct CandidateResult {
     float mu, sigma, ei;
-    bool needs_rescue;
 };
 
 __device__ __forceinline__ double ei_closed_form(double mu, double sd, double best)
@@ -27,18 +22,28 @@ __device__ __forceinline__ double ei_closed_form(double mu, double sd, double be
     return e > 0.0 ? e : 0.0;
 }
 
-// mu = k*.alpha, q = |W k*|^2 (both possibly FP32-accurate), sf2 = signal variance, best = incumbent.
+// mu = k*.alpha and q = |W k*|^2 as the engine computed them; sf2 = signal variance, best = incumbent.
 __device__ __forceinline__ CandidateResult finalize_candidate(double mu, double q, double sf2, double best)
 {
     CandidateResult r;
     double var = sf2 - q;
-    r.needs_rescue = !(var >= kRescueFraction * sf2);  // also catches NaN
     if (!(var > 0.0)) var = 0.0;
     const double sd = sqrt(var);
     r.mu = (float)mu;
     r.sigma = (float)sd;
     r.ei = (float)ei_closed_form(mu, sd, best);
     return r;
+}
+
+// First-order, random-sign estimates of the engine's own rounding error in mu and in q, from the
+// per-entry relative error eps of k*:
+//   d mu ~ 2 eps sqrt(sum_i (k*_i alpha_i)^2)
+//   d q  ~ 2 eps |W|_2 sqrt(q sum_i k*_i^2)        (from dq = 2 V.(W dk*), |V|^2 = q)
+// The flagging pass compares them with the accuracy contract once the pool's largest EI is known.
+__device__ __forceinline__ float mu_error_estimate(double eps, double a2) { return (float)(2.0 * eps * sqrt(a2)); }
+__device__ __forceinline__ float q_error_estimate(double eps, double wnorm, double q, double s2)
+{
+    return (float)(2.0 * eps * wnorm * sqrt(fmax(q, 0.0) * s2));
 }
 
 }  // namespace r3

@@ -26,19 +26,29 @@ __global__ void check_finite_kernel(const float* __restrict__ a, size_t count, i
     if (__syncthreads_or(bad) && threadIdx.x == 0) atomicOr(status, DEV_NONFINITE);
 }
 
-__global__ void min_y_kernel(const float* __restrict__ y, int n, float* best)
+__global__ void min_y_kernel(const float* __restrict__ y, int n, float* best, float* yabs)
 {
-    __shared__ float s[256];
+    __shared__ float s[256], a[256];
     const float* yg = y + (size_t)blockIdx.x * n;
-    float v = INFINITY;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) v = fminf(v, yg[i]);
+    float v = INFINITY, m = 0.f;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        v = fminf(v, yg[i]);
+        m = fmaxf(m, fabsf(yg[i]));
+    }
     s[threadIdx.x] = v;
+    a[threadIdx.x] = m;
     __syncthreads();
     for (int o = 128; o > 0; o >>= 1) {
-        if (threadIdx.x < o) s[threadIdx.x] = fminf(s[threadIdx.x], s[threadIdx.x + o]);
+        if (threadIdx.x < o) {
+            s[threadIdx.x] = fminf(s[threadIdx.x], s[threadIdx.x + o]);
+            a[threadIdx.x] = fmaxf(a[threadIdx.x], a[threadIdx.x + o]);
+        }
         __syncthreads();
     }
-    if (threadIdx.x == 0) best[blockIdx.x] = s[0];
+    if (threadIdx.x == 0) {
+        best[blockIdx.x] = s[0];
+        yabs[blockIdx.x] = a[0];
+    }
 }
 
 // ------------------------------------------------------------------------------------ Gram
@@ -290,7 +300,8 @@ __global__ void __launch_bounds__(256) trtri_gemm_kernel(const double* __restric
 
 // ------------------------------------------------------------------------------------ weights
 // u = W y (lower-triangular W, one warp per row); rows >= n give 0.
-__global__ void w_times_y_kernel(const double* __restrict__ W, const float* __restrict__ y, int n,
+template <typename T>
+__global__ void w_times_y_kernel(const double* __restrict__ W, const T* __restrict__ y, int ystride, int n,
                                  int npad, double* __restrict__ u)
 {
     const int g = blockIdx.y;
@@ -300,7 +311,7 @@ __global__ void w_times_y_kernel(const double* __restrict__ W, const float* __re
     const double* Wr = W + (size_t)g * npad * npad + (size_t)row * npad;
     double s = 0.0;
     if (row < n)
-        for (int k = lane; k <= row; k += 32) s += Wr[k] * (double)y[(size_t)g * n + k];
+        for (int k = lane; k <= row; k += 32) s += Wr[k] * (double)y[(size_t)g * ystride + k];
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     if (lane == 0) u[(size_t)g * npad + row] = s;
 }
@@ -318,6 +329,41 @@ __global__ void wt_times_u_kernel(const double* __restrict__ W, const double* __
         for (int i = j; i < n; ++i) s += Wg[(size_t)i * npad + j] * u[(size_t)g * npad + i];
     alpha64[(size_t)g * npad + j] = s;
     alpha32[(size_t)g * npad + j] = (float)s;
+}
+
+// Power iteration on W^T W: v holds the current vector (unit norm after the call), lam its norm
+// before normalisation, i.e. the current estimate of |W|_2^2.
+__global__ void power_init_kernel(double* __restrict__ v, int n, int npad)
+{
+    const int g = blockIdx.x;
+    for (int i = threadIdx.x; i < npad; i += blockDim.x)
+        v[(size_t)g * npad + i] = (i < n) ? (1.0 + 0.37 * ((i * 2654435761u >> 16) & 0xff) / 255.0) : 0.0;
+}
+
+__global__ void power_normalize_kernel(double* __restrict__ v, int npad, double* __restrict__ lam)
+{
+    __shared__ double s[256];
+    const int g = blockIdx.x;
+    double* vg = v + (size_t)g * npad;
+    double acc = 0.0;
+    for (int i = threadIdx.x; i < npad; i += 256) acc += vg[i] * vg[i];
+    s[threadIdx.x] = acc;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) s[threadIdx.x] += s[threadIdx.x + o];
+        __syncthreads();
+    }
+    const double nrm = sqrt(s[0]);
+    if (threadIdx.x == 0) lam[g] = nrm;
+    const double inv = nrm > 0.0 ? 1.0 / nrm : 0.0;
+    for (int i = threadIdx.x; i < npad; i += 256) vg[i] *= inv;
+}
+
+__global__ void power_finish_kernel(const double* __restrict__ lam, double* __restrict__ wnorm, int batch)
+{
+    // lam ~ |W|_2^2 from below; 1.5 covers slow convergence
+    const int g = blockIdx.x * blockDim.x + threadIdx.x;
+    if (g < batch) wnorm[g] = 1.5 * sqrt(lam[g]);
 }
 
 __global__ void to_float_kernel(const double* __restrict__ a, float* __restrict__ b, size_t count)
@@ -367,7 +413,7 @@ r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream)
 
     LAUNCH_OR_FAIL(check_finite_kernel, 296, 256, gp->X, (size_t)B * n * d, gp->status_d);
     LAUNCH_OR_FAIL(check_finite_kernel, 64, 256, y, (size_t)B * n, gp->status_d);
-    LAUNCH_OR_FAIL(min_y_kernel, B, 256, y, n, gp->best_d);
+    LAUNCH_OR_FAIL(min_y_kernel, B, 256, y, n, gp->best_d, gp->yabs_d);
 
     LAUNCH_OR_FAIL(gram_kernel, dim3(npad / 16, npad / 16, B), dim3(16, 16), gp->X, gp->ell_d, gp->sf2_d,
                    gp->sn2_d, n, d, npad, gp->L64);
@@ -392,7 +438,21 @@ r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream)
         LAUNCH_OR_FAIL(trtri_gemm_kernel, grid, 256, gp->W64, T, gp->W64, npad, s, npairs, 1);
     }
 
-    LAUNCH_OR_FAIL(w_times_y_kernel, dim3((npad + 7) / 8, B), 256, gp->W64, y, n, npad, u);
+    // spectral norm of W by power iteration on W^T W (alpha64/alpha32 serve as scratch first)
+    {
+        double* pv = gp->alpha64;
+        double* lam = T;  // [B] scratch
+        LAUNCH_OR_FAIL(power_init_kernel, B, 256, pv, n, npad);
+        LAUNCH_OR_FAIL(power_normalize_kernel, B, 256, pv, npad, lam);
+        for (int it = 0; it < 16; ++it) {
+            LAUNCH_OR_FAIL(w_times_y_kernel<double>, dim3((npad + 7) / 8, B), 256, gp->W64, pv, npad, n, npad, u);
+            LAUNCH_OR_FAIL(wt_times_u_kernel, dim3((npad + 127) / 128, B), 128, gp->W64, u, n, npad, pv,
+                           gp->alpha32);
+            LAUNCH_OR_FAIL(power_normalize_kernel, B, 256, pv, npad, lam);
+        }
+        LAUNCH_OR_FAIL(power_finish_kernel, (B + 255) / 256, 256, lam, gp->wnorm_d, B);
+    }
+    LAUNCH_OR_FAIL(w_times_y_kernel<float>, dim3((npad + 7) / 8, B), 256, gp->W64, y, n, n, npad, u);
     LAUNCH_OR_FAIL(wt_times_u_kernel, dim3((npad + 127) / 128, B), 128, gp->W64, u, n, npad,
                    gp->alpha64, gp->alpha32);
     LAUNCH_OR_FAIL(to_float_kernel, 1184, 256, gp->W64, gp->W32, (size_t)B * mat);

@@ -63,6 +63,8 @@ struct r3_gp {
     int npad = 0;              // n rounded up to kFitBlock; padded rows/cols are identity / zero
     int device = 0;
     std::vector<float> ell, sf2, sn2, best;   // host copies [batch][d], [batch], [batch], [batch]
+    std::vector<float> y_absmax;              // [batch] max |y|
+    std::vector<double> wnorm;                // [batch] estimate of |L^-1|_2 (power iteration x 1.5)
 
     float* X = nullptr;        // [batch][n][d]   raw observations (FP32 as given)
     float* ell_d = nullptr;    // [batch][d]      lengthscales as given
@@ -70,6 +72,8 @@ struct r3_gp {
     float* sn2_d = nullptr;    // [batch]
     float* sf2_d = nullptr;    // [batch]
     float* best_d = nullptr;   // [batch]
+    float* yabs_d = nullptr;   // [batch] max |y|
+    double* wnorm_d = nullptr; // [batch]
     double* L64 = nullptr;     // [batch][npad][npad] lower Cholesky factor (upper part zero)
     double* W64 = nullptr;     // [batch][npad][npad] W = L^-1, lower
     float* W32 = nullptr;      // [batch][npad][npad] W rounded to FP32
@@ -77,6 +81,7 @@ struct r3_gp {
     float* alpha32 = nullptr;  // [batch][npad]
     int* status_d = nullptr;   // [2]: status bits, first bad pivot index
     int* status_h = nullptr;   // pinned mirror of status_d
+    int* rescued_h = nullptr;  // pinned [64]: candidates recomputed in FP64 by the last scoring call, per GP
 
     // tensor-core operands (built by fit when the tensor engine can serve (n, d))
     void* tc = nullptr;        // r3::TensorOperands*, see r3_score_tc.cu
@@ -103,12 +108,20 @@ size_t score_simt_workspace_bytes(const r3_gp* gp, long long m);
 r3_status_t score_simt(r3_gp* gp, const float* Xcand, long long m, float* mu, float* sigma, float* ei,
                        void* ws, size_t ws_bytes, cudaStream_t stream);
 
-// FP64 rescue of the candidates whose variance is too small for FP32-level partial results
-// (r3_rescue.cu).  The engines append such candidates to a list while they write their own
-// FP32-level mu/sigma/EI; this pass recomputes those entries entirely in FP64 and overwrites them.
-//   list  [cap]  flat candidate ids g*m + j;  count[0] = entries appended (may exceed cap: clamped)
-r3_status_t rescue(r3_gp* gp, const float* Xcand, long long m, const int* count, const long long* list,
-                   long long cap, float* mu, float* sigma, float* ei, cudaStream_t stream);
+// Accuracy guard and FP64 rescue (r3_rescue.cu).  The engines write their results and, per candidate,
+// estimates of their own rounding error in mu (err_mu) and in q = |W k*|^2 (err_q); the guard then
+// lists the candidates that may miss the accuracy contract and recomputes them in FP64.
+struct GuardBuffers {
+    float* err_mu;      // [batch][m]
+    float* err_q;       // [batch][m]
+    int* list;          // [batch][m] candidate indices to recompute
+    int* count;         // [batch]
+    unsigned* maxbits;  // [batch] bit pattern of the largest EI
+};
+size_t guard_workspace_bytes(const r3_gp* gp, long long m);
+GuardBuffers guard_carve(const r3_gp* gp, long long m, void* ws);
+r3_status_t guard_and_rescue(r3_gp* gp, const float* Xcand, long long m, const GuardBuffers& b, float* mu,
+                             float* sigma, float* ei, cudaStream_t stream);
 
 // tensor-core scoring (r3_score_tc.cu)
 bool tc_supported(int n, int d);

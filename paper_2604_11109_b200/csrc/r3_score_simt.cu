@@ -15,12 +15,13 @@ namespace r3 {
 namespace {
 
 constexpr size_t kSlabBytes = 256ull << 20;
+// relative error of one k* entry on this path: FP32 differences, FMA chain, sqrtf, expf
+constexpr double kEpsSimt = 1.2e-7;
 
 struct SimtWorkspace {
     float* ks;         // [slab][npad]
-    double* mu64;      // [slab]
-    int* count;        // [1] rescue list length (padded to 16 B)
-    long long* list;   // [batch*m]
+    double* mu64;      // [slab][3]: mu, sum (k* alpha)^2, sum k*^2
+    GuardBuffers guard;
     long long slab;
 };
 
@@ -41,10 +42,8 @@ SimtWorkspace carve(const r3_gp* gp, long long m, void* ws)
     w.ks = (float*)p;
     p += (size_t)w.slab * gp->npad * sizeof(float);
     w.mu64 = (double*)p;
-    p += (size_t)w.slab * sizeof(double);
-    w.count = (int*)p;
-    p += 16;
-    w.list = (long long*)p;
+    p += (size_t)w.slab * 3 * sizeof(double);
+    w.guard = guard_carve(gp, m, p);
     return w;
 }
 
@@ -60,7 +59,7 @@ __global__ void __launch_bounds__(256) kstar_kernel(const float* __restrict__ X,
     __shared__ float sz[64][33], sx[64][33], sl[32];
     const int t = threadIdx.x, ty = t / 16, tx = t % 16;
     const long long c0 = (long long)blockIdx.x * 64;
-    double mu_acc[4] = {0.0, 0.0, 0.0, 0.0};
+    double mu_acc[4] = {0.0, 0.0, 0.0, 0.0}, a1_acc[4] = {0.0, 0.0, 0.0, 0.0}, s2_acc[4] = {0.0, 0.0, 0.0, 0.0};
     bool bad = false;
     for (int k0 = 0; k0 < npad; k0 += 64) {
         float r2[4][4] = {};
@@ -95,11 +94,11 @@ __global__ void __launch_bounds__(256) kstar_kernel(const float* __restrict__ X,
         }
         float al[4];
 #pragma unroll
-        for (int v = 0; v < 4; ++v) al[v] = alpha[k0 + tx * 4 + v];  // zero beyond n
+        for (int v = 0; v < 4; ++v) al[v] = (k0 + tx * 4 + v < npad) ? alpha[k0 + tx * 4 + v] : 0.f;  // zero beyond n
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             float kv[4];
-            float part = 0.f;
+            float part = 0.f, apart = 0.f, spart = 0.f;
 #pragma unroll
             for (int v = 0; v < 4; ++v) {
                 float s = sqrtf(5.0f * r2[u][v]);
@@ -107,20 +106,32 @@ __global__ void __launch_bounds__(256) kstar_kernel(const float* __restrict__ X,
                 if (k0 + tx * 4 + v >= n) val = 0.f;
                 kv[v] = val;
                 part = fmaf(val, al[v], part);
+                apart = fmaf(val * al[v], val * al[v], apart);
+                spart = fmaf(val, val, spart);
             }
             mu_acc[u] += (double)part;
+            a1_acc[u] += (double)apart;
+            s2_acc[u] += (double)spart;
             const long long c = c0 + ty + 16 * u;
-            if (c < mc)
+            if (c < mc && k0 + tx * 4 < npad)
                 *reinterpret_cast<float4*>(ks + (size_t)c * npad + k0 + tx * 4) =
                     make_float4(kv[0], kv[1], kv[2], kv[3]);
         }
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-        double v = mu_acc[u];
-        for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        double v = mu_acc[u], a = a1_acc[u], s = s2_acc[u];
+        for (int o = 8; o > 0; o >>= 1) {
+            v += __shfl_xor_sync(0xffffffffu, v, o);
+            a += __shfl_xor_sync(0xffffffffu, a, o);
+            s += __shfl_xor_sync(0xffffffffu, s, o);
+        }
         const long long c = c0 + ty + 16 * u;
-        if (tx == 0 && c < mc) mu64[c] = v;
+        if (tx == 0 && c < mc) {
+            mu64[3 * c + 0] = v;
+            mu64[3 * c + 1] = a;
+            mu64[3 * c + 2] = s;
+        }
     }
     if (__syncthreads_or(bad) && t == 0) atomicOr(status, DEV_NONFINITE);
 }
@@ -131,10 +142,10 @@ __global__ void __launch_bounds__(256) kstar_kernel(const float* __restrict__ X,
 __global__ void __launch_bounds__(256) trigemm_sq_kernel(const float* __restrict__ W,   // [npad][npad]
                                                          const float* __restrict__ ks,  // [slab][npad]
                                                          const double* __restrict__ mu64, int npad,
-                                                         long long mc, double sf2, double best,
+                                                         long long mc, double sf2, double best, double eps_k, double wnorm,
                                                          float* __restrict__ mu, float* __restrict__ sigma,
-                                                         float* __restrict__ ei, long long flat0,
-                                                         int* count, long long* list, long long cap)
+                                                         float* __restrict__ ei, float* __restrict__ err_mu,
+                                                         float* __restrict__ err_q)
 {
     __shared__ __align__(16) float sw[16][132];
     __shared__ __align__(16) float sk[16][132];
@@ -190,14 +201,12 @@ __global__ void __launch_bounds__(256) trigemm_sq_kernel(const float* __restrict
             double q = 0.0;
 #pragma unroll
             for (int r = 0; r < 16; ++r) q += sq[r][t];
-            CandidateResult res = finalize_candidate(mu64[c], q, sf2, best);
+            const CandidateResult res = finalize_candidate(mu64[3 * c], q, sf2, best);
             mu[c] = res.mu;
             sigma[c] = res.sigma;
             ei[c] = res.ei;
-            if (res.needs_rescue) {
-                int slot = atomicAdd(count, 1);
-                if (slot < cap) list[slot] = flat0 + c;
-            }
+            err_mu[c] = mu_error_estimate(eps_k, mu64[3 * c + 1]);
+            err_q[c] = q_error_estimate(eps_k, wnorm, q, mu64[3 * c + 2]);
         }
     }
 }
@@ -207,8 +216,8 @@ __global__ void __launch_bounds__(256) trigemm_sq_kernel(const float* __restrict
 size_t score_simt_workspace_bytes(const r3_gp* gp, long long m)
 {
     const long long slab = slab_candidates(gp->npad, m);
-    return (size_t)slab * gp->npad * sizeof(float) + (size_t)slab * sizeof(double) + 16 +
-           (size_t)gp->batch * m * sizeof(long long);
+    return (size_t)slab * gp->npad * sizeof(float) + (size_t)slab * 3 * sizeof(double) +
+           guard_workspace_bytes(gp, m);
 }
 
 r3_status_t score_simt(r3_gp* gp, const float* Xcand, long long m, float* mu, float* sigma, float* ei,
@@ -220,8 +229,6 @@ r3_status_t score_simt(r3_gp* gp, const float* Xcand, long long m, float* mu, fl
     }
     SimtWorkspace w = carve(gp, m, ws);
     const int n = gp->n, d = gp->d, npad = gp->npad;
-    const long long cap = (long long)gp->batch * m;
-    R3_CUDA_TRY(cudaMemsetAsync(w.count, 0, sizeof(int), stream));
     for (int g = 0; g < gp->batch; ++g) {
         for (long long s0 = 0; s0 < m; s0 += w.slab) {
             const long long mc = (m - s0) < w.slab ? (m - s0) : w.slab;
@@ -234,12 +241,12 @@ r3_status_t score_simt(r3_gp* gp, const float* Xcand, long long m, float* mu, fl
             prof_begin(gp, stream);
             R3_LAUNCH(trigemm_sq_kernel, (unsigned)((mc + 127) / 128), 256, 0, stream,
                       gp->W32 + (size_t)g * npad * npad, w.ks, w.mu64, npad, mc, (double)gp->sf2[g],
-                      (double)gp->best[g], mu + off, sigma + off, ei + off, (long long)off, w.count,
-                      w.list, cap);
+                      (double)gp->best[g], kEpsSimt, gp->wnorm[g], mu + off, sigma + off, ei + off,
+                      w.guard.err_mu + off, w.guard.err_q + off);
             prof_end(gp, stream);
         }
     }
-    return rescue(gp, Xcand, m, w.count, w.list, cap, mu, sigma, ei, stream);
+    return guard_and_rescue(gp, Xcand, m, w.guard, mu, sigma, ei, stream);
 }
 
 }  // namespace r3
