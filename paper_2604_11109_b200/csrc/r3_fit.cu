@@ -316,17 +316,33 @@ __global__ void w_times_y_kernel(const double* __restrict__ W, const T* __restri
     if (lane == 0) u[(size_t)g * npad + row] = s;
 }
 
-// alpha = W^T u (one thread per column, coalesced across columns); also the FP32 copy.
-__global__ void wt_times_u_kernel(const double* __restrict__ W, const double* __restrict__ u, int n,
-                                  int npad, double* __restrict__ alpha64, float* __restrict__ alpha32)
+// alpha = W^T u in two steps so that n = 4096 still fills the GPU: the rows are cut into kRowSlabs
+// slabs, each block sums one slab for 128 columns (coalesced across columns), then the slabs are added
+// in a fixed order (deterministic).
+constexpr int kRowSlabs = 32;
+__global__ void wt_times_u_partial_kernel(const double* __restrict__ W, const double* __restrict__ u, int n,
+                                          int npad, double* __restrict__ partial)
+{
+    const int g = blockIdx.z, slab = blockIdx.y;
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= npad) return;
+    const int rows = (npad + kRowSlabs - 1) / kRowSlabs;
+    const int i0 = max(slab * rows, j), i1 = min(min((slab + 1) * rows, npad), n);
+    const double* Wg = W + (size_t)g * npad * npad;
+    double s = 0.0;
+    if (j < n)
+        for (int i = i0; i < i1; ++i) s += Wg[(size_t)i * npad + j] * u[(size_t)g * npad + i];
+    partial[((size_t)g * kRowSlabs + slab) * npad + j] = s;
+}
+
+__global__ void wt_times_u_reduce_kernel(const double* __restrict__ partial, int npad,
+                                         double* __restrict__ alpha64, float* __restrict__ alpha32)
 {
     const int g = blockIdx.y;
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= npad) return;
-    const double* Wg = W + (size_t)g * npad * npad;
     double s = 0.0;
-    if (j < n)
-        for (int i = j; i < n; ++i) s += Wg[(size_t)i * npad + j] * u[(size_t)g * npad + i];
+    for (int r = 0; r < kRowSlabs; ++r) s += partial[((size_t)g * kRowSlabs + r) * npad + j];
     alpha64[(size_t)g * npad + j] = s;
     alpha32[(size_t)g * npad + j] = (float)s;
 }
@@ -441,20 +457,24 @@ r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream)
     // spectral norm of W by power iteration on W^T W (alpha64/alpha32 serve as scratch first)
     {
         double* pv = gp->alpha64;
-        double* lam = T;  // [B] scratch
+        double* lam = T;  // [B] scratch, followed by the row-slab partial sums
+        double* part = T + B;
         LAUNCH_OR_FAIL(power_init_kernel, B, 256, pv, n, npad);
         LAUNCH_OR_FAIL(power_normalize_kernel, B, 256, pv, npad, lam);
-        for (int it = 0; it < 16; ++it) {
+        for (int it = 0; it < 12; ++it) {
             LAUNCH_OR_FAIL(w_times_y_kernel<double>, dim3((npad + 7) / 8, B), 256, gp->W64, pv, npad, n, npad, u);
-            LAUNCH_OR_FAIL(wt_times_u_kernel, dim3((npad + 127) / 128, B), 128, gp->W64, u, n, npad, pv,
-                           gp->alpha32);
+            LAUNCH_OR_FAIL(wt_times_u_partial_kernel, dim3((npad + 127) / 128, kRowSlabs, B), 128, gp->W64, u, n,
+                           npad, part);
+            LAUNCH_OR_FAIL(wt_times_u_reduce_kernel, dim3((npad + 127) / 128, B), 128, part, npad, pv, gp->alpha32);
             LAUNCH_OR_FAIL(power_normalize_kernel, B, 256, pv, npad, lam);
         }
         LAUNCH_OR_FAIL(power_finish_kernel, (B + 255) / 256, 256, lam, gp->wnorm_d, B);
     }
     LAUNCH_OR_FAIL(w_times_y_kernel<float>, dim3((npad + 7) / 8, B), 256, gp->W64, y, n, n, npad, u);
-    LAUNCH_OR_FAIL(wt_times_u_kernel, dim3((npad + 127) / 128, B), 128, gp->W64, u, n, npad,
-                   gp->alpha64, gp->alpha32);
+    LAUNCH_OR_FAIL(wt_times_u_partial_kernel, dim3((npad + 127) / 128, kRowSlabs, B), 128, gp->W64, u, n, npad,
+                   T + B);
+    LAUNCH_OR_FAIL(wt_times_u_reduce_kernel, dim3((npad + 127) / 128, B), 128, T + B, npad, gp->alpha64,
+                   gp->alpha32);
     LAUNCH_OR_FAIL(to_float_kernel, 1184, 256, gp->W64, gp->W32, (size_t)B * mat);
 
     TRY_OR_FAIL(cudaMemcpyAsync(gp->status_h, gp->status_d, 2 * sizeof(int), cudaMemcpyDeviceToHost, stream));

@@ -16,9 +16,10 @@
 // accuracy from TF32 operands.  W is lower-triangular, so pass p only needs k < (p+1) NV; k* chunks are
 // regenerated for every pass they take part in instead of being stored.
 //
-// Warp roles (256 threads): warp 0 streams chunks of scaled observations, warp 1 streams chunks of W,
-// warp 2 issues every MMA (one thread) and owns the TMEM allocation, warps 4-7 (one per TMEM lane
-// quarter) are the Matern/epilogue warps.  Stages are handed over through mbarriers; every wait is
+// Warp roles: warp 0 streams chunks of scaled observations, warp 1 streams chunks of W, warp 2 issues
+// every MMA (one thread) and owns the TMEM allocation, warps 4.. form G Matern/epilogue groups of four
+// warps (one warp per TMEM lane quarter); group g takes every G-th chunk with its own distance and k*
+// buffers, so G chunks are in flight between the two MMA streams.  Stages are handed over through mbarriers; every wait is
 // bounded: when a limit is hit the CTA raises a status bit, all roles leave their loops, in-flight
 // copies and MMAs are drained (bounded again), TMEM is freed and the kernel returns.
 //
@@ -42,7 +43,7 @@ constexpr double kEpsTc0 = 2.5e-7;
 constexpr double kEpsTc1 = 2.0e-7;
 
 struct TensorOperands {
-    int NV = 0, DP = 0, NP = 0, P = 0, xs = 0, ws = 0, tmem_cols = 0;
+    int NV = 0, G = 0, DP = 0, NP = 0, P = 0, xs = 0, ws = 0, tmem_cols = 0;
     size_t smem_bytes = 0;
     size_t wt_gp_stride = 0;   // floats per GP in wt
     float* centre = nullptr;   // [B][DP]  column means of X (zero padded)
@@ -156,13 +157,9 @@ __device__ __forceinline__ float tf32_hi(float x)
     return __uint_as_float(u);
 }
 
-// Shared-memory matrix descriptor: no swizzle, K-major; lbo = bytes between the two 16-byte k-slices
-// of one MMA, sbo = bytes between 8-row groups.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo)
-{
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) |
-           (1ull << 46);
-}
+// Shared-memory matrix descriptors are the no-swizzle K-major form: bits 0-13 start address >> 4,
+// bits 16-29 the byte distance between the two 16-byte k-slices of one MMA >> 4, bits 32-45 the byte
+// distance between 8-row groups >> 4, bit 46 the descriptor version.
 // Instruction descriptor: FP32 accumulate, TF32 x TF32, both K-major, M = 128, N = n.
 __device__ __forceinline__ constexpr uint32_t instr_desc(uint32_t n)
 {
@@ -174,43 +171,61 @@ struct SmemMap {
     uint32_t z, k, x, w, bar;
     uint32_t x_stage, w_stage;
 };
-__host__ __device__ inline SmemMap smem_map(int DP, int NV, int xs, int ws)
+__host__ __device__ inline SmemMap smem_map(int DP, int NV, int G, int xs, int ws)
 {
     SmemMap s;
-    s.z = 0;                                  // 2 planes x [DP/4][128][4] floats
-    s.k = s.z + 2u * DP * 512u;               // 2 buffers x 2 planes x [KC/4][128][4]
-    s.x = s.k + 2u * 2u * (KC / 4) * 2048u;   // xs stages x 2 planes x [DP/4][KC][4]
+    s.z = 0;                                       // 2 planes x [DP/4][128][4] floats
+    s.k = s.z + 2u * DP * 512u;                    // G buffers x 2 planes x [KC/4][128][4]
+    s.x = s.k + (uint32_t)G * 16384u;              // xs stages x 2 planes x [DP/4][KC][4]
     s.x_stage = 2u * DP * KC * 4u;
-    s.w = s.x + (uint32_t)xs * s.x_stage;     // ws stages x 2 planes x [KC/4][NV][4]
+    s.w = s.x + (uint32_t)xs * s.x_stage;          // ws stages x 2 planes x [KC/4][NV][4]
     s.w_stage = 2u * KC * NV * 4u;
     s.bar = s.w + (uint32_t)ws * s.w_stage;
     return s;
 }
-constexpr uint32_t kBarBytes = 512;
+constexpr uint32_t kBarBytes = 1024;   // barriers, flags, TMEM slot, candidate norms
 
 // barrier slots (8 bytes each) inside the barrier block
 enum : uint32_t {
-    BAR_X_FULL = 0, BAR_X_EMPTY = 4, BAR_W_FULL = 8, BAR_W_EMPTY = 12, BAR_D_FULL = 16, BAR_D_EMPTY = 18,
-    BAR_K_FULL = 20, BAR_K_EMPTY = 22, BAR_V_FULL = 24, BAR_V_EMPTY = 25, BAR_Z_READY = 26, BAR_MMA_DONE = 27,
-    BAR_COUNT = 28
+    BAR_X_FULL = 0, BAR_X_EMPTY = 4, BAR_W_FULL = 8, BAR_W_EMPTY = 12, BAR_D_FULL = 16, BAR_D_EMPTY = 20,
+    BAR_K_FULL = 24, BAR_K_EMPTY = 28, BAR_V_FULL = 32, BAR_V_EMPTY = 33, BAR_Z_READY = 34, BAR_MMA_DONE = 35,
+    BAR_RED_READY = 36, BAR_COUNT = 37
 };
+constexpr uint32_t kFlagOffset = BAR_COUNT * 8;       // int abort, int drain-abort, uint32 tmem base
+constexpr uint32_t kZnOffset = 512;                   // float[128] squared norms of the scaled candidates
 
-template <int NV>
-__global__ void __launch_bounds__(256, 1) score_tc_kernel(const TcParams prm)
+__device__ __forceinline__ uint64_t pack64(uint32_t lo, uint32_t hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ float sqrt_approx(float x)
+{
+    float r;
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+
+// NV: rows of W per pass (TMEM columns of the V accumulator).  G: number of Matern warp groups; group
+// g owns items t = g (mod G) of the chunk sequence together with distance buffer g and k* buffer g.
+template <int NV, int G>
+__global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcParams prm)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* sm = smem_raw + (base - raw);
-    const SmemMap map = smem_map(prm.DP, NV, prm.xs, prm.ws);
+    const SmemMap map = smem_map(prm.DP, NV, G, prm.xs, prm.ws);
     const uint32_t bars = base + map.bar;
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + map.bar + BAR_COUNT * 8);
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + map.bar + BAR_COUNT * 8 + 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + map.bar + kFlagOffset);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + map.bar + kFlagOffset + 8);
+    float* zn_s = reinterpret_cast<float*>(sm + map.bar + kZnOffset);
     auto bar = [&](uint32_t slot) { return bars + slot * 8u; };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int CPP = NV / KC;                  // chunks per pass width
-    constexpr uint32_t TMEM_COLS = (NV + 2 * KC) <= 256 ? 256u : 512u;
+    constexpr uint32_t TMEM_COLS = (NV + G * KC) <= 256 ? 256u : 512u;
     const int DP = prm.DP, P = prm.P, xs = prm.xs, ws = prm.ws;
 
     if (threadIdx.x == 0) {
@@ -219,17 +234,16 @@ __global__ void __launch_bounds__(256, 1) score_tc_kernel(const TcParams prm)
             mbar_init(bar(BAR_X_EMPTY + i), 1);
             mbar_init(bar(BAR_W_FULL + i), 1);
             mbar_init(bar(BAR_W_EMPTY + i), 1);
-        }
-        for (int i = 0; i < 2; ++i) {
             mbar_init(bar(BAR_D_FULL + i), 1);
             mbar_init(bar(BAR_D_EMPTY + i), 128);
             mbar_init(bar(BAR_K_FULL + i), 128);
             mbar_init(bar(BAR_K_EMPTY + i), 1);
         }
         mbar_init(bar(BAR_V_FULL), 1);
-        mbar_init(bar(BAR_V_EMPTY), 128);
+        mbar_init(bar(BAR_V_EMPTY), 128 * G);
         mbar_init(bar(BAR_Z_READY), 128);
         mbar_init(bar(BAR_MMA_DONE), 1);
+        mbar_init(bar(BAR_RED_READY), 128 * G);
         abort_flag[0] = 0;
         abort_flag[1] = 0;   // private flag of the bounded drain waits
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -295,7 +309,13 @@ __global__ void __launch_bounds__(256, 1) score_tc_kernel(const TcParams prm)
         // ------------------------------------------------------------ MMA issuer
         constexpr uint32_t IDESC_D = instr_desc(KC);
         constexpr uint32_t IDESC_V = instr_desc(NV);
-        const uint32_t zH = base + map.z, zL = zH + (uint32_t)DP * 512u;
+        // descriptor words: lo = start>>4 | (lbo>>4)<<16, hi = sbo>>4 | version bit
+        constexpr uint32_t HI = (128u >> 4) | (1u << 14);
+        const uint32_t zH_lo = ((base + map.z) >> 4) | ((2048u >> 4) << 16);
+        const uint32_t zL_lo = zH_lo + (((uint32_t)DP * 512u) >> 4);
+        const uint32_t x_lo0 = ((base + map.x) >> 4) | (((KC * 16u) >> 4) << 16);
+        const uint32_t k_lo0 = ((base + map.k) >> 4) | ((2048u >> 4) << 16);
+        const uint32_t w_lo0 = ((base + map.w) >> 4) | (((NV * 16u) >> 4) << 16);
         const int ksteps_d = DP / 8;
         long long t = 0;      // item counter (rings)
         long long pv = 0;     // pass counter (V accumulator hand-over)
@@ -303,17 +323,19 @@ __global__ void __launch_bounds__(256, 1) score_tc_kernel(const TcParams prm)
         bool ok = true;
 
         auto issue_distance = [&](long long tu) -> bool {
-            const int s = (int)(tu % xs), b = (int)(tu & 1);
+            const int s = (int)(tu % xs), b = (int)(tu % G);
+            const long long j = tu / G;
             if (!mbar_wait(bar(BAR_X_FULL + s), (uint32_t)((tu / xs) & 1), abort_flag)) return false;
-            if (!mbar_wait(bar(BAR_D_EMPTY + b), (uint32_t)(((tu >> 1) & 1) ^ 1), abort_flag)) return false;
+            if (!mbar_wait(bar(BAR_D_EMPTY + b), (uint32_t)((j & 1) ^ 1), abort_flag)) return false;
             tc_fence_after();
-            const uint32_t xH = base + map.x + s * map.x_stage, xL = xH + (uint32_t)DP * KC * 4u;
+            const uint32_t xH_lo = x_lo0 + ((s * map.x_stage) >> 4), xL_lo = xH_lo + (((uint32_t)DP * KC * 4u) >> 4);
             const uint32_t dcol = tmem + NV + b * KC;
             uint32_t acc = 0;
+#pragma unroll
             for (int combo = 0; combo < 3; ++combo) {
-                const uint32_t a0 = combo == 2 ? zL : zH, b0 = combo == 1 ? xL : xH;
-                for (int j = 0; j < ksteps_d; ++j) {
-                    tc_mma_tf32(dcol, smem_desc(a0 + j * 4096u, 2048u, 128u), smem_desc(b0 + j * (2u * KC * 16u), KC * 16u, 128u),
+                const uint32_t a0 = combo == 2 ? zL_lo : zH_lo, b0 = combo == 1 ? xL_lo : xH_lo;
+                for (int jj = 0; jj < ksteps_d; ++jj) {
+                    tc_mma_tf32(dcol, pack64(a0 + jj * (4096u >> 4), HI), pack64(b0 + jj * ((2u * KC * 16u) >> 4), HI),
                                 IDESC_D, acc);
                     acc = 1;
                 }
@@ -327,26 +349,28 @@ __global__ void __launch_bounds__(256, 1) score_tc_kernel(const TcParams prm)
             if (!(ok = mbar_wait(bar(BAR_Z_READY), (uint32_t)(tile_iter & 1), abort_flag))) break;
             tc_fence_after();
             const long long t_tile0 = t;
-            for (int u = 0; ok && u < 2 && u < items_per_tile; ++u) ok = issue_distance(t_tile0 + u);
+            for (int u = 0; ok && u < G && u < items_per_tile; ++u) ok = issue_distance(t_tile0 + u);
             for (int p = 0; ok && p < P; ++p) {
                 const int nchunk = (p + 1) * CPP;
                 for (int c = 0; ok && c < nchunk; ++c, ++t) {
-                    const int b = (int)(t & 1), s = (int)(t % ws);
+                    const int b = (int)(t % G), s = (int)(t % ws);
+                    const long long j = t / G;
                     if (c == 0) {
                         if (!(ok = mbar_wait(bar(BAR_V_EMPTY), (uint32_t)((pv & 1) ^ 1), abort_flag))) break;
                     }
-                    if (!(ok = mbar_wait(bar(BAR_K_FULL + b), (uint32_t)((t >> 1) & 1), abort_flag))) break;
+                    if (!(ok = mbar_wait(bar(BAR_K_FULL + b), (uint32_t)(j & 1), abort_flag))) break;
                     if (!(ok = mbar_wait(bar(BAR_W_FULL + s), (uint32_t)((t / ws) & 1), abort_flag))) break;
                     tc_fence_after();
-                    const uint32_t aH = base + map.k + b * 16384u, aL = aH + 8192u;
-                    const uint32_t bH = base + map.w + s * map.w_stage, bL = bH + (uint32_t)KC * NV * 4u;
+                    const uint32_t aH = k_lo0 + ((b * 16384u) >> 4), aL = aH + (8192u >> 4);
+                    const uint32_t bH = w_lo0 + ((s * map.w_stage) >> 4), bL = bH + (((uint32_t)KC * NV * 4u) >> 4);
+#pragma unroll
                     for (int combo = 0; combo < 3; ++combo) {
                         const uint32_t a0 = combo == 2 ? aL : aH, b0 = combo == 1 ? bL : bH;
 #pragma unroll
-                        for (int j = 0; j < KC / 8; ++j)
-                            tc_mma_tf32(tmem, smem_desc(a0 + j * 4096u, 2048u, 128u),
-                                        smem_desc(b0 + j * (2u * NV * 16u), NV * 16u, 128u), IDESC_V,
-                                        (c > 0 || combo > 0 || j > 0) ? 1u : 0u);
+                        for (int jj = 0; jj < KC / 8; ++jj)
+                            tc_mma_tf32(tmem, pack64(a0 + jj * (4096u >> 4), HI),
+                                        pack64(b0 + jj * ((2u * NV * 16u) >> 4), HI), IDESC_V,
+                                        (c > 0 || combo > 0 || jj > 0) ? 1u : 0u);
                     }
                     tc_commit(bar(BAR_W_EMPTY + s));
                     tc_commit(bar(BAR_K_EMPTY + b));
@@ -354,7 +378,7 @@ __global__ void __launch_bounds__(256, 1) score_tc_kernel(const TcParams prm)
                         tc_commit(bar(BAR_V_FULL));
                         ++pv;
                     }
-                    const long long ahead = t + 2;
+                    const long long ahead = t + G;
                     if (ahead - t_tile0 < items_per_tile) ok = issue_distance(ahead);
                 }
             }
@@ -363,21 +387,26 @@ __global__ void __launch_bounds__(256, 1) score_tc_kernel(const TcParams prm)
         tc_commit(bar(BAR_MMA_DONE));
         mbar_wait(bar(BAR_MMA_DONE), 0, abort_flag + 1);
     } else if (warp >= 4) {
-        // ------------------------------------------------------------ Matern / epilogue warps
-        const int q4 = warp - 4;                 // TMEM lane quarter == warp % 4
+        // ------------------------------------------------------------ Matern / epilogue warp groups
+        const int grp = (warp - 4) >> 2;         // 0..G-1
+        const int q4 = warp & 3;                 // TMEM lane quarter == warp % 4
         const int row = q4 * 32 + lane;          // candidate row in the tile == TMEM lane
         const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
-        long long t = 0, pv = 0;
+        long long t = grp;                       // next own item (global numbering)
+        long long t_tile0 = 0;                   // first item of the current tile
+        long long pv = 0, tile_iter = 0;
         bool ok = true;
         bool bad = false;
-        for (long long tile = first_tile; ok && tile < prm.total_tiles; tile += tile_step) {
+        // scratch for the end-of-tile reduction lives in k* buffer 0 (dead once the last pass is done)
+        double* red = reinterpret_cast<double*>(sm + map.k);
+        for (long long tile = first_tile; ok && tile < prm.total_tiles; tile += tile_step, ++tile_iter) {
             const int g = (int)(tile / prm.tiles_per_gp);
             const long long cand = (tile % prm.tiles_per_gp) * TILE_M + row;
             const bool valid = cand < prm.m;
             const float sf2 = prm.sf2[g];
-            // ---- scale the candidate, split it, store it as the A operand of the distance MMA
-            float zn = 0.f;
-            {
+            if (grp == G - 1) {
+                // ---- scale the candidate, split it, store it as the A operand of the distance MMA
+                float zn = 0.f;
                 const float* zrow = prm.xcand + ((size_t)g * prm.m + (valid ? cand : 0)) * prm.d;
                 const float* cen = prm.centre + (size_t)g * DP;
                 const float* scl = prm.scale + (size_t)g * DP;
@@ -408,25 +437,39 @@ __global__ void __launch_bounds__(256, 1) score_tc_kernel(const TcParams prm)
                     *reinterpret_cast<float4*>(sm + map.z + (uint32_t)DP * 512u + (uint32_t)j4 * 2048u + row * 16) =
                         make_float4(lo[0], lo[1], lo[2], lo[3]);
                 }
+                zn_s[row] = zn;
+                fence_proxy_async();
+                mbar_arrive(bar(BAR_Z_READY));
             }
-            fence_proxy_async();
-            mbar_arrive(bar(BAR_Z_READY));
+            ok = mbar_wait(bar(BAR_Z_READY), (uint32_t)(tile_iter & 1), abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            const float zn = zn_s[row];
 
             const float* xn_g = prm.xnorm + (size_t)g * prm.NP;
             const float* al_g = prm.alpha + (size_t)g * prm.NP;
             double mu_acc = 0.0, a2_acc = 0.0, s2_acc = 0.0, q_acc = 0.0;
+            int pass_base = 0;   // items of this tile before pass p
             for (int p = 0; ok && p < P; ++p) {
                 const int nchunk = (p + 1) * CPP;
-                for (int c = 0; c < nchunk; ++c, ++t) {
-                    const int b = (int)(t & 1);
-                    ok = mbar_wait(bar(BAR_D_FULL + b), (uint32_t)((t >> 1) & 1), abort_flag);
+                // own items of this pass: global t with t - t_tile0 - pass_base in [0, nchunk)
+                while (t - t_tile0 - pass_base < nchunk) {
+                    const int c = (int)(t - t_tile0 - pass_base);
+                    const long long j = t / G;
+                    // the next own chunk's norms and weights: pull them towards L1 while this one is worked on
+                    if (lane < 2) {
+                        const int cn = c + G < nchunk ? c + G : (c + G - nchunk);
+                        const float* pf = (lane == 0 ? xn_g : al_g) + cn * KC;
+                        asm volatile("prefetch.global.L1 [%0];" ::"l"(pf));
+                    }
+                    ok = mbar_wait(bar(BAR_D_FULL + grp), (uint32_t)(j & 1), abort_flag);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     tc_fence_after();
                     float dot[KC];
-                    tc_ld16(lane_addr + NV + b * KC, dot);
+                    tc_ld16(lane_addr + NV + grp * KC, dot);
                     tc_fence_before();
-                    mbar_arrive(bar(BAR_D_EMPTY + b));
+                    mbar_arrive(bar(BAR_D_EMPTY + grp));
                     const bool fresh = c >= p * CPP;   // first time this chunk is generated for the tile
                     float kv[KC];
                     float mpart = 0.f, apart = 0.f, spart = 0.f;
@@ -438,7 +481,7 @@ __global__ void __launch_bounds__(256, 1) score_tc_kernel(const TcParams prm)
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const float r2 = fmaxf(fmaf(-2.f, dot[4 * q + e], zn + xn[e]), 0.f);
-                            const float s = sqrtf(5.f * r2);
+                            const float s = sqrt_approx(5.f * r2);
                             const float v = sf2 * fmaf(s, fmaf(s, 1.f / 3.f, 1.f), 1.f) * __expf(-s);
                             kv[4 * q + e] = v;
                             const float va = v * al[e];
@@ -452,10 +495,10 @@ __global__ void __launch_bounds__(256, 1) score_tc_kernel(const TcParams prm)
                         a2_acc += (double)apart;
                         s2_acc += (double)spart;
                     }
-                    ok = mbar_wait(bar(BAR_K_EMPTY + b), (uint32_t)(((t >> 1) & 1) ^ 1), abort_flag);
+                    ok = mbar_wait(bar(BAR_K_EMPTY + grp), (uint32_t)((j & 1) ^ 1), abort_flag);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
-                    uint8_t* kb = sm + map.k + b * 16384u + row * 16;
+                    uint8_t* kb = sm + map.k + grp * 16384u + row * 16;
 #pragma unroll
                     for (int q = 0; q < KC / 4; ++q) {
                         float hi[4], lo[4];
@@ -468,16 +511,18 @@ __global__ void __launch_bounds__(256, 1) score_tc_kernel(const TcParams prm)
                         *reinterpret_cast<float4*>(kb + 8192u + q * 2048u) = make_float4(lo[0], lo[1], lo[2], lo[3]);
                     }
                     fence_proxy_async();
-                    mbar_arrive(bar(BAR_K_FULL + b));
+                    mbar_arrive(bar(BAR_K_FULL + grp));
+                    t += G;
                 }
                 if (!ok) break;
-                // ---- end of pass: q += sum_i V^2
+                pass_base += nchunk;
+                // ---- end of pass: q += sum_i V^2 over this group's share of the columns
                 ok = mbar_wait(bar(BAR_V_FULL), (uint32_t)(pv & 1), abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tc_fence_after();
 #pragma unroll 1
-                for (int c0 = 0; c0 < NV; c0 += 16) {
+                for (int c0 = grp * 16; c0 < NV; c0 += 16 * G) {
                     float v[16];
                     tc_ld16(lane_addr + c0, v);
                     float part = 0.f;
@@ -490,7 +535,27 @@ __global__ void __launch_bounds__(256, 1) score_tc_kernel(const TcParams prm)
                 ++pv;
             }
             if (!ok) break;
-            if (valid) {
+            t_tile0 += items_per_tile;
+            // ---- combine the groups' partial sums; group 0 finishes the candidate
+            if (G > 1) {
+                double* mine = red + ((size_t)grp * TILE_M + row) * 4;
+                mine[0] = mu_acc; mine[1] = a2_acc; mine[2] = s2_acc; mine[3] = q_acc;
+                mbar_arrive(bar(BAR_RED_READY));
+                if (grp == 0) {   // only the finishing group waits; the others move on to the next tile
+                    ok = mbar_wait(bar(BAR_RED_READY), (uint32_t)(tile_iter & 1), abort_flag);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                }
+            }
+            if (grp == 0 && valid) {
+                if (G > 1) {
+                    mu_acc = a2_acc = s2_acc = q_acc = 0.0;
+#pragma unroll
+                    for (int gg = 0; gg < G; ++gg) {
+                        const double* o = red + ((size_t)gg * TILE_M + row) * 4;
+                        mu_acc += o[0]; a2_acc += o[1]; s2_acc += o[2]; q_acc += o[3];
+                    }
+                }
                 const size_t f = (size_t)g * prm.m + cand;
                 const CandidateResult res = finalize_candidate(mu_acc, q_acc, (double)sf2, (double)prm.best[g]);
                 prm.mu[f] = res.mu;
@@ -645,17 +710,18 @@ r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream)
     t->NP = round_up(n, t->NV);
     t->P = t->NP / t->NV;
     t->xs = 2;
+    t->G = t->NV == 256 ? 3 : 2;
     const size_t budget = 227 * 1024 - 1024 - kBarBytes;
     for (t->ws = MAX_STAGES; t->ws >= 2; --t->ws) {
-        const SmemMap mp = smem_map(t->DP, t->NV, t->xs, t->ws);
+        const SmemMap mp = smem_map(t->DP, t->NV, t->G, t->xs, t->ws);
         if (mp.bar <= budget) break;
     }
     if (t->ws < 2) {
         tc_release(gp);   // does not fit: the SIMT engine serves this shape
         return R3_OK;
     }
-    t->smem_bytes = smem_map(t->DP, t->NV, t->xs, t->ws).bar + kBarBytes + 1024;
-    t->tmem_cols = (t->NV + 2 * KC) <= 256 ? 256 : 512;
+    t->smem_bytes = smem_map(t->DP, t->NV, t->G, t->xs, t->ws).bar + kBarBytes + 1024;
+    t->tmem_cols = (t->NV + t->G * KC) <= 256 ? 256 : 512;
     const int CPP = t->NV / KC;
     const size_t tiles = (size_t)CPP * t->P * (t->P + 1) / 2;
     t->wt_gp_stride = tiles * (2 * (size_t)KC * t->NV);
@@ -683,9 +749,9 @@ r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream)
     if ((e = cudaGetLastError()) != cudaSuccess) return fail("operand preparation launch", e);
     if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return fail("operand preparation", e);
     if (t->NV == 256)
-        e = cudaFuncSetAttribute(score_tc_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t->smem_bytes);
+        e = cudaFuncSetAttribute(score_tc_kernel<256, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t->smem_bytes);
     else
-        e = cudaFuncSetAttribute(score_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t->smem_bytes);
+        e = cudaFuncSetAttribute(score_tc_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t->smem_bytes);
     if (e != cudaSuccess) return fail("cudaFuncSetAttribute", e);
     return R3_OK;
 }
@@ -739,9 +805,9 @@ r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, floa
     const unsigned grid = (unsigned)(prm.total_tiles < sms ? prm.total_tiles : sms);
     prof_begin(gp, stream);
     if (t->NV == 256)
-        R3_LAUNCH(score_tc_kernel<256>, grid, 256, t->smem_bytes, stream, prm);
+        R3_LAUNCH((score_tc_kernel<256, 3>), grid, 128 + 128 * 3, t->smem_bytes, stream, prm);
     else
-        R3_LAUNCH(score_tc_kernel<128>, grid, 256, t->smem_bytes, stream, prm);
+        R3_LAUNCH((score_tc_kernel<128, 2>), grid, 128 + 128 * 2, t->smem_bytes, stream, prm);
     prof_end(gp, stream);
     return guard_and_rescue(gp, Xcand, m, gb, mu, sigma, ei, stream);
 }
