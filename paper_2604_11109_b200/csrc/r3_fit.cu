@@ -397,12 +397,13 @@ r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream)
 {
     const int B = gp->batch, n = gp->n, d = gp->d, npad = gp->npad;
     const size_t mat = (size_t)npad * npad;
-    double *Dinv = nullptr, *T = nullptr, *u = nullptr;
+    double *Dinv = nullptr, *T = nullptr, *u = nullptr, *slabs = nullptr;
     R3_CUDA_TRY(cudaMalloc(&Dinv, sizeof(double) * B * (size_t)(npad / NB) * NB * NB));
     auto fail = [&](r3_status_t st) {
         cudaFree(Dinv);
         cudaFree(T);
         cudaFree(u);
+        cudaFree(slabs);
         return st;
     };
 #define TRY_OR_FAIL(expr)                                                                          \
@@ -426,6 +427,7 @@ r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream)
 
     TRY_OR_FAIL(cudaMalloc(&T, sizeof(double) * B * mat));
     TRY_OR_FAIL(cudaMalloc(&u, sizeof(double) * B * npad));
+    TRY_OR_FAIL(cudaMalloc(&slabs, sizeof(double) * ((size_t)B + (size_t)B * kRowSlabs * npad)));
 
     LAUNCH_OR_FAIL(check_finite_kernel, 296, 256, gp->X, (size_t)B * n * d, gp->status_d);
     LAUNCH_OR_FAIL(check_finite_kernel, 64, 256, y, (size_t)B * n, gp->status_d);
@@ -457,8 +459,8 @@ r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream)
     // spectral norm of W by power iteration on W^T W (alpha64/alpha32 serve as scratch first)
     {
         double* pv = gp->alpha64;
-        double* lam = T;  // [B] scratch, followed by the row-slab partial sums
-        double* part = T + B;
+        double* lam = slabs;  // [B], followed by the row-slab partial sums
+        double* part = slabs + B;
         LAUNCH_OR_FAIL(power_init_kernel, B, 256, pv, n, npad);
         LAUNCH_OR_FAIL(power_normalize_kernel, B, 256, pv, npad, lam);
         for (int it = 0; it < 12; ++it) {
@@ -472,8 +474,8 @@ r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream)
     }
     LAUNCH_OR_FAIL(w_times_y_kernel<float>, dim3((npad + 7) / 8, B), 256, gp->W64, y, n, n, npad, u);
     LAUNCH_OR_FAIL(wt_times_u_partial_kernel, dim3((npad + 127) / 128, kRowSlabs, B), 128, gp->W64, u, n, npad,
-                   T + B);
-    LAUNCH_OR_FAIL(wt_times_u_reduce_kernel, dim3((npad + 127) / 128, B), 128, T + B, npad, gp->alpha64,
+                   slabs + B);
+    LAUNCH_OR_FAIL(wt_times_u_reduce_kernel, dim3((npad + 127) / 128, B), 128, slabs + B, npad, gp->alpha64,
                    gp->alpha32);
     LAUNCH_OR_FAIL(to_float_kernel, 1184, 256, gp->W64, gp->W32, (size_t)B * mat);
 

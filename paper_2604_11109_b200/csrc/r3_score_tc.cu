@@ -1,31 +1,46 @@
-// Tensor-core scoring engine for sm_100a: tcgen05 MMAs (kind::tf32, 3xTF32 split) with TMEM
-// accumulators, operands staged by bulk asynchronous copies, everything fused in one kernel so that
-// the cross-covariance k* never leaves the SM.
+// Tensor-core scoring engine for sm_100a: tcgen05 MMAs (kind::f16 on two-term FP16 splits, FP32
+// accumulation in TMEM), operands staged by bulk asynchronous copies, everything fused in one kernel
+// so that the cross-covariance k* never leaves the SM.
 //
 // One CTA owns a tile of 128 candidates; a TMEM lane IS a candidate.  For that tile it walks the rows
 // of W = L^-1 in passes of NV rows (the V accumulator: 128 lanes x NV TMEM columns) and, inside a pass,
-// the observations in chunks of KC = 16:
+// the observations in chunks of KC = 32:
 //
-//   distance MMA   D[cand][k] = z~ . x~_k   (A = scaled candidates, B = scaled observations, depth d)
-//   Matern warps   r^2 = |z~|^2 + |x~_k|^2 - 2 D, k* = sf2 M52(r): read D from TMEM, write k* (hi/lo
-//                  TF32 planes) as the next A operand into shared memory; mu += k* alpha on the way
-//   variance MMA   V[cand][i] += k*[cand][k] W[i][k]   (B = pre-tiled chunk of W, hi/lo planes)
+//   distance MMA   D[cand][k] = z~ . x~_k   (A = scaled candidates, kept in TMEM for the whole tile;
+//                  B = scaled observations, depth d), for KD observations at a time.  An MMA whose A
+//                  operand comes from shared memory costs ~130 cycles however narrow it is (the A
+//                  tile is fetched again every time); with A in TMEM a narrow MMA is cheap
+//   Matern warps   r^2 = |z~|^2 + |x~_k|^2 - 2 D, k* = sf2 M52(r): read D from TMEM, write k* (scaled,
+//                  FP16 hi/lo planes) as the next A operand into shared memory; mu += k* alpha on the way
+//   variance MMA   V[cand][i] += k*[cand][k] W[i][k]   (B = pre-tiled chunk of W, scaled FP16 hi/lo planes)
 //   end of pass    q += sum_i V[cand][i]^2 read back from TMEM; after the last pass sigma, EI, outputs
 //
-// Each product is three MMAs (hi*hi + hi*lo + lo*hi) accumulating in FP32, which restores FP32-level
-// accuracy from TF32 operands.  W is lower-triangular, so pass p only needs k < (p+1) NV; k* chunks are
-// regenerated for every pass they take part in instead of being stored.
+// Precision.  Every product is three MMAs (hi*hi + hi*lo + lo*hi): x = hi + lo with hi = fp16(x) and
+// lo = fp16(x - hi) carries 22 significant bits, and the tensor core accumulates in FP32, so the
+// result is FP32-grade at twice the TF32 rate and half the operand bytes.  k* and W are multiplied by
+// powers of two before the split (so that the low parts stay normal numbers) and the accumulator is
+// scaled back exactly.  The scaled coordinates of the distance product must fit FP16's range; a
+// history that does not is left to the SIMT engine and a candidate that does not is recomputed in FP64.
 //
-// Warp roles: warp 0 streams chunks of scaled observations, warp 1 streams chunks of W, warp 2 issues
-// every MMA (one thread) and owns the TMEM allocation, warps 4.. form G Matern/epilogue groups of four
-// warps (one warp per TMEM lane quarter); group g takes every G-th chunk with its own distance and k*
-// buffers, so G chunks are in flight between the two MMA streams.  Stages are handed over through mbarriers; every wait is
-// bounded: when a limit is hit the CTA raises a status bit, all roles leave their loops, in-flight
-// copies and MMAs are drained (bounded again), TMEM is freed and the kernel returns.
+// W is lower-triangular, so pass p only needs k < (p+1) NV; k* chunks are regenerated for every pass
+// they take part in instead of being stored.
+//
+// Warp roles: warp 0 streams the operands (lane 0: scaled observations, lane 1: chunks of W), warp 1
+// issues the distance MMAs, warp 2 issues the variance MMAs and owns the TMEM allocation (one thread
+// each), warps 4.. form G Matern/epilogue groups of four warps (one warp per TMEM lane quarter); group
+// g takes every G-th chunk with its own k* buffer, so G chunks are in flight between the two MMA
+// streams.  Stages are handed over through mbarriers; every wait is bounded: when a limit is hit the
+// CTA raises a status bit, all roles leave their loops, in-flight copies and MMAs are drained (bounded
+// again), TMEM is freed and the kernel returns.
 //
 // Operand layouts are the no-swizzle K-major "core matrix" form: 8 rows x 16 bytes contiguous, 8-row
 // groups 128 bytes apart, 16-byte k-slices one full panel apart.  W and the observations are stored
 // in global memory already tiled that way by the fit, so a stage is one contiguous bulk copy.
+#include <cuda_fp16.h>
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+
 #include "r3_epilogue.cuh"
 #include "r3_internal.cuh"
 
@@ -33,26 +48,38 @@ namespace r3 {
 
 namespace {
 
-constexpr int KC = 16;        // observations per chunk
+constexpr int KC = 32;        // observations per chunk of the variance product
 constexpr int TILE_M = 128;   // candidates per CTA tile
-constexpr int MAX_STAGES = 4;
+constexpr int XS = 2;         // stages of scaled observations
+constexpr int MAX_STAGES = 4; // stages of W
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;  // ~2 s
 
-// relative error of one k* entry: eps0 + eps1 * (|z~|^2 + max|x~|^2) / sqrt(d)  (distance by 3xTF32 GEMM)
+// relative error of one k* entry: eps0 + eps1 * (|z~|^2 + max|x~|^2) / sqrt(d)  (distance by split GEMM)
 constexpr double kEpsTc0 = 2.5e-7;
-constexpr double kEpsTc1 = 2.0e-7;
+constexpr double kEpsTc1 = 5.0e-8;
+// A pair (candidate, observation) whose k* (|z~|^2 + |x~|^2) exceeds kRefine sf2 has its squared distance
+// recomputed by direct differences: r^2 from the norm expansion loses (|z~|^2 + |x~|^2) / r^2 digits, and
+// the close pairs are the ones that carry the posterior.
+constexpr float kRefine = 2.0f;
+// scaled coordinates beyond this do not fit the FP16 planes of the distance product
+constexpr float kMaxScaled = 16384.f;
+// operands of the variance product are scaled to at most 2^kScaleExp before the FP16 split
+constexpr int kScaleExp = 14;
 
 struct TensorOperands {
-    int NV = 0, G = 0, DP = 0, NP = 0, P = 0, xs = 0, ws = 0, tmem_cols = 0;
+    int NV = 0, G = 0, KD = 0, DP = 0, NP = 0, P = 0, ws = 0;
     size_t smem_bytes = 0;
-    size_t wt_gp_stride = 0;   // floats per GP in wt
+    size_t wt_gp_stride = 0;   // halves per GP in wt
     float* centre = nullptr;   // [B][DP]  column means of X (zero padded)
     float* scale = nullptr;    // [B][DP]  1/lengthscale (zero padded)
-    float* xt = nullptr;       // [B][NP/KC][2][DP/4][KC][4]  scaled observations, hi/lo planes
+    __half* xt = nullptr;      // [B][NP/KD][2][DP/8][KD][8]  scaled observations, FP16 hi/lo planes
+    float* xs32 = nullptr;     // [B][NP][DP]  scaled observations in FP32 (refinement of close pairs)
     float* xnorm = nullptr;    // [B][NP]  |x~_k|^2
     float* xnmax = nullptr;    // [B]      max_k |x~_k|^2
     float* alpha = nullptr;    // [B][NP]  weights, zero padded
-    float* wt = nullptr;       // [B][tile(p,c)][2][KC/4][NV][4]  W chunks, hi/lo planes
+    __half* wt = nullptr;      // [B][tile(p,c)][2][KC/8][NV][8]  chunks of 2^eW W, FP16 hi/lo planes
+    float* kscale = nullptr;   // [B]  2^eK, applied to k* before its split
+    double* vinv2 = nullptr;   // [B]  2^(-2 (eK + eW)): scales sum V^2 back
 };
 
 struct TcParams {
@@ -60,13 +87,16 @@ struct TcParams {
     long long m;
     int batch, d;
     float *mu, *sigma, *ei, *err_mu, *err_q;
-    const float *centre, *scale, *xt, *xnorm, *xnmax, *alpha, *wt;
+    const float *centre, *scale, *xs32, *xnorm, *xnmax, *alpha, *kscale;
+    const __half *xt, *wt;
+    const double* vinv2;
     size_t wt_gp_stride;
     const float *sf2, *best;
     const double* wnorm;
-    int DP, NP, P, xs, ws;
+    int DP, NP, P, ws;
     int* status;
     long long tiles_per_gp, total_tiles;
+    long long* trace;   // optional [grid][4 roles][8] cycle counters (diagnostics)
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -127,15 +157,32 @@ __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tc_mma_tf32(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                            uint32_t accumulate)
+__device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                           uint32_t accumulate)
 {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
+}
+// A operand from TMEM (lane = row, one 32-bit column = two consecutive FP16 k-elements)
+__device__ __forceinline__ void tc_mma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+                                              uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t* r)
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(taddr), "r"(r[0]),
+                 "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
 }
 __device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v)
 {
@@ -150,50 +197,13 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v)
 #pragma unroll
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
-__device__ __forceinline__ float tf32_hi(float x)
+__device__ __forceinline__ void tc_ld8(uint32_t taddr, uint32_t* r)
 {
-    uint32_t u;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(x));
-    return __uint_as_float(u);
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr)
+                 : "memory");
 }
-
-// Shared-memory matrix descriptors are the no-swizzle K-major form: bits 0-13 start address >> 4,
-// bits 16-29 the byte distance between the two 16-byte k-slices of one MMA >> 4, bits 32-45 the byte
-// distance between 8-row groups >> 4, bit 46 the descriptor version.
-// Instruction descriptor: FP32 accumulate, TF32 x TF32, both K-major, M = 128, N = n.
-__device__ __forceinline__ constexpr uint32_t instr_desc(uint32_t n)
-{
-    return (1u << 4) | (2u << 7) | (2u << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
-}
-
-// shared-memory map (byte offsets from a 1024-aligned base)
-struct SmemMap {
-    uint32_t z, k, x, w, bar;
-    uint32_t x_stage, w_stage;
-};
-__host__ __device__ inline SmemMap smem_map(int DP, int NV, int G, int xs, int ws)
-{
-    SmemMap s;
-    s.z = 0;                                       // 2 planes x [DP/4][128][4] floats
-    s.k = s.z + 2u * DP * 512u;                    // G buffers x 2 planes x [KC/4][128][4]
-    s.x = s.k + (uint32_t)G * 16384u;              // xs stages x 2 planes x [DP/4][KC][4]
-    s.x_stage = 2u * DP * KC * 4u;
-    s.w = s.x + (uint32_t)xs * s.x_stage;          // ws stages x 2 planes x [KC/4][NV][4]
-    s.w_stage = 2u * KC * NV * 4u;
-    s.bar = s.w + (uint32_t)ws * s.w_stage;
-    return s;
-}
-constexpr uint32_t kBarBytes = 1024;   // barriers, flags, TMEM slot, candidate norms
-
-// barrier slots (8 bytes each) inside the barrier block
-enum : uint32_t {
-    BAR_X_FULL = 0, BAR_X_EMPTY = 4, BAR_W_FULL = 8, BAR_W_EMPTY = 12, BAR_D_FULL = 16, BAR_D_EMPTY = 20,
-    BAR_K_FULL = 24, BAR_K_EMPTY = 28, BAR_V_FULL = 32, BAR_V_EMPTY = 33, BAR_Z_READY = 34, BAR_MMA_DONE = 35,
-    BAR_RED_READY = 36, BAR_COUNT = 37
-};
-constexpr uint32_t kFlagOffset = BAR_COUNT * 8;       // int abort, int drain-abort, uint32 tmem base
-constexpr uint32_t kZnOffset = 512;                   // float[128] squared norms of the scaled candidates
-
 __device__ __forceinline__ uint64_t pack64(uint32_t lo, uint32_t hi)
 {
     uint64_t r;
@@ -206,17 +216,121 @@ __device__ __forceinline__ float sqrt_approx(float x)
     asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
     return r;
 }
+// (a, b) -> FP16 hi parts and FP16 low parts, each packed as half2
+__device__ __forceinline__ void split2(float a, float b, __half2& hi, __half2& lo)
+{
+    hi = __floats2half2_rn(a, b);
+    const float2 back = __half22float2(hi);
+    lo = __floats2half2_rn(a - back.x, b - back.y);
+}
+
+// Shared-memory matrix descriptors are the no-swizzle K-major form: bits 0-13 start address >> 4,
+// bits 16-29 the byte distance between the two 16-byte k-slices of one MMA >> 4, bits 32-45 the byte
+// distance between 8-row groups (128) >> 4, bit 46 the descriptor version.
+constexpr uint32_t kDescHi = (128u >> 4) | (1u << 14);
+// Instruction descriptor: FP32 accumulate, FP16 x FP16 (format code 0), both K-major, M = 128, N = n.
+__device__ __forceinline__ constexpr uint32_t instr_desc_f16(uint32_t n)
+{
+    return (1u << 4) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+// shared-memory map (byte offsets from a 1024-aligned base)
+struct SmemMap {
+    uint32_t z, k, x, w, bar;
+    uint32_t x_stage, w_stage;
+};
+__host__ __device__ inline SmemMap smem_map(int DP, int NV, int G, int KD, int ws)
+{
+    SmemMap s;
+    s.z = 0;                                       // (the scaled candidates live in TMEM)
+    s.k = 0;                                       // G buffers x 2 planes x [KC/8][128][8] halves
+    s.x = s.k + (uint32_t)G * 16384u;              // XS stages x 2 planes x [DP/8][KD][8] halves
+    s.x_stage = 2u * DP * KD * 2u;
+    s.w = s.x + (uint32_t)XS * s.x_stage;          // ws stages x 2 planes x [KC/8][NV][8] halves
+    s.w_stage = 2u * KC * NV * 2u;
+    s.bar = s.w + (uint32_t)ws * s.w_stage;
+    return s;
+}
+constexpr uint32_t kBarBytes = 1024;   // barriers, flags, TMEM slot, candidate norms
+
+// barrier slots (8 bytes each) inside the barrier block
+enum : uint32_t {
+    BAR_X_FULL = 0, BAR_X_EMPTY = 2, BAR_W_FULL = 4, BAR_W_EMPTY = 8, BAR_D_FULL = 12, BAR_D_EMPTY = 14,
+    BAR_K_FULL = 16, BAR_K_EMPTY = 20, BAR_V_FULL = 24, BAR_V_EMPTY = 25, BAR_Z_READY = 26, BAR_RED_READY = 27,
+    BAR_MMA_DONE = 28,  // two slots: distance issuer, variance issuer
+    BAR_COUNT = 30
+};
+constexpr uint32_t kFlagOffset = BAR_COUNT * 8;       // int abort, int drain-abort, uint32 tmem base
+constexpr uint32_t kZnOffset = 512;                   // float[128] squared norms of the scaled candidates
+
+#define TICK(cat)                                                                          \
+    do {                                                                                   \
+        if (prm.trace) {                                                                   \
+            const long long now__ = clock64();                                             \
+            tacc[cat] += now__ - tlast;                                                    \
+            tlast = now__;                                                                 \
+        }                                                                                  \
+    } while (0)
+
+// Out-of-line (cold) path of the Matern warps: for the pairs marked in `close`, replace k* by the value
+// computed from r^2 = sum_j (z~_j - x~_j)^2, with z~ = hi + lo read back from the TMEM planes at z_taddr
+// and x~ in FP32 from global memory.  Called by all 32 lanes of a warp together (TMEM loads are
+// warp-wide); a lane without marked pairs only takes part in the loads.
+__device__ __noinline__ void refine_close_pairs(float* kv, uint32_t close, uint32_t z_taddr, int DP,
+                                                const float* __restrict__ xrow0, float sf2)
+{
+    float r2x[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) r2x[i] = 0.f;
+    for (int j16 = 0; j16 < DP / 16; ++j16) {
+        uint32_t zh[8], zl[8];
+        tc_ld8(z_taddr + j16 * 8, zh);
+        tc_ld8(z_taddr + DP / 2 + j16 * 8, zl);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        float z[16];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&zh[e]));
+            const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&zl[e]));
+            z[2 * e] = a.x + b.x;
+            z[2 * e + 1] = a.y + b.y;
+        }
+        for (uint32_t rest = close; rest; rest &= rest - 1) {
+            const int i = __ffs(rest) - 1;
+            const float4* xp = reinterpret_cast<const float4*>(xrow0 + (size_t)i * DP + j16 * 16);
+            float acc = 0.f;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float4 x4 = __ldg(xp + e);
+                float df = z[4 * e] - x4.x;
+                acc = fmaf(df, df, acc);
+                df = z[4 * e + 1] - x4.y;
+                acc = fmaf(df, df, acc);
+                df = z[4 * e + 2] - x4.z;
+                acc = fmaf(df, df, acc);
+                df = z[4 * e + 3] - x4.w;
+                acc = fmaf(df, df, acc);
+            }
+            r2x[i] += acc;
+        }
+    }
+    for (uint32_t rest = close; rest; rest &= rest - 1) {
+        const int i = __ffs(rest) - 1;
+        const float s = sqrtf(5.f * r2x[i]);
+        kv[i] = sf2 * fmaf(s, fmaf(s, 1.f / 3.f, 1.f), 1.f) * __expf(-s);
+    }
+}
 
 // NV: rows of W per pass (TMEM columns of the V accumulator).  G: number of Matern warp groups; group
-// g owns items t = g (mod G) of the chunk sequence together with distance buffer g and k* buffer g.
-template <int NV, int G>
+// g owns chunks t = g (mod G) and k* buffer g.  KD: observations per distance product.
+template <int NV, int G, int KD>
 __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcParams prm)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* sm = smem_raw + (base - raw);
-    const SmemMap map = smem_map(prm.DP, NV, G, prm.xs, prm.ws);
+    const SmemMap map = smem_map(prm.DP, NV, G, KD, prm.ws);
     const uint32_t bars = base + map.bar;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + map.bar + kFlagOffset);
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + map.bar + kFlagOffset + 8);
@@ -225,25 +339,32 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int CPP = NV / KC;                  // chunks per pass width
-    constexpr uint32_t TMEM_COLS = (NV + G * KC) <= 256 ? 256u : 512u;
-    const int DP = prm.DP, P = prm.P, xs = prm.xs, ws = prm.ws;
+    constexpr int SL = KD / KC;                   // chunks per distance product
+    // TMEM columns: V accumulator [0, NV), two distance buffers [NV, NV + 2 KD), scaled candidates
+    // (FP16 hi plane, then lo plane, DP/2 columns each) from NV + 2 KD
+    constexpr uint32_t TMEM_COLS = 512u;
+    constexpr uint32_t ZCOL = NV + 2 * KD;
+    const int DP = prm.DP, P = prm.P, ws = prm.ws;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < MAX_STAGES; ++i) {
+        for (int i = 0; i < XS; ++i) {
             mbar_init(bar(BAR_X_FULL + i), 1);
             mbar_init(bar(BAR_X_EMPTY + i), 1);
+            mbar_init(bar(BAR_D_FULL + i), 1);
+            mbar_init(bar(BAR_D_EMPTY + i), 128 * SL);
+        }
+        for (int i = 0; i < MAX_STAGES; ++i) {
             mbar_init(bar(BAR_W_FULL + i), 1);
             mbar_init(bar(BAR_W_EMPTY + i), 1);
-            mbar_init(bar(BAR_D_FULL + i), 1);
-            mbar_init(bar(BAR_D_EMPTY + i), 128);
             mbar_init(bar(BAR_K_FULL + i), 128);
             mbar_init(bar(BAR_K_EMPTY + i), 1);
         }
         mbar_init(bar(BAR_V_FULL), 1);
         mbar_init(bar(BAR_V_EMPTY), 128 * G);
         mbar_init(bar(BAR_Z_READY), 128);
-        mbar_init(bar(BAR_MMA_DONE), 1);
         mbar_init(bar(BAR_RED_READY), 128 * G);
+        mbar_init(bar(BAR_MMA_DONE), 1);
+        mbar_init(bar(BAR_MMA_DONE + 1), 1);
         abort_flag[0] = 0;
         abort_flag[1] = 0;   // private flag of the bounded drain waits
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -264,137 +385,169 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
     // tiles of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ...
     const long long first_tile = blockIdx.x, tile_step = gridDim.x;
     const int items_per_tile = CPP * P * (P + 1) / 2;
+    long long tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    long long tlast = prm.trace ? clock64() : 0;
 
     if (warp == 0 && lane == 0) {
         // ------------------------------------------------------------ producer: scaled observations
         const uint32_t bytes = map.x_stage;
-        long long t = 0;
+        long long issued = 0;
+        int st = 0;
+        uint32_t ph = 0;   // stage ring: (stage, phase) advance together, no divisions in the loop
         bool ok = true;
         for (long long tile = first_tile; ok && tile < prm.total_tiles; tile += tile_step) {
             const int g = (int)(tile / prm.tiles_per_gp);
-            const float* src = prm.xt + (size_t)g * (prm.NP / KC) * (bytes / 4);
+            const __half* src = prm.xt + (size_t)g * (prm.NP / KD) * (bytes / 2);
             for (int p = 0; ok && p < P; ++p)
-                for (int c = 0; c < (p + 1) * CPP; ++c, ++t) {
-                    const int s = (int)(t % xs);
-                    if (!(ok = mbar_wait(bar(BAR_X_EMPTY + s), (uint32_t)(((t / xs) & 1) ^ 1), abort_flag))) break;
-                    mbar_arrive_expect_tx(bar(BAR_X_FULL + s), bytes);
-                    bulk_g2s(base + map.x + s * bytes, src + (size_t)c * (bytes / 4), bytes, bar(BAR_X_FULL + s));
+                for (int c = 0; c < (p + 1) * (NV / KD); ++c, ++issued) {
+                    if (!(ok = mbar_wait(bar(BAR_X_EMPTY + st), ph ^ 1u, abort_flag))) break;
+                    mbar_arrive_expect_tx(bar(BAR_X_FULL + st), bytes);
+                    bulk_g2s(base + map.x + st * bytes, src + (size_t)c * (bytes / 2), bytes, bar(BAR_X_FULL + st));
+                    if (++st == XS) { st = 0; ph ^= 1u; }
                 }
         }
-        if (!ok)  // aborting: let the copies still in flight land before the CTA goes away
-            for (long long u = (t > xs ? t - xs : 0); u < t; ++u)
-                mbar_wait(bar(BAR_X_FULL + (int)(u % xs)), (uint32_t)((u / xs) & 1), abort_flag + 1);
-    } else if (warp == 1 && lane == 0) {
+        if (!ok) {  // aborting: let the copies still in flight land before the CTA goes away
+            const int pending = (int)(issued < XS ? issued : XS);
+            for (int u = 0; u < pending; ++u) {
+                if (--st < 0) { st = XS - 1; ph ^= 1u; }
+                mbar_wait(bar(BAR_X_FULL + st), ph, abort_flag + 1);
+            }
+        }
+    } else if (warp == 0 && lane == 1) {
         // ------------------------------------------------------------ producer: chunks of W
         const uint32_t bytes = map.w_stage;
-        long long t = 0;
+        long long issued = 0;
+        int st = 0;
+        uint32_t ph = 0;
         bool ok = true;
         for (long long tile = first_tile; ok && tile < prm.total_tiles; tile += tile_step) {
             const int g = (int)(tile / prm.tiles_per_gp);
-            const float* src = prm.wt + (size_t)g * prm.wt_gp_stride;
+            const __half* src = prm.wt + (size_t)g * prm.wt_gp_stride;
             for (int p = 0; ok && p < P; ++p) {
-                const float* psrc = src + (size_t)(CPP * p * (p + 1) / 2) * (bytes / 4);
-                for (int c = 0; c < (p + 1) * CPP; ++c, ++t) {
-                    const int s = (int)(t % ws);
-                    if (!(ok = mbar_wait(bar(BAR_W_EMPTY + s), (uint32_t)(((t / ws) & 1) ^ 1), abort_flag))) break;
-                    mbar_arrive_expect_tx(bar(BAR_W_FULL + s), bytes);
-                    bulk_g2s(base + map.w + s * bytes, psrc + (size_t)c * (bytes / 4), bytes, bar(BAR_W_FULL + s));
+                const __half* psrc = src + (size_t)(CPP * p * (p + 1) / 2) * (bytes / 2);
+                for (int c = 0; c < (p + 1) * CPP; ++c, ++issued) {
+                    if (!(ok = mbar_wait(bar(BAR_W_EMPTY + st), ph ^ 1u, abort_flag))) break;
+                    mbar_arrive_expect_tx(bar(BAR_W_FULL + st), bytes);
+                    bulk_g2s(base + map.w + st * bytes, psrc + (size_t)c * (bytes / 2), bytes, bar(BAR_W_FULL + st));
+                    if (++st == ws) { st = 0; ph ^= 1u; }
                 }
             }
         }
-        if (!ok)
-            for (long long u = (t > ws ? t - ws : 0); u < t; ++u)
-                mbar_wait(bar(BAR_W_FULL + (int)(u % ws)), (uint32_t)((u / ws) & 1), abort_flag + 1);
+        if (!ok) {
+            const int pending = (int)(issued < ws ? issued : ws);
+            for (int u = 0; u < pending; ++u) {
+                if (--st < 0) { st = ws - 1; ph ^= 1u; }
+                mbar_wait(bar(BAR_W_FULL + st), ph, abort_flag + 1);
+            }
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ------------------------------------------------------------ MMA issuer: distance products
+        constexpr uint32_t IDESC_D = instr_desc_f16(KD);
+        // descriptor low word = start >> 4 | (k-slice distance >> 4) << 16
+        const uint32_t zH = tmem + ZCOL, zL = zH + (uint32_t)DP / 2;
+        const uint32_t x_lo0 = ((base + map.x) >> 4) | (((KD * 16u) >> 4) << 16);
+        const int ksteps = DP / 16;
+        long long tile_iter = 0;
+        int st = 0, db = 0;
+        uint32_t ph = 0, d_ph = 0;   // X stage ring; parity of the distance-buffer pair
+        bool ok = true;
+        for (long long tile = first_tile; ok && tile < prm.total_tiles; tile += tile_step, ++tile_iter) {
+            TICK(7);
+            if (!(ok = mbar_wait(bar(BAR_Z_READY), (uint32_t)(tile_iter & 1), abort_flag))) break;
+            TICK(3);
+            tc_fence_after();
+            for (int u = 0; u < items_per_tile / SL; ++u) {
+                TICK(7);
+                if (!(ok = mbar_wait(bar(BAR_X_FULL + st), ph, abort_flag))) break;
+                TICK(0);
+                if (!(ok = mbar_wait(bar(BAR_D_EMPTY + db), d_ph ^ 1u, abort_flag))) break;
+                TICK(1);
+                tc_fence_after();
+                const uint32_t xH_lo = x_lo0 + ((st * map.x_stage) >> 4), xL_lo = xH_lo + (((uint32_t)DP * KD * 2u) >> 4);
+                const uint32_t dcol = tmem + NV + db * KD;
+                uint32_t acc = 0;
+#pragma unroll
+                for (int combo = 0; combo < 3; ++combo) {
+                    const uint32_t a0 = combo == 2 ? zL : zH, b0 = combo == 1 ? xL_lo : xH_lo;
+                    for (int jj = 0; jj < ksteps; ++jj) {
+                        tc_mma_f16_ts(dcol, a0 + jj * 8u, pack64(b0 + jj * ((2u * KD * 16u) >> 4), kDescHi), IDESC_D, acc);
+                        acc = 1;
+                    }
+                }
+                tc_commit(bar(BAR_X_EMPTY + st));
+                tc_commit(bar(BAR_D_FULL + db));
+                TICK(2);
+                if (++st == XS) { st = 0; ph ^= 1u; }
+                if (++db == 2) { db = 0; d_ph ^= 1u; }
+            }
+        }
+        // every MMA issued by this thread must have completed before TMEM is freed
+        tc_commit(bar(BAR_MMA_DONE));
+        mbar_wait(bar(BAR_MMA_DONE), 0, abort_flag + 1);
+        if (prm.trace)
+            for (int i = 0; i < 8; ++i) prm.trace[((size_t)blockIdx.x * 4 + 3) * 8 + i] = tacc[i];
     } else if (warp == 2 && lane == 0) {
-        // ------------------------------------------------------------ MMA issuer
-        constexpr uint32_t IDESC_D = instr_desc(KC);
-        constexpr uint32_t IDESC_V = instr_desc(NV);
-        // descriptor words: lo = start>>4 | (lbo>>4)<<16, hi = sbo>>4 | version bit
-        constexpr uint32_t HI = (128u >> 4) | (1u << 14);
-        const uint32_t zH_lo = ((base + map.z) >> 4) | ((2048u >> 4) << 16);
-        const uint32_t zL_lo = zH_lo + (((uint32_t)DP * 512u) >> 4);
-        const uint32_t x_lo0 = ((base + map.x) >> 4) | (((KC * 16u) >> 4) << 16);
+        // ------------------------------------------------------------ MMA issuer: variance product
+        constexpr uint32_t IDESC_V = instr_desc_f16(NV);
         const uint32_t k_lo0 = ((base + map.k) >> 4) | ((2048u >> 4) << 16);
         const uint32_t w_lo0 = ((base + map.w) >> 4) | (((NV * 16u) >> 4) << 16);
-        const int ksteps_d = DP / 8;
-        long long t = 0;      // item counter (rings)
-        long long pv = 0;     // pass counter (V accumulator hand-over)
-        long long tile_iter = 0;
+        uint32_t v_ph = 0;    // parity of the pass counter (V accumulator hand-over)
+        int w_s = 0, k_s = 0;
+        uint32_t w_ph = 0, k_ph = 0;
         bool ok = true;
-
-        auto issue_distance = [&](long long tu) -> bool {
-            const int s = (int)(tu % xs), b = (int)(tu % G);
-            const long long j = tu / G;
-            if (!mbar_wait(bar(BAR_X_FULL + s), (uint32_t)((tu / xs) & 1), abort_flag)) return false;
-            if (!mbar_wait(bar(BAR_D_EMPTY + b), (uint32_t)((j & 1) ^ 1), abort_flag)) return false;
-            tc_fence_after();
-            const uint32_t xH_lo = x_lo0 + ((s * map.x_stage) >> 4), xL_lo = xH_lo + (((uint32_t)DP * KC * 4u) >> 4);
-            const uint32_t dcol = tmem + NV + b * KC;
-            uint32_t acc = 0;
-#pragma unroll
-            for (int combo = 0; combo < 3; ++combo) {
-                const uint32_t a0 = combo == 2 ? zL_lo : zH_lo, b0 = combo == 1 ? xL_lo : xH_lo;
-                for (int jj = 0; jj < ksteps_d; ++jj) {
-                    tc_mma_tf32(dcol, pack64(a0 + jj * (4096u >> 4), HI), pack64(b0 + jj * ((2u * KC * 16u) >> 4), HI),
-                                IDESC_D, acc);
-                    acc = 1;
-                }
-            }
-            tc_commit(bar(BAR_X_EMPTY + s));
-            tc_commit(bar(BAR_D_FULL + b));
-            return true;
-        };
-
-        for (long long tile = first_tile; ok && tile < prm.total_tiles; tile += tile_step, ++tile_iter) {
-            if (!(ok = mbar_wait(bar(BAR_Z_READY), (uint32_t)(tile_iter & 1), abort_flag))) break;
-            tc_fence_after();
-            const long long t_tile0 = t;
-            for (int u = 0; ok && u < G && u < items_per_tile; ++u) ok = issue_distance(t_tile0 + u);
+        for (long long tile = first_tile; ok && tile < prm.total_tiles; tile += tile_step) {
             for (int p = 0; ok && p < P; ++p) {
                 const int nchunk = (p + 1) * CPP;
-                for (int c = 0; ok && c < nchunk; ++c, ++t) {
-                    const int b = (int)(t % G), s = (int)(t % ws);
-                    const long long j = t / G;
+                for (int c = 0; ok && c < nchunk; ++c) {
+                    const int b = k_s, s = w_s;
+                    TICK(7);
                     if (c == 0) {
-                        if (!(ok = mbar_wait(bar(BAR_V_EMPTY), (uint32_t)((pv & 1) ^ 1), abort_flag))) break;
+                        if (!(ok = mbar_wait(bar(BAR_V_EMPTY), v_ph ^ 1u, abort_flag))) break;
                     }
-                    if (!(ok = mbar_wait(bar(BAR_K_FULL + b), (uint32_t)(j & 1), abort_flag))) break;
-                    if (!(ok = mbar_wait(bar(BAR_W_FULL + s), (uint32_t)((t / ws) & 1), abort_flag))) break;
+                    TICK(3);
+                    if (!(ok = mbar_wait(bar(BAR_K_FULL + b), k_ph, abort_flag))) break;
+                    TICK(4);
+                    if (!(ok = mbar_wait(bar(BAR_W_FULL + s), w_ph, abort_flag))) break;
+                    if (++k_s == G) { k_s = 0; k_ph ^= 1u; }
+                    if (++w_s == ws) { w_s = 0; w_ph ^= 1u; }
+                    TICK(5);
                     tc_fence_after();
                     const uint32_t aH = k_lo0 + ((b * 16384u) >> 4), aL = aH + (8192u >> 4);
-                    const uint32_t bH = w_lo0 + ((s * map.w_stage) >> 4), bL = bH + (((uint32_t)KC * NV * 4u) >> 4);
+                    const uint32_t bH = w_lo0 + ((s * map.w_stage) >> 4), bL = bH + (((uint32_t)KC * NV * 2u) >> 4);
 #pragma unroll
                     for (int combo = 0; combo < 3; ++combo) {
                         const uint32_t a0 = combo == 2 ? aL : aH, b0 = combo == 1 ? bL : bH;
 #pragma unroll
-                        for (int jj = 0; jj < KC / 8; ++jj)
-                            tc_mma_tf32(tmem, pack64(a0 + jj * (4096u >> 4), HI),
-                                        pack64(b0 + jj * ((2u * NV * 16u) >> 4), HI), IDESC_V,
-                                        (c > 0 || combo > 0 || jj > 0) ? 1u : 0u);
+                        for (int jj = 0; jj < KC / 16; ++jj)
+                            tc_mma_f16(tmem, pack64(a0 + jj * (4096u >> 4), kDescHi),
+                                       pack64(b0 + jj * ((2u * NV * 16u) >> 4), kDescHi), IDESC_V,
+                                       (c > 0 || combo > 0 || jj > 0) ? 1u : 0u);
                     }
                     tc_commit(bar(BAR_W_EMPTY + s));
                     tc_commit(bar(BAR_K_EMPTY + b));
                     if (c == nchunk - 1) {
                         tc_commit(bar(BAR_V_FULL));
-                        ++pv;
+                        v_ph ^= 1u;
                     }
-                    const long long ahead = t + G;
-                    if (ahead - t_tile0 < items_per_tile) ok = issue_distance(ahead);
+                    TICK(6);
                 }
             }
         }
-        // every MMA issued so far must have completed before TMEM is freed
-        tc_commit(bar(BAR_MMA_DONE));
-        mbar_wait(bar(BAR_MMA_DONE), 0, abort_flag + 1);
+        tc_commit(bar(BAR_MMA_DONE + 1));
+        mbar_wait(bar(BAR_MMA_DONE + 1), 0, abort_flag + 1);
+        if (prm.trace)
+            for (int i = 0; i < 8; ++i) prm.trace[((size_t)blockIdx.x * 4 + 0) * 8 + i] = tacc[i];
     } else if (warp >= 4) {
         // ------------------------------------------------------------ Matern / epilogue warp groups
         const int grp = (warp - 4) >> 2;         // 0..G-1
         const int q4 = warp & 3;                 // TMEM lane quarter == warp % 4
         const int row = q4 * 32 + lane;          // candidate row in the tile == TMEM lane
         const uint32_t lane_addr = tmem + ((uint32_t)(q4 * 32) << 16);
-        long long t = grp;                       // next own item (global numbering)
-        long long t_tile0 = 0;                   // first item of the current tile
-        long long pv = 0, tile_iter = 0;
+        long long t = grp;                       // next own chunk (global numbering)
+        long long t_tile0 = 0;                   // first chunk of the current tile
+        uint32_t own_ph = 0;                     // parity of this group's own-chunk count
+        uint32_t v_ph = 0;                       // parity of the pass counter
+        long long tile_iter = 0;
         bool ok = true;
         bool bad = false;
         // scratch for the end-of-tile reduction lives in k* buffer 0 (dead once the last pass is done)
@@ -404,122 +557,188 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
             const long long cand = (tile % prm.tiles_per_gp) * TILE_M + row;
             const bool valid = cand < prm.m;
             const float sf2 = prm.sf2[g];
+            const float kscale = prm.kscale[g];
             if (grp == G - 1) {
                 // ---- scale the candidate, split it, store it as the A operand of the distance MMA
                 float zn = 0.f;
+                bool far = false;
                 const float* zrow = prm.xcand + ((size_t)g * prm.m + (valid ? cand : 0)) * prm.d;
                 const float* cen = prm.centre + (size_t)g * DP;
                 const float* scl = prm.scale + (size_t)g * DP;
                 const bool vec = (prm.d % 4) == 0;
-                for (int j4 = 0; j4 < DP / 4; ++j4) {
-                    float z[4];
-                    if (vec && 4 * j4 < prm.d) {
-                        const float4 v = *reinterpret_cast<const float4*>(zrow + 4 * j4);
-                        z[0] = v.x; z[1] = v.y; z[2] = v.z; z[3] = v.w;
+                uint32_t zh[8], zl[8];
+                for (int j8 = 0; j8 < DP / 8; ++j8) {
+                    __half2 hi2[4], lo2[4];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int j4 = 2 * j8 + h;
+                        float z[4];
+                        if (vec && 4 * j4 < prm.d) {
+                            const float4 v = *reinterpret_cast<const float4*>(zrow + 4 * j4);
+                            z[0] = v.x; z[1] = v.y; z[2] = v.z; z[3] = v.w;
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) z[e] = (4 * j4 + e < prm.d) ? zrow[4 * j4 + e] : 0.f;
+                        }
+                        const float4 c4 = __ldg(reinterpret_cast<const float4*>(cen + 4 * j4));
+                        const float4 s4 = __ldg(reinterpret_cast<const float4*>(scl + 4 * j4));
+                        const float cc[4] = {c4.x, c4.y, c4.z, c4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
+                        float zt[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            bad |= !isfinite(z[e]);
+                            float v = valid ? (z[e] - cc[e]) * ss[e] : 0.f;
+                            if (fabsf(v) > kMaxScaled) {   // outside the FP16 planes' range: clamp, and have it recomputed
+                                v = copysignf(kMaxScaled, v);
+                                far = true;
+                            }
+                            zt[e] = v;
+                            zn = fmaf(v, v, zn);
+                        }
+                        split2(zt[0], zt[1], hi2[2 * h], lo2[2 * h]);
+                        split2(zt[2], zt[3], hi2[2 * h + 1], lo2[2 * h + 1]);
+                    }
+                    // 8 features = 4 columns of each plane; two such groups make one 8-column store
+                    if (j8 & 1) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            zh[4 + e] = *reinterpret_cast<const uint32_t*>(&hi2[e]);
+                            zl[4 + e] = *reinterpret_cast<const uint32_t*>(&lo2[e]);
+                        }
+                        tc_st8(lane_addr + ZCOL + (uint32_t)(j8 >> 1) * 8u, zh);
+                        tc_st8(lane_addr + ZCOL + (uint32_t)DP / 2 + (uint32_t)(j8 >> 1) * 8u, zl);
                     } else {
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) z[e] = (4 * j4 + e < prm.d) ? zrow[4 * j4 + e] : 0.f;
+                        for (int e = 0; e < 4; ++e) {
+                            zh[e] = *reinterpret_cast<const uint32_t*>(&hi2[e]);
+                            zl[e] = *reinterpret_cast<const uint32_t*>(&lo2[e]);
+                        }
                     }
-                    const float4 c4 = __ldg(reinterpret_cast<const float4*>(cen + 4 * j4));
-                    const float4 s4 = __ldg(reinterpret_cast<const float4*>(scl + 4 * j4));
-                    const float cc[4] = {c4.x, c4.y, c4.z, c4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
-                    float hi[4], lo[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        bad |= !isfinite(z[e]);
-                        const float zt = valid ? (z[e] - cc[e]) * ss[e] : 0.f;
-                        zn = fmaf(zt, zt, zn);
-                        hi[e] = tf32_hi(zt);
-                        lo[e] = zt - hi[e];
-                    }
-                    *reinterpret_cast<float4*>(sm + map.z + (uint32_t)j4 * 2048u + row * 16) =
-                        make_float4(hi[0], hi[1], hi[2], hi[3]);
-                    *reinterpret_cast<float4*>(sm + map.z + (uint32_t)DP * 512u + (uint32_t)j4 * 2048u + row * 16) =
-                        make_float4(lo[0], lo[1], lo[2], lo[3]);
                 }
-                zn_s[row] = zn;
-                fence_proxy_async();
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                zn_s[row] = far ? -zn : zn;   // the sign carries the out-of-range mark
+                tc_fence_before();
                 mbar_arrive(bar(BAR_Z_READY));
             }
             ok = mbar_wait(bar(BAR_Z_READY), (uint32_t)(tile_iter & 1), abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            const float zn = zn_s[row];
+            const bool far_cand = zn_s[row] < 0.f;
+            const float zn = fabsf(zn_s[row]);
 
+            const float* xs_g = prm.xs32 + (size_t)g * prm.NP * DP;
+            const float refine_at = far_cand ? INFINITY : kRefine * sf2;
             const float* xn_g = prm.xnorm + (size_t)g * prm.NP;
             const float* al_g = prm.alpha + (size_t)g * prm.NP;
             double mu_acc = 0.0, a2_acc = 0.0, s2_acc = 0.0, q_acc = 0.0;
-            int pass_base = 0;   // items of this tile before pass p
+            int pass_base = 0;   // chunks of this tile before pass p
             for (int p = 0; ok && p < P; ++p) {
                 const int nchunk = (p + 1) * CPP;
-                // own items of this pass: global t with t - t_tile0 - pass_base in [0, nchunk)
+                // own chunks of this pass: global t with t - t_tile0 - pass_base in [0, nchunk)
                 while (t - t_tile0 - pass_base < nchunk) {
                     const int c = (int)(t - t_tile0 - pass_base);
-                    const long long j = t / G;
+                    const long long U = t / SL;       // distance product and the slice of its buffer
+                    const int db = (int)(U & 1), slice = (int)(t % SL);
                     // the next own chunk's norms and weights: pull them towards L1 while this one is worked on
                     if (lane < 2) {
                         const int cn = c + G < nchunk ? c + G : (c + G - nchunk);
                         const float* pf = (lane == 0 ? xn_g : al_g) + cn * KC;
                         asm volatile("prefetch.global.L1 [%0];" ::"l"(pf));
                     }
-                    ok = mbar_wait(bar(BAR_D_FULL + grp), (uint32_t)(j & 1), abort_flag);
+                    TICK(7);
+                    ok = mbar_wait(bar(BAR_D_FULL + db), (uint32_t)((U >> 1) & 1), abort_flag);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
+                    TICK(0);
                     tc_fence_after();
-                    float dot[KC];
-                    tc_ld16(lane_addr + NV + grp * KC, dot);
-                    tc_fence_before();
-                    mbar_arrive(bar(BAR_D_EMPTY + grp));
                     const bool fresh = c >= p * CPP;   // first time this chunk is generated for the tile
-                    float kv[KC];
-                    float mpart = 0.f, apart = 0.f, spart = 0.f;
-#pragma unroll
-                    for (int q = 0; q < KC / 4; ++q) {
-                        const float4 xn4 = __ldg(reinterpret_cast<const float4*>(xn_g + c * KC + 4 * q));
-                        const float4 al4 = __ldg(reinterpret_cast<const float4*>(al_g + c * KC + 4 * q));
-                        const float xn[4] = {xn4.x, xn4.y, xn4.z, xn4.w}, al[4] = {al4.x, al4.y, al4.z, al4.w};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float r2 = fmaxf(fmaf(-2.f, dot[4 * q + e], zn + xn[e]), 0.f);
-                            const float s = sqrt_approx(5.f * r2);
-                            const float v = sf2 * fmaf(s, fmaf(s, 1.f / 3.f, 1.f), 1.f) * __expf(-s);
-                            kv[4 * q + e] = v;
-                            const float va = v * al[e];
-                            mpart += va;
-                            apart = fmaf(va, va, apart);
-                            spart = fmaf(v, v, spart);
-                        }
-                    }
-                    if (fresh) {
-                        mu_acc += (double)mpart;
-                        a2_acc += (double)apart;
-                        s2_acc += (double)spart;
-                    }
-                    ok = mbar_wait(bar(BAR_K_EMPTY + grp), (uint32_t)((j & 1) ^ 1), abort_flag);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
                     uint8_t* kb = sm + map.k + grp * 16384u + row * 16;
 #pragma unroll
-                    for (int q = 0; q < KC / 4; ++q) {
-                        float hi[4], lo[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            hi[e] = tf32_hi(kv[4 * q + e]);
-                            lo[e] = kv[4 * q + e] - hi[e];
+                    for (int h = 0; h < KC / 16; ++h) {
+                        float dot[16];
+                        tc_ld16(lane_addr + NV + db * KD + slice * KC + h * 16, dot);
+                        if (h == KC / 16 - 1) {
+                            tc_fence_before();
+                            mbar_arrive(bar(BAR_D_EMPTY + db));
                         }
-                        *reinterpret_cast<float4*>(kb + q * 2048u) = make_float4(hi[0], hi[1], hi[2], hi[3]);
-                        *reinterpret_cast<float4*>(kb + 8192u + q * 2048u) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+                        TICK(1);
+                        float kv[16];
+                        uint32_t close = 0;   // bit i: pair i needs its distance by direct differences
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const float4 xn4 = __ldg(reinterpret_cast<const float4*>(xn_g + c * KC + h * 16 + 4 * q));
+                            const float xn[4] = {xn4.x, xn4.y, xn4.z, xn4.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float r2 = fmaxf(fmaf(-2.f, dot[4 * q + e], zn + xn[e]), 0.f);
+                                const float s = sqrt_approx(5.f * r2);
+                                const float v = sf2 * fmaf(s, fmaf(s, 1.f / 3.f, 1.f), 1.f) * __expf(-s);
+                                kv[4 * q + e] = v;
+                                if (v * (zn + xn[e]) > refine_at) close |= 1u << (4 * q + e);
+                            }
+                        }
+                        if (__any_sync(0xffffffffu, close != 0)) {
+                            // rare: hand the 16 values to the out-of-line refinement through a local array so
+                            // that the hot path keeps kv in registers
+                            float tmp[16];
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) tmp[i] = kv[i];
+                            refine_close_pairs(tmp, close, lane_addr + ZCOL, DP, xs_g + (size_t)(c * KC + h * 16) * DP, sf2);
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) kv[i] = tmp[i];
+                        }
+                        if (fresh) {   // warp-uniform: the mean and the error scales see every observation once
+                            float mpart = 0.f, apart = 0.f, spart = 0.f;
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const float4 al4 = __ldg(reinterpret_cast<const float4*>(al_g + c * KC + h * 16 + 4 * q));
+                                const float al[4] = {al4.x, al4.y, al4.z, al4.w};
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const float v = kv[4 * q + e], va = v * al[e];
+                                    mpart += va;
+                                    apart = fmaf(va, va, apart);
+                                    spart = fmaf(v, v, spart);
+                                }
+                            }
+                            mu_acc += (double)mpart;
+                            a2_acc += (double)apart;
+                            s2_acc += (double)spart;
+                        }
+                        TICK(2);
+                        if (h == 0) {
+                            ok = mbar_wait(bar(BAR_K_EMPTY + grp), own_ph ^ 1u, abort_flag);
+                            ok = __all_sync(0xffffffffu, ok);
+                            if (!ok) break;
+                            TICK(3);
+                        }
+                        // 16 columns = two 16-byte k-slices of the A operand, hi and lo planes
+#pragma unroll
+                        for (int sl = 0; sl < 2; ++sl) {
+                            __half2 hi2[4], lo2[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                split2(kv[8 * sl + 2 * e] * kscale, kv[8 * sl + 2 * e + 1] * kscale, hi2[e], lo2[e]);
+                            *reinterpret_cast<uint4*>(kb + (2 * h + sl) * 2048u) = *reinterpret_cast<const uint4*>(hi2);
+                            *reinterpret_cast<uint4*>(kb + 8192u + (2 * h + sl) * 2048u) =
+                                *reinterpret_cast<const uint4*>(lo2);
+                        }
                     }
+                    if (!ok) break;
                     fence_proxy_async();
                     mbar_arrive(bar(BAR_K_FULL + grp));
+                    TICK(4);
                     t += G;
+                    own_ph ^= 1u;
                 }
                 if (!ok) break;
                 pass_base += nchunk;
                 // ---- end of pass: q += sum_i V^2 over this group's share of the columns
-                ok = mbar_wait(bar(BAR_V_FULL), (uint32_t)(pv & 1), abort_flag);
+                TICK(7);
+                ok = mbar_wait(bar(BAR_V_FULL), v_ph, abort_flag);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
+                TICK(5);
                 tc_fence_after();
 #pragma unroll 1
                 for (int c0 = grp * 16; c0 < NV; c0 += 16 * G) {
@@ -532,41 +751,42 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                 }
                 tc_fence_before();
                 mbar_arrive(bar(BAR_V_EMPTY));
-                ++pv;
+                TICK(6);
+                v_ph ^= 1u;
             }
             if (!ok) break;
             t_tile0 += items_per_tile;
             // ---- combine the groups' partial sums; group 0 finishes the candidate
-            if (G > 1) {
-                double* mine = red + ((size_t)grp * TILE_M + row) * 4;
-                mine[0] = mu_acc; mine[1] = a2_acc; mine[2] = s2_acc; mine[3] = q_acc;
-                mbar_arrive(bar(BAR_RED_READY));
-                if (grp == 0) {   // only the finishing group waits; the others move on to the next tile
-                    ok = mbar_wait(bar(BAR_RED_READY), (uint32_t)(tile_iter & 1), abort_flag);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                }
-            }
-            if (grp == 0 && valid) {
-                if (G > 1) {
+            double* mine = red + ((size_t)grp * TILE_M + row) * 4;
+            mine[0] = mu_acc; mine[1] = a2_acc; mine[2] = s2_acc; mine[3] = q_acc;
+            mbar_arrive(bar(BAR_RED_READY));
+            if (grp == 0) {   // only the finishing group waits; the others move on to the next tile
+                ok = mbar_wait(bar(BAR_RED_READY), (uint32_t)(tile_iter & 1), abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                if (valid) {
                     mu_acc = a2_acc = s2_acc = q_acc = 0.0;
 #pragma unroll
                     for (int gg = 0; gg < G; ++gg) {
                         const double* o = red + ((size_t)gg * TILE_M + row) * 4;
                         mu_acc += o[0]; a2_acc += o[1]; s2_acc += o[2]; q_acc += o[3];
                     }
+                    q_acc *= prm.vinv2[g];   // undo the power-of-two scaling of k* and W
+                    const size_t f = (size_t)g * prm.m + cand;
+                    const CandidateResult res = finalize_candidate(mu_acc, q_acc, (double)sf2, (double)prm.best[g]);
+                    prm.mu[f] = res.mu;
+                    prm.sigma[f] = res.sigma;
+                    prm.ei[f] = res.ei;
+                    const double eps =
+                        far_cand ? 1.0 : kEpsTc0 + kEpsTc1 * (double)(zn + prm.xnmax[g]) * rsqrt((double)DP);
+                    prm.err_mu[f] = mu_error_estimate(eps, a2_acc);
+                    prm.err_q[f] = q_error_estimate(eps, prm.wnorm[g], q_acc, s2_acc);
                 }
-                const size_t f = (size_t)g * prm.m + cand;
-                const CandidateResult res = finalize_candidate(mu_acc, q_acc, (double)sf2, (double)prm.best[g]);
-                prm.mu[f] = res.mu;
-                prm.sigma[f] = res.sigma;
-                prm.ei[f] = res.ei;
-                const double eps = kEpsTc0 + kEpsTc1 * (double)(zn + prm.xnmax[g]) * rsqrt((double)DP);
-                prm.err_mu[f] = mu_error_estimate(eps, a2_acc);
-                prm.err_q[f] = q_error_estimate(eps, prm.wnorm[g], q_acc, s2_acc);
             }
         }
         if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(prm.status, DEV_NONFINITE);
+        if (prm.trace && q4 == 0 && lane == 0 && grp < 2)
+            for (int i = 0; i < 8; ++i) prm.trace[((size_t)blockIdx.x * 4 + 1 + grp) * 8 + i] = tacc[i];
     }
 
     // ---------------------------------------------------------------- teardown
@@ -602,30 +822,35 @@ __global__ void centre_kernel(const float* __restrict__ X, const float* __restri
     }
 }
 
-// One block per (chunk, GP): scaled observations as hi/lo planes in the MMA's B-operand layout,
-// their squared norms, and the padded weights.
+// One block per (distance product, GP): scaled observations as FP16 hi/lo planes in the MMA's
+// B-operand layout, their squared norms (of the FP32 values the planes represent), the padded weights,
+// and the largest scaled coordinate (the FP16 planes have a limited range).
 __global__ void xt_build_kernel(const float* __restrict__ X, const float* __restrict__ centre,
                                 const float* __restrict__ scale, const float* __restrict__ alpha32, int n, int d,
-                                int npad_fit, int DP, int NP, float* __restrict__ xt, float* __restrict__ xnorm,
-                                float* __restrict__ alpha)
+                                int npad_fit, int DP, int NP, int KD, __half* __restrict__ xt,
+                                float* __restrict__ xs32, float* __restrict__ xnorm, float* __restrict__ alpha, unsigned* __restrict__ xamax_bits)
 {
     const int g = blockIdx.y, c = blockIdx.x;
-    float* blob = xt + ((size_t)g * (NP / KC) + c) * (2 * DP * KC);
+    __half* blob = xt + ((size_t)g * (NP / KD) + c) * (2 * DP * KD);
     const float* cen = centre + (size_t)g * DP;
     const float* scl = scale + (size_t)g * DP;
-    for (int e = threadIdx.x; e < DP * KC; e += blockDim.x) {
-        const int r = e % KC, j = e / KC;
-        const int k = c * KC + r;
+    float amax = 0.f;
+    for (int e = threadIdx.x; e < DP * KD; e += blockDim.x) {
+        const int r = e % KD, j = e / KD;
+        const int k = c * KD + r;
         float xv = 0.f;
         if (k < n && j < d) xv = (float)(((double)X[((size_t)g * n + k) * d + j] - (double)cen[j]) * (double)scl[j]);
-        // round to nearest on the 13 dropped mantissa bits, as cvt.rna.tf32 does
-        const float h = __uint_as_float((__float_as_uint(xv) + 0x1000u) & 0xFFFFE000u);
-        const size_t off = ((size_t)(j / 4) * KC + r) * 4 + (j % 4);
+        amax = fmaxf(amax, fabsf(xv));
+        xs32[((size_t)g * NP + k) * DP + j] = xv;
+        const __half h = __float2half_rn(xv);
+        const size_t off = ((size_t)(j / 8) * KD + r) * 8 + (j % 8);
         blob[off] = h;
-        blob[(size_t)DP * KC + off] = xv - h;
+        blob[(size_t)DP * KD + off] = __float2half_rn(xv - __half2float(h));
     }
-    for (int r = threadIdx.x; r < KC; r += blockDim.x) {
-        const int k = c * KC + r;
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if ((threadIdx.x & 31) == 0) atomicMax(xamax_bits, __float_as_uint(amax));
+    for (int r = threadIdx.x; r < KD; r += blockDim.x) {
+        const int k = c * KD + r;
         double nrm = 0.0;
         if (k < n)
             for (int j = 0; j < d; ++j) {
@@ -651,31 +876,61 @@ __global__ void xnmax_kernel(const float* __restrict__ xnorm, int NP, float* __r
     if (threadIdx.x == 0) xnmax[blockIdx.x] = s[0];
 }
 
-// One block per (chunk c, pass p, GP): the KC x NV block of W (rows p NV.., columns c KC..) as hi/lo
-// planes in the B-operand layout; zero outside the lower triangle and outside n.
+// Largest |W| entry of each GP (bit pattern of a non-negative float, so atomicMax orders it).
+__global__ void wmax_kernel(const double* __restrict__ W64, int n, int npad_fit, unsigned* __restrict__ wmax_bits)
+{
+    const int g = blockIdx.y;
+    const double* Wg = W64 + (size_t)g * npad_fit * npad_fit;
+    float v = 0.f;
+    for (size_t e = blockIdx.x * (size_t)blockDim.x + threadIdx.x; e < (size_t)n * n; e += (size_t)gridDim.x * blockDim.x) {
+        const int i = (int)(e / n), k = (int)(e % n);
+        if (k <= i) v = fmaxf(v, fabsf((float)Wg[(size_t)i * npad_fit + k]));
+    }
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    if ((threadIdx.x & 31) == 0) atomicMax(&wmax_bits[g], __float_as_uint(v));
+}
+
+// One block per (chunk c, pass p, GP): the KC x NV block of 2^eW W (rows p NV.., columns c KC..) as
+// FP16 hi/lo planes in the B-operand layout; zero outside the lower triangle and outside n.
 __global__ void wt_build_kernel(const double* __restrict__ W64, int n, int npad_fit, int NV, size_t gp_stride,
-                                float* __restrict__ wt)
+                                const float* __restrict__ wscale, __half* __restrict__ wt)
 {
     const int c = blockIdx.x, p = blockIdx.y, g = blockIdx.z;
     const int CPP = NV / KC;
     if (c >= (p + 1) * CPP) return;
     const size_t tile = (size_t)CPP * p * (p + 1) / 2 + c;
-    float* dst = wt + (size_t)g * gp_stride + tile * (2 * KC * NV);
+    __half* dst = wt + (size_t)g * gp_stride + tile * (2 * KC * NV);
     const double* Wg = W64 + (size_t)g * npad_fit * npad_fit;
+    const double sc = (double)wscale[g];
     for (int e = threadIdx.x; e < KC * NV; e += blockDim.x) {
         const int kk = e % KC, r = e / KC;   // consecutive threads walk k: coalesced reads of a W row
         const int i = p * NV + r, k = c * KC + kk;
         float w = 0.f;
-        if (i < n && k <= i) w = (float)Wg[(size_t)i * npad_fit + k];
-        const uint32_t u = __float_as_uint(w);
-        const float h = __uint_as_float((u + 0x1000u) & 0xFFFFE000u);
-        const size_t off = ((size_t)(kk / 4) * NV + r) * 4 + (kk % 4);
+        if (i < n && k <= i) w = (float)(Wg[(size_t)i * npad_fit + k] * sc);
+        const __half h = __float2half_rn(w);
+        const size_t off = ((size_t)(kk / 8) * NV + r) * 8 + (kk % 8);
         dst[off] = h;
-        dst[(size_t)KC * NV + off] = w - h;
+        dst[(size_t)KC * NV + off] = __float2half_rn(w - __half2float(h));
     }
 }
 
 TensorOperands* ops_of(const r3_gp* gp) { return static_cast<TensorOperands*>(gp->tc); }
+
+void (*kernel_for(int NV, int G, int KD))(const TcParams)
+{
+    if (KD == 128) {
+        if (NV == 256) return G == 3 ? score_tc_kernel<256, 3, 128> : score_tc_kernel<256, 2, 128>;
+        return G == 3 ? score_tc_kernel<128, 3, 128> : score_tc_kernel<128, 2, 128>;
+    }
+    if (NV == 256) return G == 3 ? score_tc_kernel<256, 3, 64> : score_tc_kernel<256, 2, 64>;
+    return G == 3 ? score_tc_kernel<128, 3, 64> : score_tc_kernel<128, 2, 64>;
+}
+
+int env_int(const char* name, int fallback)
+{
+    const char* v = getenv(name);
+    return v ? atoi(v) : fallback;
+}
 
 }  // namespace
 
@@ -688,10 +943,13 @@ void tc_release(r3_gp* gp)
     cudaFree(t->centre);
     cudaFree(t->scale);
     cudaFree(t->xt);
+    cudaFree(t->xs32);
     cudaFree(t->xnorm);
     cudaFree(t->xnmax);
     cudaFree(t->alpha);
     cudaFree(t->wt);
+    cudaFree(t->kscale);
+    cudaFree(t->vinv2);
     delete t;
     gp->tc = nullptr;
 }
@@ -705,53 +963,112 @@ r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream)
         return R3_ERR_ALLOC;
     }
     gp->tc = t;
-    t->DP = round_up(d, 8);
-    t->NV = (t->DP <= 64 && n > 128) ? 256 : 128;
+    t->DP = round_up(d, 16);
+    t->NV = n > 128 ? 256 : 128;
     t->NP = round_up(n, t->NV);
     t->P = t->NP / t->NV;
-    t->xs = 2;
-    t->G = t->NV == 256 ? 3 : 2;
+    // shared-memory budget decides the shape: prefer three Matern groups, then wide distance products,
+    // then as many W stages as fit (at least three)
     const size_t budget = 227 * 1024 - 1024 - kBarBytes;
-    for (t->ws = MAX_STAGES; t->ws >= 2; --t->ws) {
-        const SmemMap mp = smem_map(t->DP, t->NV, t->G, t->xs, t->ws);
-        if (mp.bar <= budget) break;
-    }
-    if (t->ws < 2) {
+    const int want_kd = env_int("R3_TC_KD", 0), want_g = env_int("R3_TC_G", 0);
+    bool found = false;
+    for (int min_ws = 3; min_ws >= 2 && !found; --min_ws)
+        for (int pref = 0; pref < 4 && !found; ++pref) {
+            t->G = pref < 2 ? 3 : 2;
+            t->KD = (pref % 2 == 0) ? 64 : 128;
+            if (want_kd && t->KD != want_kd) continue;
+            if (want_g && t->G != want_g) continue;
+            if (t->NV % t->KD) continue;
+            for (t->ws = MAX_STAGES; t->ws >= 2; --t->ws)
+                if (smem_map(t->DP, t->NV, t->G, t->KD, t->ws).bar <= budget) break;
+            found = t->ws >= min_ws;
+        }
+    if (!found) {
         tc_release(gp);   // does not fit: the SIMT engine serves this shape
         return R3_OK;
     }
-    t->smem_bytes = smem_map(t->DP, t->NV, t->G, t->xs, t->ws).bar + kBarBytes + 1024;
-    t->tmem_cols = (t->NV + t->G * KC) <= 256 ? 256 : 512;
+    t->smem_bytes = smem_map(t->DP, t->NV, t->G, t->KD, t->ws).bar + kBarBytes + 1024;
     const int CPP = t->NV / KC;
     const size_t tiles = (size_t)CPP * t->P * (t->P + 1) / 2;
     t->wt_gp_stride = tiles * (2 * (size_t)KC * t->NV);
+    unsigned* wmax_bits = nullptr;
+    float* wscale_d = nullptr;
     auto fail = [&](const char* what, cudaError_t e) {
         set_error("%s failed: %s", what, cudaGetErrorString(e));
+        cudaFree(wmax_bits);
+        cudaFree(wscale_d);
         tc_release(gp);
         return e == cudaErrorMemoryAllocation ? R3_ERR_ALLOC : R3_ERR_CUDA;
+    };
+    auto decline = [&]() {   // the SIMT engine serves this history
+        cudaFree(wmax_bits);
+        cudaFree(wscale_d);
+        tc_release(gp);
+        return R3_OK;
     };
     cudaError_t e;
     if ((e = cudaMalloc(&t->centre, sizeof(float) * B * t->DP)) != cudaSuccess) return fail("cudaMalloc", e);
     if ((e = cudaMalloc(&t->scale, sizeof(float) * B * t->DP)) != cudaSuccess) return fail("cudaMalloc", e);
-    if ((e = cudaMalloc(&t->xt, sizeof(float) * B * (size_t)(t->NP / KC) * 2 * t->DP * KC)) != cudaSuccess)
+    if ((e = cudaMalloc(&t->xt, sizeof(__half) * B * (size_t)(t->NP / t->KD) * 2 * t->DP * t->KD)) != cudaSuccess)
         return fail("cudaMalloc", e);
+    if ((e = cudaMalloc(&t->xs32, sizeof(float) * B * (size_t)t->NP * t->DP)) != cudaSuccess) return fail("cudaMalloc", e);
     if ((e = cudaMalloc(&t->xnorm, sizeof(float) * B * t->NP)) != cudaSuccess) return fail("cudaMalloc", e);
-    if ((e = cudaMalloc(&t->xnmax, sizeof(float) * B)) != cudaSuccess) return fail("cudaMalloc", e);
+    if ((e = cudaMalloc(&t->xnmax, sizeof(float) * (B > 2 ? B : 2))) != cudaSuccess) return fail("cudaMalloc", e);
     if ((e = cudaMalloc(&t->alpha, sizeof(float) * B * t->NP)) != cudaSuccess) return fail("cudaMalloc", e);
-    if ((e = cudaMalloc(&t->wt, sizeof(float) * B * t->wt_gp_stride)) != cudaSuccess) return fail("cudaMalloc", e);
+    if ((e = cudaMalloc(&t->wt, sizeof(__half) * B * t->wt_gp_stride)) != cudaSuccess) return fail("cudaMalloc", e);
+    if ((e = cudaMalloc(&t->kscale, sizeof(float) * B)) != cudaSuccess) return fail("cudaMalloc", e);
+    if ((e = cudaMalloc(&t->vinv2, sizeof(double) * B)) != cudaSuccess) return fail("cudaMalloc", e);
+    if ((e = cudaMalloc(&wmax_bits, sizeof(unsigned) * B)) != cudaSuccess) return fail("cudaMalloc", e);
+    if ((e = cudaMalloc(&wscale_d, sizeof(float) * B)) != cudaSuccess) return fail("cudaMalloc", e);
 
+    // scaled observations (their largest coordinate decides whether the FP16 planes can hold them) and
+    // the largest |W| of each GP (it decides the power-of-two scale of its W planes)
+    unsigned* xamax_bits = reinterpret_cast<unsigned*>(t->xnmax);   // borrowed until xnmax_kernel overwrites it
+    if ((e = cudaMemsetAsync(xamax_bits, 0, sizeof(unsigned), stream)) != cudaSuccess) return fail("cudaMemsetAsync", e);
+    if ((e = cudaMemsetAsync(wmax_bits, 0, sizeof(unsigned) * B, stream)) != cudaSuccess) return fail("cudaMemsetAsync", e);
     centre_kernel<<<dim3(t->DP, B), 256, 0, stream>>>(gp->X, gp->inv_ell, n, d, t->DP, t->centre, t->scale);
-    xt_build_kernel<<<dim3(t->NP / KC, B), 256, 0, stream>>>(gp->X, t->centre, t->scale, gp->alpha32, n, d, gp->npad,
-                                                             t->DP, t->NP, t->xt, t->xnorm, t->alpha);
+    xt_build_kernel<<<dim3(t->NP / t->KD, B), 256, 0, stream>>>(gp->X, t->centre, t->scale, gp->alpha32, n, d, gp->npad,
+                                                                t->DP, t->NP, t->KD, t->xt, t->xs32, t->xnorm, t->alpha, xamax_bits);
+    wmax_kernel<<<dim3(296, B), 256, 0, stream>>>(gp->W64, n, gp->npad, wmax_bits);
+    g_launches += 3;
+    float xamax = 0.f;
+    std::vector<float> wmax(B);
+    if ((e = cudaMemcpyAsync(&xamax, xamax_bits, sizeof(float), cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
+        return fail("cudaMemcpyAsync", e);
+    if ((e = cudaMemcpyAsync(wmax.data(), wmax_bits, sizeof(float) * B, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
+        return fail("cudaMemcpyAsync", e);
+    if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return fail("operand preparation", e);
+    if (!(xamax <= kMaxScaled)) return decline();   // scaled coordinates beyond the FP16 planes
+    std::vector<float> wscale(B), kscale(B);
+    std::vector<double> vinv2(B);
+    for (int g = 0; g < B; ++g) {
+        int ew = 0, ek = 0;
+        frexp((double)wmax[g], &ew);               // wmax < 2^ew
+        frexp((double)gp->sf2[g], &ek);            // sf2  < 2^ek  (k* <= sf2)
+        const int sw = kScaleExp - ew, sk = kScaleExp - ek;
+        if (!(wmax[g] > 0.f) || sw < -60 || sw > 60 || sk < -60 || sk > 60) return decline();   // degenerate scales
+        wscale[g] = (float)ldexp(1.0, sw);
+        kscale[g] = (float)ldexp(1.0, sk);
+        vinv2[g] = ldexp(1.0, -2 * (sw + sk));
+    }
+    if ((e = cudaMemcpyAsync(wscale_d, wscale.data(), sizeof(float) * B, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+        return fail("cudaMemcpyAsync", e);
+    if ((e = cudaMemcpyAsync(t->kscale, kscale.data(), sizeof(float) * B, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+        return fail("cudaMemcpyAsync", e);
+    if ((e = cudaMemcpyAsync(t->vinv2, vinv2.data(), sizeof(double) * B, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+        return fail("cudaMemcpyAsync", e);
     xnmax_kernel<<<B, 256, 0, stream>>>(t->xnorm, t->NP, t->xnmax);
-    wt_build_kernel<<<dim3(t->P * CPP, t->P, B), 256, 0, stream>>>(gp->W64, n, gp->npad, t->NV, t->wt_gp_stride, t->wt);
-    g_launches += 4;
+    wt_build_kernel<<<dim3(t->P * CPP, t->P, B), 256, 0, stream>>>(gp->W64, n, gp->npad, t->NV, t->wt_gp_stride,
+                                                                   wscale_d, t->wt);
+    g_launches += 2;
     if ((e = cudaGetLastError()) != cudaSuccess) return fail("operand preparation launch", e);
     if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return fail("operand preparation", e);
-    if (t->NV == 256)
-        e = cudaFuncSetAttribute(score_tc_kernel<256, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t->smem_bytes);
-    else
-        e = cudaFuncSetAttribute(score_tc_kernel<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t->smem_bytes);
+    cudaFree(wmax_bits);
+    cudaFree(wscale_d);
+    wmax_bits = nullptr;
+    wscale_d = nullptr;
+    e = cudaFuncSetAttribute(kernel_for(t->NV, t->G, t->KD), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)t->smem_bytes);
     if (e != cudaSuccess) return fail("cudaFuncSetAttribute", e);
     return R3_OK;
 }
@@ -784,10 +1101,13 @@ r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, floa
     prm.centre = t->centre;
     prm.scale = t->scale;
     prm.xt = t->xt;
+    prm.xs32 = t->xs32;
     prm.xnorm = t->xnorm;
     prm.xnmax = t->xnmax;
     prm.alpha = t->alpha;
     prm.wt = t->wt;
+    prm.kscale = t->kscale;
+    prm.vinv2 = t->vinv2;
     prm.wt_gp_stride = t->wt_gp_stride;
     prm.sf2 = gp->sf2_d;
     prm.best = gp->best_d;
@@ -795,7 +1115,6 @@ r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, floa
     prm.DP = t->DP;
     prm.NP = t->NP;
     prm.P = t->P;
-    prm.xs = t->xs;
     prm.ws = t->ws;
     prm.status = gp->status_d;
     prm.tiles_per_gp = (m + TILE_M - 1) / TILE_M;
@@ -803,12 +1122,29 @@ r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, floa
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, gp->device);
     const unsigned grid = (unsigned)(prm.total_tiles < sms ? prm.total_tiles : sms);
+    // R3_TC_TRACE=1 prints, for the first CTA, the cycles each role spent per wait / issue category
+    prm.trace = nullptr;
+    if (getenv("R3_TC_TRACE")) {
+        if (cudaMalloc(&prm.trace, sizeof(long long) * grid * 32) != cudaSuccess) prm.trace = nullptr;
+        if (prm.trace) cudaMemset(prm.trace, 0, sizeof(long long) * grid * 32);
+    }
+    void (*kernel)(const TcParams) = kernel_for(t->NV, t->G, t->KD);
     prof_begin(gp, stream);
-    if (t->NV == 256)
-        R3_LAUNCH((score_tc_kernel<256, 3>), grid, 128 + 128 * 3, t->smem_bytes, stream, prm);
-    else
-        R3_LAUNCH((score_tc_kernel<128, 2>), grid, 128 + 128 * 2, t->smem_bytes, stream, prm);
+    R3_LAUNCH(kernel, grid, 128 + 128 * t->G, t->smem_bytes, stream, prm);
     prof_end(gp, stream);
+    if (prm.trace) {
+        std::vector<long long> h((size_t)grid * 32);
+        cudaMemcpy(h.data(), prm.trace, sizeof(long long) * grid * 32, cudaMemcpyDeviceToHost);
+        cudaFree(prm.trace);
+        const char* names[4] = {"mmaV", "matern0", "matern1", "mmaD"};
+        fprintf(stderr, "trace shape NV=%d G=%d KD=%d ws=%d DP=%d P=%d smem=%zu\n", t->NV, t->G, t->KD, t->ws, t->DP, t->P,
+                t->smem_bytes);
+        for (int r = 0; r < 4; ++r) {
+            fprintf(stderr, "trace cta0 %s:", names[r]);
+            for (int i = 0; i < 8; ++i) fprintf(stderr, " %lld", h[(size_t)r * 8 + i]);
+            fprintf(stderr, "\n");
+        }
+    }
     return guard_and_rescue(gp, Xcand, m, gb, mu, sigma, ei, stream);
 }
 
