@@ -56,7 +56,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
             return
@@ -153,7 +153,7 @@ def run_reference(args, c):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=5, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -276,16 +276,23 @@ def main():
     cands_per_launch = B * m * args.steps / max(kernel_launches, 1)
     npad = (n + 31) // 32 * 32
     if engine == "tensor":
-        # algorithmic flops per candidate of S4 (n^2, lower triangle, 2 flops per MAC on n^2/2 MACs); the kernel
-        # issues 3 TF32 MMAs per product, so issued = 3x that
-        alg_flops = float(npad) * npad
+        # Variance contraction S4: algorithmic n^2 flops per candidate (n^2/2 MACs over the lower triangle); the
+        # kernel issues three FP16 MMAs per product (hi*hi + hi*lo + lo*hi), so issued = 3x that, at the FP16/BF16
+        # tensor rate.  The distance products and the diagonal blocks' zero halves are not counted.
+        alg_flops = float(n) * n
         issued = 3.0 * alg_flops
         achieved = issued * cands_per_launch / (per_launch_ms * 1e-3) / 1e12
-        peak = peaks["bf16_tflops_sustained" if per_launch_ms > 50 else "bf16_tflops"] * NOMINAL_TF32_OVER_BF16
+        peak = peaks["bf16_tflops"]
         roofline = {"bound": "tensor", "kernel": "score_tc_kernel", "achieved": achieved, "peak": peak,
                     "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
-                    "note": f"issued 3xTF32 flops; algorithmic = achieved/3; peak = {peak_kind} bf16 x 1.1/2.25",
-                    "algorithmic_tflops": achieved / 3.0}
+                    "note": f"issued FP16 flops of the variance contraction (3 MMAs per product); peak = {peak_kind} "
+                            "bf16 burst (same tensor rate as fp16)",
+                    "algorithmic_tflops": achieved / 3.0,
+                    "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"]}
+        if c.cfg == 5 and args.m is None:
+            # dram bytes per launch from the ncu capture of this kernel on m = 32768 (profiles/score_tc_kernel_cfg5.md):
+            # 37.7 MB of pre-tiled operands read once + 259 B per candidate (241 read, 17.8 written)
+            roofline["traffic"] = 37.7e6 + 259.0 * cands_per_launch
     else:
         alg_flops = float(npad) * npad
         achieved = alg_flops * cands_per_launch / (per_launch_ms * 1e-3) / 1e12
@@ -309,7 +316,7 @@ def main():
     print(json.dumps({
         "metric": "gp_ei_candidates_scored_per_sec", "value": value, "unit": "candidates/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32" if engine == "simt" else "tf32x3", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32" if engine == "simt" else "f16x3", "data": "synthetic",
         "config": {"workload": c.name, "batch": B, "n": n, "d": d, "m": m, "k": k, "engine": engine,
                    "l2": "pool (%.0f MB) and outputs exceed the 126 MB L2" % (xc.numel() * 4 / 1e6)
                    if xc.numel() * 4 > 126e6 else "pool smaller than L2; not flushed"},
