@@ -120,6 +120,32 @@ r3_status_t r3_topk(const float* ei, int batch, long long m, int k, int* idx, fl
 unsigned long long r3_topk_scratch_bytes(int batch, long long m, int k);
 
 /*
+ * r3_topk_noalloc -- r3_topk for callers that must not allocate.  (The paper has no counterpart; this
+ * entry point exists for the way the library gets embedded.)
+ *
+ * A replay server that proposes points from inside a latency-critical loop, a host whose device
+ * memory is handed out once at start-up by another framework's arena, or any code running where
+ * cudaMalloc is off limits (it synchronises the device and can fail late) cannot give r3_topk a
+ * workspace sized at run time.  This variant keeps the workspace in a fixed array that is part of the
+ * library image: 1 MiB of device memory on every GPU that loads the library, held until the process
+ * exits.  The call itself never calls cudaMalloc, cudaFree or any allocating routine.
+ *
+ *   Same arguments and results as r3_topk (idx/val sorted by value descending, ties by index
+ *   ascending), without the scratch pair.
+ *   Limit: batch * ceil(m / 4096) * k <= 65536 (e.g. one pool of 1,048,576 values with k <= 256, or
+ *   64 pools of 65,536 values with k <= 64); larger requests return R3_ERR_UNSUPPORTED and say so.
+ *   The first call on a device looks the array's device address up (once per device, cached); make
+ *   that first call before any stream capture begins.
+ *   Every call uses the same array and nothing in it needs to start at zero -- each level of the
+ *   selection overwrites what the next one reads -- so the previous call's contents are harmless; but
+ *   two calls that overlap on the GPU (different streams, no ordering between them) race on it.
+ *   Order them, or use r3_topk with separate workspaces.
+ * Asynchronous on `cuda_stream`.
+ */
+r3_status_t r3_topk_noalloc(const float* ei, int batch, long long m, int k, int* idx, float* val,
+                            void* cuda_stream);
+
+/*
  * r3_gp_score_topk -- r3_gp_score followed by r3_topk on the EI it produced, with
  * the handle's own workspace; asynchronous on `cuda_stream`.  This is the "one
  * BO proposal round" call: idx [batch][k] are the pool members to replay next.

@@ -37,6 +37,7 @@ SIGNATURES = {
     "r3_gp_score": (_i, [_vp, _vp, _ll, _vp, _vp, _vp, _vp]),
     "r3_topk": (_i, [_vp, _i, _ll, _i, _vp, _vp, _vp, _ull, _vp]),
     "r3_topk_scratch_bytes": (_ull, [_i, _ll, _i]),
+    "r3_topk_noalloc": (_i, [_vp, _i, _ll, _i, _vp, _vp, _vp]),
     "r3_gp_score_topk": (_i, [_vp, _vp, _ll, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "r3_gp_score_topk_host": (_i, [_vp, _vp, _ll, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "r3_gp_check": (_i, [_vp, _vp]),
@@ -178,6 +179,19 @@ def r3_topk(ei, k: int, scratch=None):
                        ctypes.c_void_p(val.data_ptr()), ctypes.c_void_p(scratch.data_ptr()), scratch.numel(),
                        _stream()))
     return (idx[0], val[0]) if squeeze else (idx, val)
+
+
+def r3_topk_noalloc(ei, k: int, out):
+    """r3_topk without any allocation: the library's fixed key array is the workspace and the caller
+    supplies the outputs, out = (idx int32 [batch][k], val float32 [batch][k] or None).  For callers that
+    cannot allocate device memory at call time; limited to batch * ceil(m / 4096) * k <= 65536."""
+    if ei.dim() == 1:
+        ei = ei.unsqueeze(0)
+    batch, m = ei.shape
+    idx, val = out
+    _check(load().r3_topk_noalloc(_dev_f32(ei, "ei"), batch, m, k, ctypes.c_void_p(idx.data_ptr()),
+                                  ctypes.c_void_p(val.data_ptr()) if val is not None else ctypes.c_void_p(), _stream()))
+    return out
 
 
 def r3_topk_scratch_bytes(batch: int, m: int, k: int) -> int:

@@ -316,6 +316,22 @@ r3_status_t r3_topk(const float* ei, int batch, long long m, int k, int* idx, fl
     return st;
 }
 
+r3_status_t r3_topk_noalloc(const float* ei, int batch, long long m, int k, int* idx, float* val, void* cuda_stream)
+{
+    r3_status_t st = check_topk_args(ei, batch, m, k, idx);
+    if (st != R3_OK) return st;
+    const size_t capacity = topk_static_capacity_bytes();
+    if (topk_workspace_bytes(batch, m, k) > capacity) {
+        set_error("r3_topk_noalloc: batch * ceil(m / 4096) * k = %lld exceeds the fixed capacity of %zu keys; use r3_topk",
+                  (long long)batch * ((m + 4095) / 4096) * k, topk_static_capacity_keys());
+        return R3_ERR_UNSUPPORTED;
+    }
+    void* scratch = nullptr;
+    st = topk_static_scratch(&scratch);   // first call on a device: looks the array's address up (no allocation)
+    if (st != R3_OK) return st;
+    return topk_device(ei, batch, m, k, idx, val, scratch, capacity, (cudaStream_t)cuda_stream);
+}
+
 r3_status_t r3_gp_score_topk(r3_gp_t* gp, const float* Xcand, long long m, int k, float* mu, float* sigma,
                              float* ei, int* idx, float* val, void* cuda_stream)
 {

@@ -136,6 +136,11 @@ size_t topk_workspace_bytes(int batch, long long m, int k);
 r3_status_t topk_device(const float* ei, int batch, long long m, int k, int* idx, float* val, void* ws,
                         size_t ws_bytes, cudaStream_t stream);
 
+// fixed (never allocated) key storage for r3_topk_noalloc
+r3_status_t topk_static_scratch(void** ptr);
+size_t topk_static_capacity_keys();
+size_t topk_static_capacity_bytes();
+
 r3_status_t ensure_workspace(r3_gp* gp, size_t bytes);
 
 // Event pair around one launch of the dominant kernel (no-ops unless profiling is on).

@@ -7,6 +7,8 @@
 // and emits its k largest; levels repeat until one chunk is left, whose k largest are the answer.
 // The first level reads the EI array once (4 bytes per candidate); later levels touch k keys per
 // chunk of the level before.
+#include <mutex>
+
 #include "r3_internal.cuh"
 
 namespace r3 {
@@ -99,7 +101,40 @@ __global__ void topk_write_kernel(const unsigned long long* __restrict__ keys, c
 
 long long chunks_of(long long count) { return (count + CHUNK - 1) / CHUNK; }
 
+// Fixed key storage of r3_topk_noalloc: two ping-pong buffers of kStaticKeys keys each, resident in
+// every device that loads the library until the process exits (1 MiB, plus the 64 bytes of slack the
+// workspace size formula carries).
+constexpr size_t kStaticKeys = 65536;
+static __device__ __align__(256) unsigned long long g_topk_static_keys[2 * kStaticKeys + 8];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[kMaxDevices] = {};   // device address of g_topk_static_keys, per device ordinal
+
 }  // namespace
+
+// Device address of the static key array on the current device.  The array's name is only a host-side
+// handle: the address a kernel can use has to be asked for, once per device, with that device current.
+r3_status_t topk_static_scratch(void** ptr)
+{
+    int dev = 0;
+    R3_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) {
+        set_error("r3_topk_noalloc: device ordinal %d outside [0, %d)", dev, kMaxDevices);
+        return R3_ERR_UNSUPPORTED;
+    }
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void* p = nullptr;
+        R3_CUDA_TRY(cudaGetSymbolAddress(&p, g_topk_static_keys));
+        g_static_ptr[dev] = p;
+    }
+    *ptr = g_static_ptr[dev];
+    return R3_OK;
+}
+
+size_t topk_static_capacity_keys() { return kStaticKeys; }
+size_t topk_static_capacity_bytes() { return sizeof(unsigned long long) * (2 * kStaticKeys + 8); }
 
 size_t topk_workspace_bytes(int batch, long long m, int k)
 {
