@@ -53,7 +53,7 @@ typedef enum {
 typedef enum {
     R3_ENGINE_AUTO = 0,   /* tensor-core path where it applies, else SIMT */
     R3_ENGINE_SIMT = 1,   /* FP32 CUDA-core path (direct-difference distances) */
-    R3_ENGINE_TENSOR = 2  /* tcgen05 3xTF32 path (distance GEMM + triangular contraction) */
+    R3_ENGINE_TENSOR = 2  /* tcgen05 path: FP16-split distance product + triangular contraction, FP32 accumulate */
 } r3_engine_t;
 
 /*

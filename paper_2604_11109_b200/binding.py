@@ -17,7 +17,8 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libr3gp.so")
+# R3_LIB_PATH points the binding at another build of the same library (kernel experiments)
+LIB_PATH = os.environ.get("R3_LIB_PATH") or os.path.join(_HERE, "libr3gp.so")
 
 R3_OK = 0
 STATUS_NAMES = {

@@ -66,8 +66,7 @@ static r3_engine_t pick_engine(const r3_gp* gp)
         case R3_ENGINE_SIMT: return R3_ENGINE_SIMT;
         case R3_ENGINE_TENSOR: return tc_ok ? R3_ENGINE_TENSOR : R3_ENGINE_SIMT;
         default:
-            // small feature counts keep the direct-difference distances of the SIMT engine
-            return (tc_ok && gp->d > 16) ? R3_ENGINE_TENSOR : R3_ENGINE_SIMT;
+            return tc_ok ? R3_ENGINE_TENSOR : R3_ENGINE_SIMT;
     }
 }
 

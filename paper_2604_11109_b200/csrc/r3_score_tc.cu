@@ -54,13 +54,18 @@ constexpr int XS = 2;         // stages of scaled observations
 constexpr int MAX_STAGES = 4; // stages of W
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;  // ~2 s
 
-// relative error of one k* entry: eps0 + eps1 * (|z~|^2 + max|x~|^2) / sqrt(d)  (distance by split GEMM)
+// Scaled coordinates are x^ = (x - centre) * sqrt(5) log2(e) / lengthscale, so that u = |z^ - x^| is the
+// Matern argument in base-2 units: s = sqrt(5) r = u ln 2, exp(-s) = 2^-u, 1 + s + s^2/3 = 1 + c1 u + c2 u^2.
+constexpr double kCoordScale = 2.23606797749978969641 * 1.44269504088896340736;
+constexpr float kPolyC1 = 0.69314718055994530942f;               // ln 2
+constexpr float kPolyC2 = 0.16015101049403078f;                  // (ln 2)^2 / 3
+// relative error of one k* entry: eps0 + eps1 * (|z^|^2 + max|x^|^2) / sqrt(d)  (distance by split GEMM)
 constexpr double kEpsTc0 = 2.5e-7;
-constexpr double kEpsTc1 = 5.0e-8;
-// A pair (candidate, observation) whose k* (|z~|^2 + |x~|^2) exceeds kRefine sf2 has its squared distance
+constexpr double kEpsTc1 = 5.0e-8 / (kCoordScale * kCoordScale);
+// A pair (candidate, observation) whose k*/sf2 (|z^|^2 + |x^|^2) exceeds kRefine has its squared distance
 // recomputed by direct differences: r^2 from the norm expansion loses (|z~|^2 + |x~|^2) / r^2 digits, and
 // the close pairs are the ones that carry the posterior.
-constexpr float kRefine = 2.0f;
+constexpr float kRefine = 2.0f * (float)(kCoordScale * kCoordScale);
 // scaled coordinates beyond this do not fit the FP16 planes of the distance product
 constexpr float kMaxScaled = 16384.f;
 // operands of the variance product are scaled to at most 2^kScaleExp before the FP16 split
@@ -216,6 +221,12 @@ __device__ __forceinline__ float sqrt_approx(float x)
     asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
     return r;
 }
+__device__ __forceinline__ float exp2_approx(float x)
+{
+    float r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
 // (a, b) -> FP16 hi parts and FP16 low parts, each packed as half2
 __device__ __forceinline__ void split2(float a, float b, __half2& hi, __half2& lo)
 {
@@ -263,6 +274,10 @@ enum : uint32_t {
 constexpr uint32_t kFlagOffset = BAR_COUNT * 8;       // int abort, int drain-abort, uint32 tmem base
 constexpr uint32_t kZnOffset = 512;                   // float[128] squared norms of the scaled candidates
 
+// Per-role cycle accounting, compiled in only with -DR3_TC_TRACE (it costs issue slots on the hot path).
+#ifndef R3_TC_TRACE
+#define TICK(cat) do { } while (0)
+#else
 #define TICK(cat)                                                                          \
     do {                                                                                   \
         if (prm.trace) {                                                                   \
@@ -271,14 +286,18 @@ constexpr uint32_t kZnOffset = 512;                   // float[128] squared norm
             tlast = now__;                                                                 \
         }                                                                                  \
     } while (0)
+#endif
 
-// Out-of-line (cold) path of the Matern warps: for the pairs marked in `close`, replace k* by the value
+// Out-of-line (cold) path of the Matern warps: for the pairs whose k*/sf2 exceeds v_thresh, replace it by the value
 // computed from r^2 = sum_j (z~_j - x~_j)^2, with z~ = hi + lo read back from the TMEM planes at z_taddr
 // and x~ in FP32 from global memory.  Called by all 32 lanes of a warp together (TMEM loads are
 // warp-wide); a lane without marked pairs only takes part in the loads.
-__device__ __noinline__ void refine_close_pairs(float* kv, uint32_t close, uint32_t z_taddr, int DP,
-                                                const float* __restrict__ xrow0, float sf2)
+__device__ __noinline__ void refine_close_pairs(float* kv, float v_thresh, uint32_t z_taddr, int DP,
+                                                const float* __restrict__ xrow0)
 {
+    uint32_t close = 0;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) close |= (kv[i] > v_thresh) ? (1u << i) : 0u;
     float r2x[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) r2x[i] = 0.f;
@@ -316,8 +335,8 @@ __device__ __noinline__ void refine_close_pairs(float* kv, uint32_t close, uint3
     }
     for (uint32_t rest = close; rest; rest &= rest - 1) {
         const int i = __ffs(rest) - 1;
-        const float s = sqrtf(5.f * r2x[i]);
-        kv[i] = sf2 * fmaf(s, fmaf(s, 1.f / 3.f, 1.f), 1.f) * __expf(-s);
+        const float u = sqrtf(r2x[i]);
+        kv[i] = fmaf(u, fmaf(u, kPolyC2, kPolyC1), 1.f) * exp2f(-u);
     }
 }
 
@@ -557,7 +576,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
             const long long cand = (tile % prm.tiles_per_gp) * TILE_M + row;
             const bool valid = cand < prm.m;
             const float sf2 = prm.sf2[g];
-            const float kscale = prm.kscale[g];
+            const float kvscale = prm.kscale[g] * sf2;   // k* = sf2 * (k*/sf2), scaled for its FP16 split
             if (grp == G - 1) {
                 // ---- scale the candidate, split it, store it as the A operand of the distance MMA
                 float zn = 0.f;
@@ -627,7 +646,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
             const float zn = fabsf(zn_s[row]);
 
             const float* xs_g = prm.xs32 + (size_t)g * prm.NP * DP;
-            const float refine_at = far_cand ? INFINITY : kRefine * sf2;
+            const float v_thresh = far_cand ? INFINITY : kRefine / (zn + prm.xnmax[g]);
             const float* xn_g = prm.xnorm + (size_t)g * prm.NP;
             const float* al_g = prm.alpha + (size_t)g * prm.NP;
             double mu_acc = 0.0, a2_acc = 0.0, s2_acc = 0.0, q_acc = 0.0;
@@ -662,28 +681,27 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                             mbar_arrive(bar(BAR_D_EMPTY + db));
                         }
                         TICK(1);
-                        float kv[16];
-                        uint32_t close = 0;   // bit i: pair i needs its distance by direct differences
+                        float kv[16];   // k*/sf2
+                        float vmax = 0.f;
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
                             const float4 xn4 = __ldg(reinterpret_cast<const float4*>(xn_g + c * KC + h * 16 + 4 * q));
                             const float xn[4] = {xn4.x, xn4.y, xn4.z, xn4.w};
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
-                                const float r2 = fmaxf(fmaf(-2.f, dot[4 * q + e], zn + xn[e]), 0.f);
-                                const float s = sqrt_approx(5.f * r2);
-                                const float v = sf2 * fmaf(s, fmaf(s, 1.f / 3.f, 1.f), 1.f) * __expf(-s);
+                                const float u = sqrt_approx(fmaxf(fmaf(-2.f, dot[4 * q + e], zn + xn[e]), 0.f));
+                                const float v = fmaf(u, fmaf(u, kPolyC2, kPolyC1), 1.f) * exp2_approx(-u);
                                 kv[4 * q + e] = v;
-                                if (v * (zn + xn[e]) > refine_at) close |= 1u << (4 * q + e);
+                                vmax = fmaxf(vmax, v);
                             }
                         }
-                        if (__any_sync(0xffffffffu, close != 0)) {
+                        if (__any_sync(0xffffffffu, vmax > v_thresh)) {
                             // rare: hand the 16 values to the out-of-line refinement through a local array so
                             // that the hot path keeps kv in registers
                             float tmp[16];
 #pragma unroll
                             for (int i = 0; i < 16; ++i) tmp[i] = kv[i];
-                            refine_close_pairs(tmp, close, lane_addr + ZCOL, DP, xs_g + (size_t)(c * KC + h * 16) * DP, sf2);
+                            refine_close_pairs(tmp, v_thresh, lane_addr + ZCOL, DP, xs_g + (size_t)(c * KC + h * 16) * DP);
 #pragma unroll
                             for (int i = 0; i < 16; ++i) kv[i] = tmp[i];
                         }
@@ -701,9 +719,9 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                                     spart = fmaf(v, v, spart);
                                 }
                             }
-                            mu_acc += (double)mpart;
-                            a2_acc += (double)apart;
-                            s2_acc += (double)spart;
+                            mu_acc += (double)(mpart * sf2);
+                            a2_acc += (double)(apart * sf2 * sf2);
+                            s2_acc += (double)(spart * sf2 * sf2);
                         }
                         TICK(2);
                         if (h == 0) {
@@ -718,7 +736,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                             __half2 hi2[4], lo2[4];
 #pragma unroll
                             for (int e = 0; e < 4; ++e)
-                                split2(kv[8 * sl + 2 * e] * kscale, kv[8 * sl + 2 * e + 1] * kscale, hi2[e], lo2[e]);
+                                split2(kv[8 * sl + 2 * e] * kvscale, kv[8 * sl + 2 * e + 1] * kvscale, hi2[e], lo2[e]);
                             *reinterpret_cast<uint4*>(kb + (2 * h + sl) * 2048u) = *reinterpret_cast<const uint4*>(hi2);
                             *reinterpret_cast<uint4*>(kb + 8192u + (2 * h + sl) * 2048u) =
                                 *reinterpret_cast<const uint4*>(lo2);
@@ -818,7 +836,7 @@ __global__ void centre_kernel(const float* __restrict__ X, const float* __restri
     }
     if (threadIdx.x == 0) {
         centre[(size_t)g * DP + j] = (j < d) ? (float)(s[0] / n) : 0.f;
-        scale[(size_t)g * DP + j] = (j < d) ? inv_ell[(size_t)g * d + j] : 0.f;
+        scale[(size_t)g * DP + j] = (j < d) ? (float)((double)inv_ell[(size_t)g * d + j] * kCoordScale) : 0.f;
     }
 }
 
