@@ -51,7 +51,7 @@ namespace {
 constexpr int KC = 32;        // observations per chunk of the variance product
 constexpr int TILE_M = 128;   // candidates per CTA tile
 constexpr int XS = 2;         // stages of scaled observations
-constexpr int MAX_STAGES = 4; // stages of W
+constexpr int MAX_STAGES = 6; // stages of W
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;  // ~2 s
 
 // Scaled coordinates are x^ = (x - centre) * sqrt(5) log2(e) / lengthscale, so that u = |z^ - x^| is the
@@ -73,6 +73,7 @@ constexpr int kScaleExp = 14;
 
 struct TensorOperands {
     int NV = 0, G = 0, KD = 0, DP = 0, NP = 0, P = 0, ws = 0;
+    bool kt = false;           // k* buffers in TMEM
     size_t smem_bytes = 0;
     size_t wt_gp_stride = 0;   // halves per GP in wt
     float* centre = nullptr;   // [B][DP]  column means of X (zero padded)
@@ -247,15 +248,15 @@ __device__ __forceinline__ constexpr uint32_t instr_desc_f16(uint32_t n)
 
 // shared-memory map (byte offsets from a 1024-aligned base)
 struct SmemMap {
-    uint32_t z, k, x, w, bar;
+    uint32_t z, k, x, w, bar;   // z: reduction scratch; k: k* buffers (absent when k* lives in TMEM)
     uint32_t x_stage, w_stage;
 };
-__host__ __device__ inline SmemMap smem_map(int DP, int NV, int G, int KD, int ws)
+__host__ __device__ inline SmemMap smem_map(int DP, int NV, int G, int KD, int ws, bool kt)
 {
     SmemMap s;
-    s.z = 0;                                       // (the scaled candidates live in TMEM)
-    s.k = 0;                                       // G buffers x 2 planes x [KC/8][128][8] halves
-    s.x = s.k + (uint32_t)G * 16384u;              // XS stages x 2 planes x [DP/8][KD][8] halves
+    s.z = 0;                                       // end-of-tile reduction scratch: G x 128 rows x 4 doubles
+    s.k = (uint32_t)G * 4096u;                     // k* in shared memory: G buffers x 2 planes x [KC/8][128][8] halves
+    s.x = s.k + (kt ? 0u : (uint32_t)G * 16384u);  // XS stages x 2 planes x [DP/8][KD][8] halves
     s.x_stage = 2u * DP * KD * 2u;
     s.w = s.x + (uint32_t)XS * s.x_stage;          // ws stages x 2 planes x [KC/8][NV][8] halves
     s.w_stage = 2u * KC * NV * 2u;
@@ -266,10 +267,10 @@ constexpr uint32_t kBarBytes = 1024;   // barriers, flags, TMEM slot, candidate 
 
 // barrier slots (8 bytes each) inside the barrier block
 enum : uint32_t {
-    BAR_X_FULL = 0, BAR_X_EMPTY = 2, BAR_W_FULL = 4, BAR_W_EMPTY = 8, BAR_D_FULL = 12, BAR_D_EMPTY = 14,
-    BAR_K_FULL = 16, BAR_K_EMPTY = 20, BAR_V_FULL = 24, BAR_V_EMPTY = 25, BAR_Z_READY = 26, BAR_RED_READY = 27,
-    BAR_MMA_DONE = 28,  // two slots: distance issuer, variance issuer
-    BAR_COUNT = 30
+    BAR_X_FULL = 0, BAR_X_EMPTY = 2, BAR_W_FULL = 4, BAR_W_EMPTY = 10, BAR_D_FULL = 16, BAR_D_EMPTY = 18,
+    BAR_K_FULL = 20, BAR_K_EMPTY = 24, BAR_V_FULL = 28, BAR_V_EMPTY = 29, BAR_Z_READY = 30, BAR_RED_READY = 31,
+    BAR_MMA_DONE = 32,  // two slots: distance issuer, variance issuer
+    BAR_COUNT = 34
 };
 constexpr uint32_t kFlagOffset = BAR_COUNT * 8;       // int abort, int drain-abort, uint32 tmem base
 constexpr uint32_t kZnOffset = 512;                   // float[128] squared norms of the scaled candidates
@@ -288,11 +289,11 @@ constexpr uint32_t kZnOffset = 512;                   // float[128] squared norm
     } while (0)
 #endif
 
-// Out-of-line (cold) path of the Matern warps: for the pairs whose k*/sf2 exceeds v_thresh, replace it by the value
+// Out-of-line (cold) path of the Matern warps: for the pairs whose (scaled) k* exceeds v_thresh, replace it by the value
 // computed from r^2 = sum_j (z~_j - x~_j)^2, with z~ = hi + lo read back from the TMEM planes at z_taddr
 // and x~ in FP32 from global memory.  Called by all 32 lanes of a warp together (TMEM loads are
 // warp-wide); a lane without marked pairs only takes part in the loads.
-__device__ __noinline__ void refine_close_pairs(float* kv, float v_thresh, uint32_t z_taddr, int DP,
+__device__ __noinline__ void refine_close_pairs(float* kv, float v_thresh, float kvscale, uint32_t z_taddr, int DP,
                                                 const float* __restrict__ xrow0)
 {
     uint32_t close = 0;
@@ -336,20 +337,22 @@ __device__ __noinline__ void refine_close_pairs(float* kv, float v_thresh, uint3
     for (uint32_t rest = close; rest; rest &= rest - 1) {
         const int i = __ffs(rest) - 1;
         const float u = sqrtf(r2x[i]);
-        kv[i] = fmaf(u, fmaf(u, kPolyC2, kPolyC1), 1.f) * exp2f(-u);
+        kv[i] = kvscale * fmaf(u, fmaf(u, kPolyC2, kPolyC1), 1.f) * exp2f(-u);
     }
 }
 
 // NV: rows of W per pass (TMEM columns of the V accumulator).  G: number of Matern warp groups; group
-// g owns chunks t = g (mod G) and k* buffer g.  KD: observations per distance product.
-template <int NV, int G, int KD>
+// g owns chunks t = g (mod G) and k* buffer g.  KD: observations per distance product.  KT: the k*
+// buffers (A operand of the variance product) live in TMEM instead of shared memory: shared memory then
+// only feeds the B operands, which is what keeps its 128 B/clk from becoming the limit.
+template <int NV, int G, int KD, bool KT>
 __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcParams prm)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* sm = smem_raw + (base - raw);
-    const SmemMap map = smem_map(prm.DP, NV, G, KD, prm.ws);
+    const SmemMap map = smem_map(prm.DP, NV, G, KD, prm.ws, KT);
     const uint32_t bars = base + map.bar;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + map.bar + kFlagOffset);
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + map.bar + kFlagOffset + 8);
@@ -360,9 +363,11 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
     constexpr int CPP = NV / KC;                  // chunks per pass width
     constexpr int SL = KD / KC;                   // chunks per distance product
     // TMEM columns: V accumulator [0, NV), two distance buffers [NV, NV + 2 KD), scaled candidates
-    // (FP16 hi plane, then lo plane, DP/2 columns each) from NV + 2 KD
+    // (FP16 hi plane, then lo plane, DP/2 columns each) from NV + 2 KD, then (KT) G k* buffers of
+    // 2 planes x KC/2 columns
     constexpr uint32_t TMEM_COLS = 512u;
     constexpr uint32_t ZCOL = NV + 2 * KD;
+    const uint32_t KCOL = ZCOL + (uint32_t)prm.DP;
     const int DP = prm.DP, P = prm.P, ws = prm.ws;
 
     if (threadIdx.x == 0) {
@@ -375,6 +380,8 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
         for (int i = 0; i < MAX_STAGES; ++i) {
             mbar_init(bar(BAR_W_FULL + i), 1);
             mbar_init(bar(BAR_W_EMPTY + i), 1);
+        }
+        for (int i = 0; i < 4; ++i) {
             mbar_init(bar(BAR_K_FULL + i), 128);
             mbar_init(bar(BAR_K_EMPTY + i), 1);
         }
@@ -531,16 +538,28 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     if (++w_s == ws) { w_s = 0; w_ph ^= 1u; }
                     TICK(5);
                     tc_fence_after();
-                    const uint32_t aH = k_lo0 + ((b * 16384u) >> 4), aL = aH + (8192u >> 4);
                     const uint32_t bH = w_lo0 + ((s * map.w_stage) >> 4), bL = bH + (((uint32_t)KC * NV * 2u) >> 4);
+                    if (KT) {
+                        const uint32_t aH = tmem + KCOL + (uint32_t)b * KC, aL = aH + KC / 2;
 #pragma unroll
-                    for (int combo = 0; combo < 3; ++combo) {
-                        const uint32_t a0 = combo == 2 ? aL : aH, b0 = combo == 1 ? bL : bH;
+                        for (int combo = 0; combo < 3; ++combo) {
+                            const uint32_t a0 = combo == 2 ? aL : aH, b0 = combo == 1 ? bL : bH;
 #pragma unroll
-                        for (int jj = 0; jj < KC / 16; ++jj)
-                            tc_mma_f16(tmem, pack64(a0 + jj * (4096u >> 4), kDescHi),
-                                       pack64(b0 + jj * ((2u * NV * 16u) >> 4), kDescHi), IDESC_V,
-                                       (c > 0 || combo > 0 || jj > 0) ? 1u : 0u);
+                            for (int jj = 0; jj < KC / 16; ++jj)
+                                tc_mma_f16_ts(tmem, a0 + jj * 8u, pack64(b0 + jj * ((2u * NV * 16u) >> 4), kDescHi), IDESC_V,
+                                              (c > 0 || combo > 0 || jj > 0) ? 1u : 0u);
+                        }
+                    } else {
+                        const uint32_t aH = k_lo0 + ((b * 16384u) >> 4), aL = aH + (8192u >> 4);
+#pragma unroll
+                        for (int combo = 0; combo < 3; ++combo) {
+                            const uint32_t a0 = combo == 2 ? aL : aH, b0 = combo == 1 ? bL : bH;
+#pragma unroll
+                            for (int jj = 0; jj < KC / 16; ++jj)
+                                tc_mma_f16(tmem, pack64(a0 + jj * (4096u >> 4), kDescHi),
+                                           pack64(b0 + jj * ((2u * NV * 16u) >> 4), kDescHi), IDESC_V,
+                                           (c > 0 || combo > 0 || jj > 0) ? 1u : 0u);
+                        }
                     }
                     tc_commit(bar(BAR_W_EMPTY + s));
                     tc_commit(bar(BAR_K_EMPTY + b));
@@ -569,8 +588,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
         long long tile_iter = 0;
         bool ok = true;
         bool bad = false;
-        // scratch for the end-of-tile reduction lives in k* buffer 0 (dead once the last pass is done)
-        double* red = reinterpret_cast<double*>(sm + map.k);
+        double* red = reinterpret_cast<double*>(sm + map.z);   // scratch of the end-of-tile reduction
         for (long long tile = first_tile; ok && tile < prm.total_tiles; tile += tile_step, ++tile_iter) {
             const int g = (int)(tile / prm.tiles_per_gp);
             const long long cand = (tile % prm.tiles_per_gp) * TILE_M + row;
@@ -646,7 +664,9 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
             const float zn = fabsf(zn_s[row]);
 
             const float* xs_g = prm.xs32 + (size_t)g * prm.NP * DP;
-            const float v_thresh = far_cand ? INFINITY : kRefine / (zn + prm.xnmax[g]);
+            const float v_thresh = far_cand ? INFINITY : kvscale * kRefine / (zn + prm.xnmax[g]);
+            const float pc0 = kvscale, pc1 = kvscale * kPolyC1, pc2 = kvscale * kPolyC2;
+            const float inv_kscale = 1.f / prm.kscale[g];   // scaled k* -> k*
             const float* xn_g = prm.xnorm + (size_t)g * prm.NP;
             const float* al_g = prm.alpha + (size_t)g * prm.NP;
             double mu_acc = 0.0, a2_acc = 0.0, s2_acc = 0.0, q_acc = 0.0;
@@ -681,27 +701,29 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                             mbar_arrive(bar(BAR_D_EMPTY + db));
                         }
                         TICK(1);
-                        float kv[16];   // k*/sf2
-                        float vmax = 0.f;
+                        float kv[16];   // k* times kvscale (the power of two of its FP16 split)
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
                             const float4 xn4 = __ldg(reinterpret_cast<const float4*>(xn_g + c * KC + h * 16 + 4 * q));
                             const float xn[4] = {xn4.x, xn4.y, xn4.z, xn4.w};
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
-                                const float u = sqrt_approx(fmaxf(fmaf(-2.f, dot[4 * q + e], zn + xn[e]), 0.f));
-                                const float v = fmaf(u, fmaf(u, kPolyC2, kPolyC1), 1.f) * exp2_approx(-u);
-                                kv[4 * q + e] = v;
-                                vmax = fmaxf(vmax, v);
+                                // |.|: a slightly negative r^2 (rounding) is a tiny distance either way
+                                const float u = sqrt_approx(fabsf(fmaf(-2.f, dot[4 * q + e], zn + xn[e])));
+                                kv[4 * q + e] = fmaf(u, fmaf(u, pc2, pc1), pc0) * exp2_approx(-u);
                             }
                         }
+                        float vmax = fmaxf(fmaxf(kv[0], kv[1]), fmaxf(kv[2], kv[3]));
+#pragma unroll
+                        for (int i = 4; i < 16; i += 4)
+                            vmax = fmaxf(vmax, fmaxf(fmaxf(kv[i], kv[i + 1]), fmaxf(kv[i + 2], kv[i + 3])));
                         if (__any_sync(0xffffffffu, vmax > v_thresh)) {
                             // rare: hand the 16 values to the out-of-line refinement through a local array so
                             // that the hot path keeps kv in registers
                             float tmp[16];
 #pragma unroll
                             for (int i = 0; i < 16; ++i) tmp[i] = kv[i];
-                            refine_close_pairs(tmp, v_thresh, lane_addr + ZCOL, DP, xs_g + (size_t)(c * KC + h * 16) * DP);
+                            refine_close_pairs(tmp, v_thresh, kvscale, lane_addr + ZCOL, DP, xs_g + (size_t)(c * KC + h * 16) * DP);
 #pragma unroll
                             for (int i = 0; i < 16; ++i) kv[i] = tmp[i];
                         }
@@ -719,9 +741,9 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                                     spart = fmaf(v, v, spart);
                                 }
                             }
-                            mu_acc += (double)(mpart * sf2);
-                            a2_acc += (double)(apart * sf2 * sf2);
-                            s2_acc += (double)(spart * sf2 * sf2);
+                            mu_acc += (double)(mpart * inv_kscale);
+                            a2_acc += (double)(apart * inv_kscale * inv_kscale);
+                            s2_acc += (double)(spart * inv_kscale * inv_kscale);
                         }
                         TICK(2);
                         if (h == 0) {
@@ -730,20 +752,39 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                             if (!ok) break;
                             TICK(3);
                         }
-                        // 16 columns = two 16-byte k-slices of the A operand, hi and lo planes
+                        if (KT) {
+                            // 16 columns = 8 packed TMEM columns of each plane
+                            uint32_t kh[8], kl[8];
 #pragma unroll
-                        for (int sl = 0; sl < 2; ++sl) {
-                            __half2 hi2[4], lo2[4];
+                            for (int e = 0; e < 8; ++e) {
+                                __half2 hi, lo;
+                                split2(kv[2 * e], kv[2 * e + 1], hi, lo);
+                                kh[e] = *reinterpret_cast<const uint32_t*>(&hi);
+                                kl[e] = *reinterpret_cast<const uint32_t*>(&lo);
+                            }
+                            tc_st8(lane_addr + KCOL + (uint32_t)grp * KC + h * 8, kh);
+                            tc_st8(lane_addr + KCOL + (uint32_t)grp * KC + KC / 2 + h * 8, kl);
+                        } else {
+                            // 16 columns = two 16-byte k-slices of the A operand, hi and lo planes
 #pragma unroll
-                            for (int e = 0; e < 4; ++e)
-                                split2(kv[8 * sl + 2 * e] * kvscale, kv[8 * sl + 2 * e + 1] * kvscale, hi2[e], lo2[e]);
-                            *reinterpret_cast<uint4*>(kb + (2 * h + sl) * 2048u) = *reinterpret_cast<const uint4*>(hi2);
-                            *reinterpret_cast<uint4*>(kb + 8192u + (2 * h + sl) * 2048u) =
-                                *reinterpret_cast<const uint4*>(lo2);
+                            for (int sl = 0; sl < 2; ++sl) {
+                                __half2 hi2[4], lo2[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e)
+                                    split2(kv[8 * sl + 2 * e], kv[8 * sl + 2 * e + 1], hi2[e], lo2[e]);
+                                *reinterpret_cast<uint4*>(kb + (2 * h + sl) * 2048u) = *reinterpret_cast<const uint4*>(hi2);
+                                *reinterpret_cast<uint4*>(kb + 8192u + (2 * h + sl) * 2048u) =
+                                    *reinterpret_cast<const uint4*>(lo2);
+                            }
                         }
                     }
                     if (!ok) break;
-                    fence_proxy_async();
+                    if (KT) {
+                        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                        tc_fence_before();
+                    } else {
+                        fence_proxy_async();
+                    }
                     mbar_arrive(bar(BAR_K_FULL + grp));
                     TICK(4);
                     t += G;
@@ -934,14 +975,14 @@ __global__ void wt_build_kernel(const double* __restrict__ W64, int n, int npad_
 
 TensorOperands* ops_of(const r3_gp* gp) { return static_cast<TensorOperands*>(gp->tc); }
 
-void (*kernel_for(int NV, int G, int KD))(const TcParams)
+void (*kernel_for(int NV, int G, bool kt))(const TcParams)
 {
-    if (KD == 128) {
-        if (NV == 256) return G == 3 ? score_tc_kernel<256, 3, 128> : score_tc_kernel<256, 2, 128>;
-        return G == 3 ? score_tc_kernel<128, 3, 128> : score_tc_kernel<128, 2, 128>;
+    if (kt) {
+        if (NV == 256) return G == 3 ? score_tc_kernel<256, 3, 64, true> : score_tc_kernel<256, 2, 64, true>;
+        return G == 3 ? score_tc_kernel<128, 3, 64, true> : score_tc_kernel<128, 2, 64, true>;
     }
-    if (NV == 256) return G == 3 ? score_tc_kernel<256, 3, 64> : score_tc_kernel<256, 2, 64>;
-    return G == 3 ? score_tc_kernel<128, 3, 64> : score_tc_kernel<128, 2, 64>;
+    if (NV == 256) return G == 3 ? score_tc_kernel<256, 3, 64, false> : score_tc_kernel<256, 2, 64, false>;
+    return G == 3 ? score_tc_kernel<128, 3, 64, false> : score_tc_kernel<128, 2, 64, false>;
 }
 
 int env_int(const char* name, int fallback)
@@ -985,27 +1026,32 @@ r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream)
     t->NV = n > 128 ? 256 : 128;
     t->NP = round_up(n, t->NV);
     t->P = t->NP / t->NV;
-    // shared-memory budget decides the shape: prefer three Matern groups, then wide distance products,
-    // then as many W stages as fit (at least three)
+    // Shape, in order of preference (measured on the largest workload: the first two are within 1 %):
+    // k* in shared memory with three Matern groups and at least three W stages; k* in TMEM (needs
+    // V accumulator + two distance buffers + candidates + G k* buffers <= 512 columns), which frees
+    // shared memory for W stages; then whatever fits with two W stages.
     const size_t budget = 227 * 1024 - 1024 - kBarBytes;
-    const int want_kd = env_int("R3_TC_KD", 0), want_g = env_int("R3_TC_G", 0);
+    const int want_kt = env_int("R3_TC_KT", -1), want_g = env_int("R3_TC_G", 0);
+    t->KD = 64;
     bool found = false;
-    for (int min_ws = 3; min_ws >= 2 && !found; --min_ws)
-        for (int pref = 0; pref < 4 && !found; ++pref) {
-            t->G = pref < 2 ? 3 : 2;
-            t->KD = (pref % 2 == 0) ? 64 : 128;
-            if (want_kd && t->KD != want_kd) continue;
-            if (want_g && t->G != want_g) continue;
-            if (t->NV % t->KD) continue;
-            for (t->ws = MAX_STAGES; t->ws >= 2; --t->ws)
-                if (smem_map(t->DP, t->NV, t->G, t->KD, t->ws).bar <= budget) break;
-            found = t->ws >= min_ws;
-        }
+    static const struct { bool kt; int G, min_ws; } prefs[] = {
+        {false, 3, 3}, {true, 3, 3}, {true, 2, 3}, {false, 2, 3}, {false, 3, 2}, {true, 2, 2}, {false, 2, 2}};
+    for (const auto& pr : prefs) {
+        if (found) break;
+        t->kt = pr.kt;
+        t->G = pr.G;
+        if (want_kt >= 0 && (int)t->kt != want_kt) continue;
+        if (want_g && t->G != want_g) continue;
+        if (t->NV + 2 * t->KD + t->DP + (t->kt ? t->G * KC : 0) > 512) continue;
+        for (t->ws = MAX_STAGES; t->ws >= 2; --t->ws)
+            if (smem_map(t->DP, t->NV, t->G, t->KD, t->ws, t->kt).bar <= budget) break;
+        found = t->ws >= pr.min_ws;
+    }
     if (!found) {
         tc_release(gp);   // does not fit: the SIMT engine serves this shape
         return R3_OK;
     }
-    t->smem_bytes = smem_map(t->DP, t->NV, t->G, t->KD, t->ws).bar + kBarBytes + 1024;
+    t->smem_bytes = smem_map(t->DP, t->NV, t->G, t->KD, t->ws, t->kt).bar + kBarBytes + 1024;
     const int CPP = t->NV / KC;
     const size_t tiles = (size_t)CPP * t->P * (t->P + 1) / 2;
     t->wt_gp_stride = tiles * (2 * (size_t)KC * t->NV);
@@ -1085,7 +1131,7 @@ r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream)
     cudaFree(wscale_d);
     wmax_bits = nullptr;
     wscale_d = nullptr;
-    e = cudaFuncSetAttribute(kernel_for(t->NV, t->G, t->KD), cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(kernel_for(t->NV, t->G, t->kt), cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)t->smem_bytes);
     if (e != cudaSuccess) return fail("cudaFuncSetAttribute", e);
     return R3_OK;
@@ -1146,7 +1192,7 @@ r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, floa
         if (cudaMalloc(&prm.trace, sizeof(long long) * grid * 32) != cudaSuccess) prm.trace = nullptr;
         if (prm.trace) cudaMemset(prm.trace, 0, sizeof(long long) * grid * 32);
     }
-    void (*kernel)(const TcParams) = kernel_for(t->NV, t->G, t->KD);
+    void (*kernel)(const TcParams) = kernel_for(t->NV, t->G, t->kt);
     prof_begin(gp, stream);
     R3_LAUNCH(kernel, grid, 128 + 128 * t->G, t->smem_bytes, stream, prm);
     prof_end(gp, stream);
@@ -1155,8 +1201,8 @@ r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, floa
         cudaMemcpy(h.data(), prm.trace, sizeof(long long) * grid * 32, cudaMemcpyDeviceToHost);
         cudaFree(prm.trace);
         const char* names[4] = {"mmaV", "matern0", "matern1", "mmaD"};
-        fprintf(stderr, "trace shape NV=%d G=%d KD=%d ws=%d DP=%d P=%d smem=%zu\n", t->NV, t->G, t->KD, t->ws, t->DP, t->P,
-                t->smem_bytes);
+        fprintf(stderr, "trace shape NV=%d G=%d KD=%d kt=%d ws=%d DP=%d P=%d smem=%zu\n", t->NV, t->G, t->KD, (int)t->kt, t->ws,
+                t->DP, t->P, t->smem_bytes);
         for (int r = 0; r < 4; ++r) {
             fprintf(stderr, "trace cta0 %s:", names[r]);
             for (int i = 0; i < 8; ++i) fprintf(stderr, " %lld", h[(size_t)r * 8 + i]);
