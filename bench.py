@@ -191,6 +191,7 @@ def main():
     xc = torch.from_numpy(g["Xcand"]).cuda()
     B, m, k, n, d = c.batch, c.m, c.k, c.n, c.d
 
+    b.r3_gp_fit(X, y, g["ell"], g["sf2"], g["sn2"]).close()   # warm-up fit: module load and first-use costs
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
     ev[0].record()
     gp = b.r3_gp_fit(X, y, g["ell"], g["sf2"], g["sn2"])
