@@ -43,208 +43,11 @@
 
 #include "r3_epilogue.cuh"
 #include "r3_internal.cuh"
+#include "r3_tc_common.cuh"
 
 namespace r3 {
 
 namespace {
-
-constexpr int KC = 32;        // observations per chunk of the variance product
-constexpr int TILE_M = 128;   // candidates per CTA tile
-constexpr int XS = 2;         // stages of scaled observations
-constexpr int MAX_STAGES = 6; // stages of W
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;  // ~2 s
-
-// Scaled coordinates are x^ = (x - centre) * sqrt(5) log2(e) / lengthscale, so that u = |z^ - x^| is the
-// Matern argument in base-2 units: s = sqrt(5) r = u ln 2, exp(-s) = 2^-u, 1 + s + s^2/3 = 1 + c1 u + c2 u^2.
-constexpr double kCoordScale = 2.23606797749978969641 * 1.44269504088896340736;
-constexpr float kPolyC1 = 0.69314718055994530942f;               // ln 2
-constexpr float kPolyC2 = 0.16015101049403078f;                  // (ln 2)^2 / 3
-// relative error of one k* entry: eps0 + eps1 * (|z^|^2 + max|x^|^2) / sqrt(d)  (distance by split GEMM)
-constexpr double kEpsTc0 = 2.5e-7;
-constexpr double kEpsTc1 = 5.0e-8 / (kCoordScale * kCoordScale);
-// A pair (candidate, observation) whose k*/sf2 (|z^|^2 + |x^|^2) exceeds kRefine has its squared distance
-// recomputed by direct differences: r^2 from the norm expansion loses (|z~|^2 + |x~|^2) / r^2 digits, and
-// the close pairs are the ones that carry the posterior.
-constexpr float kRefine = 2.0f * (float)(kCoordScale * kCoordScale);
-// scaled coordinates beyond this do not fit the FP16 planes of the distance product
-constexpr float kMaxScaled = 16384.f;
-// operands of the variance product are scaled to at most 2^kScaleExp before the FP16 split
-constexpr int kScaleExp = 14;
-
-struct TensorOperands {
-    int NV = 0, G = 0, KD = 0, DP = 0, NP = 0, P = 0, ws = 0;
-    bool kt = false;           // k* buffers in TMEM
-    size_t smem_bytes = 0;
-    size_t wt_gp_stride = 0;   // halves per GP in wt
-    float* centre = nullptr;   // [B][DP]  column means of X (zero padded)
-    float* scale = nullptr;    // [B][DP]  1/lengthscale (zero padded)
-    __half* xt = nullptr;      // [B][NP/KD][2][DP/8][KD][8]  scaled observations, FP16 hi/lo planes
-    float* xs32 = nullptr;     // [B][NP][DP]  scaled observations in FP32 (refinement of close pairs)
-    float* xnorm = nullptr;    // [B][NP]  |x~_k|^2
-    float* xnmax = nullptr;    // [B]      max_k |x~_k|^2
-    float* alpha = nullptr;    // [B][NP]  weights, zero padded
-    __half* wt = nullptr;      // [B][tile(p,c)][2][KC/8][NV][8]  chunks of 2^eW W, FP16 hi/lo planes
-    float* kscale = nullptr;   // [B]  2^eK, applied to k* before its split
-    double* vinv2 = nullptr;   // [B]  2^(-2 (eK + eW)): scales sum V^2 back
-};
-
-struct TcParams {
-    const float* xcand;
-    long long m;
-    int batch, d;
-    float *mu, *sigma, *ei, *err_mu, *err_q;
-    const float *centre, *scale, *xs32, *xnorm, *xnmax, *alpha, *kscale;
-    const __half *xt, *wt;
-    const double* vinv2;
-    size_t wt_gp_stride;
-    const float *sf2, *best;
-    const double* wnorm;
-    int DP, NP, P, ws;
-    int* status;
-    long long tiles_per_gp, total_tiles;
-    long long* trace;   // optional [grid][4 roles][8] cycle counters (diagnostics)
-};
-
-// ------------------------------------------------------------------------------------------------
-// PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok;
-}
-// Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
-            *abort_flag = 1;
-            return false;
-        }
-    }
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                 "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
-__device__ __forceinline__ void fence_proxy_async()
-{
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                           uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// A operand from TMEM (lane = row, one 32-bit column = two consecutive FP16 k-elements)
-__device__ __forceinline__ void tc_mma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
-                                              uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t* r)
-{
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(taddr), "r"(r[0]),
-                 "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
-                 : "memory");
-}
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v)
-{
-    uint32_t r[16];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr)
-        : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-}
-__device__ __forceinline__ void tc_ld8(uint32_t taddr, uint32_t* r)
-{
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-                 : "r"(taddr)
-                 : "memory");
-}
-__device__ __forceinline__ uint64_t pack64(uint32_t lo, uint32_t hi)
-{
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
-    return r;
-}
-__device__ __forceinline__ float sqrt_approx(float x)
-{
-    float r;
-    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
-    return r;
-}
-__device__ __forceinline__ float exp2_approx(float x)
-{
-    float r;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
-    return r;
-}
-// (a, b) -> FP16 hi parts and FP16 low parts, each packed as half2
-__device__ __forceinline__ void split2(float a, float b, __half2& hi, __half2& lo)
-{
-    hi = __floats2half2_rn(a, b);
-    const float2 back = __half22float2(hi);
-    lo = __floats2half2_rn(a - back.x, b - back.y);
-}
-
-// Shared-memory matrix descriptors are the no-swizzle K-major form: bits 0-13 start address >> 4,
-// bits 16-29 the byte distance between the two 16-byte k-slices of one MMA >> 4, bits 32-45 the byte
-// distance between 8-row groups (128) >> 4, bit 46 the descriptor version.
-constexpr uint32_t kDescHi = (128u >> 4) | (1u << 14);
-// Instruction descriptor: FP32 accumulate, FP16 x FP16 (format code 0), both K-major, M = 128, N = n.
-__device__ __forceinline__ constexpr uint32_t instr_desc_f16(uint32_t n)
-{
-    return (1u << 4) | ((n >> 3) << 17) | ((128u >> 4) << 24);
-}
 
 // shared-memory map (byte offsets from a 1024-aligned base)
 struct SmemMap {
@@ -275,71 +78,6 @@ enum : uint32_t {
 constexpr uint32_t kFlagOffset = BAR_COUNT * 8;       // int abort, int drain-abort, uint32 tmem base
 constexpr uint32_t kZnOffset = 512;                   // float[128] squared norms of the scaled candidates
 
-// Per-role cycle accounting, compiled in only with -DR3_TC_TRACE (it costs issue slots on the hot path).
-#ifndef R3_TC_TRACE
-#define TICK(cat) do { } while (0)
-#else
-#define TICK(cat)                                                                          \
-    do {                                                                                   \
-        if (prm.trace) {                                                                   \
-            const long long now__ = clock64();                                             \
-            tacc[cat] += now__ - tlast;                                                    \
-            tlast = now__;                                                                 \
-        }                                                                                  \
-    } while (0)
-#endif
-
-// Out-of-line (cold) path of the Matern warps: for the pairs whose (scaled) k* exceeds v_thresh, replace it by the value
-// computed from r^2 = sum_j (z~_j - x~_j)^2, with z~ = hi + lo read back from the TMEM planes at z_taddr
-// and x~ in FP32 from global memory.  Called by all 32 lanes of a warp together (TMEM loads are
-// warp-wide); a lane without marked pairs only takes part in the loads.
-__device__ __noinline__ void refine_close_pairs(float* kv, float v_thresh, float kvscale, uint32_t z_taddr, int DP,
-                                                const float* __restrict__ xrow0)
-{
-    uint32_t close = 0;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) close |= (kv[i] > v_thresh) ? (1u << i) : 0u;
-    float r2x[16];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) r2x[i] = 0.f;
-    for (int j16 = 0; j16 < DP / 16; ++j16) {
-        uint32_t zh[8], zl[8];
-        tc_ld8(z_taddr + j16 * 8, zh);
-        tc_ld8(z_taddr + DP / 2 + j16 * 8, zl);
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        float z[16];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&zh[e]));
-            const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&zl[e]));
-            z[2 * e] = a.x + b.x;
-            z[2 * e + 1] = a.y + b.y;
-        }
-        for (uint32_t rest = close; rest; rest &= rest - 1) {
-            const int i = __ffs(rest) - 1;
-            const float4* xp = reinterpret_cast<const float4*>(xrow0 + (size_t)i * DP + j16 * 16);
-            float acc = 0.f;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float4 x4 = __ldg(xp + e);
-                float df = z[4 * e] - x4.x;
-                acc = fmaf(df, df, acc);
-                df = z[4 * e + 1] - x4.y;
-                acc = fmaf(df, df, acc);
-                df = z[4 * e + 2] - x4.z;
-                acc = fmaf(df, df, acc);
-                df = z[4 * e + 3] - x4.w;
-                acc = fmaf(df, df, acc);
-            }
-            r2x[i] += acc;
-        }
-    }
-    for (uint32_t rest = close; rest; rest &= rest - 1) {
-        const int i = __ffs(rest) - 1;
-        const float u = sqrtf(r2x[i]);
-        kv[i] = kvscale * fmaf(u, fmaf(u, kPolyC2, kPolyC1), 1.f) * exp2f(-u);
-    }
-}
 
 // NV: rows of W per pass (TMEM columns of the V accumulator).  G: number of Matern warp groups; group
 // g owns chunks t = g (mod G) and k* buffer g.  KD: observations per distance product.  KT: the k*
@@ -471,7 +209,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
         constexpr uint32_t IDESC_D = instr_desc_f16(KD);
         // descriptor low word = start >> 4 | (k-slice distance >> 4) << 16
         const uint32_t zH = tmem + ZCOL, zL = zH + (uint32_t)DP / 2;
-        const uint32_t x_lo0 = ((base + map.x) >> 4) | (((KD * 16u) >> 4) << 16);
+        const uint32_t x_lo0 = desc_addr(base + map.x) | (((KD * 16u) >> 4) << 16);
         const int ksteps = DP / 16;
         long long tile_iter = 0;
         int st = 0, db = 0;
@@ -515,8 +253,8 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
     } else if (warp == 2 && lane == 0) {
         // ------------------------------------------------------------ MMA issuer: variance product
         constexpr uint32_t IDESC_V = instr_desc_f16(NV);
-        const uint32_t k_lo0 = ((base + map.k) >> 4) | ((2048u >> 4) << 16);
-        const uint32_t w_lo0 = ((base + map.w) >> 4) | (((NV * 16u) >> 4) << 16);
+        const uint32_t k_lo0 = desc_addr(base + map.k) | ((2048u >> 4) << 16);
+        const uint32_t w_lo0 = desc_addr(base + map.w) | (((NV * 16u) >> 4) << 16);
         uint32_t v_ph = 0;    // parity of the pass counter (V accumulator hand-over)
         int w_s = 0, k_s = 0;
         uint32_t w_ph = 0, k_ph = 0;
@@ -692,6 +430,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     tc_fence_after();
                     const bool fresh = c >= p * CPP;   // first time this chunk is generated for the tile
                     uint8_t* kb = sm + map.k + grp * 16384u + row * 16;
+                    uint32_t kh[KC / 16][8], kl[KC / 16][8];
 #pragma unroll
                     for (int h = 0; h < KC / 16; ++h) {
                         float dot[16];
@@ -745,36 +484,35 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                             a2_acc += (double)(apart * inv_kscale * inv_kscale);
                             s2_acc += (double)(spart * inv_kscale * inv_kscale);
                         }
-                        TICK(2);
-                        if (h == 0) {
-                            ok = mbar_wait(bar(BAR_K_EMPTY + grp), own_ph ^ 1u, abort_flag);
-                            ok = __all_sync(0xffffffffu, ok);
-                            if (!ok) break;
-                            TICK(3);
+                        // split into the two FP16 planes; the stores wait until the whole chunk is computed
+                        // so that the arithmetic does not sit between the buffer's release and its refill
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            __half2 hi, lo;
+                            split2(kv[2 * e], kv[2 * e + 1], hi, lo);
+                            kh[h][e] = *reinterpret_cast<const uint32_t*>(&hi);
+                            kl[h][e] = *reinterpret_cast<const uint32_t*>(&lo);
                         }
+                    }
+                    TICK(2);
+                    ok = mbar_wait(bar(BAR_K_EMPTY + grp), own_ph ^ 1u, abort_flag);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    TICK(3);
+#pragma unroll
+                    for (int h = 0; h < KC / 16; ++h) {
                         if (KT) {
                             // 16 columns = 8 packed TMEM columns of each plane
-                            uint32_t kh[8], kl[8];
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) {
-                                __half2 hi, lo;
-                                split2(kv[2 * e], kv[2 * e + 1], hi, lo);
-                                kh[e] = *reinterpret_cast<const uint32_t*>(&hi);
-                                kl[e] = *reinterpret_cast<const uint32_t*>(&lo);
-                            }
-                            tc_st8(lane_addr + KCOL + (uint32_t)grp * KC + h * 8, kh);
-                            tc_st8(lane_addr + KCOL + (uint32_t)grp * KC + KC / 2 + h * 8, kl);
+                            tc_st8(lane_addr + KCOL + (uint32_t)grp * KC + h * 8, kh[h]);
+                            tc_st8(lane_addr + KCOL + (uint32_t)grp * KC + KC / 2 + h * 8, kl[h]);
                         } else {
                             // 16 columns = two 16-byte k-slices of the A operand, hi and lo planes
 #pragma unroll
                             for (int sl = 0; sl < 2; ++sl) {
-                                __half2 hi2[4], lo2[4];
-#pragma unroll
-                                for (int e = 0; e < 4; ++e)
-                                    split2(kv[8 * sl + 2 * e], kv[8 * sl + 2 * e + 1], hi2[e], lo2[e]);
-                                *reinterpret_cast<uint4*>(kb + (2 * h + sl) * 2048u) = *reinterpret_cast<const uint4*>(hi2);
+                                *reinterpret_cast<uint4*>(kb + (2 * h + sl) * 2048u) =
+                                    make_uint4(kh[h][4 * sl], kh[h][4 * sl + 1], kh[h][4 * sl + 2], kh[h][4 * sl + 3]);
                                 *reinterpret_cast<uint4*>(kb + 8192u + (2 * h + sl) * 2048u) =
-                                    *reinterpret_cast<const uint4*>(lo2);
+                                    make_uint4(kl[h][4 * sl], kl[h][4 * sl + 1], kl[h][4 * sl + 2], kl[h][4 * sl + 3]);
                             }
                         }
                     }
@@ -1192,9 +930,18 @@ r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, floa
         if (cudaMalloc(&prm.trace, sizeof(long long) * grid * 32) != cudaSuccess) prm.trace = nullptr;
         if (prm.trace) cudaMemset(prm.trace, 0, sizeof(long long) * grid * 32);
     }
-    void (*kernel)(const TcParams) = kernel_for(t->NV, t->G, t->kt);
+    // The paired kernel (two CTAs of a cluster share a tile and the k* chunks) serves histories with at least
+    // two passes; R3_TC_PAIR=0/1 overrides the choice.
+    int pair_ws = 0;
+    const bool pair = env_int("R3_TC_PAIR", 0) != 0 && tc_pair_fits(t, &pair_ws);
     prof_begin(gp, stream);
-    R3_LAUNCH(kernel, grid, 128 + 128 * t->G, t->smem_bytes, stream, prm);
+    if (pair) {
+        const r3_status_t st = launch_tc_pair(t, prm, sms, stream);
+        if (st != R3_OK) return st;
+    } else {
+        void (*kernel)(const TcParams) = kernel_for(t->NV, t->G, t->kt);
+        R3_LAUNCH(kernel, grid, 128 + 128 * t->G, t->smem_bytes, stream, prm);
+    }
     prof_end(gp, stream);
     if (prm.trace) {
         std::vector<long long> h((size_t)grid * 32);
@@ -1203,11 +950,12 @@ r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, floa
         const char* names[4] = {"mmaV", "matern0", "matern1", "mmaD"};
         fprintf(stderr, "trace shape NV=%d G=%d KD=%d kt=%d ws=%d DP=%d P=%d smem=%zu\n", t->NV, t->G, t->KD, (int)t->kt, t->ws,
                 t->DP, t->P, t->smem_bytes);
-        for (int r = 0; r < 4; ++r) {
-            fprintf(stderr, "trace cta0 %s:", names[r]);
-            for (int i = 0; i < 8; ++i) fprintf(stderr, " %lld", h[(size_t)r * 8 + i]);
-            fprintf(stderr, "\n");
-        }
+        for (int cta = 0; cta < (pair ? 2 : 1); ++cta)
+            for (int r = 0; r < 4; ++r) {
+                fprintf(stderr, "trace cta%d %s:", cta, names[r]);
+                for (int i = 0; i < 8; ++i) fprintf(stderr, " %lld", h[((size_t)cta * 4 + r) * 8 + i]);
+                fprintf(stderr, "\n");
+            }
     }
     return guard_and_rescue(gp, Xcand, m, gb, mu, sigma, ei, stream);
 }
