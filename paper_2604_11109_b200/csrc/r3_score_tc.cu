@@ -252,7 +252,6 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
             for (int i = 0; i < 8; ++i) prm.trace[((size_t)blockIdx.x * 4 + 3) * 8 + i] = tacc[i];
     } else if (warp == 2 && lane == 0) {
         // ------------------------------------------------------------ MMA issuer: variance product
-        constexpr uint32_t IDESC_V = instr_desc_f16(NV);
         const uint32_t k_lo0 = desc_addr(base + map.k) | ((2048u >> 4) << 16);
         const uint32_t w_lo0 = desc_addr(base + map.w) | (((NV * 16u) >> 4) << 16);
         uint32_t v_ph = 0;    // parity of the pass counter (V accumulator hand-over)
@@ -276,7 +275,12 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     if (++w_s == ws) { w_s = 0; w_ph ^= 1u; }
                     TICK(5);
                     tc_fence_after();
-                    const uint32_t bH = w_lo0 + ((s * map.w_stage) >> 4), bL = bH + (((uint32_t)KC * NV * 2u) >> 4);
+                    // In the pass's diagonal block the rows of W above the chunk's columns are zero (W is lower
+                    // triangular): the MMAs start at the first row that can be non-zero and get narrower.
+                    const uint32_t skip = c > p * CPP ? (uint32_t)(c - p * CPP) * KC : 0u;
+                    const uint32_t idesc_v = instr_desc_f16(NV - skip);
+                    const uint32_t vcol = tmem + skip;
+                    const uint32_t bH = w_lo0 + ((s * map.w_stage) >> 4) + skip, bL = bH + (((uint32_t)KC * NV * 2u) >> 4);
                     if (KT) {
                         const uint32_t aH = tmem + KCOL + (uint32_t)b * KC, aL = aH + KC / 2;
 #pragma unroll
@@ -284,7 +288,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                             const uint32_t a0 = combo == 2 ? aL : aH, b0 = combo == 1 ? bL : bH;
 #pragma unroll
                             for (int jj = 0; jj < KC / 16; ++jj)
-                                tc_mma_f16_ts(tmem, a0 + jj * 8u, pack64(b0 + jj * ((2u * NV * 16u) >> 4), kDescHi), IDESC_V,
+                                tc_mma_f16_ts(vcol, a0 + jj * 8u, pack64(b0 + jj * ((2u * NV * 16u) >> 4), kDescHi), idesc_v,
                                               (c > 0 || combo > 0 || jj > 0) ? 1u : 0u);
                         }
                     } else {
@@ -294,8 +298,8 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                             const uint32_t a0 = combo == 2 ? aL : aH, b0 = combo == 1 ? bL : bH;
 #pragma unroll
                             for (int jj = 0; jj < KC / 16; ++jj)
-                                tc_mma_f16(tmem, pack64(a0 + jj * (4096u >> 4), kDescHi),
-                                           pack64(b0 + jj * ((2u * NV * 16u) >> 4), kDescHi), IDESC_V,
+                                tc_mma_f16(vcol, pack64(a0 + jj * (4096u >> 4), kDescHi),
+                                           pack64(b0 + jj * ((2u * NV * 16u) >> 4), kDescHi), idesc_v,
                                            (c > 0 || combo > 0 || jj > 0) ? 1u : 0u);
                         }
                     }
@@ -431,15 +435,17 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     const bool fresh = c >= p * CPP;   // first time this chunk is generated for the tile
                     uint8_t* kb = sm + map.k + grp * 16384u + row * 16;
                     uint32_t kh[KC / 16][8], kl[KC / 16][8];
+                    // both halves of the chunk's dot products in one round trip to TMEM, then the buffer is free
+                    float dots[KC / 16][16];
+#pragma unroll
+                    for (int h = 0; h < KC / 16; ++h) tc_ld16_issue(lane_addr + NV + db * KD + slice * KC + h * 16, dots[h]);
+                    tc_wait_ld32(dots[0], dots[1]);
+                    tc_fence_before();
+                    mbar_arrive(bar(BAR_D_EMPTY + db));
+                    TICK(1);
 #pragma unroll
                     for (int h = 0; h < KC / 16; ++h) {
-                        float dot[16];
-                        tc_ld16(lane_addr + NV + db * KD + slice * KC + h * 16, dot);
-                        if (h == KC / 16 - 1) {
-                            tc_fence_before();
-                            mbar_arrive(bar(BAR_D_EMPTY + db));
-                        }
-                        TICK(1);
+                        const float* dot = dots[h];
                         float kv[16];   // k* times kvscale (the power of two of its FP16 split)
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
@@ -538,13 +544,23 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                 TICK(5);
                 tc_fence_after();
 #pragma unroll 1
-                for (int c0 = grp * 16; c0 < NV; c0 += 16 * G) {
-                    float v[16];
-                    tc_ld16(lane_addr + c0, v);
-                    float part = 0.f;
+                for (int c0 = grp * 16; c0 < NV; c0 += 32 * G) {   // two column blocks per round trip to TMEM
+                    const int c1 = c0 + 16 * G;
+                    float v[16], w[16];
+                    float part0 = 0.f, part1 = 0.f;
+                    if (c1 < NV) {
+                        tc_ld16_issue(lane_addr + c0, v);
+                        tc_ld16_issue(lane_addr + c1, w);
+                        tc_wait_ld32(v, w);
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) part = fmaf(v[i], v[i], part);
-                    q_acc += (double)part;
+                        for (int i = 0; i < 16; ++i) part1 = fmaf(w[i], w[i], part1);
+                    } else {
+                        tc_ld16(lane_addr + c0, v);
+                    }
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) part0 = fmaf(v[i], v[i], part0);
+                    q_acc += (double)part0;
+                    q_acc += (double)part1;
                 }
                 tc_fence_before();
                 mbar_arrive(bar(BAR_V_EMPTY));

@@ -105,12 +105,6 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
         }
     }
 }
-__device__ __forceinline__ void st_cluster_v4(uint32_t cluster_addr, uint4 v)
-{
-    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "r"(v.x), "r"(v.y), "r"(v.z),
-                 "r"(v.w)
-                 : "memory");
-}
 __device__ __forceinline__ void mbar_arrive_expect_tx_cluster(uint32_t cluster_bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.release.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_bar), "r"(bytes)
@@ -487,14 +481,17 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
                     const bool fresh = c >= 2 * j * CPP2;   // first super-pass that generates this chunk
                     uint8_t* kb = sm + map.k + b * 16384u + row * 16;
                     uint32_t kh[KC / 16][8], kl[KC / 16][8];
+                    // both halves of the chunk's dot products in one round trip to TMEM, then the buffer is free
+                    float dots[KC / 16][16];
+#pragma unroll
+                    for (int h = 0; h < KC / 16; ++h) tc_ld16_issue(lane_addr + NV2 + db * KD2 + grp * KC + h * 16, dots[h]);
+                    tc_wait_ld32(dots[0], dots[1]);
+                    tc_fence_before();
+                    mbar_arrive(bar(PB_D_EMPTY + db));
+                    TICK(1);
 #pragma unroll
                     for (int h = 0; h < KC / 16; ++h) {
-                        float dot[16];
-                        tc_ld16(lane_addr + NV2 + db * KD2 + grp * KC + h * 16, dot);
-                        if (h == KC / 16 - 1) {
-                            tc_fence_before();
-                            mbar_arrive(bar(PB_D_EMPTY + db));
-                        }
+                        const float* dot = dots[h];
                         float kv[16];
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
