@@ -150,6 +150,177 @@ def run_reference(args, c):
     }))
 
 
+def run_tpe(args, c):
+    """Parzen-estimator scoring of the workload's pool (one history, GP 0): fit once, then per step one
+    r3_tpe_score over the pool and one r3_topk of the scores.  `--impl reference` times the FP64 oracle."""
+    from paper_2604_11109_b200 import workloads as w
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    g = w.generate_gp(c, 0)
+    levels = w.tpe_levels(c)
+    n, d, m, k = c.n, c.d, c.m, c.k
+    evals = float(sum(n + 2 for l in levels if l == 0))      # exponentials per candidate
+    base = {"metric": "tpe_candidates_scored_per_sec", "unit": "candidates/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "data": "synthetic",
+            "config": {"workload": c.name + "-tpe", "n": n, "d": d, "m": m, "k": k, "gamma": 0.25,
+                       "ordinal_dims": int((levels == 0).sum()), "categorical_dims": int((levels != 0).sum())}}
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        from oracle import tpe_oracle as T
+        model = T.tpe_fit(g["X"], g["y"], levels, 0.25, 1.0)
+        per_step = min(m, 256 if n >= 2048 else 4096)
+        t0 = None
+        for i in range(args.warmup + args.steps):
+            if i == args.warmup:
+                t0 = time.perf_counter()
+            lo = (i * per_step) % max(m - per_step + 1, 1)
+            T.tpe_topk(T.tpe_score(model, g["Xcand"][lo:lo + per_step]), min(k, per_step))
+        el = time.perf_counter() - t0
+        value = per_step * args.steps / el
+        sample = f"{per_step} candidates per step of {c.name} (n={n}, d={d}), fit excluded"
+        base.update({"impl": "reference", "value": value, "ms_per_step": 1e3 * el / args.steps, "dtype": "f64",
+                     "cpu_baseline": {"value": value, "unit": "candidates/s", "cores": 1, "kind": "oracle",
+                                      "sample": sample},
+                     "e2e": {"value": value, "unit": "candidates/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                     "gpu_launches": 0})
+        print(json.dumps(base))
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2604_11109_b200 import binding as b
+    from paper_2604_11109_b200.sharding import merge_topk
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    pool = g["Xcand"] if rank == 0 else w.generate_gp(c, rank)["Xcand"]   # weak scaling: one pool per rank
+    X, y, xc = torch.from_numpy(g["X"]).cuda(), torch.from_numpy(g["y"]).cuda(), torch.from_numpy(pool).cuda()
+    b.r3_tpe_fit(X, y, levels).close()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    ev[0].record()
+    tpe = b.r3_tpe_fit(X, y, levels, 0.25, 1.0)
+    ev[1].record()
+    torch.cuda.synchronize()
+    fit_ms = ev[0].elapsed_time(ev[1])
+    score = torch.empty((m,), device="cuda")
+    scratch = torch.empty((b.r3_topk_scratch_bytes(1, m, k),), dtype=torch.uint8, device="cuda")
+    kernel_ms = []
+
+    def step(timed=False):
+        if timed:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+        b.r3_tpe_score(tpe, xc, score)
+        if timed:
+            e1.record()
+            kernel_ms.append((e0, e1))
+        idx, val = b.r3_topk(score, k, scratch)
+        if world > 1:
+            merge_topk(val, idx, k, rank * m, topk_fn=lambda v, kk: b.r3_topk(v, kk)[0])
+        return idx, val
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    b.r3_tpe_check(tpe)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    b.r3_launch_count_reset()
+    barrier()
+    ev[2].record()
+    for _ in range(args.steps):
+        step(True)
+    ev[3].record()
+    barrier()
+    launches = b.r3_launch_count()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = ev[2].elapsed_time(ev[3])
+    if world > 1:
+        t = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    k_ms = sum(a.elapsed_time(z) for a, z in kernel_ms) / len(kernel_ms)
+
+    # end to end: pool from pinned host memory, selected indices and values back to the host
+    xh = torch.from_numpy(pool).pin_memory()
+    ih, vh = torch.empty((k,), dtype=torch.int32).pin_memory(), torch.empty((k,)).pin_memory()
+    xd = torch.empty_like(xc)
+
+    def e2e_step():
+        xd.copy_(xh, non_blocking=True)
+        b.r3_tpe_score(tpe, xd, score)
+        idx, val = b.r3_topk(score, k, scratch)
+        ih.copy_(idx, non_blocking=True)
+        vh.copy_(val, non_blocking=True)
+
+    e2e_steps = max(2, min(args.steps, 5))
+    e2e_step()
+    barrier()
+    ev[0].record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    ev[1].record()
+    barrier()
+    e2e_ms = ev[0].elapsed_time(ev[1]) / e2e_steps
+    if world > 1:
+        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    if rank != 0:
+        tpe.close()
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    sm_mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
+    peak = 148 * 16 * sm_mhz * 1e6 / 1e12
+    achieved = evals * m / (k_ms * 1e-3) / 1e12
+    cpu = None
+    if not args.no_cpu_baseline:
+        from oracle import tpe_oracle as T
+        model = T.tpe_fit(g["X"], g["y"], levels, 0.25, 1.0)
+        chunk, done, t0 = (256 if n >= 2048 else 4096), 0, time.perf_counter()
+        while True:
+            lo = done % max(m - chunk, 1)
+            T.tpe_score(model, pool[lo:lo + chunk])
+            done += min(chunk, m - lo)
+            el = time.perf_counter() - t0
+            if el >= 10.0 or done >= m:
+                break
+        cpu = {"value": done / el, "unit": "candidates/s", "cores": 1, "kind": "oracle",
+               "sample": f"{done} candidates of {c.name} in {el:.1f} s (numpy FP64, fit excluded)"}
+    base.update({
+        "value": world * m / (ms_per_step * 1e-3), "n_gpus": world, "ms_per_step": ms_per_step, "dtype": "f32",
+        "fit_ms": fit_ms, "clocks": clocks,
+        "config": dict(base["config"], l2="pool (%.0f MB) exceeds the 126 MB L2" % (xc.numel() * 4 / 1e6)
+                       if xc.numel() * 4 > 126e6 else "pool smaller than L2; not flushed"),
+        "e2e": {"value": world * m / (e2e_ms * 1e-3), "unit": "candidates/s", "h2d_bytes_per_step": int(xh.numel() * 4),
+                "d2h_bytes_per_step": int(k * 8), "ms_per_step": e2e_ms},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "alu", "kernel": "tpe_score_kernel", "achieved": achieved, "peak": peak,
+                     "unit": "Texp2/s", "frac": achieved / peak, "traffic": None,
+                     "note": "one MUFU.EX2 per (candidate, ordinal dimension, component); peak = 148 SMs x 16 MUFU "
+                             "results per clock x max SM clock",
+                     "kernel_ms_per_launch": k_ms, "kernel_share_of_step": k_ms / ms_per_step},
+        "cpu_baseline": cpu, "peaks": "derived",
+    })
+    print(json.dumps(base))
+    tpe.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -160,11 +331,16 @@ def main():
     ap.add_argument("--engine", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--m", type=int, default=None, help="override the pool size (profiling of small cases)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--surrogate", default="gp", choices=["gp", "tpe"],
+                    help="gp: the headline GP-EI path; tpe: Parzen-estimator scoring of the same pools")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" and args.m is None else args.warmup
 
     from paper_2604_11109_b200 import workloads as w
     c = w.get_config(args.config, m=args.m)
+    if args.surrogate == "tpe":
+        run_tpe(args, c)
+        return
     if args.impl == "reference":
         run_reference(args, c)
         return

@@ -203,6 +203,77 @@ void r3_launch_count_reset(void);
 
 void r3_gp_free(r3_gp_t* gp);
 
+/* ------------------------------------------------------------------------------------------------
+ * Tree-structured Parzen Estimator (TPE) candidate scoring.
+ *
+ * Section VII-C: inside the replay server the paper's experiments tune pass order and launch
+ * parameters with parallel Tree Parzen Estimation for 30 iterations.  The paper prints no formula,
+ * quantile, bandwidth rule or prior for it; the definition implemented here is this library's own
+ * statement of the estimator, steps (T1)-(T4):
+ *
+ *   (T1) n_good = min(max(1, ceil(gamma*n)), n); sort the history by y ascending (ties: lower
+ *        index); the first n_good observations are the "good" set, the rest the "bad" set.
+ *   (T2) ordinal / continuous dimension (levels[j] == 0), per set with s values: a mixture of s + 1
+ *        normal densities truncated to [0, 1] -- one per value (weight 1) and a prior (weight
+ *        prior_weight, mean 1/2, sigma 1).  With the s + 1 means sorted ascending (the prior after
+ *        equal values), a value's sigma is the larger gap to its neighbours, clipped to
+ *        [1/min(100, s + 1), 1].
+ *   (T3) categorical dimension (levels[j] == C, 2 <= C <= 64): level v = clamp(floor(x*(C-1) + 1/2),
+ *        0, C-1) with the product and the sum each rounded to FP32;
+ *        P(v) = (count_v + prior_weight/C) / (s + prior_weight).
+ *   (T4) score(x) = sum_j [ ln l_j(x_j) - ln g_j(x_j) ], l from the good set, g from the bad set.
+ *        Larger is better; pass the scores to r3_topk to pick the next points.
+ *
+ * Features are expected in [0, 1] (normalised); values outside are evaluated with the same formulas.
+ */
+typedef struct r3_tpe r3_tpe_t; /* opaque; owns device memory */
+
+/*
+ * r3_tpe_fit -- steps (T1)-(T3) on the device: order of the history, mixtures and level tables.
+ *
+ *   X       device [n][d]   observed configurations, row-major
+ *   y       device [n]      observed values (smaller is better)
+ *   levels  host   [d]      0 = ordinal/continuous, C in [2, 64] = categorical with C levels
+ *   1 <= n <= 4096, 1 <= d <= 256, 0 < gamma <= 1, prior_weight > 0
+ *   out     receives the handle (NULL on error)
+ *
+ * Synchronises `cuda_stream` before returning; a NaN/Inf in X or y returns R3_ERR_NONFINITE.
+ */
+r3_status_t r3_tpe_fit(const float* X, const float* y, const int* levels, int n, int d, float gamma,
+                       float prior_weight, void* cuda_stream, r3_tpe_t** out);
+
+/*
+ * r3_tpe_score -- step (T4) for every candidate of a pool.
+ *
+ *   Xcand  device [m][d], 1 <= m < 2^31        score  device [m] (FP32, caller-allocated)
+ *
+ * Asynchronous on `cuda_stream`; does not synchronise and does not allocate.  A non-finite candidate
+ * is latched in the handle and reported by r3_tpe_check.
+ */
+r3_status_t r3_tpe_score(r3_tpe_t* tpe, const float* Xcand, long long m, float* score, void* cuda_stream);
+
+/* Synchronises the stream and returns (and clears) the status latched by device code since the last
+ * check: R3_OK or R3_ERR_NONFINITE. */
+r3_status_t r3_tpe_check(r3_tpe_t* tpe, void* cuda_stream);
+
+/*
+ * r3_tpe_get_model -- copy the fitted model to host memory (for inspection and tests); synchronises.
+ * Any output pointer may be NULL.
+ *
+ *   n_good  host [1]
+ *   order   host [n]              history indices by y ascending
+ *   comps   host [d][n + 2][4]    per dimension the good set's components then the bad set's
+ *                                 (n_good + 1 and n - n_good + 1 of them, each set sorted by mean):
+ *                                 {mean, log2(e)/(2 sigma^2), log2(weight/(sigma Z sqrt(2 pi))), sigma};
+ *                                 all zero for a categorical dimension
+ *   table   host [d][64]          ln P_good(v) - ln P_bad(v) per level v of a categorical
+ *                                 dimension; zero elsewhere
+ */
+r3_status_t r3_tpe_get_model(r3_tpe_t* tpe, int* n_good, int* order, float* comps, float* table);
+
+/* Frees the handle and its device memory; NULL is allowed. */
+void r3_tpe_free(r3_tpe_t* tpe);
+
 const char* r3_status_string(r3_status_t status);
 const char* r3_last_error(void);
 int r3_version(void);

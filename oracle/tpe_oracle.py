@@ -14,9 +14,11 @@ listed here and each function says which step it is.
 
 Definition (features are normalised to [0, 1]; smaller y is better):
 
-  (T1) split      n_good = min(max(1, ceil(gamma * n)), n).  Sort the history by y
-                  ascending, ties by lower index; the first n_good observations
-                  are the "good" set, the rest the "bad" set (possibly empty).
+  (T1) split      n_good = min(max(1, ceil(gamma * n)), n), with gamma first rounded
+                  to FP32 (the type it has at the library's boundary) and the
+                  product taken in FP64.  Sort the history by y ascending, ties by
+                  lower index; the first n_good observations are the "good" set,
+                  the rest the "bad" set (possibly empty).
   (T2) ordinal / continuous dimension (levels == 0), for one set with values
                   p_1..p_s: the mixture has s + 1 components -- one per value
                   (weight 1, mean p_i) and a prior (weight prior_weight, mean
@@ -83,7 +85,7 @@ def split(y: np.ndarray, gamma: float):
     """(T1): the order of the history and the size of the good set."""
     y = np.asarray(y, dtype=np.float64)
     n = y.shape[0]
-    n_good = min(max(1, int(math.ceil(gamma * n))), n)
+    n_good = min(max(1, int(math.ceil(float(np.float32(gamma)) * n))), n)
     order = np.argsort(y, kind="stable")
     return order, n_good
 

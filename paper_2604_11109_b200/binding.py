@@ -38,6 +38,12 @@ SIGNATURES = {
     "r3_gp_score": (_i, [_vp, _vp, _ll, _vp, _vp, _vp, _vp]),
     "r3_topk": (_i, [_vp, _i, _ll, _i, _vp, _vp, _vp, _ull, _vp]),
     "r3_topk_scratch_bytes": (_ull, [_i, _ll, _i]),
+    "r3_tpe_fit": (_i, [_vp, _vp, ctypes.POINTER(ctypes.c_int), _i, _i, ctypes.c_float, ctypes.c_float, _vp,
+                        ctypes.POINTER(_vp)]),
+    "r3_tpe_score": (_i, [_vp, _vp, _ll, _vp, _vp]),
+    "r3_tpe_check": (_i, [_vp, _vp]),
+    "r3_tpe_get_model": (_i, [_vp, ctypes.POINTER(ctypes.c_int), _vp, _vp, _vp]),
+    "r3_tpe_free": (None, [_vp]),
     "r3_topk_noalloc": (_i, [_vp, _i, _ll, _i, _vp, _vp, _vp]),
     "r3_gp_score_topk": (_i, [_vp, _vp, _ll, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "r3_gp_score_topk_host": (_i, [_vp, _vp, _ll, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -288,6 +294,76 @@ def r3_launch_count_reset():
 
 def r3_gp_free(gp: GP):
     gp.close()
+
+
+class TPE:
+    """Owner of one ``r3_tpe_t*``; freed on ``close()`` or garbage collection."""
+
+    def __init__(self, handle: int, n: int, d: int):
+        self._h = ctypes.c_void_p(handle)
+        self.n, self.d = n, d
+
+    @property
+    def handle(self):
+        if not self._h:
+            raise ValueError("TPE handle already freed")
+        return self._h
+
+    def close(self):
+        if self._h:
+            load().r3_tpe_free(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def r3_tpe_fit(X, y, levels, gamma: float = 0.25, prior_weight: float = 1.0) -> TPE:
+    """X [n][d] and y [n] CUDA float32; levels host int array [d] (0 = ordinal, C >= 2 = categorical)."""
+    n, d = X.shape
+    if tuple(y.shape) != (n,):
+        raise ValueError("y must be [n]")
+    lv = np.ascontiguousarray(np.asarray(levels, dtype=np.int32))
+    if lv.shape != (d,):
+        raise ValueError("levels must be [d]")
+    out = ctypes.c_void_p()
+    _check(load().r3_tpe_fit(_dev_f32(X, "X"), _dev_f32(y, "y"), lv.ctypes.data_as(ctypes.POINTER(ctypes.c_int)), n, d,
+                             float(gamma), float(prior_weight), _stream(), ctypes.byref(out)))
+    return TPE(out.value, n, d)
+
+
+def r3_tpe_score(tpe: TPE, Xcand, out=None):
+    """Log-density ratio of every candidate: Xcand [m][d] CUDA float32 -> score [m]."""
+    import torch
+    m, d = Xcand.shape
+    if d != tpe.d:
+        raise ValueError("Xcand must be [m][d]")
+    if out is None:
+        out = torch.empty((m,), dtype=torch.float32, device=Xcand.device)
+    _check(load().r3_tpe_score(tpe.handle, _dev_f32(Xcand, "Xcand"), m, _dev_f32(out, "score"), _stream()))
+    return out
+
+
+def r3_tpe_check(tpe: TPE):
+    _check(load().r3_tpe_check(tpe.handle, _stream()))
+
+
+def r3_tpe_get_model(tpe: TPE):
+    """Host copies of the fitted model: (n_good, order [n], comps [d][n+2][4], table [d][64])."""
+    n_good = ctypes.c_int()
+    order = np.empty((tpe.n,), dtype=np.int32)
+    comps = np.empty((tpe.d, tpe.n + 2, 4), dtype=np.float32)
+    table = np.empty((tpe.d, 64), dtype=np.float32)
+    _check(load().r3_tpe_get_model(tpe.handle, ctypes.byref(n_good), ctypes.c_void_p(order.ctypes.data),
+                                   ctypes.c_void_p(comps.ctypes.data), ctypes.c_void_p(table.ctypes.data)))
+    return n_good.value, order, comps, table
+
+
+def r3_tpe_free(tpe: TPE):
+    tpe.close()
 
 
 def r3_version() -> int:

@@ -15,7 +15,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libr3gp.so")
-SOURCES = ["r3_api.cu", "r3_fit.cu", "r3_score_simt.cu", "r3_rescue.cu", "r3_score_tc.cu", "r3_score_tc2.cu", "r3_topk.cu"]
+SOURCES = ["r3_api.cu", "r3_fit.cu", "r3_score_simt.cu", "r3_rescue.cu", "r3_score_tc.cu", "r3_score_tc2.cu", "r3_topk.cu",
+           "r3_tpe.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
 

@@ -1,0 +1,449 @@
+// Tree-structured Parzen Estimator: fit (order of the history, per-dimension mixtures and level
+// tables) and candidate scoring (log-density ratio), steps (T1)-(T4) of the definition in r3.h.
+//
+// Fit is small (n <= 4096): one block sorts the history by y, then one block per dimension sorts each
+// set's values (bitonic network in shared memory), derives the bandwidths from the neighbour gaps in
+// FP64 and stores every component as {mean, a, b, sigma} with
+//     a = log2(e) / (2 sigma^2),   b = log2( weight / (sum of weights * sigma * Z * sqrt(2 pi)) ),
+// so that the scoring kernel evaluates a component as exp2(b - a (x - mean)^2): one subtraction, one
+// multiplication, one fused multiply-add, one MUFU.EX2 and one addition per (candidate, component).
+// Scoring is bound by the MUFU unit (16 results per clock per SM); the components of a dimension are
+// staged through shared memory and every thread carries one or two candidates.
+#include <math.h>
+
+#include <new>
+#include <vector>
+
+#include "r3_internal.cuh"
+
+struct r3_tpe {
+    int n = 0, d = 0, n_good = 0, device = 0;
+    float prior_weight = 1.f;
+    std::vector<int> levels;
+    int* levels_d = nullptr;   // [d]
+    int* order_d = nullptr;    // [n] history indices by y ascending
+    float4* comps_d = nullptr; // [d][n + 2]: good set's components, then the bad set's
+    float* table_d = nullptr;  // [d][64] ln P_good - ln P_bad per level
+    int* status_d = nullptr;   // status bits
+    int* status_h = nullptr;   // pinned mirror
+};
+
+namespace r3 {
+
+namespace {
+
+constexpr int kTpeMaxN = 4096;
+constexpr int kTpeMaxLevels = 64;
+constexpr int kSortThreads = 1024;
+constexpr int kScoreThreads = 256;
+constexpr int kStage = 512;   // components per shared-memory stage
+
+// Unsigned integer with the same order as the float (-0 and +0 equal).
+__device__ __forceinline__ unsigned ordered_bits(float v)
+{
+    if (v == 0.0f) v = 0.0f;
+    const unsigned u = __float_as_uint(v);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float from_ordered_bits(unsigned u)
+{
+    return __uint_as_float((u & 0x80000000u) ? (u & 0x7FFFFFFFu) : ~u);
+}
+
+// Ascending bitonic sort of `count` (a power of two) 64-bit keys in shared memory.
+__device__ void bitonic_sort_asc(unsigned long long* s, int count)
+{
+    for (int size = 2; size <= count; size <<= 1) {
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            __syncthreads();
+            for (int t = threadIdx.x; t < count / 2; t += blockDim.x) {
+                const int lo = 2 * t - (t & (stride - 1));
+                const int hi = lo + stride;
+                const bool asc = ((lo & size) == 0);
+                const unsigned long long a = s[lo], b = s[hi];
+                if ((a > b) == asc) {
+                    s[lo] = b;
+                    s[hi] = a;
+                }
+            }
+        }
+    }
+    __syncthreads();
+}
+
+__device__ __forceinline__ int pow2_at_least(int v)
+{
+    int p = 1;
+    while (p < v) p <<= 1;
+    return p;
+}
+
+// (T1) order[i] = index of the i-th smallest y, ties by lower index.
+__global__ void __launch_bounds__(kSortThreads) tpe_order_kernel(const float* __restrict__ y, int n,
+                                                                 int* __restrict__ order, int* __restrict__ status)
+{
+    __shared__ unsigned long long keys[kTpeMaxN];
+    const int count = pow2_at_least(n);
+    bool bad = false;
+    for (int i = threadIdx.x; i < count; i += blockDim.x) {
+        unsigned long long k = ~0ull;
+        if (i < n) {
+            const float v = y[i];
+            bad |= !isfinite(v);
+            k = ((unsigned long long)ordered_bits(v) << 32) | (unsigned)i;
+        }
+        keys[i] = k;
+    }
+    if (bad) atomicOr(status, DEV_NONFINITE);
+    bitonic_sort_asc(keys, count);
+    for (int i = threadIdx.x; i < n; i += blockDim.x) order[i] = (int)(keys[i] & 0xFFFFFFFFull);
+}
+
+// (T2), (T3): one block per dimension, both sets in turn.
+__global__ void __launch_bounds__(kSortThreads) tpe_mixture_kernel(const float* __restrict__ X,
+                                                                   const int* __restrict__ order, int n, int d,
+                                                                   int n_good, const int* __restrict__ levels,
+                                                                   double prior_weight, float4* __restrict__ comps,
+                                                                   float* __restrict__ table, int* __restrict__ status)
+{
+    extern __shared__ unsigned long long keys[];   // pow2 >= n + 1 keys
+    __shared__ int counts[kTpeMaxLevels];
+    __shared__ double lnp_good[kTpeMaxLevels];
+    const int j = blockIdx.x;
+    const int C = levels[j];
+    bool bad = false;
+    for (int set = 0; set < 2; ++set) {
+        const int s = set == 0 ? n_good : n - n_good;
+        const int first = set == 0 ? 0 : n_good;            // position in `order`
+        float4* out = comps + (size_t)j * (n + 2) + (set == 0 ? 0 : n_good + 1);
+        if (C > 0) {
+            // ---- (T3) smoothed level frequencies
+            for (int v = threadIdx.x; v < kTpeMaxLevels; v += blockDim.x) counts[v] = 0;
+            __syncthreads();
+            for (int i = threadIdx.x; i < s; i += blockDim.x) {
+                const float x = X[(size_t)order[first + i] * d + j];
+                bad |= !isfinite(x);
+                const float lv = floorf(__fadd_rn(__fmul_rn(x, (float)(C - 1)), 0.5f));
+                const int v = (int)fminf(fmaxf(lv, 0.f), (float)(C - 1));
+                atomicAdd(&counts[isfinite(x) ? v : 0], 1);
+            }
+            __syncthreads();
+            for (int v = threadIdx.x; v < C; v += blockDim.x) {
+                const double lnp = log(((double)counts[v] + prior_weight / C) / ((double)s + prior_weight));
+                if (set == 0)
+                    lnp_good[v] = lnp;
+                else
+                    table[(size_t)j * kTpeMaxLevels + v] = (float)(lnp_good[v] - lnp);
+            }
+            __syncthreads();
+            continue;
+        }
+        // ---- (T2) sort the s values and the prior mean; the prior (index s) goes after equal values
+        const int count = pow2_at_least(s + 1);
+        for (int i = threadIdx.x; i < count; i += blockDim.x) {
+            unsigned long long k = ~0ull;
+            if (i < s) {
+                const float x = X[(size_t)order[first + i] * d + j];
+                bad |= !isfinite(x);
+                k = ((unsigned long long)ordered_bits(isfinite(x) ? x : 0.f) << 32) | (unsigned)i;
+            } else if (i == s) {
+                k = ((unsigned long long)ordered_bits(0.5f) << 32) | (unsigned)s;
+            }
+            keys[i] = k;
+        }
+        bitonic_sort_asc(keys, count);
+        const double sigma_lo = 1.0 / fmin(100.0, (double)s + 1.0);
+        const double wsum = (double)s + prior_weight;
+        for (int t = threadIdx.x; t <= s; t += blockDim.x) {
+            const unsigned long long k = keys[t];
+            const bool is_prior = (int)(k & 0xFFFFFFFFull) == s;
+            const double mu = (double)from_ordered_bits((unsigned)(k >> 32));
+            double sigma = 1.0;
+            if (!is_prior) {
+                double gap = -1.0;
+                if (t > 0) gap = fmax(gap, mu - (double)from_ordered_bits((unsigned)(keys[t - 1] >> 32)));
+                if (t < s) gap = fmax(gap, (double)from_ordered_bits((unsigned)(keys[t + 1] >> 32)) - mu);
+                sigma = fmin(fmax(gap, sigma_lo), 1.0);
+            }
+            const double w = is_prior ? prior_weight : 1.0;
+            const double Z = 0.5 * erfc(-(1.0 - mu) / sigma * 0.70710678118654752440) -
+                             0.5 * erfc(-(0.0 - mu) / sigma * 0.70710678118654752440);
+            const double a = 1.4426950408889634074 / (2.0 * sigma * sigma);
+            const double b = log2(w / (wsum * sigma * Z * 2.5066282746310005024));
+            out[t] = make_float4((float)mu, (float)a, (float)b, (float)sigma);
+        }
+        __syncthreads();
+    }
+    if (bad) atomicOr(status, DEV_NONFINITE);
+}
+
+__device__ __forceinline__ float ex2_fast(float x)
+{
+    float r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ float lg2_fast(float x)
+{
+    float r;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+
+// sum over `count` components of exp2(b - a (x - mean)^2) for R candidates at once.  The components are
+// staged through shared memory by the whole block (all of its threads must call this together): one
+// broadcast LDS.128 per component instead of a global load per thread was worth 14 % on the full pool.
+template <int R>
+__device__ __forceinline__ void mixture_sums_staged(const float4* __restrict__ comp, int count, const float (&x)[R],
+                                                    float (&sum)[R], float4* stage)
+{
+    // four partial sums per candidate: independent add chains, and half the rounding of one long sum
+    float part[4][R];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int r = 0; r < R; ++r) part[u][r] = 0.f;
+    for (int c0 = 0; c0 < count; c0 += kStage) {
+        const int nc = min(kStage, count - c0);
+        __syncthreads();
+        for (int i = threadIdx.x; i < nc; i += kScoreThreads) stage[i] = __ldg(comp + c0 + i);
+        __syncthreads();
+        int c = 0;
+        for (; c + 4 <= nc; c += 4) {
+            float4 q[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) q[u] = stage[c + u];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    const float t = x[r] - q[u].x;
+                    part[u][r] += ex2_fast(fmaf(-t, t * q[u].y, q[u].z));
+                }
+            }
+        }
+        for (; c < nc; ++c) {
+            const float4 q = stage[c];
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const float t = x[r] - q.x;
+                part[c & 3][r] += ex2_fast(fmaf(-t, t * q.y, q.z));
+            }
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) sum[r] = (part[0][r] + part[1][r]) + (part[2][r] + part[3][r]);
+}
+
+// (T4) score of every candidate.  A block covers R * blockDim.x consecutive candidates; thread t holds
+// candidates t, t + blockDim.x, ... of the block's range so that the result stores coalesce.
+template <int R>
+__global__ void __launch_bounds__(kScoreThreads) tpe_score_kernel(const float* __restrict__ Xc, long long m, int n,
+                                                                  int d, int n_good, const int* __restrict__ levels,
+                                                                  const float4* __restrict__ comps,
+                                                                  const float* __restrict__ table,
+                                                                  float* __restrict__ score, int* __restrict__ status)
+{
+    const long long tiles = (m + (long long)R * kScoreThreads - 1) / ((long long)R * kScoreThreads);
+    bool bad = false;
+    __shared__ float4 stage[kStage];
+    for (long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+        const long long base = tile * (long long)R * kScoreThreads + threadIdx.x;
+        const float* row[R];
+        bool valid[R];
+        float acc[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const long long cand = base + (long long)r * kScoreThreads;
+            valid[r] = cand < m;
+            row[r] = Xc + (size_t)(valid[r] ? cand : 0) * d;
+            acc[r] = 0.f;
+        }
+        for (int j = 0; j < d; ++j) {
+            float x[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                x[r] = row[r][j];
+                bad |= valid[r] && !isfinite(x[r]);
+            }
+            const int C = __ldg(levels + j);
+            if (C > 0) {
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    const float lv = floorf(__fadd_rn(__fmul_rn(x[r], (float)(C - 1)), 0.5f));
+                    const int v = isfinite(x[r]) ? (int)fminf(fmaxf(lv, 0.f), (float)(C - 1)) : 0;
+                    acc[r] += __ldg(table + (size_t)j * kTpeMaxLevels + v);
+                }
+            } else {
+                const float4* cj = comps + (size_t)j * (n + 2);
+                float sl[R], sg[R];
+                mixture_sums_staged<R>(cj, n_good + 1, x, sl, stage);
+                mixture_sums_staged<R>(cj + n_good + 1, n - n_good + 1, x, sg, stage);
+#pragma unroll
+                for (int r = 0; r < R; ++r) acc[r] += 0.69314718f * (lg2_fast(sl[r]) - lg2_fast(sg[r]));
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+            if (valid[r]) score[base + (long long)r * kScoreThreads] = acc[r];
+    }
+    if (bad) atomicOr(status, DEV_NONFINITE);
+}
+
+void tpe_destroy(r3_tpe* t)
+{
+    if (!t) return;
+    cudaFree(t->levels_d);
+    cudaFree(t->order_d);
+    cudaFree(t->comps_d);
+    cudaFree(t->table_d);
+    cudaFree(t->status_d);
+    if (t->status_h) cudaFreeHost(t->status_h);
+    delete t;
+}
+
+r3_status_t tpe_fit_impl(r3_tpe* t, const float* X, const float* y, cudaStream_t stream)
+{
+    const int n = t->n, d = t->d;
+    R3_CUDA_TRY(cudaGetDevice(&t->device));
+    R3_CUDA_TRY(cudaMalloc(&t->levels_d, sizeof(int) * d));
+    R3_CUDA_TRY(cudaMalloc(&t->order_d, sizeof(int) * n));
+    R3_CUDA_TRY(cudaMalloc(&t->comps_d, sizeof(float4) * (size_t)d * (n + 2)));
+    R3_CUDA_TRY(cudaMalloc(&t->table_d, sizeof(float) * (size_t)d * kTpeMaxLevels));
+    R3_CUDA_TRY(cudaMalloc(&t->status_d, sizeof(int)));
+    R3_CUDA_TRY(cudaMallocHost(&t->status_h, sizeof(int)));
+    R3_CUDA_TRY(cudaMemcpyAsync(t->levels_d, t->levels.data(), sizeof(int) * d, cudaMemcpyHostToDevice, stream));
+    R3_CUDA_TRY(cudaMemsetAsync(t->comps_d, 0, sizeof(float4) * (size_t)d * (n + 2), stream));
+    R3_CUDA_TRY(cudaMemsetAsync(t->table_d, 0, sizeof(float) * (size_t)d * kTpeMaxLevels, stream));
+    R3_CUDA_TRY(cudaMemsetAsync(t->status_d, 0, sizeof(int), stream));
+    R3_LAUNCH(tpe_order_kernel, 1, kSortThreads, 0, stream, y, n, t->order_d, t->status_d);
+    int count = 1;
+    while (count < n + 1) count <<= 1;
+    const size_t smem = sizeof(unsigned long long) * (size_t)count;
+    if (smem > 48 * 1024)
+        R3_CUDA_TRY(cudaFuncSetAttribute(tpe_mixture_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    R3_LAUNCH(tpe_mixture_kernel, d, kSortThreads, smem, stream, X, t->order_d, n, d, t->n_good, t->levels_d,
+              (double)t->prior_weight, t->comps_d, t->table_d, t->status_d);
+    R3_CUDA_TRY(cudaMemcpyAsync(t->status_h, t->status_d, sizeof(int), cudaMemcpyDeviceToHost, stream));
+    R3_CUDA_TRY(cudaStreamSynchronize(stream));
+    if (*t->status_h & DEV_NONFINITE) {
+        set_error("r3_tpe_fit: X or y contains NaN or Inf");
+        return R3_ERR_NONFINITE;
+    }
+    return R3_OK;
+}
+
+}  // namespace
+
+}  // namespace r3
+
+using namespace r3;
+
+extern "C" {
+
+r3_status_t r3_tpe_fit(const float* X, const float* y, const int* levels, int n, int d, float gamma,
+                       float prior_weight, void* cuda_stream, r3_tpe_t** out)
+{
+    if (out) *out = nullptr;
+    if (!X || !y || !levels || !out) {
+        set_error("r3_tpe_fit: NULL argument");
+        return R3_ERR_INVALID_ARG;
+    }
+    if (n < 1 || n > kTpeMaxN || d < 1 || d > kMaxD) {
+        set_error("r3_tpe_fit: need 1 <= n <= %d and 1 <= d <= %d (got n=%d, d=%d)", kTpeMaxN, kMaxD, n, d);
+        return R3_ERR_INVALID_ARG;
+    }
+    if (!(gamma > 0.f && gamma <= 1.f) || !(prior_weight > 0.f) || !isfinite(prior_weight)) {
+        set_error("r3_tpe_fit: need 0 < gamma <= 1 and a finite prior_weight > 0");
+        return R3_ERR_INVALID_ARG;
+    }
+    for (int j = 0; j < d; ++j)
+        if (levels[j] != 0 && (levels[j] < 2 || levels[j] > kTpeMaxLevels)) {
+            set_error("r3_tpe_fit: levels[%d] = %d; allowed are 0 and 2..%d", j, levels[j], kTpeMaxLevels);
+            return R3_ERR_INVALID_ARG;
+        }
+    r3_tpe* t = new (std::nothrow) r3_tpe;
+    if (!t) {
+        set_error("r3_tpe_fit: out of host memory");
+        return R3_ERR_ALLOC;
+    }
+    t->n = n;
+    t->d = d;
+    t->prior_weight = prior_weight;
+    const long long ng = (long long)ceil((double)gamma * (double)n);
+    t->n_good = (int)(ng < 1 ? 1 : (ng > n ? n : ng));
+    t->levels.assign(levels, levels + d);
+    const r3_status_t st = tpe_fit_impl(t, X, y, (cudaStream_t)cuda_stream);
+    if (st != R3_OK) {
+        tpe_destroy(t);
+        return st;
+    }
+    *out = t;
+    return R3_OK;
+}
+
+r3_status_t r3_tpe_score(r3_tpe_t* tpe, const float* Xcand, long long m, float* score, void* cuda_stream)
+{
+    if (!tpe || !Xcand || !score) {
+        set_error("r3_tpe_score: NULL argument");
+        return R3_ERR_INVALID_ARG;
+    }
+    if (m < 1 || m >= (1ll << 31)) {
+        set_error("r3_tpe_score: need 1 <= m < 2^31 (got %lld)", m);
+        return R3_ERR_INVALID_ARG;
+    }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    // Two candidates per thread (one shared-memory read serves both) when that still gives every SM
+    // several blocks; one per thread for small pools.  More per thread measured slower on the full pool
+    // (fewer, longer blocks balance worse over the 148 SMs).
+    const long long tiles2 = (m + 2ll * kScoreThreads - 1) / (2ll * kScoreThreads);
+    if (tiles2 >= 148ll * 4) {
+        const unsigned grid = (unsigned)(tiles2 < 148ll * 64 ? tiles2 : 148ll * 64);
+        R3_LAUNCH(tpe_score_kernel<2>, grid, kScoreThreads, 0, stream, Xcand, m, tpe->n, tpe->d, tpe->n_good,
+                  tpe->levels_d, tpe->comps_d, tpe->table_d, score, tpe->status_d);
+    } else {
+        const long long tiles1 = (m + kScoreThreads - 1) / kScoreThreads;
+        R3_LAUNCH(tpe_score_kernel<1>, (unsigned)tiles1, kScoreThreads, 0, stream, Xcand, m, tpe->n, tpe->d,
+                  tpe->n_good, tpe->levels_d, tpe->comps_d, tpe->table_d, score, tpe->status_d);
+    }
+    return R3_OK;
+}
+
+r3_status_t r3_tpe_check(r3_tpe_t* tpe, void* cuda_stream)
+{
+    if (!tpe) {
+        set_error("r3_tpe_check: NULL handle");
+        return R3_ERR_INVALID_ARG;
+    }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    R3_CUDA_TRY(cudaMemcpyAsync(tpe->status_h, tpe->status_d, sizeof(int), cudaMemcpyDeviceToHost, stream));
+    R3_CUDA_TRY(cudaMemsetAsync(tpe->status_d, 0, sizeof(int), stream));
+    R3_CUDA_TRY(cudaStreamSynchronize(stream));
+    if (*tpe->status_h & DEV_NONFINITE) {
+        set_error("r3_tpe_score: a candidate contains NaN or Inf");
+        return R3_ERR_NONFINITE;
+    }
+    return R3_OK;
+}
+
+r3_status_t r3_tpe_get_model(r3_tpe_t* tpe, int* n_good, int* order, float* comps, float* table)
+{
+    if (!tpe) {
+        set_error("r3_tpe_get_model: NULL handle");
+        return R3_ERR_INVALID_ARG;
+    }
+    R3_CUDA_TRY(cudaDeviceSynchronize());
+    if (n_good) *n_good = tpe->n_good;
+    if (order) R3_CUDA_TRY(cudaMemcpy(order, tpe->order_d, sizeof(int) * tpe->n, cudaMemcpyDeviceToHost));
+    if (comps)
+        R3_CUDA_TRY(cudaMemcpy(comps, tpe->comps_d, sizeof(float4) * (size_t)tpe->d * (tpe->n + 2),
+                               cudaMemcpyDeviceToHost));
+    if (table)
+        R3_CUDA_TRY(cudaMemcpy(table, tpe->table_d, sizeof(float) * (size_t)tpe->d * kTpeMaxLevels,
+                               cudaMemcpyDeviceToHost));
+    return R3_OK;
+}
+
+void r3_tpe_free(r3_tpe_t* tpe) { tpe_destroy(tpe); }
+
+}  // extern "C"

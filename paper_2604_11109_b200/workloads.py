@@ -117,6 +117,15 @@ def feature_levels(c: Config):
     return lv
 
 
+def tpe_levels(c: Config) -> np.ndarray:
+    """Kind of each feature for the Parzen estimator: 0 = ordinal (more than two admissible values),
+    2 = a binary flag, treated as a two-level categorical.  The permutation features of config 4 are
+    all ordinal."""
+    if c.cfg == 4:
+        return np.zeros(c.d, dtype=np.int32)
+    return np.array([0 if len(l) > 2 else 2 for l in feature_levels(c)], dtype=np.int32)
+
+
 def _draw_level_idx(rng, levels, count):
     return np.stack([rng.integers(0, len(l), size=count) for l in levels], axis=1)
 

@@ -1,0 +1,210 @@
+"""GPU parity of TPE candidate scoring: the CUDA library through its C ABI against the FP64 oracle.
+
+Integer results (the order of the history, the good-set size, the selected top-k where the oracle's
+gap exceeds the tolerance) must match exactly.  Floating point: the fitted model is computed in FP64
+on both sides and stored in FP32 on the device (relative 2e-7 on a mean, bandwidth or coefficient);
+the score is a sum over d dimensions of differences of log-sums evaluated in FP32 with MUFU
+exponentials.  One log-sum is off by about 5e-7 (rounding of the exponents, 2^-24 of a magnitude
+up to 10, and the MUFU results) plus 3e-8 * sqrt(n) (FP32 accumulation of up to n + 1 positive
+terms); the 2 * d_ord log-sums of a score err independently, so the score is held to four standard
+deviations of that,
+
+    |score - oracle| <= 4 * sqrt(2 * d_ord) * (5e-7 + 3e-8 * sqrt(n)) + 5e-6 * |oracle|,
+
+d_ord the number of ordinal dimensions (at least 1).
+"""
+import numpy as np
+import pytest
+
+from oracle import tpe_oracle as T
+from paper_2604_11109_b200 import binding as b
+from paper_2604_11109_b200 import workloads as w
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+RTOL = 5e-6
+
+
+def atol(n, levels):
+    d_ord = max(1, int((np.asarray(levels) == 0).sum()))
+    return 4.0 * np.sqrt(2.0 * d_ord) * (5e-7 + 3e-8 * np.sqrt(n))
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def rand_case(seed, n, d, m, frac_cat=0.4, continuous=True):
+    rng = np.random.default_rng(seed)
+    levels = np.zeros(d, dtype=np.int32)
+    X = np.empty((n, d))
+    Xc = np.empty((m, d))
+    for j in range(d):
+        if rng.random() < frac_cat:
+            C = int(rng.integers(2, 9))
+            levels[j] = C
+            X[:, j] = rng.integers(0, C, size=n) / (C - 1)
+            Xc[:, j] = rng.integers(0, C, size=m) / (C - 1)
+        elif continuous and rng.random() < 0.5:
+            X[:, j] = rng.random(n)
+            Xc[:, j] = rng.random(m)
+        else:
+            L = int(rng.integers(3, 17))
+            X[:, j] = rng.integers(0, L, size=n) / (L - 1)
+            Xc[:, j] = rng.integers(0, L, size=m) / (L - 1)
+    y = np.round(rng.normal(0, 1, n), 1)      # rounded: ties in y
+    return X.astype(np.float32), y.astype(np.float32), levels, Xc.astype(np.float32)
+
+
+def check_model(tpe, model, n, d):
+    n_good, order, comps, table = b.r3_tpe_get_model(tpe)
+    assert n_good == model.n_good
+    assert order.tolist() == model.order.tolist()
+    for j in range(d):
+        if model.levels[j]:
+            C = int(model.levels[j])
+            want = np.log(model.good[j].prob) - np.log(model.bad[j].prob)
+            np.testing.assert_allclose(table[j, :C], want, rtol=1e-6, atol=1e-6)
+            assert not comps[j].any()
+            continue
+        off = 0
+        for mix in (model.good[j], model.bad[j]):
+            cnt = mix.mu.shape[0]
+            got = comps[j, off:off + cnt].astype(np.float64)
+            off += cnt
+            # the device keeps each set sorted by mean, the prior after equal values
+            srt = np.lexsort((np.arange(cnt), mix.mu))
+            np.testing.assert_array_equal(got[:, 0], mix.mu[srt])
+            # equal means may come in any order; their bandwidths as a multiset must agree
+            key_got = np.lexsort((got[:, 3], got[:, 0]))
+            key_ref = np.lexsort((mix.sigma[srt], mix.mu[srt]))
+            np.testing.assert_allclose(got[key_got, 3], mix.sigma[srt][key_ref], rtol=2e-7)
+            a = np.log2(np.e) / (2 * mix.sigma ** 2)
+            bb = np.log2(mix.weight / (mix.sigma * mix.Z * np.sqrt(2 * np.pi)))
+            np.testing.assert_allclose(np.sort(got[:, 1]), np.sort(a), rtol=3e-7)
+            np.testing.assert_allclose(np.sort(got[:, 2]), np.sort(bb), rtol=3e-7, atol=3e-7)
+        assert not table[j].any()
+
+
+def check_score(got, want, ATOL):
+    err = np.abs(got.astype(np.float64) - want)
+    tol = ATOL + RTOL * np.abs(want)
+    worst = float((err / tol).max())
+    assert worst <= 1.0, f"score error {worst:.2f} x tolerance (max abs {err.max():.3e})"
+    return worst
+
+
+def check_topk(score_gpu, idx_gpu, want, k, ATOL):
+    """Exact where the oracle separates rank k from rank k + 1 by more than the tolerance."""
+    ref = T.tpe_topk(want, min(k + 1, want.shape[0]))
+    tol = ATOL + RTOL * np.abs(want[ref]).max()
+    sel = want[idx_gpu]
+    assert len(set(idx_gpu.tolist())) == k
+    if ref.shape[0] > k and want[ref[k - 1]] - want[ref[k]] > 2 * tol:
+        assert set(idx_gpu.tolist()) == set(ref[:k].tolist())
+    # every selected candidate is within tolerance of belonging; order by the device's own scores
+    assert sel.min() >= want[ref[k - 1]] - 2 * tol
+    s = score_gpu[idx_gpu]
+    assert np.all(s[:-1] >= s[1:])
+    eq = s[:-1] == s[1:]
+    assert np.all(idx_gpu[:-1][eq] < idx_gpu[1:][eq])
+
+
+@pytest.mark.parametrize("seed,n,d,m,gamma,w0", [
+    (0, 1, 1, 5, 0.25, 1.0),            # one observation: the bad set is the prior alone
+    (1, 2, 3, 17, 1.0, 1.0),            # gamma = 1: everything is good
+    (2, 37, 5, 1025, 0.25, 1.0),        # one candidate past a block's range
+    (3, 200, 7, 4099, 0.15, 2.5),
+    (4, 513, 13, 3000, 0.5, 0.3),
+    (5, 4096, 3, 2048, 0.25, 1.0),      # largest history
+])
+def test_small_cases(seed, n, d, m, gamma, w0):
+    X, y, levels, Xc = rand_case(seed, n, d, m)
+    model = T.tpe_fit(X, y, levels, gamma, w0)
+    tpe = b.r3_tpe_fit(dev(X), dev(y), levels, gamma, w0)
+    check_model(tpe, model, n, d)
+    got = b.r3_tpe_score(tpe, dev(Xc)).cpu().numpy()
+    b.r3_tpe_check(tpe)
+    want = T.tpe_score(model, Xc)
+    check_score(got, want, atol(n, levels))
+    k = min(8, m)
+    idx, val = b.r3_topk(dev(got), k)
+    check_topk(got, idx.cpu().numpy().astype(np.int64), want, k, atol(n, levels))
+    tpe.close()
+
+
+def test_all_categorical_and_all_ordinal():
+    for frac in (0.0, 1.0):
+        X, y, levels, Xc = rand_case(40 + int(frac), 150, 6, 777, frac_cat=frac)
+        model = T.tpe_fit(X, y, levels, 0.25, 1.0)
+        tpe = b.r3_tpe_fit(dev(X), dev(y), levels, 0.25, 1.0)
+        check_model(tpe, model, 150, 6)
+        check_score(b.r3_tpe_score(tpe, dev(Xc)).cpu().numpy(), T.tpe_score(model, Xc), atol(150, levels))
+        tpe.close()
+
+
+def test_candidates_outside_the_unit_interval():
+    X, y, levels, Xc = rand_case(50, 90, 4, 600, frac_cat=0.25)
+    Xc = (Xc * 1.3 - 0.15).astype(np.float32)
+    model = T.tpe_fit(X, y, levels, 0.25, 1.0)
+    tpe = b.r3_tpe_fit(dev(X), dev(y), levels, 0.25, 1.0)
+    check_score(b.r3_tpe_score(tpe, dev(Xc)).cpu().numpy(), T.tpe_score(model, Xc), atol(90, levels))
+    tpe.close()
+
+
+@pytest.mark.parametrize("cfg,sample", [(1, 4096), (2, 8192), (5, 1024)])
+def test_workloads_full_size(cfg, sample):
+    """The launch configuration the benchmark times, on the whole pool; the oracle on a seeded sample."""
+    c = w.get_config(cfg)
+    g = w.generate_gp(c, 0)
+    levels = w.tpe_levels(c)
+    model = T.tpe_fit(g["X"], g["y"], levels, 0.25, 1.0)
+    tpe = b.r3_tpe_fit(dev(g["X"]), dev(g["y"]), levels, 0.25, 1.0)
+    check_model(tpe, model, c.n, c.d)
+    got = b.r3_tpe_score(tpe, dev(g["Xcand"])).cpu().numpy()
+    b.r3_tpe_check(tpe)
+    assert np.isfinite(got).all()
+    sel = w.sample_indices(c, sample)
+    want = T.tpe_score(model, g["Xcand"][sel])
+    check_score(got[sel], want, atol(c.n, levels))
+    # top-k of the sampled pool, decided by the device on its own scores of the same candidates
+    k = min(c.k, 32)
+    idx, _ = b.r3_topk(dev(got[sel]), k)
+    check_topk(got[sel], idx.cpu().numpy().astype(np.int64), want, k, atol(c.n, levels))
+    # the full pool's selection is sorted, distinct and at least as good as the sample's best
+    idx_full, val_full = b.r3_topk(dev(got), k)
+    v = val_full.cpu().numpy()
+    assert np.all(v[:-1] >= v[1:]) and v[0] >= got[sel].max()
+    tpe.close()
+
+
+def test_errors():
+    X, y, levels, Xc = rand_case(60, 20, 3, 50)
+    ybad = y.copy()
+    ybad[3] = np.nan
+    with pytest.raises(b.R3Error) as e:
+        b.r3_tpe_fit(dev(X), dev(ybad), levels)
+    assert e.value.status == 2
+    Xbad = X.copy()
+    Xbad[5, 1] = np.inf
+    with pytest.raises(b.R3Error) as e:
+        b.r3_tpe_fit(dev(Xbad), dev(y), levels)
+    assert e.value.status == 2
+    for bad_levels in ([1, 0, 0], [0, 65, 0], [0, -2, 0]):
+        with pytest.raises(b.R3Error) as e:
+            b.r3_tpe_fit(dev(X), dev(y), np.array(bad_levels, dtype=np.int32))
+        assert e.value.status == 1
+    for gamma, w0 in ((0.0, 1.0), (1.5, 1.0), (0.25, 0.0)):
+        with pytest.raises(b.R3Error) as e:
+            b.r3_tpe_fit(dev(X), dev(y), levels, gamma, w0)
+        assert e.value.status == 1
+    tpe = b.r3_tpe_fit(dev(X), dev(y), levels)
+    Xc[7, 0] = np.nan
+    b.r3_tpe_score(tpe, dev(Xc))
+    with pytest.raises(b.R3Error) as e:
+        b.r3_tpe_check(tpe)
+    assert e.value.status == 2
+    b.r3_tpe_score(tpe, dev(np.nan_to_num(Xc)))
+    b.r3_tpe_check(tpe)      # the latch was cleared
+    tpe.close()

@@ -123,7 +123,7 @@ def test_score_prefers_the_good_cluster():
 def _brute_force(X, y, levels, gamma, w0, cand):
     """The definition again in plain loops and scalars (tiny inputs only)."""
     n, d = len(X), len(X[0])
-    n_good = min(max(1, math.ceil(gamma * n)), n)
+    n_good = min(max(1, math.ceil(float(np.float32(gamma)) * n)), n)   # gamma is FP32 at the boundary
     order = sorted(range(n), key=lambda i: (y[i], i))
     sets = [order[:n_good], order[n_good:]]
     out = []
