@@ -39,6 +39,10 @@ Definition (features are normalised to [0, 1]; smaller y is better):
                   candidate (the ratio l/g is monotone in Expected Improvement
                   under the estimator's model).
 
+Parity unpinned against the paper: it prints no formula or worked example for
+this estimator, so the pins below tie the oracle to its stated definition and to
+the mathematics only.
+
 Pins (tests/test_tpe_oracle_pins.py): every mixture integrates to 1 over [0, 1]
 by adaptive quadrature; the components equal SciPy's truncated normal; a
 hand-worked split, bandwidth and clipping example; categorical probabilities
