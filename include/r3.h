@@ -193,6 +193,26 @@ r3_status_t r3_gp_last_rescued(r3_gp_t* gp, void* cuda_stream, long long* total)
 r3_status_t r3_gp_profile(r3_gp_t* gp, int enable);
 r3_status_t r3_gp_profile_read(r3_gp_t* gp, double* kernel_ms, long long* launches);
 
+/*
+ * r3_gp_append -- add k observations to every GP of the handle without refactoring the history.
+ *
+ * One BO round ends with k replayed points; conditioning on them is a rank-k extension of the factor,
+ * O(k n^2), instead of the O(n^3) of a new r3_gp_fit (the loop of Section IV: propose, replay, update).
+ * With K' = [[K, B], [B^T, C]]:  L21 = (L^-1 B)^T,  L22 L22^T = C - L21 L21^T,  W' = L'^-1 by blocks,
+ * alpha' = K'^-1 y'.  The handle afterwards equals, up to FP64 rounding, the one r3_gp_fit returns for
+ * the concatenated history with the same hyper-parameters; best becomes min(y') (an incumbent set
+ * with r3_gp_set_best is replaced) and the scoring engine is chosen again for the new size.
+ *
+ *   Xnew  device [batch][k][d]     ynew  device [batch][k]      1 <= k <= 128,  n + k <= 8192
+ *
+ * Synchronises `cuda_stream`.  On any error (R3_ERR_NONFINITE, R3_ERR_NOT_PD with the failing pivot in
+ * r3_last_error, allocation failure) the handle is unchanged and still usable.
+ */
+r3_status_t r3_gp_append(r3_gp_t* gp, const float* Xnew, const float* ynew, int k, void* cuda_stream);
+
+/* Number of observations per GP currently in the handle. */
+int r3_gp_size(const r3_gp_t* gp);
+
 /* Copy fit results to host arrays (diagnostics and tests): alpha [batch][n] FP64,
  * L [batch][n][n] FP64 lower-triangular (upper part zero).  Either may be NULL. */
 r3_status_t r3_gp_get_factor(const r3_gp_t* gp, double* alpha, double* L);
@@ -273,6 +293,15 @@ r3_status_t r3_tpe_get_model(r3_tpe_t* tpe, int* n_good, int* order, float* comp
 
 /* Frees the handle and its device memory; NULL is allowed. */
 void r3_tpe_free(r3_tpe_t* tpe);
+
+/*
+ * Device memory the library has freed is kept (per device, at most 2 GiB, blocks of 1 MiB and more) and
+ * handed out again by later calls, because allocating and freeing the 100 MB arrays of a fit costs more
+ * than the kernels of an append.  r3_trim_cache returns the kept blocks of the current device to the
+ * driver; r3_cached_bytes reports how much is kept.
+ */
+void r3_trim_cache(void);
+unsigned long long r3_cached_bytes(void);
 
 const char* r3_status_string(r3_status_t status);
 const char* r3_last_error(void);

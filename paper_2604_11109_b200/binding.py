@@ -38,6 +38,10 @@ SIGNATURES = {
     "r3_gp_score": (_i, [_vp, _vp, _ll, _vp, _vp, _vp, _vp]),
     "r3_topk": (_i, [_vp, _i, _ll, _i, _vp, _vp, _vp, _ull, _vp]),
     "r3_topk_scratch_bytes": (_ull, [_i, _ll, _i]),
+    "r3_trim_cache": (None, []),
+    "r3_cached_bytes": (_ull, []),
+    "r3_gp_append": (_i, [_vp, _vp, _vp, _i, _vp]),
+    "r3_gp_size": (_i, [_vp]),
     "r3_tpe_fit": (_i, [_vp, _vp, ctypes.POINTER(ctypes.c_int), _i, _i, ctypes.c_float, ctypes.c_float, _vp,
                         ctypes.POINTER(_vp)]),
     "r3_tpe_score": (_i, [_vp, _vp, _ll, _vp, _vp]),
@@ -235,6 +239,21 @@ def r3_gp_score_topk_host(gp: GP, Xcand_host, k: int, out):
     return out
 
 
+def r3_gp_append(gp: GP, Xnew, ynew):
+    """Add k observations per GP: Xnew [batch][k][d] (or [k][d]) and ynew [batch][k] CUDA float32."""
+    if Xnew.dim() == 2:
+        Xnew, ynew = Xnew.unsqueeze(0), ynew.unsqueeze(0)
+    batch, k, d = Xnew.shape
+    if batch != gp.batch or d != gp.d or tuple(ynew.shape) != (batch, k):
+        raise ValueError("Xnew must be [batch][k][d] and ynew [batch][k]")
+    _check(load().r3_gp_append(gp.handle, _dev_f32(Xnew, "Xnew"), _dev_f32(ynew, "ynew"), k, _stream()))
+    gp.n = r3_gp_size(gp)
+
+
+def r3_gp_size(gp: GP) -> int:
+    return int(load().r3_gp_size(gp.handle))
+
+
 def r3_gp_check(gp: GP):
     _check(load().r3_gp_check(gp.handle, _stream()))
 
@@ -364,6 +383,15 @@ def r3_tpe_get_model(tpe: TPE):
 
 def r3_tpe_free(tpe: TPE):
     tpe.close()
+
+
+def r3_trim_cache():
+    """Return the device memory the library keeps for reuse to the driver."""
+    load().r3_trim_cache()
+
+
+def r3_cached_bytes() -> int:
+    return int(load().r3_cached_bytes())
 
 
 def r3_version() -> int:

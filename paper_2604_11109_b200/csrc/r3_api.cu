@@ -26,11 +26,11 @@ r3_status_t ensure_workspace(r3_gp* gp, size_t bytes)
     if (bytes <= gp->ws_bytes) return R3_OK;
     // growing synchronises the device: wait for work that may still use the old buffer
     R3_CUDA_TRY(cudaDeviceSynchronize());
-    if (gp->ws) cudaFree(gp->ws);
+    if (gp->ws) dev_free(gp->ws);
     gp->ws = nullptr;
     gp->ws_bytes = 0;
     const size_t want = (bytes + (1u << 20)) & ~((size_t)(1u << 20) - 1);
-    R3_CUDA_TRY(cudaMalloc(&gp->ws, want));
+    R3_CUDA_TRY(dev_malloc(&gp->ws, want));
     gp->ws_bytes = want;
     return R3_OK;
 }
@@ -131,24 +131,25 @@ void r3_gp_free(r3_gp_t* gp)
 {
     if (!gp) return;
     tc_release(gp);
-    cudaFree(gp->X);
-    cudaFree(gp->ell_d);
-    cudaFree(gp->inv_ell);
-    cudaFree(gp->sn2_d);
-    cudaFree(gp->sf2_d);
-    cudaFree(gp->best_d);
-    cudaFree(gp->yabs_d);
-    cudaFree(gp->wnorm_d);
-    cudaFree(gp->L64);
-    cudaFree(gp->W64);
-    cudaFree(gp->W32);
-    cudaFree(gp->alpha64);
-    cudaFree(gp->alpha32);
-    cudaFree(gp->status_d);
+    dev_free(gp->X);
+    dev_free(gp->y);
+    dev_free(gp->ell_d);
+    dev_free(gp->inv_ell);
+    dev_free(gp->sn2_d);
+    dev_free(gp->sf2_d);
+    dev_free(gp->best_d);
+    dev_free(gp->yabs_d);
+    dev_free(gp->wnorm_d);
+    dev_free(gp->L64);
+    dev_free(gp->W64);
+    dev_free(gp->W32);
+    dev_free(gp->alpha64);
+    dev_free(gp->alpha32);
+    dev_free(gp->status_d);
     if (gp->status_h) cudaFreeHost(gp->status_h);
     if (gp->rescued_h) cudaFreeHost(gp->rescued_h);
     for (cudaEvent_t e : gp->events) cudaEventDestroy(e);
-    cudaFree(gp->ws);
+    dev_free(gp->ws);
     delete gp;
 }
 
@@ -210,20 +211,21 @@ r3_status_t r3_gp_fit(const float* X, const float* y, const float* lengthscales,
     for (size_t i = 0; i < inv.size(); ++i) inv[i] = (float)(1.0 / (double)gp->ell[i]);
 
     const size_t mat = (size_t)gp->npad * gp->npad;
-    TRY_BAIL(cudaMalloc(&gp->X, sizeof(float) * batch * (size_t)n * d));
-    TRY_BAIL(cudaMalloc(&gp->ell_d, sizeof(float) * batch * d));
-    TRY_BAIL(cudaMalloc(&gp->inv_ell, sizeof(float) * batch * d));
-    TRY_BAIL(cudaMalloc(&gp->sn2_d, sizeof(float) * batch));
-    TRY_BAIL(cudaMalloc(&gp->sf2_d, sizeof(float) * batch));
-    TRY_BAIL(cudaMalloc(&gp->best_d, sizeof(float) * batch));
-    TRY_BAIL(cudaMalloc(&gp->yabs_d, sizeof(float) * batch));
-    TRY_BAIL(cudaMalloc(&gp->wnorm_d, sizeof(double) * batch));
-    TRY_BAIL(cudaMalloc(&gp->L64, sizeof(double) * batch * mat));
-    TRY_BAIL(cudaMalloc(&gp->W64, sizeof(double) * batch * mat));
-    TRY_BAIL(cudaMalloc(&gp->W32, sizeof(float) * batch * mat));
-    TRY_BAIL(cudaMalloc(&gp->alpha64, sizeof(double) * batch * gp->npad));
-    TRY_BAIL(cudaMalloc(&gp->alpha32, sizeof(float) * batch * gp->npad));
-    TRY_BAIL(cudaMalloc(&gp->status_d, 2 * sizeof(int)));
+    TRY_BAIL(dev_malloc(&gp->X, sizeof(float) * batch * (size_t)n * d));
+    TRY_BAIL(dev_malloc(&gp->y, sizeof(float) * batch * (size_t)n));
+    TRY_BAIL(dev_malloc(&gp->ell_d, sizeof(float) * batch * d));
+    TRY_BAIL(dev_malloc(&gp->inv_ell, sizeof(float) * batch * d));
+    TRY_BAIL(dev_malloc(&gp->sn2_d, sizeof(float) * batch));
+    TRY_BAIL(dev_malloc(&gp->sf2_d, sizeof(float) * batch));
+    TRY_BAIL(dev_malloc(&gp->best_d, sizeof(float) * batch));
+    TRY_BAIL(dev_malloc(&gp->yabs_d, sizeof(float) * batch));
+    TRY_BAIL(dev_malloc(&gp->wnorm_d, sizeof(double) * batch));
+    TRY_BAIL(dev_malloc(&gp->L64, sizeof(double) * batch * mat));
+    TRY_BAIL(dev_malloc(&gp->W64, sizeof(double) * batch * mat));
+    TRY_BAIL(dev_malloc(&gp->W32, sizeof(float) * batch * mat));
+    TRY_BAIL(dev_malloc(&gp->alpha64, sizeof(double) * batch * gp->npad));
+    TRY_BAIL(dev_malloc(&gp->alpha32, sizeof(float) * batch * gp->npad));
+    TRY_BAIL(dev_malloc(&gp->status_d, 2 * sizeof(int)));
     TRY_BAIL(cudaMallocHost(&gp->status_h, 2 * sizeof(int)));
     TRY_BAIL(cudaMallocHost(&gp->rescued_h, 64 * sizeof(int)));
     for (int i = 0; i < 64; ++i) gp->rescued_h[i] = 0;
@@ -231,6 +233,7 @@ r3_status_t r3_gp_fit(const float* X, const float* y, const float* lengthscales,
     gp->status_h[1] = INT_MAX;
     TRY_BAIL(cudaMemcpyAsync(gp->status_d, gp->status_h, 2 * sizeof(int), cudaMemcpyHostToDevice, stream));
     TRY_BAIL(cudaMemcpyAsync(gp->X, X, sizeof(float) * batch * (size_t)n * d, cudaMemcpyDeviceToDevice, stream));
+    TRY_BAIL(cudaMemcpyAsync(gp->y, y, sizeof(float) * batch * (size_t)n, cudaMemcpyDeviceToDevice, stream));
     TRY_BAIL(cudaMemcpyAsync(gp->ell_d, gp->ell.data(), sizeof(float) * batch * d, cudaMemcpyHostToDevice, stream));
     TRY_BAIL(cudaMemcpyAsync(gp->inv_ell, inv.data(), sizeof(float) * batch * d, cudaMemcpyHostToDevice, stream));
     TRY_BAIL(cudaMemcpyAsync(gp->sn2_d, gp->sn2.data(), sizeof(float) * batch, cudaMemcpyHostToDevice, stream));
@@ -264,6 +267,48 @@ r3_status_t r3_gp_fit(const float* X, const float* y, const float* lengthscales,
     *out = gp;
     return R3_OK;
 }
+
+r3_status_t r3_gp_append(r3_gp_t* gp, const float* Xnew, const float* ynew, int k, void* cuda_stream)
+{
+    if (!gp || !Xnew || !ynew) {
+        set_error("r3_gp_append: NULL argument");
+        return R3_ERR_INVALID_ARG;
+    }
+    if (k < 1 || k > kAppendMax || gp->n + k > kMaxN) {
+        set_error("r3_gp_append: need 1 <= k <= %d and n + k <= %d (n=%d, k=%d)", kAppendMax, kMaxN, gp->n, k);
+        return R3_ERR_INVALID_ARG;
+    }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    r3_status_t st = append_device(gp, Xnew, ynew, k, stream);
+    const int bits = gp->status_h ? gp->status_h[0] : 0;
+    const int pivot = gp->status_h ? gp->status_h[1] : 0;
+    if (st == R3_OK && (bits & (DEV_NONFINITE | DEV_NOT_PD))) {
+        // the handle was not touched; clear the latch so that it stays usable
+        gp->status_h[0] = 0;
+        gp->status_h[1] = INT_MAX;
+        R3_CUDA_TRY(cudaMemcpyAsync(gp->status_d, gp->status_h, 2 * sizeof(int), cudaMemcpyHostToDevice, stream));
+        R3_CUDA_TRY(cudaStreamSynchronize(stream));
+        if (bits & DEV_NONFINITE) {
+            set_error("r3_gp_append: Xnew or ynew contains a non-finite value");
+            return R3_ERR_NONFINITE;
+        }
+        set_error("r3_gp_append: pivot %d of the extended K + noise*I is not positive (duplicate rows with zero noise?)",
+                  pivot);
+        return R3_ERR_NOT_PD;
+    }
+    if (st != R3_OK) return st;
+    R3_CUDA_TRY(cudaMemcpy(gp->best.data(), gp->best_d, sizeof(float) * gp->batch, cudaMemcpyDeviceToHost));
+    R3_CUDA_TRY(cudaMemcpy(gp->y_absmax.data(), gp->yabs_d, sizeof(float) * gp->batch, cudaMemcpyDeviceToHost));
+    R3_CUDA_TRY(cudaMemcpy(gp->wnorm.data(), gp->wnorm_d, sizeof(double) * gp->batch, cudaMemcpyDeviceToHost));
+    tc_release(gp);
+    if (tc_supported(gp->n, gp->d)) {
+        st = tc_prepare(gp, stream);
+        if (st != R3_OK) return st;
+    }
+    return R3_OK;
+}
+
+int r3_gp_size(const r3_gp_t* gp) { return gp ? gp->n : 0; }
 
 r3_status_t r3_gp_score(r3_gp_t* gp, const float* Xcand, long long m, float* mu, float* sigma, float* ei,
                         void* cuda_stream)
@@ -304,10 +349,10 @@ r3_status_t r3_topk(const float* ei, int batch, long long m, int k, int* idx, fl
     if (scratch) return topk_device(ei, batch, m, k, idx, val, scratch, (size_t)scratch_bytes, stream);
     void* ws = nullptr;
     const size_t bytes = topk_workspace_bytes(batch, m, k);
-    R3_CUDA_TRY(cudaMalloc(&ws, bytes));
+    R3_CUDA_TRY(dev_malloc(&ws, bytes));
     st = topk_device(ei, batch, m, k, idx, val, ws, bytes, stream);
     cudaError_t e = cudaStreamSynchronize(stream);
-    cudaFree(ws);
+    dev_free(ws);
     if (st == R3_OK && e != cudaSuccess) {
         set_error("r3_topk: %s", cudaGetErrorString(e));
         st = R3_ERR_CUDA;

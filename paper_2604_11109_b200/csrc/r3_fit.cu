@@ -389,6 +389,31 @@ __global__ void to_float_kernel(const double* __restrict__ a, float* __restrict_
         b[i] = (float)a[i];
 }
 
+// From W and y: the estimate of |W|_2 (power iteration on W^T W; alpha64/alpha32 serve as scratch first),
+// alpha = W^T (W y) in FP64 and FP32, and W rounded to FP32.  u: [B][npad] scratch; slabs: [B + B*kRowSlabs*npad].
+r3_status_t finish_weights(int B, int n, int npad, const double* W64, const float* y, double* alpha64, float* alpha32,
+                           float* W32, double* wnorm_d, double* u, double* slabs, cudaStream_t stream)
+{
+    double* pv = alpha64;
+    double* lam = slabs;  // [B], followed by the row-slab partial sums
+    double* part = slabs + B;
+    R3_LAUNCH(power_init_kernel, B, 256, 0, stream, pv, n, npad);
+    R3_LAUNCH(power_normalize_kernel, B, 256, 0, stream, pv, npad, lam);
+    for (int it = 0; it < 12; ++it) {
+        R3_LAUNCH(w_times_y_kernel<double>, dim3((npad + 7) / 8, B), 256, 0, stream, W64, pv, npad, n, npad, u);
+        R3_LAUNCH(wt_times_u_partial_kernel, dim3((npad + 127) / 128, kRowSlabs, B), 128, 0, stream, W64, u, n, npad,
+                  part);
+        R3_LAUNCH(wt_times_u_reduce_kernel, dim3((npad + 127) / 128, B), 128, 0, stream, part, npad, pv, alpha32);
+        R3_LAUNCH(power_normalize_kernel, B, 256, 0, stream, pv, npad, lam);
+    }
+    R3_LAUNCH(power_finish_kernel, (B + 255) / 256, 256, 0, stream, lam, wnorm_d, B);
+    R3_LAUNCH(w_times_y_kernel<float>, dim3((npad + 7) / 8, B), 256, 0, stream, W64, y, n, n, npad, u);
+    R3_LAUNCH(wt_times_u_partial_kernel, dim3((npad + 127) / 128, kRowSlabs, B), 128, 0, stream, W64, u, n, npad, part);
+    R3_LAUNCH(wt_times_u_reduce_kernel, dim3((npad + 127) / 128, B), 128, 0, stream, part, npad, alpha64, alpha32);
+    R3_LAUNCH(to_float_kernel, 1184, 256, 0, stream, W64, W32, (size_t)B * npad * npad);
+    return R3_OK;
+}
+
 }  // namespace
 
 // Runs the whole fit on `stream`.  gp->X, ell (device copies) and the scalar arrays are already in
@@ -398,12 +423,12 @@ r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream)
     const int B = gp->batch, n = gp->n, d = gp->d, npad = gp->npad;
     const size_t mat = (size_t)npad * npad;
     double *Dinv = nullptr, *T = nullptr, *u = nullptr, *slabs = nullptr;
-    R3_CUDA_TRY(cudaMalloc(&Dinv, sizeof(double) * B * (size_t)(npad / NB) * NB * NB));
+    R3_CUDA_TRY(dev_malloc(&Dinv, sizeof(double) * B * (size_t)(npad / NB) * NB * NB));
     auto fail = [&](r3_status_t st) {
-        cudaFree(Dinv);
-        cudaFree(T);
-        cudaFree(u);
-        cudaFree(slabs);
+        dev_free(Dinv);
+        dev_free(T);
+        dev_free(u);
+        dev_free(slabs);
         return st;
     };
 #define TRY_OR_FAIL(expr)                                                                          \
@@ -425,9 +450,9 @@ r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream)
         }                                                                                          \
     } while (0)
 
-    TRY_OR_FAIL(cudaMalloc(&T, sizeof(double) * B * mat));
-    TRY_OR_FAIL(cudaMalloc(&u, sizeof(double) * B * npad));
-    TRY_OR_FAIL(cudaMalloc(&slabs, sizeof(double) * ((size_t)B + (size_t)B * kRowSlabs * npad)));
+    TRY_OR_FAIL(dev_malloc(&T, sizeof(double) * B * mat));
+    TRY_OR_FAIL(dev_malloc(&u, sizeof(double) * B * npad));
+    TRY_OR_FAIL(dev_malloc(&slabs, sizeof(double) * ((size_t)B + (size_t)B * kRowSlabs * npad)));
 
     LAUNCH_OR_FAIL(check_finite_kernel, 296, 256, gp->X, (size_t)B * n * d, gp->status_d);
     LAUNCH_OR_FAIL(check_finite_kernel, 64, 256, y, (size_t)B * n, gp->status_d);
@@ -456,34 +481,315 @@ r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream)
         LAUNCH_OR_FAIL(trtri_gemm_kernel, grid, 256, gp->W64, T, gp->W64, npad, s, npairs, 1);
     }
 
-    // spectral norm of W by power iteration on W^T W (alpha64/alpha32 serve as scratch first)
     {
-        double* pv = gp->alpha64;
-        double* lam = slabs;  // [B], followed by the row-slab partial sums
-        double* part = slabs + B;
-        LAUNCH_OR_FAIL(power_init_kernel, B, 256, pv, n, npad);
-        LAUNCH_OR_FAIL(power_normalize_kernel, B, 256, pv, npad, lam);
-        for (int it = 0; it < 12; ++it) {
-            LAUNCH_OR_FAIL(w_times_y_kernel<double>, dim3((npad + 7) / 8, B), 256, gp->W64, pv, npad, n, npad, u);
-            LAUNCH_OR_FAIL(wt_times_u_partial_kernel, dim3((npad + 127) / 128, kRowSlabs, B), 128, gp->W64, u, n,
-                           npad, part);
-            LAUNCH_OR_FAIL(wt_times_u_reduce_kernel, dim3((npad + 127) / 128, B), 128, part, npad, pv, gp->alpha32);
-            LAUNCH_OR_FAIL(power_normalize_kernel, B, 256, pv, npad, lam);
-        }
-        LAUNCH_OR_FAIL(power_finish_kernel, (B + 255) / 256, 256, lam, gp->wnorm_d, B);
+        const r3_status_t st = finish_weights(B, n, npad, gp->W64, y, gp->alpha64, gp->alpha32, gp->W32, gp->wnorm_d, u,
+                                              slabs, stream);
+        if (st != R3_OK) return fail(st);
     }
-    LAUNCH_OR_FAIL(w_times_y_kernel<float>, dim3((npad + 7) / 8, B), 256, gp->W64, y, n, n, npad, u);
-    LAUNCH_OR_FAIL(wt_times_u_partial_kernel, dim3((npad + 127) / 128, kRowSlabs, B), 128, gp->W64, u, n, npad,
-                   slabs + B);
-    LAUNCH_OR_FAIL(wt_times_u_reduce_kernel, dim3((npad + 127) / 128, B), 128, slabs + B, npad, gp->alpha64,
-                   gp->alpha32);
-    LAUNCH_OR_FAIL(to_float_kernel, 1184, 256, gp->W64, gp->W32, (size_t)B * mat);
-
     TRY_OR_FAIL(cudaMemcpyAsync(gp->status_h, gp->status_d, 2 * sizeof(int), cudaMemcpyDeviceToHost, stream));
     TRY_OR_FAIL(cudaStreamSynchronize(stream));
 #undef TRY_OR_FAIL
 #undef LAUNCH_OR_FAIL
     fail(R3_OK);  // frees the temporaries
+    return R3_OK;
+}
+
+// =====================================================================================================
+// r3_gp_append: k more observations per GP without refactoring what is already factored.
+//
+// With K' = [[K, B], [B^T, C]] (B = k(X, Xnew), C = k(Xnew, Xnew) + noise*I) and K = L L^T, W = L^-1:
+//     L21 = (W B)^T,   S = C - L21 L21^T = L22 L22^T,   L' = [[L, 0], [L21, L22]],
+//     W22 = L22^-1,    W21 = -W22 (L21 W),              W' = [[W, 0], [W21, W22]],
+// then alpha' = W'^T (W' y') as in the fit.  Two k x n x n/2 products in FP64 dominate: O(k n^2) against
+// the fit's O(n^3 / 3).  The results equal a fit of the concatenated history up to rounding.
+namespace {
+
+// k <= kAppendMax (r3_internal.cuh): S and W22 are handled by one block per GP
+
+// Copy the leading n0 x n0 blocks of the old matrices into the (zeroed) new ones and put the identity
+// on the padding rows.
+__global__ void embed_kernel(const double* __restrict__ src, int np0, double* __restrict__ dst, int np1, int n0, int n1)
+{
+    const int g = blockIdx.y;
+    const int i = blockIdx.x;
+    const double* s = src + (size_t)g * np0 * np0 + (size_t)i * np0;
+    double* t = dst + (size_t)g * np1 * np1 + (size_t)i * np1;
+    if (i < n0) {
+        for (int c = threadIdx.x; c <= i; c += blockDim.x) t[c] = s[c];
+    } else if (i >= n1 && threadIdx.x == 0) {
+        t[i] = 1.0;
+    }
+}
+
+// Rows of the new observations of K' (lower triangle): row n0 + i, columns 0 .. n0 + i.
+__global__ void cross_gram_kernel(const float* __restrict__ X, const float* __restrict__ ell,
+                                  const float* __restrict__ sf2, const float* __restrict__ sn2, int n0, int n1, int d,
+                                  int np1, double* __restrict__ K)
+{
+    const int g = blockIdx.z, i = n0 + blockIdx.y;
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c > i) return;
+    const float* Xg = X + (size_t)g * n1 * d;
+    const float* xi = Xg + (size_t)i * d;
+    const float* xc = Xg + (size_t)c * d;
+    const float* lg = ell + (size_t)g * d;
+    double r2 = 0.0;
+    for (int j = 0; j < d; ++j) {
+        const double diff = ((double)xi[j] - (double)xc[j]) / (double)lg[j];
+        r2 += diff * diff;
+    }
+    const double s = sqrt(5.0) * sqrt(r2);
+    double v = (double)sf2[g] * (1.0 + s + s * s / 3.0) * exp(-s);
+    if (c == i) v += (double)sn2[g];
+    K[(size_t)g * np1 * np1 + (size_t)i * np1 + c] = v;
+}
+
+// C[M x N] = A[M x R] * op(Wm) with the lower-triangular Wm (upper part stored as zeros):
+//   NT = true :  C[i][c] = sum_{r <= c} A[i][r] * Wm[c][r]      (A * Wm^T)
+//   NT = false:  C[i][c] = sum_{r >= c} A[i][r] * Wm[r][c]      (A * Wm)
+// FP64, 32 x 64 tile per block of 256 threads (2 x 4 per thread), reduction in steps of 16 over the part of
+// r that can be non-zero for the tile's columns.
+template <bool NT>
+__global__ void __launch_bounds__(256) tri_gemm_kernel(const double* __restrict__ A, int lda, size_t strideA,
+                                                       const double* __restrict__ Wm, int ldw, size_t strideW,
+                                                       double* __restrict__ C, int ldc, size_t strideC, int M, int N)
+{
+    __shared__ double As[32][17], Bs[16][65];
+    const int g = blockIdx.z;
+    A += (size_t)g * strideA;
+    Wm += (size_t)g * strideW;
+    C += (size_t)g * strideC;
+    const int i0 = blockIdx.y * 32, c0 = blockIdx.x * 64;
+    const int t = threadIdx.x, ty = t / 16, tx = t % 16;
+    double acc[2][4] = {};
+    const int r_begin = NT ? 0 : (c0 / 16) * 16;
+    const int r_end = NT ? min(c0 + 64, N) : N;
+    for (int r0 = r_begin; r0 < r_end; r0 += 16) {
+        for (int e = t; e < 32 * 16; e += 256) {
+            const int i = e / 16, r = e % 16;
+            As[i][r] = (i0 + i < M && r0 + r < N) ? A[(size_t)(i0 + i) * lda + r0 + r] : 0.0;
+        }
+        for (int e = t; e < 16 * 64; e += 256) {
+            if (NT) {
+                const int c = e / 16, r = e % 16;   // consecutive threads walk r: 128 contiguous bytes per row of Wm
+                Bs[r][c] = (c0 + c < N && r0 + r < N) ? Wm[(size_t)(c0 + c) * ldw + r0 + r] : 0.0;
+            } else {
+                const int r = e / 64, c = e % 64;
+                Bs[r][c] = (c0 + c < N && r0 + r < N) ? Wm[(size_t)(r0 + r) * ldw + c0 + c] : 0.0;
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int r = 0; r < 16; ++r) {
+            const double a0 = As[ty * 2][r], a1 = As[ty * 2 + 1][r];
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                const double b = Bs[r][tx * 4 + v];
+                acc[0][v] = fma(a0, b, acc[0][v]);
+                acc[1][v] = fma(a1, b, acc[1][v]);
+            }
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int u = 0; u < 2; ++u)
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            const int i = i0 + ty * 2 + u, c = c0 + tx * 4 + v;
+            if (i < M && c < N) C[(size_t)i * ldc + c] = acc[u][v];
+        }
+}
+
+// S[i][j] = C[i][j] - sum_c L21[i][c] L21[j][c] for j <= i, written over the C block of L' (one warp per entry).
+__global__ void schur_kernel(const double* __restrict__ L21, int n0, int k, double* __restrict__ Lnew, int np1)
+{
+    const int g = blockIdx.z, i = blockIdx.y;
+    const int j = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
+    const int lane = threadIdx.x % 32;
+    if (j > i) return;
+    const double* a = L21 + ((size_t)g * k + i) * n0;
+    const double* b = L21 + ((size_t)g * k + j) * n0;
+    double s = 0.0;
+    for (int c = lane; c < n0; c += 32) s = fma(a[c], b[c], s);
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) Lnew[(size_t)g * np1 * np1 + (size_t)(n0 + i) * np1 + n0 + j] -= s;
+}
+
+// In-place Cholesky of the k x k block at (n0, n0) of L' and its inverse into W' (one block per GP, k <= 128).
+__global__ void __launch_bounds__(256) small_chol_inv_kernel(double* __restrict__ Lnew, double* __restrict__ Wnew,
+                                                              int np1, int n0, int k, int* __restrict__ status)
+{
+    const int g = blockIdx.x;
+    double* S = Lnew + (size_t)g * np1 * np1 + (size_t)n0 * np1 + n0;   // S[i][j] at S[i * np1 + j]
+    double* V = Wnew + (size_t)g * np1 * np1 + (size_t)n0 * np1 + n0;
+    __shared__ double piv_s;
+    for (int j = 0; j < k; ++j) {
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            double piv = S[(size_t)j * np1 + j];
+            if (!(piv > 0.0)) {
+                atomicOr(&status[0], DEV_NOT_PD);
+                atomicMin(&status[1], n0 + j);
+                piv = 1.0;
+            }
+            piv_s = sqrt(piv);
+        }
+        __syncthreads();
+        const double l = piv_s;
+        for (int i = j + threadIdx.x; i < k; i += blockDim.x)
+            S[(size_t)i * np1 + j] = (i == j) ? l : S[(size_t)i * np1 + j] / l;
+        __syncthreads();
+        const int w = k - j - 1;
+        for (int e = threadIdx.x; e < w * w; e += blockDim.x) {
+            const int i = j + 1 + e / w, c = j + 1 + e % w;
+            if (c <= i) S[(size_t)i * np1 + c] -= S[(size_t)i * np1 + j] * S[(size_t)c * np1 + j];
+        }
+    }
+    __syncthreads();
+    // inverse by forward substitution, one column per thread: L22 v = e_c
+    for (int c = threadIdx.x; c < k; c += blockDim.x) {
+        V[(size_t)c * np1 + c] = 1.0 / S[(size_t)c * np1 + c];
+        for (int i = c + 1; i < k; ++i) {
+            double s = 0.0;
+            for (int j = c; j < i; ++j) s = fma(S[(size_t)i * np1 + j], V[(size_t)j * np1 + c], s);
+            V[(size_t)i * np1 + c] = -s / S[(size_t)i * np1 + i];
+        }
+    }
+}
+
+// Rows of L' : copy L21 [k][n0] into rows n0.. of L'.  Rows of W' : W21 = -W22 T2.
+__global__ void place_l21_kernel(const double* __restrict__ L21, int n0, int k, double* __restrict__ Lnew, int np1)
+{
+    const int g = blockIdx.z, i = blockIdx.y;
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c < n0) Lnew[(size_t)g * np1 * np1 + (size_t)(n0 + i) * np1 + c] = L21[((size_t)g * k + i) * n0 + c];
+}
+
+__global__ void w21_kernel(const double* __restrict__ T2, int n0, int k, double* __restrict__ Wnew, int np1)
+{
+    const int g = blockIdx.z, i = blockIdx.y;
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= n0) return;
+    const double* W22 = Wnew + (size_t)g * np1 * np1 + (size_t)(n0 + i) * np1 + n0;   // row i of W22
+    const double* T = T2 + (size_t)g * k * n0;
+    double s = 0.0;
+    for (int j = 0; j <= i; ++j) s = fma(W22[j], T[(size_t)j * n0 + c], s);
+    Wnew[(size_t)g * np1 * np1 + (size_t)(n0 + i) * np1 + c] = -s;
+}
+
+struct AppendBuffers {
+    float *X = nullptr, *y = nullptr, *W32 = nullptr, *alpha32 = nullptr, *best = nullptr;   // best: [2][B]
+    double *L64 = nullptr, *W64 = nullptr, *alpha64 = nullptr, *T1 = nullptr, *T2 = nullptr, *u = nullptr,
+           *slabs = nullptr, *wnorm = nullptr;
+    void release()
+    {
+        dev_free(X); dev_free(y); dev_free(W32); dev_free(alpha32); dev_free(L64); dev_free(W64); dev_free(alpha64);
+        dev_free(T1); dev_free(T2); dev_free(u); dev_free(slabs); dev_free(best); dev_free(wnorm);
+        *this = AppendBuffers();
+    }
+};
+
+}  // namespace
+
+r3_status_t append_device(r3_gp* gp, const float* Xnew, const float* ynew, int k, cudaStream_t stream)
+{
+    const size_t xnew_gp_stride = (size_t)k * gp->d, ynew_gp_stride = (size_t)k;
+    const int B = gp->batch, d = gp->d, n0 = gp->n, n1 = n0 + k, np0 = gp->npad, np1 = round_up(n1, NB);
+    const size_t mat1 = (size_t)np1 * np1;
+    AppendBuffers nb;
+    auto fail = [&](r3_status_t st) {
+        nb.release();
+        return st;
+    };
+#define TRY_OR_FAIL(expr)                                                                          \
+    do {                                                                                           \
+        cudaError_t e__ = (expr);                                                                  \
+        if (e__ != cudaSuccess) {                                                                  \
+            set_error("%s failed: %s", #expr, cudaGetErrorString(e__));                            \
+            return fail(e__ == cudaErrorMemoryAllocation ? R3_ERR_ALLOC : R3_ERR_CUDA);            \
+        }                                                                                          \
+    } while (0)
+#define LAUNCH_OR_FAIL(kernel, grid, block, ...)                                                   \
+    do {                                                                                           \
+        kernel<<<(grid), (block), 0, stream>>>(__VA_ARGS__);                                       \
+        ++g_launches;                                                                              \
+        cudaError_t e__ = cudaGetLastError();                                                      \
+        if (e__ != cudaSuccess) {                                                                  \
+            set_error("launch of %s failed: %s", #kernel, cudaGetErrorString(e__));                \
+            return fail(R3_ERR_CUDA);                                                              \
+        }                                                                                          \
+    } while (0)
+    TRY_OR_FAIL(dev_malloc(&nb.X, sizeof(float) * B * (size_t)n1 * d));
+    TRY_OR_FAIL(dev_malloc(&nb.y, sizeof(float) * B * (size_t)n1));
+    TRY_OR_FAIL(dev_malloc(&nb.L64, sizeof(double) * B * mat1));
+    TRY_OR_FAIL(dev_malloc(&nb.W64, sizeof(double) * B * mat1));
+    TRY_OR_FAIL(dev_malloc(&nb.W32, sizeof(float) * B * mat1));
+    TRY_OR_FAIL(dev_malloc(&nb.alpha64, sizeof(double) * B * np1));
+    TRY_OR_FAIL(dev_malloc(&nb.alpha32, sizeof(float) * B * np1));
+    TRY_OR_FAIL(dev_malloc(&nb.T1, sizeof(double) * B * (size_t)k * n0));
+    TRY_OR_FAIL(dev_malloc(&nb.T2, sizeof(double) * B * (size_t)k * n0));
+    TRY_OR_FAIL(dev_malloc(&nb.u, sizeof(double) * B * np1));
+    TRY_OR_FAIL(dev_malloc(&nb.slabs, sizeof(double) * ((size_t)B + (size_t)B * kRowSlabs * np1)));
+    TRY_OR_FAIL(dev_malloc(&nb.best, sizeof(float) * 2 * B));
+    TRY_OR_FAIL(dev_malloc(&nb.wnorm, sizeof(double) * B));
+    LAUNCH_OR_FAIL(check_finite_kernel, 64, 256, Xnew, (size_t)B * k * d, gp->status_d);
+    LAUNCH_OR_FAIL(check_finite_kernel, 64, 256, ynew, (size_t)B * k, gp->status_d);
+
+    // histories: old rows then new rows, per GP
+    TRY_OR_FAIL(cudaMemcpy2DAsync(nb.X, sizeof(float) * (size_t)n1 * d, gp->X, sizeof(float) * (size_t)n0 * d,
+                                  sizeof(float) * (size_t)n0 * d, B, cudaMemcpyDeviceToDevice, stream));
+    TRY_OR_FAIL(cudaMemcpy2DAsync(nb.X + (size_t)n0 * d, sizeof(float) * (size_t)n1 * d, Xnew,
+                                  sizeof(float) * xnew_gp_stride, sizeof(float) * (size_t)k * d, B,
+                                  cudaMemcpyDeviceToDevice, stream));
+    TRY_OR_FAIL(cudaMemcpy2DAsync(nb.y, sizeof(float) * n1, gp->y, sizeof(float) * n0, sizeof(float) * n0, B,
+                                  cudaMemcpyDeviceToDevice, stream));
+    TRY_OR_FAIL(cudaMemcpy2DAsync(nb.y + n0, sizeof(float) * n1, ynew, sizeof(float) * ynew_gp_stride, sizeof(float) * k,
+                                  B, cudaMemcpyDeviceToDevice, stream));
+    TRY_OR_FAIL(cudaMemsetAsync(nb.L64, 0, sizeof(double) * B * mat1, stream));
+    TRY_OR_FAIL(cudaMemsetAsync(nb.W64, 0, sizeof(double) * B * mat1, stream));
+    LAUNCH_OR_FAIL(embed_kernel, dim3(np1, B), 128, gp->L64, np0, nb.L64, np1, n0, n1);
+    LAUNCH_OR_FAIL(embed_kernel, dim3(np1, B), 128, gp->W64, np0, nb.W64, np1, n0, n1);
+    LAUNCH_OR_FAIL(min_y_kernel, B, 256, nb.y, n1, nb.best, nb.best + B);
+
+    // new rows of K', then L21 = B^T W^T
+    LAUNCH_OR_FAIL(cross_gram_kernel, dim3((n1 + 127) / 128, k, B), 128, nb.X, gp->ell_d, gp->sf2_d, gp->sn2_d, n0, n1,
+                   d, np1, nb.L64);
+    const dim3 ggrid((n0 + 63) / 64, (k + 31) / 32, B);
+    LAUNCH_OR_FAIL(tri_gemm_kernel<true>, ggrid, 256, nb.L64 + (size_t)n0 * np1, np1, mat1, nb.W64, np1, mat1, nb.T1,
+                   n0, (size_t)k * n0, k, n0);
+    LAUNCH_OR_FAIL(place_l21_kernel, dim3((n0 + 127) / 128, k, B), 128, nb.T1, n0, k, nb.L64, np1);
+    LAUNCH_OR_FAIL(schur_kernel, dim3((k + 7) / 8, k, B), 256, nb.T1, n0, k, nb.L64, np1);
+    LAUNCH_OR_FAIL(small_chol_inv_kernel, B, 256, nb.L64, nb.W64, np1, n0, k, gp->status_d);
+    // W21 = -W22 (L21 W)
+    LAUNCH_OR_FAIL(tri_gemm_kernel<false>, ggrid, 256, nb.T1, n0, (size_t)k * n0, nb.W64, np1, mat1, nb.T2, n0,
+                   (size_t)k * n0, k, n0);
+    LAUNCH_OR_FAIL(w21_kernel, dim3((n0 + 127) / 128, k, B), 128, nb.T2, n0, k, nb.W64, np1);
+    {
+        const r3_status_t st = finish_weights(B, n1, np1, nb.W64, nb.y, nb.alpha64, nb.alpha32, nb.W32, nb.wnorm,
+                                              nb.u, nb.slabs, stream);
+        if (st != R3_OK) return fail(st);
+    }
+    TRY_OR_FAIL(cudaMemcpyAsync(gp->status_h, gp->status_d, 2 * sizeof(int), cudaMemcpyDeviceToHost, stream));
+    TRY_OR_FAIL(cudaStreamSynchronize(stream));
+#undef TRY_OR_FAIL
+#undef LAUNCH_OR_FAIL
+    if (gp->status_h[0] & (DEV_NOT_PD | DEV_NONFINITE)) return fail(R3_OK);   // the caller reports; nothing swapped
+    // success: the new arrays replace the old ones
+    if (cudaMemcpy(gp->best_d, nb.best, sizeof(float) * B, cudaMemcpyDeviceToDevice) != cudaSuccess ||
+        cudaMemcpy(gp->yabs_d, nb.best + B, sizeof(float) * B, cudaMemcpyDeviceToDevice) != cudaSuccess ||
+        cudaMemcpy(gp->wnorm_d, nb.wnorm, sizeof(double) * B, cudaMemcpyDeviceToDevice) != cudaSuccess) {
+        set_error("r3_gp_append: copying the incumbent failed");
+        return fail(R3_ERR_CUDA);
+    }
+    dev_free(gp->X); dev_free(gp->y); dev_free(gp->L64); dev_free(gp->W64); dev_free(gp->W32);
+    dev_free(gp->alpha64); dev_free(gp->alpha32);
+    gp->X = nb.X; gp->y = nb.y; gp->L64 = nb.L64; gp->W64 = nb.W64; gp->W32 = nb.W32;
+    gp->alpha64 = nb.alpha64; gp->alpha32 = nb.alpha32;
+    nb.X = nullptr; nb.y = nullptr; nb.L64 = nullptr; nb.W64 = nullptr; nb.W32 = nullptr;
+    nb.alpha64 = nullptr; nb.alpha32 = nullptr;
+    nb.release();
+    gp->n = n1;
+    gp->npad = np1;
     return R3_OK;
 }
 

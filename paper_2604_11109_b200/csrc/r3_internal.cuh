@@ -51,6 +51,18 @@ constexpr int kFitBlock = 32;   // Cholesky / inverse block size; n is padded to
 constexpr int kMaxN = 8192;
 constexpr int kMaxD = 256;
 constexpr int kMaxK = 1024;
+constexpr int kAppendMax = 128;   // observations per r3_gp_append call
+
+// device-memory cache (r3_alloc.cu): cudaMalloc/cudaFree with freed blocks kept for reuse
+cudaError_t dev_malloc_bytes(void** p, size_t bytes);
+template <typename T>
+inline cudaError_t dev_malloc(T** p, size_t bytes)
+{
+    return dev_malloc_bytes(reinterpret_cast<void**>(p), bytes);
+}
+void dev_free(void* p);
+void trim_cache();
+size_t cached_bytes();
 
 inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
 inline long long round_up_ll(long long a, long long b) { return (a + b - 1) / b * b; }
@@ -67,6 +79,7 @@ struct r3_gp {
     std::vector<double> wnorm;                // [batch] estimate of |L^-1|_2 (power iteration x 1.5)
 
     float* X = nullptr;        // [batch][n][d]   raw observations (FP32 as given)
+    float* y = nullptr;        // [batch][n]      observed values as given (kept for r3_gp_append)
     float* ell_d = nullptr;    // [batch][d]      lengthscales as given
     float* inv_ell = nullptr;  // [batch][d]      1/lengthscale
     float* sn2_d = nullptr;    // [batch]
@@ -102,6 +115,9 @@ namespace r3 {
 
 // fit (r3_fit.cu)
 r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream);
+// Appends k observations per GP (r3_gp_append): extends L, W, alpha, X, y in O(k n^2); synchronises.  On
+// any error the handle is left as it was.
+r3_status_t append_device(r3_gp* gp, const float* Xnew, const float* ynew, int k, cudaStream_t stream);
 
 // SIMT scoring (r3_score_simt.cu)
 size_t score_simt_workspace_bytes(const r3_gp* gp, long long m);

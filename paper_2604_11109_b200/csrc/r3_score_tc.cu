@@ -753,16 +753,16 @@ void tc_release(r3_gp* gp)
 {
     TensorOperands* t = ops_of(gp);
     if (!t) return;
-    cudaFree(t->centre);
-    cudaFree(t->scale);
-    cudaFree(t->xt);
-    cudaFree(t->xs32);
-    cudaFree(t->xnorm);
-    cudaFree(t->xnmax);
-    cudaFree(t->alpha);
-    cudaFree(t->wt);
-    cudaFree(t->kscale);
-    cudaFree(t->vinv2);
+    dev_free(t->centre);
+    dev_free(t->scale);
+    dev_free(t->xt);
+    dev_free(t->xs32);
+    dev_free(t->xnorm);
+    dev_free(t->xnmax);
+    dev_free(t->alpha);
+    dev_free(t->wt);
+    dev_free(t->kscale);
+    dev_free(t->vinv2);
     delete t;
     gp->tc = nullptr;
 }
@@ -813,31 +813,31 @@ r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream)
     float* wscale_d = nullptr;
     auto fail = [&](const char* what, cudaError_t e) {
         set_error("%s failed: %s", what, cudaGetErrorString(e));
-        cudaFree(wmax_bits);
-        cudaFree(wscale_d);
+        dev_free(wmax_bits);
+        dev_free(wscale_d);
         tc_release(gp);
         return e == cudaErrorMemoryAllocation ? R3_ERR_ALLOC : R3_ERR_CUDA;
     };
     auto decline = [&]() {   // the SIMT engine serves this history
-        cudaFree(wmax_bits);
-        cudaFree(wscale_d);
+        dev_free(wmax_bits);
+        dev_free(wscale_d);
         tc_release(gp);
         return R3_OK;
     };
     cudaError_t e;
-    if ((e = cudaMalloc(&t->centre, sizeof(float) * B * t->DP)) != cudaSuccess) return fail("cudaMalloc", e);
-    if ((e = cudaMalloc(&t->scale, sizeof(float) * B * t->DP)) != cudaSuccess) return fail("cudaMalloc", e);
-    if ((e = cudaMalloc(&t->xt, sizeof(__half) * B * (size_t)(t->NP / t->KD) * 2 * t->DP * t->KD)) != cudaSuccess)
+    if ((e = dev_malloc(&t->centre, sizeof(float) * B * t->DP)) != cudaSuccess) return fail("cudaMalloc", e);
+    if ((e = dev_malloc(&t->scale, sizeof(float) * B * t->DP)) != cudaSuccess) return fail("cudaMalloc", e);
+    if ((e = dev_malloc(&t->xt, sizeof(__half) * B * (size_t)(t->NP / t->KD) * 2 * t->DP * t->KD)) != cudaSuccess)
         return fail("cudaMalloc", e);
-    if ((e = cudaMalloc(&t->xs32, sizeof(float) * B * (size_t)t->NP * t->DP)) != cudaSuccess) return fail("cudaMalloc", e);
-    if ((e = cudaMalloc(&t->xnorm, sizeof(float) * B * t->NP)) != cudaSuccess) return fail("cudaMalloc", e);
-    if ((e = cudaMalloc(&t->xnmax, sizeof(float) * (B > 2 ? B : 2))) != cudaSuccess) return fail("cudaMalloc", e);
-    if ((e = cudaMalloc(&t->alpha, sizeof(float) * B * t->NP)) != cudaSuccess) return fail("cudaMalloc", e);
-    if ((e = cudaMalloc(&t->wt, sizeof(__half) * B * t->wt_gp_stride)) != cudaSuccess) return fail("cudaMalloc", e);
-    if ((e = cudaMalloc(&t->kscale, sizeof(float) * B)) != cudaSuccess) return fail("cudaMalloc", e);
-    if ((e = cudaMalloc(&t->vinv2, sizeof(double) * B)) != cudaSuccess) return fail("cudaMalloc", e);
-    if ((e = cudaMalloc(&wmax_bits, sizeof(unsigned) * B)) != cudaSuccess) return fail("cudaMalloc", e);
-    if ((e = cudaMalloc(&wscale_d, sizeof(float) * B)) != cudaSuccess) return fail("cudaMalloc", e);
+    if ((e = dev_malloc(&t->xs32, sizeof(float) * B * (size_t)t->NP * t->DP)) != cudaSuccess) return fail("cudaMalloc", e);
+    if ((e = dev_malloc(&t->xnorm, sizeof(float) * B * t->NP)) != cudaSuccess) return fail("cudaMalloc", e);
+    if ((e = dev_malloc(&t->xnmax, sizeof(float) * (B > 2 ? B : 2))) != cudaSuccess) return fail("cudaMalloc", e);
+    if ((e = dev_malloc(&t->alpha, sizeof(float) * B * t->NP)) != cudaSuccess) return fail("cudaMalloc", e);
+    if ((e = dev_malloc(&t->wt, sizeof(__half) * B * t->wt_gp_stride)) != cudaSuccess) return fail("cudaMalloc", e);
+    if ((e = dev_malloc(&t->kscale, sizeof(float) * B)) != cudaSuccess) return fail("cudaMalloc", e);
+    if ((e = dev_malloc(&t->vinv2, sizeof(double) * B)) != cudaSuccess) return fail("cudaMalloc", e);
+    if ((e = dev_malloc(&wmax_bits, sizeof(unsigned) * B)) != cudaSuccess) return fail("cudaMalloc", e);
+    if ((e = dev_malloc(&wscale_d, sizeof(float) * B)) != cudaSuccess) return fail("cudaMalloc", e);
 
     // scaled observations (their largest coordinate decides whether the FP16 planes can hold them) and
     // the largest |W| of each GP (it decides the power-of-two scale of its W planes)
@@ -881,8 +881,8 @@ r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream)
     g_launches += 2;
     if ((e = cudaGetLastError()) != cudaSuccess) return fail("operand preparation launch", e);
     if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return fail("operand preparation", e);
-    cudaFree(wmax_bits);
-    cudaFree(wscale_d);
+    dev_free(wmax_bits);
+    dev_free(wscale_d);
     wmax_bits = nullptr;
     wscale_d = nullptr;
     e = cudaFuncSetAttribute(kernel_for(t->NV, t->G, t->kt), cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -943,7 +943,7 @@ r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, floa
     // R3_TC_TRACE=1 prints, for the first CTA, the cycles each role spent per wait / issue category
     prm.trace = nullptr;
     if (getenv("R3_TC_TRACE")) {
-        if (cudaMalloc(&prm.trace, sizeof(long long) * grid * 32) != cudaSuccess) prm.trace = nullptr;
+        if (dev_malloc(&prm.trace, sizeof(long long) * grid * 32) != cudaSuccess) prm.trace = nullptr;
         if (prm.trace) cudaMemset(prm.trace, 0, sizeof(long long) * grid * 32);
     }
     // The paired kernel (two CTAs of a cluster share a tile and the k* chunks) serves histories with at least
@@ -962,7 +962,7 @@ r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, floa
     if (prm.trace) {
         std::vector<long long> h((size_t)grid * 32);
         cudaMemcpy(h.data(), prm.trace, sizeof(long long) * grid * 32, cudaMemcpyDeviceToHost);
-        cudaFree(prm.trace);
+        dev_free(prm.trace);
         const char* names[4] = {"mmaV", "matern0", "matern1", "mmaD"};
         fprintf(stderr, "trace shape NV=%d G=%d KD=%d kt=%d ws=%d DP=%d P=%d smem=%zu\n", t->NV, t->G, t->KD, (int)t->kt, t->ws,
                 t->DP, t->P, t->smem_bytes);
