@@ -193,6 +193,37 @@ def topk(ei_values, k: int):
     return idx, val
 
 
+def propose(X, y, ell, sf2: float, sn2: float, Xcand, q: int, lie: str = "believer"):
+    """Greedy batch of q distinct pool members by fantasies ("parallel" BO, Section IV: several points of one
+    search are replayed at once).  The paper gives no rule for choosing them; this is the usual sequential one,
+    written as its definition:
+
+      repeat q times:  fit the (augmented) history; score the pool with the incumbent fixed at the best
+      OBSERVED value; pick the not-yet-picked candidate of largest EI (ties: lower index); append it to the
+      history with a fantasised value -- its posterior mean ("believer") or the incumbent ("liar") -- rounded
+      to FP32 like any observation.
+
+    Returns (indices int64 [q], EI of each pick at the time it was picked, FP64 [q]).
+    """
+    if lie not in ("believer", "liar"):
+        raise ValueError("lie must be 'believer' or 'liar'")
+    Xa, ya, Xcand = _f32(X).copy(), _f32(y).copy(), _f32(Xcand)
+    best0 = float(ya.min())
+    picked, values = [], []
+    for _ in range(q):
+        f = fit(Xa, ya, ell, sf2, sn2)
+        mu, _, e = score(f, Xcand, best=best0)
+        e = e.copy()
+        e[picked] = -np.inf
+        j = int(np.argmax(e))          # first maximum: the lower index wins ties
+        picked.append(j)
+        values.append(float(e[j]))
+        value = mu[j] if lie == "believer" else best0
+        Xa = np.concatenate([Xa, Xcand[j:j + 1]])
+        ya = np.concatenate([ya, np.array([value], dtype=np.float32)])
+    return np.array(picked, dtype=np.int64), np.array(values)
+
+
 def fit_batch(X, y, ell, sf2, sn2):
     """Steps (2)-(3) for [batch] independent GPs; returns a list of Fit."""
     X, y, ell = _f32(X), _f32(y), _f32(ell)
