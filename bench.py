@@ -388,6 +388,16 @@ def main():
             torch.cuda.synchronize()
             append_ms = ev[0].elapsed_time(ev[1])
             g0.close()
+    # a parallel round's proposal: q = k distinct candidates by fantasies (believer), shortlist chosen by the library
+    qp = min(k, 256)
+    propose_ms, propose_cert = None, None
+    for rep in range(2):
+        torch.cuda.synchronize()
+        ev[0].record()
+        _, _, cert = b.r3_gp_propose(gp, xc, qp)
+        ev[1].record()
+        torch.cuda.synchronize()
+        propose_ms, propose_cert = ev[0].elapsed_time(ev[1]), bool(cert.all())
     if args.engine != "auto":
         b.r3_gp_set_engine(gp, {"simt": b.ENGINE_SIMT, "tensor": b.ENGINE_TENSOR}[args.engine])
     engine = {b.ENGINE_SIMT: "simt", b.ENGINE_TENSOR: "tensor"}[b.r3_gp_engine(gp)]
@@ -511,7 +521,8 @@ def main():
         "config": {"workload": c.name, "batch": B, "n": n, "d": d, "m": m, "k": k, "engine": engine,
                    "l2": "pool (%.0f MB) and outputs exceed the 126 MB L2" % (xc.numel() * 4 / 1e6)
                    if xc.numel() * 4 > 126e6 else "pool smaller than L2; not flushed"},
-        "fit_ms": fit_ms, "append_ms": append_ms, "append_k": ka, "clocks": clocks,
+        "fit_ms": fit_ms, "append_ms": append_ms, "append_k": ka, "propose_ms": propose_ms,
+        "propose_q": qp, "propose_certified": propose_cert, "clocks": clocks,
         "e2e": {"value": world * B * m / (e2e_ms * 1e-3), "unit": "candidates/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "matches_device_run": bool(same)},
         "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu, "peaks": peak_kind,

@@ -194,6 +194,34 @@ r3_status_t r3_gp_profile(r3_gp_t* gp, int enable);
 r3_status_t r3_gp_profile_read(r3_gp_t* gp, double* kernel_ms, long long* launches);
 
 /*
+ * r3_gp_propose -- q distinct pool members to replay in parallel, chosen greedily by fantasies.
+ *
+ * Section IV runs a parallel search: several points are in flight at once.  The paper gives no rule
+ * for choosing them; this is the usual sequential one.  q times: take the not-yet-picked candidate
+ * of largest EI (incumbent fixed at the best observed value; ties to the lower index), then
+ * condition the GP on it with a fantasised value rounded to FP32 -- its posterior mean
+ * (lie = 0, "believer") or the incumbent (lie = 1, "liar").  The handle itself is not changed.
+ *
+ * Conditioning on one point is a rank-one update of every candidate's mean and variance, so the pool
+ * is scored once (as r3_gp_score does) and the q picks run on a shortlist of the `shortlist` best
+ * candidates of that scoring, recomputed in FP64.  With the believer's value EI can only drop from
+ * pick to pick, so the shortlist loses nothing as long as every pick's EI stays above the best EI left
+ * outside it: certified[g] = 1 says that this held for GP g (or that the shortlist was the whole
+ * pool).  With lie = 1 a shortlist smaller than the pool is a heuristic and certified is 0.
+ *
+ *   Xcand      device [batch][m][d]
+ *   q          1 <= q <= min(m, 256)
+ *   shortlist  0 = automatic (max(8 q, 256), at most m and 1023), else q <= shortlist <= min(m, 1023)
+ *   idx        device [batch][q] int32, in pick order
+ *   ei_pick    device [batch][q] EI of each pick when it was picked, or NULL
+ *   certified  host   [batch], or NULL
+ *
+ * Synchronises `cuda_stream`; allocates temporary device memory.
+ */
+r3_status_t r3_gp_propose(r3_gp_t* gp, const float* Xcand, long long m, int q, int shortlist, int lie, int* idx,
+                          float* ei_pick, int* certified, void* cuda_stream);
+
+/*
  * r3_gp_append -- add k observations to every GP of the handle without refactoring the history.
  *
  * One BO round ends with k replayed points; conditioning on them is a rank-k extension of the factor,

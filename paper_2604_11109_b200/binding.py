@@ -40,6 +40,7 @@ SIGNATURES = {
     "r3_topk_scratch_bytes": (_ull, [_i, _ll, _i]),
     "r3_trim_cache": (None, []),
     "r3_cached_bytes": (_ull, []),
+    "r3_gp_propose": (_i, [_vp, _vp, _ll, _i, _i, _i, _vp, _vp, ctypes.POINTER(ctypes.c_int), _vp]),
     "r3_gp_append": (_i, [_vp, _vp, _vp, _i, _vp]),
     "r3_gp_size": (_i, [_vp]),
     "r3_tpe_fit": (_i, [_vp, _vp, ctypes.POINTER(ctypes.c_int), _i, _i, ctypes.c_float, ctypes.c_float, _vp,
@@ -237,6 +238,20 @@ def r3_gp_score_topk_host(gp: GP, Xcand_host, k: int, out):
     _check(load().r3_gp_score_topk_host(gp.handle, hp(Xcand_host), m, k, hp(mu), hp(sigma), hp(ei), hp(idx), hp(val),
                                         _stream()))
     return out
+
+
+def r3_gp_propose(gp: GP, Xcand, q: int, shortlist: int = 0, lie: str = "believer"):
+    """q pool members per GP chosen greedily by fantasies: returns (idx int32 [batch][q], EI at pick time
+    float32 [batch][q], certified bool [batch])."""
+    import torch
+    Xcand, m = _pool(gp, Xcand)
+    idx = torch.empty((gp.batch, q), dtype=torch.int32, device=Xcand.device)
+    val = torch.empty((gp.batch, q), dtype=torch.float32, device=Xcand.device)
+    cert = (ctypes.c_int * gp.batch)()
+    _check(load().r3_gp_propose(gp.handle, _dev_f32(Xcand, "Xcand"), m, int(q), int(shortlist),
+                                {"believer": 0, "liar": 1}[lie], ctypes.c_void_p(idx.data_ptr()),
+                                ctypes.c_void_p(val.data_ptr()), cert, _stream()))
+    return idx, val, np.array([bool(c) for c in cert])
 
 
 def r3_gp_append(gp: GP, Xnew, ynew):

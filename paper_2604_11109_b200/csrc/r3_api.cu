@@ -268,6 +268,100 @@ r3_status_t r3_gp_fit(const float* X, const float* y, const float* lengthscales,
     return R3_OK;
 }
 
+r3_status_t r3_gp_propose(r3_gp_t* gp, const float* Xcand, long long m, int q, int shortlist, int lie, int* idx,
+                          float* ei_pick, int* certified, void* cuda_stream)
+{
+    if (!gp || !Xcand || !idx) {
+        set_error("r3_gp_propose: NULL argument");
+        return R3_ERR_INVALID_ARG;
+    }
+    if (m < 1 || m >= (1ll << 31) || q < 1 || q > 256 || q > m || (lie != 0 && lie != 1)) {
+        set_error("r3_gp_propose: need 1 <= m < 2^31, 1 <= q <= min(m, 256), lie in {0, 1} (m=%lld q=%d lie=%d)", m, q,
+                  lie);
+        return R3_ERR_INVALID_ARG;
+    }
+    const int rmax = (int)(m < 1023 ? m : 1023);
+    int R = shortlist;
+    if (R == 0) {
+        R = 8 * q > 256 ? 8 * q : 256;
+        if (R > rmax) R = rmax;
+    }
+    if (R < q || R > rmax) {
+        set_error("r3_gp_propose: shortlist=%d outside [q, min(m, 1023)]", shortlist);
+        return R3_ERR_INVALID_ARG;
+    }
+    const int B = gp->batch;
+    const int Rk = (long long)R < m ? R + 1 : R;   // one more than the shortlist: the certificate's bound
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    r3_status_t st = ensure_workspace(gp, score_workspace_bytes(gp, m));
+    if (st != R3_OK) return st;
+    float *scores = nullptr, *sval = nullptr;
+    int* sidx = nullptr;
+    void *tws = nullptr, *pws = nullptr;
+    const size_t bm = (size_t)B * m, tbytes = topk_workspace_bytes(B, m, Rk);
+    auto done = [&](r3_status_t s) {
+        cudaStreamSynchronize(stream);
+        dev_free(scores); dev_free(sval); dev_free(sidx); dev_free(tws); dev_free(pws);
+        return s;
+    };
+#define TRY_DONE(expr)                                                                             \
+    do {                                                                                           \
+        cudaError_t e__ = (expr);                                                                  \
+        if (e__ != cudaSuccess) {                                                                  \
+            set_error("%s failed: %s", #expr, cudaGetErrorString(e__));                            \
+            return done(e__ == cudaErrorMemoryAllocation ? R3_ERR_ALLOC : R3_ERR_CUDA);            \
+        }                                                                                          \
+    } while (0)
+    TRY_DONE(dev_malloc(&scores, sizeof(float) * 3 * bm));
+    TRY_DONE(dev_malloc(&sval, sizeof(float) * (size_t)B * Rk));
+    TRY_DONE(dev_malloc(&sidx, sizeof(int) * (size_t)B * Rk));
+    TRY_DONE(dev_malloc(&tws, tbytes));
+    TRY_DONE(dev_malloc(&pws, propose_workspace_bytes(gp->npad, R, q)));
+    float *mu = scores, *sigma = scores + bm, *ei = scores + 2 * bm;
+    st = run_score(gp, Xcand, m, mu, sigma, ei, gp->ws, gp->ws_bytes, stream);
+    if (st != R3_OK) return done(st);
+    st = topk_device(ei, B, m, Rk, sidx, sval, tws, tbytes, stream);
+    if (st != R3_OK) return done(st);
+    for (int g = 0; g < B; ++g) {
+        st = propose_shortlist(gp, g, Xcand + (size_t)g * m * gp->d, sidx + (size_t)g * Rk, R, q, lie,
+                               idx + (size_t)g * q, ei_pick ? ei_pick + (size_t)g * q : nullptr, pws, stream);
+        if (st != R3_OK) return done(st);
+    }
+    // certificate and latched device status
+    std::vector<float> hval((size_t)B * Rk), hpick;
+    TRY_DONE(cudaMemcpyAsync(hval.data(), sval, sizeof(float) * hval.size(), cudaMemcpyDeviceToHost, stream));
+    TRY_DONE(cudaMemcpyAsync(gp->status_h, gp->status_d, 2 * sizeof(int), cudaMemcpyDeviceToHost, stream));
+    if (ei_pick) {
+        hpick.resize((size_t)B * q);
+        TRY_DONE(cudaMemcpyAsync(hpick.data(), ei_pick, sizeof(float) * hpick.size(), cudaMemcpyDeviceToHost, stream));
+    }
+    TRY_DONE(cudaStreamSynchronize(stream));
+#undef TRY_DONE
+    if (gp->status_h[0] & DEV_NOT_PD) {
+        gp->status_h[0] &= ~DEV_NOT_PD;
+        cudaMemcpy(gp->status_d, gp->status_h, sizeof(int), cudaMemcpyHostToDevice);
+        set_error("r3_gp_propose: a picked candidate has zero variance and the noise is zero (it duplicates an "
+                  "observation); nothing to condition on");
+        return done(R3_ERR_NOT_PD);
+    }
+    if (certified) {
+        for (int g = 0; g < B; ++g) {
+            if (Rk == R) {
+                certified[g] = 1;   // the shortlist is the whole pool
+            } else if (lie != 0 || !ei_pick) {
+                certified[g] = 0;
+            } else {
+                // the first excluded candidate's initial EI (FP32, within the scoring tolerance of 1e-5 max EI)
+                const double bound = hval[(size_t)g * Rk + R], top = hval[(size_t)g * Rk];
+                double lowest = hpick[(size_t)g * q];
+                for (int t = 1; t < q; ++t) lowest = hpick[(size_t)g * q + t] < lowest ? hpick[(size_t)g * q + t] : lowest;
+                certified[g] = lowest >= bound + 4e-5 * top ? 1 : 0;
+            }
+        }
+    }
+    return done(R3_OK);
+}
+
 r3_status_t r3_gp_append(r3_gp_t* gp, const float* Xnew, const float* ynew, int k, void* cuda_stream)
 {
     if (!gp || !Xnew || !ynew) {

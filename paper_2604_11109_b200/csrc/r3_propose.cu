@@ -1,0 +1,207 @@
+// Greedy batch proposal by fantasies ("parallel" search of Section IV: several points of one search are
+// replayed at once).  Definition: q times -- pick the not-yet-picked candidate of largest EI (incumbent
+// fixed at the best observed value), then condition the GP on that point with a fantasised value (its
+// posterior mean, "believer", or the incumbent, "liar").
+//
+// Refitting and rescoring the pool q times would cost q full scoring passes.  Conditioning on one point
+// is a rank-one change of the posterior:
+//     c(x) = cov(x, x_t),  s = var(x_t) + noise,
+//     mu(x) += c(x) (value - mu(x_t)) / s,     var(x) -= c(x)^2 / s,
+//     cov(x, x_t) = k(x, x_t) - v(x).v(x_t) - sum_{earlier picks u} c_u(x) c_u(x_t) / s_u,   v(x) = W k*(x),
+// and with the believer's value the means never move while the variances only shrink, so EI (fixed
+// incumbent) only drops: a candidate outside the R best of the first scoring can be picked only if some
+// pick's EI falls below the (R+1)-th initial EI.  So: one full scoring, top-(R+1), then the q picks on the
+// shortlist alone, in FP64 (k*, v = W k* by one triangular product, the moments recomputed), two small
+// launches per pick.  The (R+1)-th initial EI is returned as the certificate's bound.
+#include "r3_epilogue.cuh"
+#include "r3_gemm64.cuh"
+#include "r3_internal.cuh"
+
+namespace r3 {
+
+namespace {
+
+// Ks[r][i] = k(x_i, candidate sidx[r]) in FP64 by direct differences; zero in the padding columns.
+__global__ void shortlist_kstar_kernel(const float* __restrict__ X, const float* __restrict__ ell, double sf2, int n,
+                                       int d, int npad, const float* __restrict__ Xcand, const int* __restrict__ sidx,
+                                       double* __restrict__ Ks)
+{
+    const int r = blockIdx.y;
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= npad) return;
+    double v = 0.0;
+    if (i < n) {
+        const float* z = Xcand + (size_t)sidx[r] * d;
+        const float* x = X + (size_t)i * d;
+        double r2 = 0.0;
+        for (int j = 0; j < d; ++j) {
+            const double diff = ((double)x[j] - (double)z[j]) / (double)ell[j];
+            r2 += diff * diff;
+        }
+        const double s = sqrt(5.0) * sqrt(r2);
+        v = sf2 * (1.0 + s + s * s / 3.0) * exp(-s);
+    }
+    Ks[(size_t)r * npad + i] = v;
+}
+
+// mu[r] = Ks[r].alpha, var[r] = sf2 - |V[r]|^2 (one warp per shortlisted candidate).
+__global__ void shortlist_moments_kernel(const double* __restrict__ Ks, const double* __restrict__ V,
+                                         const double* __restrict__ alpha, int n, int npad, double sf2, int R,
+                                         double* __restrict__ mu, double* __restrict__ var, int* __restrict__ picked)
+{
+    const int r = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
+    const int lane = threadIdx.x % 32;
+    if (r >= R) return;
+    double m = 0.0, q = 0.0;
+    for (int i = lane; i < n; i += 32) {
+        m = fma(Ks[(size_t)r * npad + i], alpha[i], m);
+        const double v = V[(size_t)r * npad + i];
+        q = fma(v, v, q);
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        m += __shfl_xor_sync(0xffffffffu, m, o);
+        q += __shfl_xor_sync(0xffffffffu, q, o);
+    }
+    if (lane == 0) {
+        mu[r] = m;
+        var[r] = sf2 - q;
+        picked[r] = 0;
+    }
+}
+
+// One block: EI of every unpicked shortlisted candidate, the largest (ties: lower pool index) is pick t.
+__global__ void __launch_bounds__(1024) pick_kernel(const double* __restrict__ mu, const double* __restrict__ var,
+                                                    int* __restrict__ picked, const int* __restrict__ sidx, int R,
+                                                    double best, double sn2, int liar, int t, int* __restrict__ sel,
+                                                    double* __restrict__ S, double* __restrict__ delta,
+                                                    int* __restrict__ idx_out, float* __restrict__ ei_out,
+                                                    int* __restrict__ status)
+{
+    __shared__ double se[1024];
+    __shared__ int sr[1024];
+    const int r = threadIdx.x;
+    double e = -1.0;
+    if (r < R && !picked[r]) e = ei_closed_form(mu[r], sqrt(fmax(var[r], 0.0)), best);
+    se[r] = e;
+    sr[r] = r;
+    __syncthreads();
+    for (int o = 512; o > 0; o >>= 1) {
+        if (r < o) {
+            const double a = se[r], b = se[r + o];
+            const int ra = sr[r], rb = sr[r + o];
+            // an entry that is not a candidate (e < 0) always loses; equal EI: the lower pool index wins
+            const bool take_b = (b > a) || (b == a && b >= 0.0 && sidx[rb] < sidx[ra]);
+            if (take_b) {
+                se[r] = b;
+                sr[r] = rb;
+            }
+        }
+        __syncthreads();
+    }
+    if (r == 0) {
+        const int j = sr[0];
+        sel[t] = j;
+        picked[j] = 1;
+        idx_out[t] = sidx[j];
+        if (ei_out) ei_out[t] = (float)se[0];
+        const double s = fmax(var[j], 0.0) + sn2;
+        if (!(s > 0.0)) {   // a candidate on top of an observation with zero noise: nothing to condition on
+            atomicOr(status, DEV_NOT_PD);
+            S[t] = INFINITY;
+            delta[t] = 0.0;
+        } else {
+            S[t] = s;
+            // the fantasised value enters the history as an observation, i.e. rounded to FP32
+            const double value = liar ? best : (double)(float)mu[j];
+            delta[t] = (value - mu[j]) / s;
+        }
+    }
+}
+
+// One warp per shortlisted candidate r: c = cov(x_r, x_pick) under the posterior before pick t, then the
+// rank-one update of its mean and variance.  C[t][r] keeps c for the later picks.
+__global__ void condition_kernel(const float* __restrict__ Xcand, const int* __restrict__ sidx,
+                                 const float* __restrict__ ell, double sf2, int d, const double* __restrict__ V, int n,
+                                 int npad, double* __restrict__ C, const double* __restrict__ S,
+                                 const double* __restrict__ delta, const int* __restrict__ sel, int t, int R,
+                                 double* __restrict__ mu, double* __restrict__ var)
+{
+    const int r = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
+    const int lane = threadIdx.x % 32;
+    if (r >= R) return;
+    const int j = sel[t];
+    const float* xr = Xcand + (size_t)sidx[r] * d;
+    const float* xj = Xcand + (size_t)sidx[j] * d;
+    double r2 = 0.0, dot = 0.0, prev = 0.0;
+    for (int f = lane; f < d; f += 32) {
+        const double diff = ((double)xr[f] - (double)xj[f]) / (double)ell[f];
+        r2 = fma(diff, diff, r2);
+    }
+    for (int i = lane; i < n; i += 32) dot = fma(V[(size_t)r * npad + i], V[(size_t)j * npad + i], dot);
+    for (int u = lane; u < t; u += 32) prev += C[(size_t)u * R + r] * C[(size_t)u * R + j] / S[u];
+    for (int o = 16; o > 0; o >>= 1) {
+        r2 += __shfl_xor_sync(0xffffffffu, r2, o);
+        dot += __shfl_xor_sync(0xffffffffu, dot, o);
+        prev += __shfl_xor_sync(0xffffffffu, prev, o);
+    }
+    if (lane == 0) {
+        const double s = sqrt(5.0) * sqrt(r2);
+        const double c = sf2 * (1.0 + s + s * s / 3.0) * exp(-s) - dot - prev;
+        C[(size_t)t * R + r] = c;
+        mu[r] += c * delta[t];
+        var[r] -= c * c / S[t];
+    }
+}
+
+}  // namespace
+
+size_t propose_workspace_bytes(int npad, int R, int q)
+{
+    return sizeof(double) * (2 * (size_t)R * npad + (size_t)q * R + 2 * (size_t)R + 2 * (size_t)q) +
+           sizeof(int) * ((size_t)R + q) + 256;
+}
+
+// The q picks of GP g.  sidx: device [R] pool indices of the shortlist (by initial EI, descending);
+// idx_out / ei_out: device [q].  ws: propose_workspace_bytes(npad, R, q) bytes.
+r3_status_t propose_shortlist(r3_gp* gp, int g, const float* Xcand_g, const int* sidx, int R, int q, int liar,
+                              int* idx_out, float* ei_out, void* ws, cudaStream_t stream)
+{
+    const int n = gp->n, d = gp->d, npad = gp->npad;
+    char* p = (char*)ws;
+    auto carve = [&](size_t bytes) {
+        char* r = p;
+        p += (bytes + 15) / 16 * 16;
+        return r;
+    };
+    double* Ks = (double*)carve(sizeof(double) * (size_t)R * npad);
+    double* V = (double*)carve(sizeof(double) * (size_t)R * npad);
+    double* C = (double*)carve(sizeof(double) * (size_t)q * R);
+    double* mu = (double*)carve(sizeof(double) * R);
+    double* var = (double*)carve(sizeof(double) * R);
+    double* S = (double*)carve(sizeof(double) * q);
+    double* delta = (double*)carve(sizeof(double) * q);
+    int* picked = (int*)carve(sizeof(int) * R);
+    int* sel = (int*)carve(sizeof(int) * q);
+    const float* Xg = gp->X + (size_t)g * n * d;
+    const float* ellg = gp->ell_d + (size_t)g * d;
+    const double* Wg = gp->W64 + (size_t)g * npad * npad;
+    const double sf2 = (double)gp->sf2[g], sn2 = (double)gp->sn2[g], best = (double)gp->best[g];
+
+    R3_LAUNCH(shortlist_kstar_kernel, dim3((npad + 127) / 128, R), 128, 0, stream, Xg, ellg, sf2, n, d, npad, Xcand_g,
+              sidx, Ks);
+    // V = Ks W^T (v_r = W k*_r): the same triangular product as the append step of the fit
+    R3_LAUNCH(tri_gemm_kernel<true>, dim3((n + 63) / 64, (R + 31) / 32, 1), 256, 0, stream, Ks, npad, (size_t)0, Wg,
+              npad, (size_t)0, V, npad, (size_t)0, R, n);
+    R3_LAUNCH(shortlist_moments_kernel, (R + 7) / 8, 256, 0, stream, Ks, V, gp->alpha64 + (size_t)g * npad, n, npad, sf2,
+              R, mu, var, picked);
+    for (int t = 0; t < q; ++t) {
+        R3_LAUNCH(pick_kernel, 1, 1024, 0, stream, mu, var, picked, sidx, R, best, sn2, liar, t, sel, S, delta, idx_out,
+                  ei_out, gp->status_d);
+        if (t + 1 < q)
+            R3_LAUNCH(condition_kernel, (R + 7) / 8, 256, 0, stream, Xcand_g, sidx, ellg, sf2, d, V, n, npad, C, S, delta,
+                      sel, t, R, mu, var);
+    }
+    return R3_OK;
+}
+
+}  // namespace r3
