@@ -492,8 +492,8 @@ def main():
                     "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"]}
         if c.cfg == 5 and args.m is None:
             # dram bytes per launch from the ncu capture of this kernel on m = 32768 (profiles/score_tc_kernel_cfg5.md):
-            # 37.7 MB of pre-tiled operands read once + 259 B per candidate (241 read, 17.8 written)
-            roofline["traffic"] = 37.7e6 + 259.0 * cands_per_launch
+            # 37.7 MB of pre-tiled operands read once + 263 B per candidate (244 read, 18.6 written)
+            roofline["traffic"] = 37.7e6 + 263.0 * cands_per_launch
     else:
         alg_flops = float(npad) * npad
         achieved = alg_flops * cands_per_launch / (per_launch_ms * 1e-3) / 1e12
