@@ -224,6 +224,41 @@ def propose(X, y, ell, sf2: float, sn2: float, Xcand, q: int, lie: str = "believ
     return np.array(picked, dtype=np.int64), np.array(values)
 
 
+def lml(X, y, ell, sf2: float, sn2: float):
+    """Log marginal likelihood of the history and its gradient with respect to the LOGARITHMS of the
+    hyper-parameters, in the order (log ell_1 .. log ell_d, log sf2, log sn2) -- what a hyper-parameter fit of
+    the surrogate maximises (the paper passes no rule; this is the textbook evidence of a zero-mean GP):
+
+        K = Kf + sn2 I,  alpha = K^-1 y,
+        lml = -1/2 y.alpha - 1/2 log|K| - n/2 log(2 pi),
+        d lml / d theta = 1/2 trace((alpha alpha^T - K^-1) dK/dtheta),
+        dK/dlog ell_j = sf2 exp(-s) (5/3)(1 + s) u_j^2   (u_j = (x_j - z_j)/ell_j, s = sqrt(5 sum u^2)),
+        dK/dlog sf2 = Kf,   dK/dlog sn2 = sn2 I.
+
+    Plain numpy FP64 with LAPACK's Cholesky and inverse as steps; n^2 d memory, so for test sizes only.
+    Returns (lml, gradient [d + 2]).
+    """
+    X, y, ell = _f32(X).astype(np.float64), _f32(y).astype(np.float64), _f32(ell).astype(np.float64)
+    sf2, sn2 = float(np.float32(sf2)), float(np.float32(sn2))
+    n, d = X.shape
+    U = (X[:, None, :] - X[None, :, :]) / ell[None, None, :]
+    s = np.sqrt(5.0 * (U * U).sum(axis=2))
+    e = np.exp(-s)
+    Kf = sf2 * (1.0 + s + s * s / 3.0) * e
+    K = Kf + sn2 * np.eye(n)
+    L = np.linalg.cholesky(K)
+    alpha = np.linalg.solve(L.T, np.linalg.solve(L, y))
+    value = -0.5 * float(y @ alpha) - float(np.log(np.diag(L)).sum()) - 0.5 * n * np.log(2.0 * np.pi)
+    M = np.outer(alpha, alpha) - np.linalg.inv(K)
+    G = sf2 * e * (5.0 / 3.0) * (1.0 + s)
+    grad = np.empty(d + 2)
+    for j in range(d):
+        grad[j] = 0.5 * float((M * G * U[:, :, j] ** 2).sum())
+    grad[d] = 0.5 * float((M * Kf).sum())
+    grad[d + 1] = 0.5 * sn2 * float(np.trace(M))
+    return value, grad
+
+
 def fit_batch(X, y, ell, sf2, sn2):
     """Steps (2)-(3) for [batch] independent GPs; returns a list of Fit."""
     X, y, ell = _f32(X), _f32(y), _f32(ell)
