@@ -194,6 +194,23 @@ r3_status_t r3_gp_profile(r3_gp_t* gp, int enable);
 r3_status_t r3_gp_profile_read(r3_gp_t* gp, double* kernel_ms, long long* launches);
 
 /*
+ * r3_gp_lml -- log marginal likelihood of each GP's history under its current hyper-parameters, and
+ * its gradient with respect to their logarithms: the objective of a hyper-parameter fit (the paper
+ * passes lengthscales and variances in and says nothing about choosing them).
+ *
+ *   lml  = -1/2 y.alpha - 1/2 log|K| - n/2 log(2 pi),         K = k(X,X) + noise_var I, alpha = K^-1 y
+ *   grad = 1/2 trace((alpha alpha^T - K^-1) dK/dtheta)  for theta = (log lengthscale_1..d,
+ *          log signal_var, log noise_var), with dK/dlog lengthscale_j = signal_var e^-s (5/3)(1+s) u_j^2,
+ *          u_j = (x_j - z_j)/lengthscale_j, s = sqrt(5 sum_j u_j^2).
+ *
+ *   lml   host [batch]  FP64            grad  host [batch][d + 2]  FP64, or NULL
+ *
+ * FP64 on the device from the factor the handle holds (K^-1 = W^T W costs n^3/3 multiply-adds);
+ * synchronises `cuda_stream`; allocates temporary device memory.
+ */
+r3_status_t r3_gp_lml(r3_gp_t* gp, double* lml, double* grad, void* cuda_stream);
+
+/*
  * r3_gp_propose -- q distinct pool members to replay in parallel, chosen greedily by fantasies.
  *
  * Section IV runs a parallel search: several points are in flight at once.  The paper gives no rule

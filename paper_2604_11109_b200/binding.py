@@ -40,6 +40,7 @@ SIGNATURES = {
     "r3_topk_scratch_bytes": (_ull, [_i, _ll, _i]),
     "r3_trim_cache": (None, []),
     "r3_cached_bytes": (_ull, []),
+    "r3_gp_lml": (_i, [_vp, _vp, _vp, _vp]),
     "r3_gp_propose": (_i, [_vp, _vp, _ll, _i, _i, _i, _vp, _vp, ctypes.POINTER(ctypes.c_int), _vp]),
     "r3_gp_append": (_i, [_vp, _vp, _vp, _i, _vp]),
     "r3_gp_size": (_i, [_vp]),
@@ -238,6 +239,14 @@ def r3_gp_score_topk_host(gp: GP, Xcand_host, k: int, out):
     _check(load().r3_gp_score_topk_host(gp.handle, hp(Xcand_host), m, k, hp(mu), hp(sigma), hp(ei), hp(idx), hp(val),
                                         _stream()))
     return out
+
+
+def r3_gp_lml(gp: GP):
+    """(lml [batch], gradient [batch][d + 2] in (log lengthscales, log signal_var, log noise_var)), FP64."""
+    lml = np.empty((gp.batch,), dtype=np.float64)
+    grad = np.empty((gp.batch, gp.d + 2), dtype=np.float64)
+    _check(load().r3_gp_lml(gp.handle, ctypes.c_void_p(lml.ctypes.data), ctypes.c_void_p(grad.ctypes.data), _stream()))
+    return lml, grad
 
 
 def r3_gp_propose(gp: GP, Xcand, q: int, shortlist: int = 0, lie: str = "believer"):

@@ -268,6 +268,24 @@ r3_status_t r3_gp_fit(const float* X, const float* y, const float* lengthscales,
     return R3_OK;
 }
 
+r3_status_t r3_gp_lml(r3_gp_t* gp, double* lml, double* grad, void* cuda_stream)
+{
+    if (!gp || !lml) {
+        set_error("r3_gp_lml: NULL argument");
+        return R3_ERR_INVALID_ARG;
+    }
+    const int B = gp->batch, d = gp->d;
+    std::vector<double> out((size_t)B * (d + 3));
+    const r3_status_t st = lml_device(gp, out.data(), (cudaStream_t)cuda_stream);
+    if (st != R3_OK) return st;
+    for (int g = 0; g < B; ++g) {
+        lml[g] = out[(size_t)g * (d + 3)];
+        if (grad)
+            for (int j = 0; j < d + 2; ++j) grad[(size_t)g * (d + 2) + j] = out[(size_t)g * (d + 3) + 1 + j];
+    }
+    return R3_OK;
+}
+
 r3_status_t r3_gp_propose(r3_gp_t* gp, const float* Xcand, long long m, int q, int shortlist, int lie, int* idx,
                           float* ei_pick, int* certified, void* cuda_stream)
 {

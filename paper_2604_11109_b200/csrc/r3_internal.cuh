@@ -152,6 +152,9 @@ size_t topk_workspace_bytes(int batch, long long m, int k);
 r3_status_t topk_device(const float* ei, int batch, long long m, int k, int* idx, float* val, void* ws,
                         size_t ws_bytes, cudaStream_t stream);
 
+// log marginal likelihood and gradient (r3_lml.cu): out_h host [batch][d + 3]
+r3_status_t lml_device(r3_gp* gp, double* out_h, cudaStream_t stream);
+
 // greedy batch proposal on a shortlist (r3_propose.cu)
 size_t propose_workspace_bytes(int npad, int R, int q);
 r3_status_t propose_shortlist(r3_gp* gp, int g, const float* Xcand_g, const int* sidx, int R, int q, int liar,
