@@ -353,11 +353,12 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                         const int j4 = 2 * j8 + h;
                         float z[4];
                         if (vec && 4 * j4 < prm.d) {
-                            const float4 v = *reinterpret_cast<const float4*>(zrow + 4 * j4);
+                            // read once: streaming load, so that the pool does not push W out of L2
+                            const float4 v = __ldcs(reinterpret_cast<const float4*>(zrow + 4 * j4));
                             z[0] = v.x; z[1] = v.y; z[2] = v.z; z[3] = v.w;
                         } else {
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) z[e] = (4 * j4 + e < prm.d) ? zrow[4 * j4 + e] : 0.f;
+                            for (int e = 0; e < 4; ++e) z[e] = (4 * j4 + e < prm.d) ? __ldcs(zrow + 4 * j4 + e) : 0.f;
                         }
                         const float4 c4 = __ldg(reinterpret_cast<const float4*>(cen + 4 * j4));
                         const float4 s4 = __ldg(reinterpret_cast<const float4*>(scl + 4 * j4));
@@ -587,9 +588,9 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     q_acc *= prm.vinv2[g];   // undo the power-of-two scaling of k* and W
                     const size_t f = (size_t)g * prm.m + cand;
                     const CandidateResult res = finalize_candidate(mu_acc, q_acc, (double)sf2, (double)prm.best[g]);
-                    prm.mu[f] = res.mu;
-                    prm.sigma[f] = res.sigma;
-                    prm.ei[f] = res.ei;
+                    __stcs(prm.mu + f, res.mu);
+                    __stcs(prm.sigma + f, res.sigma);
+                    __stcs(prm.ei + f, res.ei);
                     const double eps =
                         far_cand ? 1.0 : kEpsTc0 + kEpsTc1 * (double)(zn + prm.xnmax[g]) * rsqrt((double)DP);
                     prm.err_mu[f] = mu_error_estimate(eps, a2_acc);
