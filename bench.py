@@ -158,14 +158,15 @@ def run_tpe(args, c):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     g = w.generate_gp(c, 0)
-    levels = w.tpe_levels(c)
+    levels = w.tpe_levels(c, grid=args.tpe_grid)
     n, d, m, k = c.n, c.d, c.m, c.k
     evals = float(sum(n + 2 for l in levels if l == 0))      # exponentials per candidate
     base = {"metric": "tpe_candidates_scored_per_sec", "unit": "candidates/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "data": "synthetic",
             "config": {"workload": c.name + "-tpe", "n": n, "d": d, "m": m, "k": k, "gamma": 0.25,
-                       "ordinal_dims": int((levels == 0).sum()), "categorical_dims": int((levels != 0).sum())}}
+                       "ordinal_dims": int((levels == 0).sum()), "grid_dims": int((levels < 0).sum()),
+                       "categorical_dims": int((levels > 0).sum())}}
     if args.impl == "reference":
         if rank != 0:
             return
@@ -284,8 +285,23 @@ def run_tpe(args, c):
             dist.destroy_process_group()
         return
     sm_mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
-    peak = 148 * 16 * sm_mhz * 1e6 / 1e12
-    achieved = evals * m / (k_ms * 1e-3) / 1e12
+    peaks, peak_kind = load_peaks()
+    mufu_peak = 148 * 16 * sm_mhz * 1e6 / 1e12
+    hbm_bytes = float(m) * (4 * d + 4)
+    if evals * m / (mufu_peak * 1e12) >= hbm_bytes / (peaks["hbm_gbs"] * 1e9):
+        achieved = evals * m / (k_ms * 1e-3) / 1e12
+        roofline = {"bound": "alu", "kernel": "tpe_score_kernel", "achieved": achieved, "peak": mufu_peak,
+                    "unit": "Texp2/s", "frac": achieved / mufu_peak, "traffic": None,
+                    "note": "one MUFU.EX2 per (candidate, ordinal dimension, component); peak = 148 SMs x 16 MUFU "
+                            "results per clock x max SM clock"}
+    else:
+        achieved = hbm_bytes / (k_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": "tpe_score_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                    "note": f"4d + 4 bytes per candidate (pool read once, one score written); peak = {peak_kind} copy "
+                            "bandwidth"}
+    roofline["kernel_ms_per_launch"] = k_ms
+    roofline["kernel_share_of_step"] = k_ms / ms_per_step
     cpu = None
     if not args.no_cpu_baseline:
         from oracle import tpe_oracle as T
@@ -308,12 +324,8 @@ def run_tpe(args, c):
         "e2e": {"value": world * m / (e2e_ms * 1e-3), "unit": "candidates/s", "h2d_bytes_per_step": int(xh.numel() * 4),
                 "d2h_bytes_per_step": int(k * 8), "ms_per_step": e2e_ms},
         "gpu_launches": int(launches),
-        "roofline": {"bound": "alu", "kernel": "tpe_score_kernel", "achieved": achieved, "peak": peak,
-                     "unit": "Texp2/s", "frac": achieved / peak, "traffic": None,
-                     "note": "one MUFU.EX2 per (candidate, ordinal dimension, component); peak = 148 SMs x 16 MUFU "
-                             "results per clock x max SM clock",
-                     "kernel_ms_per_launch": k_ms, "kernel_share_of_step": k_ms / ms_per_step},
-        "cpu_baseline": cpu, "peaks": "derived",
+        "roofline": roofline,
+        "cpu_baseline": cpu, "peaks": peak_kind,
     })
     print(json.dumps(base))
     tpe.close()
@@ -331,6 +343,8 @@ def main():
     ap.add_argument("--engine", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--m", type=int, default=None, help="override the pool size (profiling of small cases)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tpe-grid", action="store_true",
+                    help="tpe: declare equally spaced ordinal features as grids (tabulated at fit time)")
     ap.add_argument("--surrogate", default="gp", choices=["gp", "tpe"],
                     help="gp: the headline GP-EI path; tpe: Parzen-estimator scoring of the same pools")
     args = ap.parse_args()

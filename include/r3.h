@@ -286,6 +286,10 @@ void r3_gp_free(r3_gp_t* gp);
  *   (T3) categorical dimension (levels[j] == C, 2 <= C <= 64): level v = clamp(floor(x*(C-1) + 1/2),
  *        0, C-1) with the product and the sum each rounded to FP32;
  *        P(v) = (count_v + prior_weight/C) / (s + prior_weight).
+ *   (T3g) ordinal dimension on a known grid (levels[j] == -L, 2 <= L <= 64; admissible values v/(L-1)):
+ *        the mixture of (T2), evaluated at the candidate's nearest grid value (level as in (T3), value
+ *        v/(L-1) rounded to FP32).  The L log-density ratios are tabulated by r3_tpe_fit, so such a
+ *        dimension costs one look-up per candidate instead of n + 2 exponentials.
  *   (T4) score(x) = sum_j [ ln l_j(x_j) - ln g_j(x_j) ], l from the good set, g from the bad set.
  *        Larger is better; pass the scores to r3_topk to pick the next points.
  *
@@ -298,7 +302,8 @@ typedef struct r3_tpe r3_tpe_t; /* opaque; owns device memory */
  *
  *   X       device [n][d]   observed configurations, row-major
  *   y       device [n]      observed values (smaller is better)
- *   levels  host   [d]      0 = ordinal/continuous, C in [2, 64] = categorical with C levels
+ *   levels  host   [d]      0 = ordinal/continuous, C in [2, 64] = categorical with C levels,
+ *                           -L in [-64, -2] = ordinal on the grid v/(L-1)
  *   1 <= n <= 4096, 1 <= d <= 256, 0 < gamma <= 1, prior_weight > 0
  *   out     receives the handle (NULL on error)
  *
@@ -331,8 +336,8 @@ r3_status_t r3_tpe_check(r3_tpe_t* tpe, void* cuda_stream);
  *                                 (n_good + 1 and n - n_good + 1 of them, each set sorted by mean):
  *                                 {mean, log2(e)/(2 sigma^2), log2(weight/(sigma Z sqrt(2 pi))), sigma};
  *                                 all zero for a categorical dimension
- *   table   host [d][64]          ln P_good(v) - ln P_bad(v) per level v of a categorical
- *                                 dimension; zero elsewhere
+ *   table   host [d][64]          ln P_good(v) - ln P_bad(v) per level v of a categorical dimension,
+ *                                 ln l(v/(L-1)) - ln g(v/(L-1)) per grid value of a grid dimension; zero elsewhere
  */
 r3_status_t r3_tpe_get_model(r3_tpe_t* tpe, int* n_good, int* order, float* comps, float* table);
 

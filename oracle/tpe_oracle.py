@@ -34,6 +34,13 @@ Definition (features are normalised to [0, 1]; smaller y is better):
                   v = clamp(floor(x * (C - 1) + 1/2), 0, C - 1), that product and
                   sum taken in FP32 (the precision the device decides it in);
                   P(v) = (count_v + prior_weight / C) / (s + prior_weight).
+  (T3g) ordinal dimension on a known grid (levels == -L, 2 <= L <= 64: the admissible
+                  values are v/(L-1), v = 0..L-1, as for block sizes, unroll factors
+                  or sixteen-level features): the mixture is (T2)'s, and a candidate is
+                  evaluated at its nearest grid value -- level v as in (T3), value
+                  v/(L-1) taken in FP64 and rounded to FP32, which is the FP32 number an
+                  on-grid candidate holds.  For candidates on the grid this IS (T2); it
+                  lets an implementation tabulate the L densities once.
   (T4) score      sum over dimensions of ln l_j(x_j) - ln g_j(x_j), l from the
                   good set and g from the bad set.  A larger score is a better
                   candidate (the ratio l/g is monotone in Expected Improvement
@@ -67,6 +74,7 @@ def _Phi(z: float) -> float:
 class Mixture:
     """Parzen mixture of one dimension and one set (T2), or a probability table (T3)."""
     levels: int
+    grid: int = 0                # (T3g): evaluate at the nearest of `grid` equally spaced values
     mu: np.ndarray = field(default_factory=lambda: np.zeros(0))      # [s + 1] component means, prior last
     sigma: np.ndarray = field(default_factory=lambda: np.zeros(0))   # [s + 1]
     weight: np.ndarray = field(default_factory=lambda: np.zeros(0))  # [s + 1], normalised to sum 1
@@ -149,9 +157,10 @@ def tpe_fit(X: np.ndarray, y: np.ndarray, levels, gamma: float = 0.25, prior_wei
     good, bad = [], []
     for j in range(d):
         col = X[:, j]
-        if levels[j] == 0:
+        if levels[j] <= 0:
             good.append(parzen(col[gi], prior_weight))
             bad.append(parzen(col[bi], prior_weight))
+            good[-1].grid = bad[-1].grid = int(-levels[j])
         else:
             good.append(categorical(col[gi], int(levels[j]), prior_weight))
             bad.append(categorical(col[bi], int(levels[j]), prior_weight))
@@ -162,6 +171,9 @@ def density(mix: Mixture, x: np.ndarray) -> np.ndarray:
     """Value of one dimension's mixture (T2) or level probability (T3) at the points x."""
     if mix.levels:
         return mix.prob[level_of(x, mix.levels)]
+    if mix.grid:
+        L = mix.grid
+        x = (level_of(x, L).astype(np.float64) / (L - 1)).astype(np.float32)
     x = np.asarray(x, dtype=np.float64)[:, None]
     t = (x - mix.mu[None, :]) / mix.sigma[None, :]
     comp = np.exp(-0.5 * t * t) / (_SQRT_2PI * mix.sigma[None, :] * mix.Z[None, :])

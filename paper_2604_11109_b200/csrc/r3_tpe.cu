@@ -10,6 +10,7 @@
 // Scoring is bound by the MUFU unit (16 results per clock per SM); the components of a dimension are
 // staged through shared memory and every thread carries one or two candidates.
 #include <math.h>
+#include <stdlib.h>
 
 #include <new>
 #include <vector>
@@ -106,11 +107,14 @@ __global__ void __launch_bounds__(kSortThreads) tpe_mixture_kernel(const float* 
                                                                    double prior_weight, float4* __restrict__ comps,
                                                                    float* __restrict__ table, int* __restrict__ status)
 {
-    extern __shared__ unsigned long long keys[];   // pow2 >= n + 1 keys
+    extern __shared__ unsigned long long keys[];   // pow2 >= n + 1 keys, then (grid dimensions) 2 (n + 1) doubles
     __shared__ int counts[kTpeMaxLevels];
     __shared__ double lnp_good[kTpeMaxLevels];
+    __shared__ double wsum_s[32];
     const int j = blockIdx.x;
-    const int C = levels[j];
+    const int code = levels[j];
+    const int C = code > 0 ? code : 0;      // categorical levels
+    const int G = code < 0 ? -code : 0;     // grid values of an ordinal dimension
     bool bad = false;
     for (int set = 0; set < 2; ++set) {
         const int s = set == 0 ? n_good : n - n_good;
@@ -171,8 +175,38 @@ __global__ void __launch_bounds__(kSortThreads) tpe_mixture_kernel(const float* 
             const double a = 1.4426950408889634074 / (2.0 * sigma * sigma);
             const double b = log2(w / (wsum * sigma * Z * 2.5066282746310005024));
             out[t] = make_float4((float)mu, (float)a, (float)b, (float)sigma);
+            if (G > 0) {
+                double* par = reinterpret_cast<double*>(keys + count);
+                par[2 * t] = sigma;
+                par[2 * t + 1] = w / (wsum * sigma * Z * 2.5066282746310005024);
+            }
         }
         __syncthreads();
+        if (G > 0) {
+            // (T3g) the mixture at each of the G grid values, in FP64; the warps' sums are added in order
+            const double* par = reinterpret_cast<const double*>(keys + count);
+            for (int v = 0; v < G; ++v) {
+                const double xg = (double)(float)((double)v / (double)(G - 1));
+                double acc = 0.0;
+                for (int t = threadIdx.x; t <= s; t += blockDim.x) {
+                    const double z = (xg - (double)from_ordered_bits((unsigned)(keys[t] >> 32))) / par[2 * t];
+                    acc += par[2 * t + 1] * exp(-0.5 * z * z);
+                }
+                for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+                if ((threadIdx.x & 31) == 0) wsum_s[threadIdx.x / 32] = acc;
+                __syncthreads();
+                if (threadIdx.x == 0) {
+                    double tot = 0.0;
+                    for (int w = 0; w < (int)blockDim.x / 32; ++w) tot += wsum_s[w];
+                    const double lnd = log(tot);
+                    if (set == 0)
+                        lnp_good[v] = lnd;
+                    else
+                        table[(size_t)j * kTpeMaxLevels + v] = (float)(lnp_good[v] - lnd);
+                }
+                __syncthreads();
+            }
+        }
     }
     if (bad) atomicOr(status, DEV_NONFINITE);
 }
@@ -266,7 +300,8 @@ __global__ void __launch_bounds__(kScoreThreads) tpe_score_kernel(const float* _
                 x[r] = row[r][j];
                 bad |= valid[r] && !isfinite(x[r]);
             }
-            const int C = __ldg(levels + j);
+            const int code = __ldg(levels + j);
+            const int C = code < 0 ? -code : code;   // categorical levels, or grid values of an ordinal dimension
             if (C > 0) {
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
@@ -286,6 +321,80 @@ __global__ void __launch_bounds__(kScoreThreads) tpe_score_kernel(const float* _
 #pragma unroll
         for (int r = 0; r < R; ++r)
             if (valid[r]) score[base + (long long)r * kScoreThreads] = acc[r];
+    }
+    if (bad) atomicOr(status, DEV_NONFINITE);
+}
+
+// (T4) when every dimension is tabulated (categorical or grid) and d is a multiple of 4: the score is
+// d look-ups per candidate and the kernel is a streaming read of the pool.  LPC lanes share a candidate
+// (each takes every LPC-th group of four features, a 16-byte load), so that a warp reads whole rows
+// contiguously; their partial sums meet by shuffles.  A lane always serves the same features, so the block
+// keeps a copy of the tables laid out by lane -- entry (iteration, feature-in-group, level) of lane l at
+// word ((it*4 + e)*64 + level)*32 + l -- which makes every look-up conflict-free.  Four candidates per
+// lane group are in flight.
+template <int LPC>
+__global__ void __launch_bounds__(256) tpe_table_score_kernel(const float* __restrict__ Xc, long long m, int d,
+                                                              const int* __restrict__ levels,
+                                                              const float* __restrict__ table,
+                                                              float* __restrict__ score, int* __restrict__ status)
+{
+    constexpr int CPW = 32 / LPC;          // candidates per warp and step
+    constexpr int UNROLL = 4;
+    extern __shared__ float tsm[];         // [iters][4][64][32] tables by lane, then [iters][4][32] level scales
+    const int d4 = d / 4;
+    const int iters = (d4 + LPC - 1) / LPC;
+    float* scale_sm = tsm + (size_t)iters * 4 * kTpeMaxLevels * 32;
+    for (int w = threadIdx.x; w < iters * 4 * kTpeMaxLevels * 32; w += blockDim.x) {
+        const int l = w % 32, v = (w / 32) % kTpeMaxLevels, e = (w / (32 * kTpeMaxLevels)) % 4;
+        const int it = w / (32 * kTpeMaxLevels * 4);
+        const int j4 = l % LPC + it * LPC;
+        tsm[w] = j4 < d4 ? table[(size_t)(4 * j4 + e) * kTpeMaxLevels + v] : 0.f;
+    }
+    for (int w = threadIdx.x; w < iters * 4 * 32; w += blockDim.x) {
+        const int l = w % 32, e = (w / 32) % 4, it = w / 128;
+        const int j4 = l % LPC + it * LPC;
+        const int code = j4 < d4 ? levels[4 * j4 + e] : 2;
+        scale_sm[w] = (float)((code < 0 ? -code : code) - 1);
+    }
+    __syncthreads();
+    const int lane = threadIdx.x % 32, sub = lane % LPC;
+    const long long warp = (long long)blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
+    const long long nwarps = (long long)gridDim.x * (blockDim.x / 32);
+    bool bad = false;
+    for (long long c0 = warp * CPW * UNROLL; c0 < m; c0 += nwarps * CPW * UNROLL) {
+        float acc[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) acc[u] = 0.f;
+        for (int it = 0; it < iters; ++it) {
+            const int j4 = sub + it * LPC;
+            float4 x[UNROLL];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const long long cand = c0 + u * CPW + lane / LPC;
+                x[u] = (cand < m && j4 < d4) ? __ldcs(reinterpret_cast<const float4*>(Xc + (size_t)cand * d) + j4)
+                                             : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float cm1 = scale_sm[(it * 4 + e) * 32 + lane];
+                const float* tl = tsm + (size_t)(it * 4 + e) * kTpeMaxLevels * 32 + lane;
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u) {
+                    const float xe = e == 0 ? x[u].x : (e == 1 ? x[u].y : (e == 2 ? x[u].z : x[u].w));
+                    bad |= !isfinite(xe);
+                    const float lv = floorf(__fadd_rn(__fmul_rn(xe, cm1), 0.5f));
+                    const int v = isfinite(xe) ? (int)fminf(fmaxf(lv, 0.f), cm1) : 0;
+                    acc[u] += tl[v * 32];
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+#pragma unroll
+            for (int o = LPC / 2; o > 0; o >>= 1) acc[u] += __shfl_xor_sync(0xffffffffu, acc[u], o);
+            const long long cand = c0 + u * CPW + lane / LPC;
+            if (sub == 0 && cand < m) score[cand] = acc[u];
+        }
     }
     if (bad) atomicOr(status, DEV_NONFINITE);
 }
@@ -319,7 +428,7 @@ r3_status_t tpe_fit_impl(r3_tpe* t, const float* X, const float* y, cudaStream_t
     R3_LAUNCH(tpe_order_kernel, 1, kSortThreads, 0, stream, y, n, t->order_d, t->status_d);
     int count = 1;
     while (count < n + 1) count <<= 1;
-    const size_t smem = sizeof(unsigned long long) * (size_t)count;
+    const size_t smem = sizeof(unsigned long long) * (size_t)count + sizeof(double) * 2 * ((size_t)n + 2);
     if (smem > 48 * 1024)
         R3_CUDA_TRY(cudaFuncSetAttribute(tpe_mixture_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     R3_LAUNCH(tpe_mixture_kernel, d, kSortThreads, smem, stream, X, t->order_d, n, d, t->n_good, t->levels_d,
@@ -358,8 +467,9 @@ r3_status_t r3_tpe_fit(const float* X, const float* y, const int* levels, int n,
         return R3_ERR_INVALID_ARG;
     }
     for (int j = 0; j < d; ++j)
-        if (levels[j] != 0 && (levels[j] < 2 || levels[j] > kTpeMaxLevels)) {
-            set_error("r3_tpe_fit: levels[%d] = %d; allowed are 0 and 2..%d", j, levels[j], kTpeMaxLevels);
+        if (levels[j] != 0 && (abs(levels[j]) < 2 || abs(levels[j]) > kTpeMaxLevels)) {
+            set_error("r3_tpe_fit: levels[%d] = %d; allowed are 0, 2..%d and -%d..-2", j, levels[j], kTpeMaxLevels,
+                      kTpeMaxLevels);
             return R3_ERR_INVALID_ARG;
         }
     r3_tpe* t = new (std::nothrow) r3_tpe;
@@ -393,6 +503,31 @@ r3_status_t r3_tpe_score(r3_tpe_t* tpe, const float* Xcand, long long m, float* 
         return R3_ERR_INVALID_ARG;
     }
     cudaStream_t stream = (cudaStream_t)cuda_stream;
+    bool all_tables = (tpe->d % 4) == 0 && (reinterpret_cast<uintptr_t>(Xcand) % 16) == 0;
+    for (int j = 0; j < tpe->d && all_tables; ++j) all_tables = tpe->levels[j] != 0;
+    if (all_tables) {
+        // every dimension is a look-up: stream the pool with whole-row loads
+        const int d4 = tpe->d / 4;
+#define R3_TPE_TABLE(LPC)                                                                                      \
+    do {                                                                                                       \
+        const int iters = (d4 + LPC - 1) / LPC;                                                                \
+        const size_t smem = sizeof(float) * (size_t)iters * 4 * 32 * (kTpeMaxLevels + 1);                      \
+        if (smem > 48 * 1024)                                                                                  \
+            R3_CUDA_TRY(cudaFuncSetAttribute(tpe_table_score_kernel<LPC>,                                      \
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));         \
+        const unsigned grid = 148 * (smem > 56 * 1024 ? 2 : 4);                                                \
+        R3_LAUNCH(tpe_table_score_kernel<LPC>, grid, 256, smem, stream, Xcand, m, tpe->d, tpe->levels_d,       \
+                  tpe->table_d, score, tpe->status_d);                                                         \
+    } while (0)
+        if (d4 >= 32) R3_TPE_TABLE(32);
+        else if (d4 >= 16) R3_TPE_TABLE(16);
+        else if (d4 >= 8) R3_TPE_TABLE(8);
+        else if (d4 >= 4) R3_TPE_TABLE(4);
+        else if (d4 >= 2) R3_TPE_TABLE(2);
+        else R3_TPE_TABLE(1);
+#undef R3_TPE_TABLE
+        return R3_OK;
+    }
     // Two candidates per thread (one shared-memory read serves both) when that still gives every SM
     // several blocks; one per thread for small pools.  More per thread measured slower on the full pool
     // (fewer, longer blocks balance worse over the 148 SMs).

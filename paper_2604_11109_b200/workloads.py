@@ -117,13 +117,23 @@ def feature_levels(c: Config):
     return lv
 
 
-def tpe_levels(c: Config) -> np.ndarray:
+def tpe_levels(c: Config, grid: bool = False) -> np.ndarray:
     """Kind of each feature for the Parzen estimator: 0 = ordinal (more than two admissible values),
     2 = a binary flag, treated as a two-level categorical.  The permutation features of config 4 are
-    all ordinal."""
+    all ordinal.  With ``grid`` an ordinal feature whose admissible values are v/(L-1), L <= 64, is
+    declared as such (-L)."""
     if c.cfg == 4:
         return np.zeros(c.d, dtype=np.int32)
-    return np.array([0 if len(l) > 2 else 2 for l in feature_levels(c)], dtype=np.int32)
+    out = []
+    for l in feature_levels(c):
+        L = len(l)
+        if L <= 2:
+            out.append(2)
+        elif grid and L <= 64 and np.allclose(l, np.arange(L) / (L - 1), rtol=0, atol=1e-12):
+            out.append(-L)
+        else:
+            out.append(0)
+    return np.array(out, dtype=np.int32)
 
 
 def _draw_level_idx(rng, levels, count):

@@ -53,6 +53,10 @@ def rand_case(seed, n, d, m, frac_cat=0.4, continuous=True):
             L = int(rng.integers(3, 17))
             X[:, j] = rng.integers(0, L, size=n) / (L - 1)
             Xc[:, j] = rng.integers(0, L, size=m) / (L - 1)
+            if rng.random() < 0.5:
+                levels[j] = -L          # declared as a grid: tabulated by the fit
+                if rng.random() < 0.5:  # and some candidates slightly off the grid
+                    Xc[:, j] += rng.uniform(-0.3, 0.3, m) / (L - 1)
     y = np.round(rng.normal(0, 1, n), 1)      # rounded: ties in y
     return X.astype(np.float32), y.astype(np.float32), levels, Xc.astype(np.float32)
 
@@ -62,7 +66,7 @@ def check_model(tpe, model, n, d):
     assert n_good == model.n_good
     assert order.tolist() == model.order.tolist()
     for j in range(d):
-        if model.levels[j]:
+        if model.levels[j] > 0:
             C = int(model.levels[j])
             want = np.log(model.good[j].prob) - np.log(model.bad[j].prob)
             np.testing.assert_allclose(table[j, :C], want, rtol=1e-6, atol=1e-6)
@@ -84,7 +88,13 @@ def check_model(tpe, model, n, d):
             bb = np.log2(mix.weight / (mix.sigma * mix.Z * np.sqrt(2 * np.pi)))
             np.testing.assert_allclose(np.sort(got[:, 1]), np.sort(a), rtol=3e-7)
             np.testing.assert_allclose(np.sort(got[:, 2]), np.sort(bb), rtol=3e-7, atol=3e-7)
-        assert not table[j].any()
+        if model.levels[j] < 0:
+            L = int(-model.levels[j])
+            xg = (np.arange(L) / (L - 1)).astype(np.float32)
+            want = np.log(T.density(model.good[j], xg)) - np.log(T.density(model.bad[j], xg))
+            np.testing.assert_allclose(table[j, :L], want, rtol=1e-6, atol=1e-6)
+        else:
+            assert not table[j].any()
 
 
 def check_score(got, want, ATOL):
@@ -144,6 +154,32 @@ def test_all_categorical_and_all_ordinal():
         tpe.close()
 
 
+@pytest.mark.parametrize("d,m", [(4, 1000), (8, 5000), (20, 3001), (64, 70000), (132, 2000)])
+def test_all_tabulated_dimensions_take_the_streaming_kernel(d, m):
+    """Every dimension categorical or on a grid and d a multiple of 4: scored by whole-row loads and look-ups."""
+    rng = np.random.default_rng(d)
+    n = 300
+    levels = np.empty(d, dtype=np.int32)
+    X, Xc = np.empty((n, d)), np.empty((m, d))
+    for j in range(d):
+        L = int(rng.integers(2, 33))
+        levels[j] = L if rng.random() < 0.5 else -L
+        X[:, j] = rng.integers(0, L, size=n) / (L - 1)
+        Xc[:, j] = rng.integers(0, L, size=m) / (L - 1)
+    X, Xc = X.astype(np.float32), Xc.astype(np.float32)
+    y = rng.normal(size=n).astype(np.float32)
+    model = T.tpe_fit(X, y, levels, 0.25, 1.0)
+    tpe = b.r3_tpe_fit(dev(X), dev(y), levels, 0.25, 1.0)
+    check_model(tpe, model, n, d)
+    want = T.tpe_score(model, Xc)
+    check_score(b.r3_tpe_score(tpe, dev(Xc)).cpu().numpy(), want, atol(n, levels))
+    # a pool that does not start on a 16-byte boundary goes through the general kernel: same scores
+    shifted = torch.empty(m * d + 1, dtype=torch.float32, device="cuda")[1:].view(m, d)
+    shifted.copy_(dev(Xc))
+    check_score(b.r3_tpe_score(tpe, shifted).cpu().numpy(), want, atol(n, levels))
+    tpe.close()
+
+
 def test_candidates_outside_the_unit_interval():
     X, y, levels, Xc = rand_case(50, 90, 4, 600, frac_cat=0.25)
     Xc = (Xc * 1.3 - 0.15).astype(np.float32)
@@ -153,12 +189,13 @@ def test_candidates_outside_the_unit_interval():
     tpe.close()
 
 
-@pytest.mark.parametrize("cfg,sample", [(1, 4096), (2, 8192), (5, 1024)])
-def test_workloads_full_size(cfg, sample):
+@pytest.mark.parametrize("cfg,sample,grid", [(1, 4096, False), (2, 8192, False), (5, 1024, False), (2, 8192, True),
+                                             (5, 8192, True)])
+def test_workloads_full_size(cfg, sample, grid):
     """The launch configuration the benchmark times, on the whole pool; the oracle on a seeded sample."""
     c = w.get_config(cfg)
     g = w.generate_gp(c, 0)
-    levels = w.tpe_levels(c)
+    levels = w.tpe_levels(c, grid=grid)
     model = T.tpe_fit(g["X"], g["y"], levels, 0.25, 1.0)
     tpe = b.r3_tpe_fit(dev(g["X"]), dev(g["y"]), levels, 0.25, 1.0)
     check_model(tpe, model, c.n, c.d)
@@ -191,7 +228,7 @@ def test_errors():
     with pytest.raises(b.R3Error) as e:
         b.r3_tpe_fit(dev(Xbad), dev(y), levels)
     assert e.value.status == 2
-    for bad_levels in ([1, 0, 0], [0, 65, 0], [0, -2, 0]):
+    for bad_levels in ([1, 0, 0], [0, 65, 0], [0, -1, 0], [0, -65, 0]):
         with pytest.raises(b.R3Error) as e:
             b.r3_tpe_fit(dev(X), dev(y), np.array(bad_levels, dtype=np.int32))
         assert e.value.status == 1

@@ -179,6 +179,20 @@ def test_brute_force_tiny(seed):
                                atol=1e-12)
 
 
+def test_grid_dimension_equals_the_mixture_on_grid_and_snaps_off_grid():
+    rng = np.random.default_rng(21)
+    L = 16
+    X = (rng.integers(0, L, size=(40, 1)) / (L - 1)).astype(np.float32)
+    y = rng.normal(size=40)
+    cont = T.tpe_fit(X, y, [0], gamma=0.25)
+    grid = T.tpe_fit(X, y, [-L], gamma=0.25)
+    on = (np.arange(L) / (L - 1)).astype(np.float32)[:, None]
+    np.testing.assert_array_equal(T.tpe_score(grid, on), T.tpe_score(cont, on))      # on the grid: identical
+    off = (on + np.float32(0.3 / (L - 1))).astype(np.float32)                          # nearer to the same level
+    np.testing.assert_array_equal(T.tpe_score(grid, off), T.tpe_score(cont, on))
+    assert np.abs(T.tpe_score(cont, off) - T.tpe_score(cont, on)).max() > 1e-3         # the mixture itself differs there
+
+
 def test_topk_ties_take_the_lower_index():
     s = np.array([0.5, 2.0, 2.0, -1.0, 2.0, 0.5])
     assert T.tpe_topk(s, 4).tolist() == [1, 2, 4, 0]
