@@ -83,9 +83,13 @@ constexpr uint32_t kZnOffset = 512;                   // float[128] squared norm
 // g owns chunks t = g (mod G) and k* buffer g.  KD: observations per distance product.  KT: the k*
 // buffers (A operand of the variance product) live in TMEM instead of shared memory: shared memory then
 // only feeds the B operands, which is what keeps its 128 B/clk from becoming the limit.
-template <int NV, int G, int KD, bool KT>
+// NBK: number of k* buffers.  NBK == G: group g owns buffer g.  NBK < G (k* in TMEM, where columns are
+// scarce): the buffers form a ring shared by the groups, chunk t uses buffer t mod NBK; a group that has
+// computed its chunk keeps it in registers until the ring slot is free, so the groups still run ahead.
+template <int NV, int G, int KD, bool KT, int NBK = G>
 __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcParams prm)
 {
+    static_assert(NBK == G || (KT && NBK >= 2 && NBK < G), "ring of k* buffers: TMEM only");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -255,7 +259,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
         const uint32_t k_lo0 = desc_addr(base + map.k) | ((2048u >> 4) << 16);
         const uint32_t w_lo0 = desc_addr(base + map.w) | (((NV * 16u) >> 4) << 16);
         uint32_t v_ph = 0;    // parity of the pass counter (V accumulator hand-over)
-        int w_s = 0, k_s = 0;
+        int w_s = 0, k_s = 0, e_s = 0;   // e_s: chunk number mod 4 (ring mode: which "consumed" barrier)
         uint32_t w_ph = 0, k_ph = 0;
         bool ok = true;
         for (long long tile = first_tile; ok && tile < prm.total_tiles; tile += tile_step) {
@@ -271,7 +275,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     if (!(ok = mbar_wait(bar(BAR_K_FULL + b), k_ph, abort_flag))) break;
                     TICK(4);
                     if (!(ok = mbar_wait(bar(BAR_W_FULL + s), w_ph, abort_flag))) break;
-                    if (++k_s == G) { k_s = 0; k_ph ^= 1u; }
+                    if (++k_s == NBK) { k_s = 0; k_ph ^= 1u; }
                     if (++w_s == ws) { w_s = 0; w_ph ^= 1u; }
                     TICK(5);
                     tc_fence_after();
@@ -304,7 +308,8 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                         }
                     }
                     tc_commit(bar(BAR_W_EMPTY + s));
-                    tc_commit(bar(BAR_K_EMPTY + b));
+                    tc_commit(bar(BAR_K_EMPTY + (NBK == G ? b : e_s)));
+                    e_s = (e_s + 1) & 3;
                     if (c == nchunk - 1) {
                         tc_commit(bar(BAR_V_FULL));
                         v_ph ^= 1u;
@@ -434,7 +439,10 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     TICK(0);
                     tc_fence_after();
                     const bool fresh = c >= p * CPP;   // first time this chunk is generated for the tile
-                    uint8_t* kb = sm + map.k + grp * 16384u + row * 16;
+                    // k* buffer and the parity of its hand-over: the group's own buffer, or slot t mod NBK of the ring
+                    const int kbuf = NBK == G ? grp : (int)(t % NBK);
+                    const uint32_t kpar = NBK == G ? own_ph : (uint32_t)((t / NBK) & 1);
+                    uint8_t* kb = sm + map.k + kbuf * 16384u + row * 16;
                     uint32_t kh[KC / 16][8], kl[KC / 16][8];
                     // both halves of the chunk's dot products in one round trip to TMEM, then the buffer is free
                     float dots[KC / 16][16];
@@ -502,7 +510,17 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                         }
                     }
                     TICK(2);
-                    ok = mbar_wait(bar(BAR_K_EMPTY + grp), own_ph ^ 1u, abort_flag);
+                    if (NBK == G) {
+                        ok = mbar_wait(bar(BAR_K_EMPTY + kbuf), kpar ^ 1u, abort_flag);
+                    } else if (t >= NBK) {
+                        // Ring shorter than the number of groups: slot t mod NBK is free once chunk t - NBK has
+                        // been consumed.  A parity wait is only valid at most one phase behind, and with one
+                        // barrier per slot this group could be two uses of its slot ahead of the issuer, or the
+                        // issuer two ahead of the group.  The "consumed" barriers are therefore indexed by the
+                        // chunk number mod 4: the chunks 4 apart that share a barrier are never both pending.
+                        const long long te = t - NBK;
+                        ok = mbar_wait(bar(BAR_K_EMPTY + (int)(te & 3)), (uint32_t)((te >> 2) & 1), abort_flag);
+                    }
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     TICK(3);
@@ -510,8 +528,8 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     for (int h = 0; h < KC / 16; ++h) {
                         if (KT) {
                             // 16 columns = 8 packed TMEM columns of each plane
-                            tc_st8(lane_addr + KCOL + (uint32_t)grp * KC + h * 8, kh[h]);
-                            tc_st8(lane_addr + KCOL + (uint32_t)grp * KC + KC / 2 + h * 8, kl[h]);
+                            tc_st8(lane_addr + KCOL + (uint32_t)kbuf * KC + h * 8, kh[h]);
+                            tc_st8(lane_addr + KCOL + (uint32_t)kbuf * KC + KC / 2 + h * 8, kl[h]);
                         } else {
                             // 16 columns = two 16-byte k-slices of the A operand, hi and lo planes
 #pragma unroll
@@ -530,7 +548,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     } else {
                         fence_proxy_async();
                     }
-                    mbar_arrive(bar(BAR_K_FULL + grp));
+                    mbar_arrive(bar(BAR_K_FULL + kbuf));
                     TICK(4);
                     t += G;
                     own_ph ^= 1u;
@@ -730,8 +748,10 @@ __global__ void wt_build_kernel(const double* __restrict__ W64, int n, int npad_
 
 TensorOperands* ops_of(const r3_gp* gp) { return static_cast<TensorOperands*>(gp->tc); }
 
-void (*kernel_for(int NV, int G, bool kt))(const TcParams)
+void (*kernel_for(int NV, int G, bool kt, int nbk))(const TcParams)
 {
+    if (kt && nbk == 2 && G == 3)
+        return NV == 256 ? score_tc_kernel<256, 3, 64, true, 2> : score_tc_kernel<128, 3, 64, true, 2>;
     if (kt) {
         if (NV == 256) return G == 3 ? score_tc_kernel<256, 3, 64, true> : score_tc_kernel<256, 2, 64, true>;
         return G == 3 ? score_tc_kernel<128, 3, 64, true> : score_tc_kernel<128, 2, 64, true>;
@@ -789,15 +809,19 @@ r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream)
     const int want_kt = env_int("R3_TC_KT", -1), want_g = env_int("R3_TC_G", 0);
     t->KD = 64;
     bool found = false;
-    static const struct { bool kt; int G, min_ws; } prefs[] = {
-        {false, 3, 3}, {true, 3, 3}, {true, 2, 3}, {false, 2, 3}, {false, 3, 2}, {true, 2, 2}, {false, 2, 2}};
+    static const struct { bool kt; int G, min_ws, nbk; } prefs[] = {
+        {true, 3, 3, 2},  {false, 3, 3, 3}, {true, 3, 3, 3}, {true, 2, 3, 2},
+        {false, 2, 3, 2}, {false, 3, 2, 3}, {true, 2, 2, 2}, {false, 2, 2, 2}};
+    const int want_nbk = env_int("R3_TC_NBK", 0);
     for (const auto& pr : prefs) {
         if (found) break;
         t->kt = pr.kt;
         t->G = pr.G;
+        t->nbk = pr.nbk;
         if (want_kt >= 0 && (int)t->kt != want_kt) continue;
         if (want_g && t->G != want_g) continue;
-        if (t->NV + 2 * t->KD + t->DP + (t->kt ? t->G * KC : 0) > 512) continue;
+        if (want_nbk && t->nbk != want_nbk) continue;
+        if (t->NV + 2 * t->KD + t->DP + (t->kt ? t->nbk * KC : 0) > 512) continue;
         for (t->ws = MAX_STAGES; t->ws >= 2; --t->ws)
             if (smem_map(t->DP, t->NV, t->G, t->KD, t->ws, t->kt).bar <= budget) break;
         found = t->ws >= pr.min_ws;
@@ -886,7 +910,7 @@ r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream)
     dev_free(wscale_d);
     wmax_bits = nullptr;
     wscale_d = nullptr;
-    e = cudaFuncSetAttribute(kernel_for(t->NV, t->G, t->kt), cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(kernel_for(t->NV, t->G, t->kt, t->nbk), cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)t->smem_bytes);
     if (e != cudaSuccess) return fail("cudaFuncSetAttribute", e);
     return R3_OK;
@@ -956,7 +980,7 @@ r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, floa
         const r3_status_t st = launch_tc_pair(t, prm, sms, stream);
         if (st != R3_OK) return st;
     } else {
-        void (*kernel)(const TcParams) = kernel_for(t->NV, t->G, t->kt);
+        void (*kernel)(const TcParams) = kernel_for(t->NV, t->G, t->kt, t->nbk);
         R3_LAUNCH(kernel, grid, 128 + 128 * t->G, t->smem_bytes, stream, prm);
     }
     prof_end(gp, stream);

@@ -15,6 +15,7 @@ namespace r3 {
 struct TensorOperands {
     int NV = 0, G = 0, KD = 0, DP = 0, NP = 0, P = 0, ws = 0;
     bool kt = false;           // k* buffers in TMEM
+    int nbk = 0;               // number of k* buffers (== G: one per group; smaller: a shared ring)
     size_t smem_bytes = 0;
     size_t wt_gp_stride = 0;   // halves per GP in wt
     float* centre = nullptr;   // [B][DP]  column means of X (zero padded)
