@@ -3,9 +3,8 @@
 // A value and its index are packed in one 64-bit key whose unsigned order is exactly
 // (value descending-friendly, index ascending): the float is mapped to an order-preserving unsigned
 // integer in the high word and the low word holds ~index, so "larger key" means "larger value, or
-// equal value and smaller index".  A block sorts a chunk of 4096 keys (bitonic network held in registers,
-// exchanged by warp shuffles and, for the long distances, through shared memory) and emits its k
-// largest; levels repeat until one chunk is left, whose k largest are the answer.
+// equal value and smaller index".  A block sorts a chunk of keys in shared memory (bitonic network)
+// and emits its k largest; levels repeat until one chunk is left, whose k largest are the answer.
 // The first level reads the EI array once (4 bytes per candidate); later levels touch k keys per
 // chunk of the level before.
 #include <mutex>
@@ -33,65 +32,25 @@ __device__ __forceinline__ unsigned long long make_key(float v, unsigned idx)
     return ((unsigned long long)u << 32) | (unsigned long long)(0xFFFFFFFFu - idx);
 }
 
-__device__ __forceinline__ unsigned long long shfl_xor_u64(unsigned long long v, int lane_mask)
+// Sort CHUNK keys descending in shared memory.
+__device__ __forceinline__ void bitonic_sort_desc(unsigned long long* s)
 {
-    const unsigned lo = __shfl_xor_sync(0xffffffffu, (unsigned)v, lane_mask);
-    const unsigned hi = __shfl_xor_sync(0xffffffffu, (unsigned)(v >> 32), lane_mask);
-    return ((unsigned long long)hi << 32) | lo;
-}
-
-// Bitonic sort of CHUNK = 4 * THREADS keys, descending.  Thread t owns the keys 4t .. 4t+3 in registers:
-// compare-exchanges at distance 1 and 2 stay inside a thread, distances 4 .. 64 are warp shuffles, and only
-// the distances of 128 and more (15 of the 78 steps) go through shared memory.
-__device__ __forceinline__ void bitonic_sort_desc(unsigned long long (&k)[4], unsigned long long* s)
-{
-    const int t = threadIdx.x;
-#pragma unroll 1
     for (int size = 2; size <= CHUNK; size <<= 1) {
-#pragma unroll 1
         for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            if (stride >= 128) {
-                // partner keys live in another warp
-                __syncthreads();
-#pragma unroll
-                for (int r = 0; r < 4; ++r) s[4 * t + r] = k[r];
-                __syncthreads();
-                const int pt = t ^ (stride >> 2);
-                const bool lower = (t & (stride >> 2)) == 0;
-                const bool desc = ((4 * t) & size) == 0;
-#pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    const unsigned long long o = s[4 * pt + r];
-                    const bool take_max = lower == desc;
-                    k[r] = take_max ? (k[r] > o ? k[r] : o) : (k[r] < o ? k[r] : o);
-                }
-            } else if (stride >= 4) {
-                const int lm = stride >> 2;
-                const bool lower = (t & lm) == 0;
-                const bool desc = ((4 * t) & size) == 0;
-                const bool take_max = lower == desc;
-#pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    const unsigned long long o = shfl_xor_u64(k[r], lm);
-                    k[r] = take_max ? (k[r] > o ? k[r] : o) : (k[r] < o ? k[r] : o);
-                }
-            } else {
-                // stride 1 or 2: both keys in this thread
-#pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    const int p = r ^ stride;
-                    if (p > r) {
-                        const bool desc = ((4 * t + r) & size) == 0;
-                        const unsigned long long a = k[r], b = k[p];
-                        if ((a < b) == desc) {
-                            k[r] = b;
-                            k[p] = a;
-                        }
-                    }
+            __syncthreads();
+            for (int t = threadIdx.x; t < CHUNK / 2; t += THREADS) {
+                const int lo = 2 * t - (t & (stride - 1));
+                const int hi = lo + stride;
+                const bool desc = ((lo & size) == 0);
+                const unsigned long long a = s[lo], b = s[hi];
+                if ((a < b) == desc) {
+                    s[lo] = b;
+                    s[hi] = a;
                 }
             }
         }
     }
+    __syncthreads();
 }
 
 // Level 0: keys from the EI array.  grid = (chunks, batch).
@@ -102,20 +61,13 @@ __global__ void __launch_bounds__(THREADS) topk_from_values_kernel(const float* 
     const int g = blockIdx.y;
     const long long base = (long long)blockIdx.x * CHUNK;
     const float* e = ei + (size_t)g * m;
-    // coalesced read through shared memory, then four consecutive keys per thread
     for (int t = threadIdx.x; t < CHUNK; t += THREADS) {
         const long long i = base + t;
         s[t] = (i < m) ? make_key(e[i], (unsigned)i) : 0ull;
     }
-    __syncthreads();
-    unsigned long long key[4];
-#pragma unroll
-    for (int r = 0; r < 4; ++r) key[r] = s[4 * threadIdx.x + r];
-    bitonic_sort_desc(key, s);
+    bitonic_sort_desc(s);
     unsigned long long* o = out + ((size_t)g * gridDim.x + blockIdx.x) * k;
-#pragma unroll
-    for (int r = 0; r < 4; ++r)
-        if (4 * (int)threadIdx.x + r < k) o[4 * threadIdx.x + r] = key[r];
+    for (int t = threadIdx.x; t < k; t += THREADS) o[t] = s[t];
 }
 
 // Later levels: keys from the level before.  count = keys per GP in `in`.
@@ -127,17 +79,13 @@ __global__ void __launch_bounds__(THREADS) topk_from_keys_kernel(const unsigned 
     const int g = blockIdx.y;
     const long long base = (long long)blockIdx.x * CHUNK;
     const unsigned long long* src = in + (size_t)g * count;
-    unsigned long long key[4];
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-        const long long i = base + 4 * threadIdx.x + r;
-        key[r] = (i < count) ? src[i] : 0ull;
+    for (int t = threadIdx.x; t < CHUNK; t += THREADS) {
+        const long long i = base + t;
+        s[t] = (i < count) ? src[i] : 0ull;
     }
-    bitonic_sort_desc(key, s);
+    bitonic_sort_desc(s);
     unsigned long long* o = out + ((size_t)g * gridDim.x + blockIdx.x) * k;
-#pragma unroll
-    for (int r = 0; r < 4; ++r)
-        if (4 * (int)threadIdx.x + r < k) o[4 * threadIdx.x + r] = key[r];
+    for (int t = threadIdx.x; t < k; t += THREADS) o[t] = s[t];
 }
 
 __global__ void topk_write_kernel(const unsigned long long* __restrict__ keys, const float* __restrict__ ei,
