@@ -211,6 +211,40 @@ r3_status_t r3_gp_profile_read(r3_gp_t* gp, double* kernel_ms, long long* launch
 r3_status_t r3_gp_lml(r3_gp_t* gp, double* lml, double* grad, void* cuda_stream);
 
 /*
+ * r3_gp_refit -- condition the GPs of the handle on the same histories with other hyper-parameters
+ * (arguments as for r3_gp_fit; the histories are the ones the handle holds, appended observations
+ * included).  Synchronises.  On R3_ERR_NOT_PD the handle is refitted with its previous
+ * hyper-parameters and stays usable.
+ */
+r3_status_t r3_gp_refit(r3_gp_t* gp, const float* lengthscales, const float* signal_var, const float* noise_var,
+                        void* cuda_stream);
+
+/*
+ * r3_gp_optimize -- choose the hyper-parameters of every GP of the handle by maximising its log
+ * marginal likelihood (r3_gp_lml) over theta = (log lengthscale_1..d, log signal_var, log noise_var),
+ * starting from the handle's current values.  (The paper passes hyper-parameters in and gives no rule
+ * for them; this is the usual type-II maximum likelihood.)
+ *
+ * Limited-memory BFGS (8 pairs) with a backtracking Armijo line search, one optimiser per GP, all GPs
+ * evaluated together: an evaluation is one batched refit plus one r3_gp_lml.  theta is kept inside
+ * lengthscale in [1e-3, 1e3], signal_var in [1e-6, 1e6], noise_var in [1e-8 , 1e2] by projection.
+ * A GP stops when the largest projected gradient component falls below gtol or its line search
+ * cannot improve; the call stops when every GP has stopped or after max_evals evaluations.  A trial
+ * point at which some covariance matrix is not positive definite counts as a failed step for every GP
+ * still searching (their steps are halved).
+ *
+ *   max_evals >= 1, gtol > 0
+ *   lengthscales host [batch][d], signal_var host [batch], noise_var host [batch]   outputs (FP32), any may be NULL
+ *   lml          host [batch]   the log marginal likelihood reached, or NULL
+ *   evals        host [1]       evaluations used, or NULL
+ *
+ * On return the handle is fitted with the returned hyper-parameters (never worse than the start).
+ * Synchronises.
+ */
+r3_status_t r3_gp_optimize(r3_gp_t* gp, int max_evals, double gtol, float* lengthscales, float* signal_var,
+                           float* noise_var, double* lml, int* evals, void* cuda_stream);
+
+/*
  * r3_gp_propose -- q distinct pool members to replay in parallel, chosen greedily by fantasies.
  *
  * Section IV runs a parallel search: several points are in flight at once.  The paper gives no rule

@@ -41,6 +41,8 @@ SIGNATURES = {
     "r3_trim_cache": (None, []),
     "r3_cached_bytes": (_ull, []),
     "r3_gp_lml": (_i, [_vp, _vp, _vp, _vp]),
+    "r3_gp_refit": (_i, [_vp, _fp, _fp, _fp, _vp]),
+    "r3_gp_optimize": (_i, [_vp, _i, ctypes.c_double, _vp, _vp, _vp, _vp, ctypes.POINTER(ctypes.c_int), _vp]),
     "r3_gp_propose": (_i, [_vp, _vp, _ll, _i, _i, _i, _vp, _vp, ctypes.POINTER(ctypes.c_int), _vp]),
     "r3_gp_append": (_i, [_vp, _vp, _vp, _i, _vp]),
     "r3_gp_size": (_i, [_vp]),
@@ -247,6 +249,28 @@ def r3_gp_lml(gp: GP):
     grad = np.empty((gp.batch, gp.d + 2), dtype=np.float64)
     _check(load().r3_gp_lml(gp.handle, ctypes.c_void_p(lml.ctypes.data), ctypes.c_void_p(grad.ctypes.data), _stream()))
     return lml, grad
+
+
+def r3_gp_refit(gp: GP, lengthscales, signal_var, noise_var):
+    """Condition the handle's histories on other hyper-parameters (host arrays as for r3_gp_fit)."""
+    ell, ell_p = _host_f32(lengthscales, (gp.batch, gp.d), "lengthscales")
+    sf2, sf2_p = _host_f32(signal_var, (gp.batch,), "signal_var")
+    sn2, sn2_p = _host_f32(noise_var, (gp.batch,), "noise_var")
+    _check(load().r3_gp_refit(gp.handle, ell_p, sf2_p, sn2_p, _stream()))
+
+
+def r3_gp_optimize(gp: GP, max_evals: int = 60, gtol: float = 1e-3):
+    """Maximise the log marginal likelihood over the hyper-parameters: returns (lengthscales [batch][d],
+    signal_var [batch], noise_var [batch], lml [batch], evaluations used)."""
+    ell = np.empty((gp.batch, gp.d), dtype=np.float32)
+    sf2 = np.empty((gp.batch,), dtype=np.float32)
+    sn2 = np.empty((gp.batch,), dtype=np.float32)
+    lml = np.empty((gp.batch,), dtype=np.float64)
+    used = ctypes.c_int()
+    _check(load().r3_gp_optimize(gp.handle, int(max_evals), float(gtol), ctypes.c_void_p(ell.ctypes.data),
+                                 ctypes.c_void_p(sf2.ctypes.data), ctypes.c_void_p(sn2.ctypes.data),
+                                 ctypes.c_void_p(lml.ctypes.data), ctypes.byref(used), _stream()))
+    return ell, sf2, sn2, lml, used.value
 
 
 def r3_gp_propose(gp: GP, Xcand, q: int, shortlist: int = 0, lie: str = "believer"):
