@@ -303,6 +303,51 @@ void r3_launch_count_reset(void);
 void r3_gp_free(r3_gp_t* gp);
 
 /* ------------------------------------------------------------------------------------------------
+ * The inner search as a whole (Section IV, the loop inside the replay server): fit the surrogate,
+ * propose a batch of points to replay in parallel, replay them, discard the configurations that make
+ * the kernel incorrect, add the rest to the history, repeat until a stopping rule fires, return the
+ * best configuration found.  The three stopping rules are the paper's: a maximum number of
+ * iterations, a maximum wall-clock time, a number of iterations without improvement.
+ *
+ * The replay itself is the caller's: `evaluate` gets q configurations (host, [q][d], rows of the pool)
+ * and returns a value for each (smaller is better) and whether the kernel stayed correct (valid[i] != 0).
+ * It returns 0 to go on, anything else to stop the search.
+ */
+typedef int (*r3_evaluate_fn)(const float* x, int q, int d, float* y, int* valid, void* user);
+
+typedef struct {
+    int q;               /* points proposed per round, 1..128 */
+    int max_rounds;      /* stop after this many rounds, >= 1 */
+    double max_seconds;  /* stop when this much wall-clock time has passed, <= 0: no limit */
+    int patience;        /* stop after this many rounds in a row without a better value, <= 0: no limit */
+    int optimize_every;  /* refit the hyper-parameters by r3_gp_optimize every this many rounds, <= 0: never */
+    int lie;             /* fantasised value of r3_gp_propose: 0 believer, 1 liar */
+} r3_bo_options_t;
+
+typedef enum {
+    R3_BO_MAX_ROUNDS = 0, R3_BO_MAX_SECONDS = 1, R3_BO_NO_IMPROVEMENT = 2, R3_BO_POOL_EXHAUSTED = 3,
+    R3_BO_HISTORY_FULL = 4, R3_BO_STOPPED_BY_CALLER = 5
+} r3_bo_stop_t;
+
+/*
+ * r3_bo_run -- the loop above on one GP.
+ *
+ *   X0, y0     device [n0][d], [n0]   initial history (n0 >= 1)
+ *   lengthscales host [d], signal_var, noise_var: starting hyper-parameters
+ *   pool       device [m][d]          candidate configurations; the call works on a private copy from which
+ *                                     every proposed row is removed, so no configuration is replayed twice
+ *   best_x     host [d], best_y host [1]: the best valid configuration seen (initial history included)
+ *   rounds, evaluated, discarded, stop_reason: host [1] each, any may be NULL
+ *   gp_out     if not NULL receives the final handle (the caller frees it); otherwise it is freed
+ *
+ * Every proposal is made by r3_gp_propose, every update by r3_gp_append.  Synchronises.
+ */
+r3_status_t r3_bo_run(const float* X0, const float* y0, int n0, int d, const float* lengthscales, float signal_var,
+                      float noise_var, const float* pool, long long m, const r3_bo_options_t* options,
+                      r3_evaluate_fn evaluate, void* user, float* best_x, float* best_y, int* rounds, int* evaluated,
+                      int* discarded, int* stop_reason, r3_gp_t** gp_out, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------------
  * Tree-structured Parzen Estimator (TPE) candidate scoring.
  *
  * Section VII-C: inside the replay server the paper's experiments tune pass order and launch

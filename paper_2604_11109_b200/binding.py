@@ -33,6 +33,14 @@ _vp, _i, _ll, _ull = ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong, ctypes.c_
 _fp = ctypes.POINTER(ctypes.c_float)
 
 # name -> (restype, argtypes); every symbol include/r3.h declares
+class BoOptions(ctypes.Structure):
+    _fields_ = [("q", ctypes.c_int), ("max_rounds", ctypes.c_int), ("max_seconds", ctypes.c_double),
+                ("patience", ctypes.c_int), ("optimize_every", ctypes.c_int), ("lie", ctypes.c_int)]
+
+
+EVALUATE_FN = ctypes.CFUNCTYPE(ctypes.c_int, ctypes.POINTER(ctypes.c_float), ctypes.c_int, ctypes.c_int,
+                               ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int), ctypes.c_void_p)
+
 SIGNATURES = {
     "r3_gp_fit": (_i, [_vp, _vp, _fp, _fp, _fp, _i, _i, _i, _vp, ctypes.POINTER(_vp)]),
     "r3_gp_score": (_i, [_vp, _vp, _ll, _vp, _vp, _vp, _vp]),
@@ -41,6 +49,9 @@ SIGNATURES = {
     "r3_trim_cache": (None, []),
     "r3_cached_bytes": (_ull, []),
     "r3_gp_lml": (_i, [_vp, _vp, _vp, _vp]),
+    "r3_bo_run": (_i, [_vp, _vp, _i, _i, _fp, ctypes.c_float, ctypes.c_float, _vp, _ll, ctypes.POINTER(BoOptions),
+                       EVALUATE_FN, _vp, _fp, _fp, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int),
+                       ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int), ctypes.POINTER(_vp), _vp]),
     "r3_gp_refit": (_i, [_vp, _fp, _fp, _fp, _vp]),
     "r3_gp_optimize": (_i, [_vp, _i, ctypes.c_double, _vp, _vp, _vp, _vp, ctypes.POINTER(ctypes.c_int), _vp]),
     "r3_gp_propose": (_i, [_vp, _vp, _ll, _i, _i, _i, _vp, _vp, ctypes.POINTER(ctypes.c_int), _vp]),
@@ -249,6 +260,57 @@ def r3_gp_lml(gp: GP):
     grad = np.empty((gp.batch, gp.d + 2), dtype=np.float64)
     _check(load().r3_gp_lml(gp.handle, ctypes.c_void_p(lml.ctypes.data), ctypes.c_void_p(grad.ctypes.data), _stream()))
     return lml, grad
+
+
+STOP_REASONS = ("max_rounds", "max_seconds", "no_improvement", "pool_exhausted", "history_full", "stopped_by_caller")
+
+
+def r3_bo_run(X0, y0, lengthscales, signal_var, noise_var, pool, evaluate, q=8, max_rounds=10, max_seconds=0.0,
+              patience=0, optimize_every=0, lie="believer", keep_handle=False):
+    """The whole inner search on one GP.  ``evaluate(x)`` gets a float32 array [q][d] of configurations and
+    returns (y [q], valid [q]) or (y, valid, stop).  Returns a dict with best_x, best_y, rounds, evaluated,
+    discarded, stop_reason (and ``gp`` when keep_handle)."""
+    n0, d = X0.shape
+    m = int(pool.shape[0])
+    ell, ell_p = _host_f32(lengthscales, (d,), "lengthscales")
+    opts = BoOptions(int(q), int(max_rounds), float(max_seconds), int(patience), int(optimize_every),
+                     {"believer": 0, "liar": 1}[lie])
+    failure = []
+
+    def trampoline(xp, qq, dd, yp, vp, _user):
+        try:
+            x = np.ctypeslib.as_array(xp, shape=(qq, dd)).copy()
+            out = evaluate(x)
+            y, valid = np.asarray(out[0], dtype=np.float32), np.asarray(out[1])
+            for i in range(qq):
+                yp[i] = float(y[i])
+                vp[i] = int(bool(valid[i]))
+            return int(bool(out[2])) if len(out) > 2 else 0
+        except Exception as exc:  # an exception must not cross the C boundary
+            failure.append(exc)
+            for i in range(qq):
+                vp[i] = 0      # nothing of this round enters the history
+            return 1
+
+    cb = EVALUATE_FN(trampoline)
+    best_x = np.empty((d,), dtype=np.float32)
+    best_y = ctypes.c_float()
+    rounds, evaluated, discarded, reason = ctypes.c_int(), ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+    handle = ctypes.c_void_p()
+    _check(load().r3_bo_run(_dev_f32(X0, "X0"), _dev_f32(y0, "y0"), n0, d, ell_p, float(signal_var), float(noise_var),
+                            _dev_f32(pool, "pool"), m, ctypes.byref(opts), cb, None, best_x.ctypes.data_as(_fp),
+                            ctypes.byref(best_y), ctypes.byref(rounds), ctypes.byref(evaluated), ctypes.byref(discarded),
+                            ctypes.byref(reason), ctypes.byref(handle) if keep_handle else None, _stream()))
+    if failure:
+        if keep_handle and handle.value:
+            load().r3_gp_free(handle)
+        raise failure[0]
+    out = {"best_x": best_x, "best_y": float(best_y.value), "rounds": rounds.value, "evaluated": evaluated.value,
+           "discarded": discarded.value, "stop_reason": STOP_REASONS[reason.value]}
+    if keep_handle:
+        n = int(load().r3_gp_size(handle))
+        out["gp"] = GP(handle.value, 1, n, d)
+    return out
 
 
 def r3_gp_refit(gp: GP, lengthscales, signal_var, noise_var):

@@ -16,7 +16,8 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libr3gp.so")
 SOURCES = ["r3_api.cu", "r3_fit.cu", "r3_score_simt.cu", "r3_rescue.cu", "r3_score_tc.cu", "r3_score_tc2.cu", "r3_topk.cu",
-           "r3_tpe.cu", "r3_alloc.cu", "r3_propose.cu", "r3_lml.cu", "r3_optimize.cu"]
+           "r3_tpe.cu", "r3_alloc.cu", "r3_propose.cu", "r3_lml.cu", "r3_optimize.cu",
+           "r3_driver.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
 

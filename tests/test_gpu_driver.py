@@ -1,0 +1,132 @@
+"""GPU tests of r3_bo_run, the inner search as one call (fit, propose a batch, replay through a callback,
+discard incorrect configurations, append, stop by one of the paper's three rules).
+
+Parity: the whole trajectory -- which configurations are sent to the callback, round after round --
+must be the one the oracle produces when the same loop is driven by its own definitions (refit of the
+augmented history, rescoring, greedy batch by fantasies).
+"""
+import time
+
+import numpy as np
+import pytest
+
+from oracle import gp_oracle as o
+from paper_2604_11109_b200 import binding as b
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def objective(x):
+    x = np.asarray(x, dtype=np.float64)
+    return (np.sin(5.0 * x[:, 0]) + ((x - 0.35) ** 2).sum(axis=1) * 2.0).astype(np.float32)
+
+
+def setup(seed, n0, d, m):
+    rng = np.random.default_rng(seed)
+    X0 = rng.uniform(0, 1, (n0, d)).astype(np.float32)
+    pool = rng.uniform(0, 1, (m, d)).astype(np.float32)
+    return X0, objective(X0), pool, np.full(d, 0.4, np.float32), np.float32(1.0), np.float32(1e-3)
+
+
+def oracle_loop(X0, y0, pool, ell, sf2, sn2, q, rounds, lie, is_valid):
+    X, y, pool = X0.copy(), y0.copy(), pool.copy()
+    sent = []
+    for _ in range(rounds):
+        qq = min(q, pool.shape[0])
+        idx, _ = o.propose(X, y, ell, sf2, sn2, pool, qq, lie)
+        rows = pool[idx]
+        sent.append(rows.copy())
+        vals, ok = objective(rows), is_valid(rows)
+        X = np.concatenate([X, rows[ok]])
+        y = np.concatenate([y, vals[ok]])
+        pool = np.delete(pool, idx, axis=0)
+    return sent, X, y
+
+
+@pytest.mark.parametrize("lie", ["believer", "liar"])
+def test_trajectory_matches_the_oracle_loop(lie):
+    X0, y0, pool, ell, sf2, sn2 = setup(0, 12, 3, 400)
+    is_valid = lambda r: r[:, 1] < 0.8                       # "incorrect kernels" in one corner of the space
+    sent = []
+
+    def evaluate(x):
+        sent.append(x.copy())
+        return objective(x), is_valid(x)
+
+    res = b.r3_bo_run(dev(X0), dev(y0), ell, sf2, sn2, dev(pool), evaluate, q=4, max_rounds=5, lie=lie,
+                      keep_handle=True)
+    ref_sent, Xr, yr = oracle_loop(X0, y0, pool, ell, sf2, sn2, 4, 5, lie, is_valid)
+    assert res["rounds"] == 5 and res["stop_reason"] == "max_rounds" and res["evaluated"] == 20
+    for got, want in zip(sent, ref_sent):
+        np.testing.assert_array_equal(got, want)
+    assert res["discarded"] == sum(int((~is_valid(r)).sum()) for r in ref_sent)
+    # the handle at the end holds exactly the valid observations, and the best of them is reported
+    gp = res["gp"]
+    assert b.r3_gp_size(gp) == yr.shape[0]
+    alpha, L = b.r3_gp_get_factor(gp)
+    f = o.fit(Xr, yr, ell, sf2, sn2)
+    assert np.allclose(L[0], f.L, rtol=1e-8, atol=1e-10)
+    assert res["best_y"] == yr.min()
+    np.testing.assert_array_equal(res["best_x"], Xr[int(np.argmin(yr))])
+    gp.close()
+
+
+def test_stopping_rules():
+    X0, y0, pool, ell, sf2, sn2 = setup(1, 10, 2, 300)
+    flat = lambda x: (np.full(x.shape[0], 5.0, np.float32), np.ones(x.shape[0], bool))      # never improves
+    res = b.r3_bo_run(dev(X0), dev(y0), ell, sf2, sn2, dev(pool), flat, q=3, max_rounds=50, patience=4)
+    assert res["stop_reason"] == "no_improvement" and res["rounds"] == 4
+    assert res["best_y"] == y0.min()
+
+    def slow(x):
+        time.sleep(0.05)
+        return objective(x), np.ones(x.shape[0], bool)
+
+    res = b.r3_bo_run(dev(X0), dev(y0), ell, sf2, sn2, dev(pool), slow, q=2, max_rounds=1000, max_seconds=0.3)
+    assert res["stop_reason"] == "max_seconds" and 1 <= res["rounds"] <= 7
+
+    calls = []
+
+    def stop_after_two(x):
+        calls.append(1)
+        return objective(x), np.ones(x.shape[0], bool), len(calls) >= 2
+
+    res = b.r3_bo_run(dev(X0), dev(y0), ell, sf2, sn2, dev(pool), stop_after_two, q=2, max_rounds=10)
+    assert res["stop_reason"] == "stopped_by_caller" and res["rounds"] == 2 and res["evaluated"] == 4
+
+    tiny = pool[:10]
+    seen = []
+
+    def record(x):
+        seen.append(x.copy())
+        return objective(x), np.ones(x.shape[0], bool)
+
+    res = b.r3_bo_run(dev(X0), dev(y0), ell, sf2, sn2, dev(tiny), record, q=4, max_rounds=10)
+    assert res["stop_reason"] == "pool_exhausted" and res["evaluated"] == 10
+    allrows = np.concatenate(seen)
+    assert len({r.tobytes() for r in allrows}) == 10          # every configuration replayed exactly once
+
+
+def test_search_improves_and_refits_hyper_parameters():
+    X0, y0, pool, ell, sf2, sn2 = setup(2, 8, 2, 5000)
+    res = b.r3_bo_run(dev(X0), dev(y0), ell, sf2, sn2, dev(pool), lambda x: (objective(x), np.ones(len(x), bool)),
+                      q=8, max_rounds=6, optimize_every=2)
+    assert res["rounds"] == 6 and res["evaluated"] == 48
+    assert res["best_y"] < y0.min()
+    # 48 replays should land within a small distance of the pool's best value
+    assert res["best_y"] <= np.sort(objective(pool))[25]
+
+
+def test_an_exception_in_the_callback_surfaces():
+    X0, y0, pool, ell, sf2, sn2 = setup(3, 6, 2, 100)
+
+    def broken(x):
+        raise RuntimeError("replay failed")
+
+    with pytest.raises(RuntimeError):
+        b.r3_bo_run(dev(X0), dev(y0), ell, sf2, sn2, dev(pool), broken, q=2, max_rounds=3)
