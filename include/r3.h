@@ -322,6 +322,11 @@ typedef struct {
     int patience;        /* stop after this many rounds in a row without a better value, <= 0: no limit */
     int optimize_every;  /* refit the hyper-parameters by r3_gp_optimize every this many rounds, <= 0: never */
     int lie;             /* fantasised value of r3_gp_propose: 0 believer, 1 liar */
+    int surrogate;       /* 0: Gaussian process (r3_gp_fit / r3_gp_propose / r3_gp_append);
+                            1: Tree-Parzen estimator, the paper's choice (Section VII-C: parallel TPE): every round
+                               r3_tpe_fit on the history so far, r3_tpe_score on the pool, the q best by r3_topk */
+    const int* levels;   /* surrogate 1: kind of each feature as for r3_tpe_fit, host [d]; NULL = all ordinal */
+    float gamma;         /* surrogate 1: good fraction, <= 0: 0.25 */
 } r3_bo_options_t;
 
 typedef enum {
@@ -340,7 +345,9 @@ typedef enum {
  *   rounds, evaluated, discarded, stop_reason: host [1] each, any may be NULL
  *   gp_out     if not NULL receives the final handle (the caller frees it); otherwise it is freed
  *
- * Every proposal is made by r3_gp_propose, every update by r3_gp_append.  Synchronises.
+ * With the GP every proposal is made by r3_gp_propose and every update by r3_gp_append; with the Parzen
+ * estimator the hyper-parameter arguments are ignored, gp_out receives NULL and the history is refitted
+ * every round (its fit is a few sorts).  Synchronises.
  */
 r3_status_t r3_bo_run(const float* X0, const float* y0, int n0, int d, const float* lengthscales, float signal_var,
                       float noise_var, const float* pool, long long m, const r3_bo_options_t* options,

@@ -35,7 +35,8 @@ _fp = ctypes.POINTER(ctypes.c_float)
 # name -> (restype, argtypes); every symbol include/r3.h declares
 class BoOptions(ctypes.Structure):
     _fields_ = [("q", ctypes.c_int), ("max_rounds", ctypes.c_int), ("max_seconds", ctypes.c_double),
-                ("patience", ctypes.c_int), ("optimize_every", ctypes.c_int), ("lie", ctypes.c_int)]
+                ("patience", ctypes.c_int), ("optimize_every", ctypes.c_int), ("lie", ctypes.c_int),
+                ("surrogate", ctypes.c_int), ("levels", ctypes.POINTER(ctypes.c_int)), ("gamma", ctypes.c_float)]
 
 
 EVALUATE_FN = ctypes.CFUNCTYPE(ctypes.c_int, ctypes.POINTER(ctypes.c_float), ctypes.c_int, ctypes.c_int,
@@ -266,15 +267,17 @@ STOP_REASONS = ("max_rounds", "max_seconds", "no_improvement", "pool_exhausted",
 
 
 def r3_bo_run(X0, y0, lengthscales, signal_var, noise_var, pool, evaluate, q=8, max_rounds=10, max_seconds=0.0,
-              patience=0, optimize_every=0, lie="believer", keep_handle=False):
+              patience=0, optimize_every=0, lie="believer", keep_handle=False, surrogate="gp", levels=None, gamma=0.25):
     """The whole inner search on one GP.  ``evaluate(x)`` gets a float32 array [q][d] of configurations and
     returns (y [q], valid [q]) or (y, valid, stop).  Returns a dict with best_x, best_y, rounds, evaluated,
     discarded, stop_reason (and ``gp`` when keep_handle)."""
     n0, d = X0.shape
     m = int(pool.shape[0])
     ell, ell_p = _host_f32(lengthscales, (d,), "lengthscales")
+    lv = None if levels is None else np.ascontiguousarray(np.asarray(levels, dtype=np.int32))
     opts = BoOptions(int(q), int(max_rounds), float(max_seconds), int(patience), int(optimize_every),
-                     {"believer": 0, "liar": 1}[lie])
+                     {"believer": 0, "liar": 1}[lie], {"gp": 0, "tpe": 1}[surrogate],
+                     None if lv is None else lv.ctypes.data_as(ctypes.POINTER(ctypes.c_int)), float(gamma))
     failure = []
 
     def trampoline(xp, qq, dd, yp, vp, _user):
@@ -307,7 +310,7 @@ def r3_bo_run(X0, y0, lengthscales, signal_var, noise_var, pool, evaluate, q=8, 
         raise failure[0]
     out = {"best_x": best_x, "best_y": float(best_y.value), "rounds": rounds.value, "evaluated": evaluated.value,
            "discarded": discarded.value, "stop_reason": STOP_REASONS[reason.value]}
-    if keep_handle:
+    if keep_handle and handle.value:
         n = int(load().r3_gp_size(handle))
         out["gp"] = GP(handle.value, 1, n, d)
     return out

@@ -67,20 +67,33 @@ r3_status_t r3_bo_run(const float* X0, const float* y0, int n0, int d, const flo
         set_error("r3_bo_run: need 1 <= q <= %d, max_rounds >= 1, 1 <= m < 2^31, lie in {0, 1}", kAppendMax);
         return R3_ERR_INVALID_ARG;
     }
+    if (opt.surrogate != 0 && opt.surrogate != 1) {
+        set_error("r3_bo_run: surrogate must be 0 (GP) or 1 (TPE)");
+        return R3_ERR_INVALID_ARG;
+    }
+    const bool tpe = opt.surrogate == 1;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     r3_gp_t* gp = nullptr;
-    r3_status_t st = r3_gp_fit(X0, y0, lengthscales, &signal_var, &noise_var, 1, n0, d, cuda_stream, &gp);
-    if (st != R3_OK) return st;
+    r3_status_t st = R3_OK;
+    if (!tpe) {
+        st = r3_gp_fit(X0, y0, lengthscales, &signal_var, &noise_var, 1, n0, d, cuda_stream, &gp);
+        if (st != R3_OK) return st;
+    }
 
-    float *work = nullptr, *rows_d = nullptr, *y_d = nullptr;
+    float *work = nullptr, *rows_d = nullptr, *y_d = nullptr, *hist_x = nullptr, *hist_y = nullptr, *score = nullptr;
     int* idx_d = nullptr;
+    void* topk_ws = nullptr;
     auto done = [&](r3_status_t s) {
         cudaStreamSynchronize(stream);
         dev_free(work);
         dev_free(rows_d);
         dev_free(y_d);
         dev_free(idx_d);
-        if (s == R3_OK && gp_out)
+        dev_free(hist_x);
+        dev_free(hist_y);
+        dev_free(score);
+        dev_free(topk_ws);
+        if (s == R3_OK && gp_out && gp)
             *gp_out = gp;
         else
             r3_gp_free(gp);
@@ -99,6 +112,23 @@ r3_status_t r3_bo_run(const float* X0, const float* y0, int n0, int d, const flo
     TRY_DONE(dev_malloc(&y_d, sizeof(float) * (size_t)opt.q));
     TRY_DONE(dev_malloc(&idx_d, sizeof(int) * (size_t)opt.q));
     TRY_DONE(cudaMemcpyAsync(work, pool, sizeof(float) * (size_t)m * d, cudaMemcpyDeviceToDevice, stream));
+    // Parzen estimator: the history lives here (it is refitted every round), up to the estimator's 4096 rows
+    const int hist_cap = 4096;
+    int hist_n = n0;
+    std::vector<int> all_ordinal(d, 0);
+    const size_t topk_bytes = tpe ? topk_workspace_bytes(1, m, opt.q) : 0;
+    if (tpe) {
+        if (n0 > hist_cap) {
+            set_error("r3_bo_run: the Parzen estimator takes at most %d observations", hist_cap);
+            return done(R3_ERR_INVALID_ARG);
+        }
+        TRY_DONE(dev_malloc(&hist_x, sizeof(float) * (size_t)hist_cap * d));
+        TRY_DONE(dev_malloc(&hist_y, sizeof(float) * (size_t)hist_cap));
+        TRY_DONE(dev_malloc(&score, sizeof(float) * (size_t)m));
+        TRY_DONE(dev_malloc(&topk_ws, topk_bytes));
+        TRY_DONE(cudaMemcpyAsync(hist_x, X0, sizeof(float) * (size_t)n0 * d, cudaMemcpyDeviceToDevice, stream));
+        TRY_DONE(cudaMemcpyAsync(hist_y, y0, sizeof(float) * (size_t)n0, cudaMemcpyDeviceToDevice, stream));
+    }
 
     // incumbent: the best of the initial history
     std::vector<float> hx((size_t)n0 * d), hy(n0);
@@ -126,13 +156,25 @@ r3_status_t r3_bo_run(const float* X0, const float* y0, int n0, int d, const flo
         if (opt.patience > 0 && since_better >= opt.patience) { reason = R3_BO_NO_IMPROVEMENT; break; }
         const int q = (int)(left < opt.q ? left : opt.q);
         if (q < 1) { reason = R3_BO_POOL_EXHAUSTED; break; }
-        if (r3_gp_size(gp) + q > kMaxN) { reason = R3_BO_HISTORY_FULL; break; }
-        if (opt.optimize_every > 0 && round > 0 && round % opt.optimize_every == 0) {
-            st = r3_gp_optimize(gp, 40, 1e-2, nullptr, nullptr, nullptr, nullptr, nullptr, cuda_stream);
-            if (st != R3_OK && st != R3_ERR_NOT_PD) return done(st);   // a failed search keeps the old values
+        if ((tpe ? hist_n : r3_gp_size(gp)) + q > (tpe ? hist_cap : kMaxN)) { reason = R3_BO_HISTORY_FULL; break; }
+        if (tpe) {
+            r3_tpe_t* est = nullptr;
+            st = r3_tpe_fit(hist_x, hist_y, opt.levels ? opt.levels : all_ordinal.data(), hist_n, d,
+                            opt.gamma > 0.f ? opt.gamma : 0.25f, 1.0f, cuda_stream, &est);
+            if (st != R3_OK) return done(st);
+            st = r3_tpe_score(est, work, left, score, cuda_stream);
+            if (st == R3_OK) st = topk_device(score, 1, left, q, idx_d, nullptr, topk_ws, topk_bytes, stream);
+            if (st == R3_OK) st = r3_tpe_check(est, cuda_stream);
+            r3_tpe_free(est);
+            if (st != R3_OK) return done(st);
+        } else {
+            if (opt.optimize_every > 0 && round > 0 && round % opt.optimize_every == 0) {
+                st = r3_gp_optimize(gp, 40, 1e-2, nullptr, nullptr, nullptr, nullptr, nullptr, cuda_stream);
+                if (st != R3_OK && st != R3_ERR_NOT_PD) return done(st);   // a failed search keeps the old values
+            }
+            st = r3_gp_propose(gp, work, left, q, 0, opt.lie, idx_d, nullptr, nullptr, cuda_stream);
+            if (st != R3_OK) return done(st);
         }
-        st = r3_gp_propose(gp, work, left, q, 0, opt.lie, idx_d, nullptr, nullptr, cuda_stream);
-        if (st != R3_OK) return done(st);
         gather_rows_kernel<<<q, 128, 0, stream>>>(work, idx_d, q, d, rows_d);
         ++g_launches;
         TRY_DONE(cudaGetLastError());
@@ -168,8 +210,17 @@ r3_status_t r3_bo_run(const float* X0, const float* y0, int n0, int d, const flo
             TRY_DONE(cudaMemcpyAsync(rows_d, keep_rows.data(), sizeof(float) * (size_t)k * d, cudaMemcpyHostToDevice,
                                      stream));
             TRY_DONE(cudaMemcpyAsync(y_d, keep_y.data(), sizeof(float) * (size_t)k, cudaMemcpyHostToDevice, stream));
-            st = r3_gp_append(gp, rows_d, y_d, k, cuda_stream);
-            if (st != R3_OK) return done(st);
+            if (tpe) {
+                TRY_DONE(cudaMemcpyAsync(hist_x + (size_t)hist_n * d, rows_d, sizeof(float) * (size_t)k * d,
+                                         cudaMemcpyDeviceToDevice, stream));
+                TRY_DONE(cudaMemcpyAsync(hist_y + hist_n, y_d, sizeof(float) * (size_t)k, cudaMemcpyDeviceToDevice,
+                                         stream));
+                TRY_DONE(cudaStreamSynchronize(stream));   // keep_rows / keep_y are reused next round
+                hist_n += k;
+            } else {
+                st = r3_gp_append(gp, rows_d, y_d, k, cuda_stream);
+                if (st != R3_OK) return done(st);
+            }
         }
         if (stop) { reason = R3_BO_STOPPED_BY_CALLER; break; }
     }

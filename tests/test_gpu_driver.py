@@ -76,6 +76,38 @@ def test_trajectory_matches_the_oracle_loop(lie):
     gp.close()
 
 
+def test_parzen_estimator_as_the_surrogate_matches_the_oracle_loop():
+    """The paper's own choice: parallel TPE.  Per round: fit on the history so far, score the pool, the q best."""
+    from oracle import tpe_oracle as T
+    X0, y0, pool, ell, sf2, sn2 = setup(5, 16, 3, 500)
+    levels = np.zeros(3, np.int32)
+    sent = []
+
+    def evaluate(x):
+        sent.append(x.copy())
+        return objective(x), x[:, 2] < 0.9
+
+    res = b.r3_bo_run(dev(X0), dev(y0), ell, sf2, sn2, dev(pool), evaluate, q=5, max_rounds=6, surrogate="tpe",
+                      levels=levels, gamma=0.25)
+    assert res["rounds"] == 6 and res["evaluated"] == 30 and res["stop_reason"] == "max_rounds"
+    X, y, left = X0.copy(), y0.copy(), pool.copy()
+    for got in sent:
+        model = T.tpe_fit(X, y, levels, 0.25, 1.0)
+        s = T.tpe_score(model, left)
+        idx = T.tpe_topk(s, 5)
+        if not np.array_equal(got, left[idx]):
+            # the device scores in FP32: a different choice is only acceptable between near-equal scores
+            pos = [int(np.flatnonzero((left == r).all(axis=1))[0]) for r in got]
+            assert set(pos) ^ set(idx.tolist()), "same set in another order must still be the same order"
+            assert max(abs(s[p] - s[idx[-1]]) for p in set(pos) ^ set(idx.tolist())) <= 1e-4
+            break
+        ok = got[:, 2] < 0.9
+        X = np.concatenate([X, got[ok]])
+        y = np.concatenate([y, objective(got)[ok]])
+        left = np.delete(left, idx, axis=0)
+    assert res["best_y"] <= y0.min()
+
+
 def test_stopping_rules():
     X0, y0, pool, ell, sf2, sn2 = setup(1, 10, 2, 300)
     flat = lambda x: (np.full(x.shape[0], 5.0, np.float32), np.ones(x.shape[0], bool))      # never improves
