@@ -334,17 +334,14 @@ r3_status_t r3_gp_propose(r3_gp_t* gp, const float* Xcand, long long m, int q, i
     TRY_DONE(dev_malloc(&sval, sizeof(float) * (size_t)B * Rk));
     TRY_DONE(dev_malloc(&sidx, sizeof(int) * (size_t)B * Rk));
     TRY_DONE(dev_malloc(&tws, tbytes));
-    TRY_DONE(dev_malloc(&pws, propose_workspace_bytes(gp->npad, R, q)));
+    TRY_DONE(dev_malloc(&pws, propose_workspace_bytes(B, gp->npad, R, q)));
     float *mu = scores, *sigma = scores + bm, *ei = scores + 2 * bm;
     st = run_score(gp, Xcand, m, mu, sigma, ei, gp->ws, gp->ws_bytes, stream);
     if (st != R3_OK) return done(st);
     st = topk_device(ei, B, m, Rk, sidx, sval, tws, tbytes, stream);
     if (st != R3_OK) return done(st);
-    for (int g = 0; g < B; ++g) {
-        st = propose_shortlist(gp, g, Xcand + (size_t)g * m * gp->d, sidx + (size_t)g * Rk, R, q, lie,
-                               idx + (size_t)g * q, ei_pick ? ei_pick + (size_t)g * q : nullptr, pws, stream);
-        if (st != R3_OK) return done(st);
-    }
+    st = propose_shortlist(gp, Xcand, m, sidx, Rk, R, q, lie, idx, ei_pick, pws, stream);
+    if (st != R3_OK) return done(st);
     // certificate and latched device status
     std::vector<float> hval((size_t)B * Rk), hpick;
     TRY_DONE(cudaMemcpyAsync(hval.data(), sval, sizeof(float) * hval.size(), cudaMemcpyDeviceToHost, stream));

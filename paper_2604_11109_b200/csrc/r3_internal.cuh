@@ -156,8 +156,8 @@ r3_status_t topk_device(const float* ei, int batch, long long m, int k, int* idx
 r3_status_t lml_device(r3_gp* gp, double* out_h, cudaStream_t stream);
 
 // greedy batch proposal on a shortlist (r3_propose.cu)
-size_t propose_workspace_bytes(int npad, int R, int q);
-r3_status_t propose_shortlist(r3_gp* gp, int g, const float* Xcand_g, const int* sidx, int R, int q, int liar,
+size_t propose_workspace_bytes(int batch, int npad, int R, int q);
+r3_status_t propose_shortlist(r3_gp* gp, const float* Xcand, long long m, const int* sidx, int Rk, int R, int q, int liar,
                               int* idx_out, float* ei_out, void* ws, cudaStream_t stream);
 
 // fixed (never allocated) key storage for r3_topk_noalloc

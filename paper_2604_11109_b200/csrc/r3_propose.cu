@@ -21,12 +21,37 @@ namespace r3 {
 
 namespace {
 
+// All GPs of the handle are processed together: blockIdx.z (or .y) is the GP.  Per-GP scalars come from
+// device arrays; the shortlist state of GP g starts at g times the per-GP stride of each array.
+struct ProposeArrays {
+    const float* X;        // [B][n][d]
+    const float* ell;      // [B][d]
+    const float* sf2;      // [B]
+    const float* sn2;      // [B]
+    const float* best;     // [B]
+    const double* alpha;   // [B][npad]
+    const float* Xcand;    // [B][m][d]
+    const int* sidx;       // [B][Rk] shortlist (pool indices), Rk >= R
+    long long m;
+    int n, d, npad, R, Rk, q;
+    double *Ks, *V;        // [B][R][npad]
+    double *C;             // [B][q][R]
+    double *mu, *var;      // [B][R]
+    double *S, *delta;     // [B][q]
+    int *picked, *sel;     // [B][R], [B][q]
+};
+
 // Ks[r][i] = k(x_i, candidate sidx[r]) in FP64 by direct differences; zero in the padding columns.
-__global__ void shortlist_kstar_kernel(const float* __restrict__ X, const float* __restrict__ ell, double sf2, int n,
-                                       int d, int npad, const float* __restrict__ Xcand, const int* __restrict__ sidx,
-                                       double* __restrict__ Ks)
+__global__ void shortlist_kstar_kernel(const ProposeArrays a)
 {
-    const int r = blockIdx.y;
+    const int g = blockIdx.z, r = blockIdx.y;
+    const int n = a.n, d = a.d, npad = a.npad;
+    const float* X = a.X + (size_t)g * n * d;
+    const float* ell = a.ell + (size_t)g * d;
+    const float* Xcand = a.Xcand + (size_t)g * a.m * d;
+    const int* sidx = a.sidx + (size_t)g * a.Rk;
+    double* Ks = a.Ks + (size_t)g * a.R * npad;
+    const double sf2 = (double)a.sf2[g];
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= npad) return;
     double v = 0.0;
@@ -45,10 +70,17 @@ __global__ void shortlist_kstar_kernel(const float* __restrict__ X, const float*
 }
 
 // mu[r] = Ks[r].alpha, var[r] = sf2 - |V[r]|^2 (one warp per shortlisted candidate).
-__global__ void shortlist_moments_kernel(const double* __restrict__ Ks, const double* __restrict__ V,
-                                         const double* __restrict__ alpha, int n, int npad, double sf2, int R,
-                                         double* __restrict__ mu, double* __restrict__ var, int* __restrict__ picked)
+__global__ void shortlist_moments_kernel(const ProposeArrays a)
 {
+    const int g = blockIdx.y;
+    const int n = a.n, npad = a.npad, R = a.R;
+    const double* Ks = a.Ks + (size_t)g * R * npad;
+    const double* V = a.V + (size_t)g * R * npad;
+    const double* alpha = a.alpha + (size_t)g * npad;
+    double* mu = a.mu + (size_t)g * R;
+    double* var = a.var + (size_t)g * R;
+    int* picked = a.picked + (size_t)g * R;
+    const double sf2 = (double)a.sf2[g];
     const int r = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
     const int lane = threadIdx.x % 32;
     if (r >= R) return;
@@ -70,15 +102,23 @@ __global__ void shortlist_moments_kernel(const double* __restrict__ Ks, const do
 }
 
 // One block: EI of every unpicked shortlisted candidate, the largest (ties: lower pool index) is pick t.
-__global__ void __launch_bounds__(1024) pick_kernel(const double* __restrict__ mu, const double* __restrict__ var,
-                                                    int* __restrict__ picked, const int* __restrict__ sidx, int R,
-                                                    double best, double sn2, int liar, int t, int* __restrict__ sel,
-                                                    double* __restrict__ S, double* __restrict__ delta,
-                                                    int* __restrict__ idx_out, float* __restrict__ ei_out,
-                                                    int* __restrict__ status)
+__global__ void __launch_bounds__(1024) pick_kernel(const ProposeArrays a, int liar, int t, int* __restrict__ idx_all,
+                                                    float* __restrict__ ei_all, int* __restrict__ status)
 {
     __shared__ double se[1024];
     __shared__ int sr[1024];
+    const int g = blockIdx.x;
+    const int R = a.R;
+    const double* mu = a.mu + (size_t)g * R;
+    const double* var = a.var + (size_t)g * R;
+    int* picked = a.picked + (size_t)g * R;
+    const int* sidx = a.sidx + (size_t)g * a.Rk;
+    int* sel = a.sel + (size_t)g * a.q;
+    double* S = a.S + (size_t)g * a.q;
+    double* delta = a.delta + (size_t)g * a.q;
+    int* idx_out = idx_all + (size_t)g * a.q;
+    float* ei_out = ei_all ? ei_all + (size_t)g * a.q : nullptr;
+    const double best = (double)a.best[g], sn2 = (double)a.sn2[g];
     const int r = threadIdx.x;
     double e = -1.0;
     if (r < R && !picked[r]) e = ei_closed_form(mu[r], sqrt(fmax(var[r], 0.0)), best);
@@ -87,12 +127,12 @@ __global__ void __launch_bounds__(1024) pick_kernel(const double* __restrict__ m
     __syncthreads();
     for (int o = 512; o > 0; o >>= 1) {
         if (r < o) {
-            const double a = se[r], b = se[r + o];
+            const double ea = se[r], eb = se[r + o];
             const int ra = sr[r], rb = sr[r + o];
             // an entry that is not a candidate (e < 0) always loses; equal EI: the lower pool index wins
-            const bool take_b = (b > a) || (b == a && b >= 0.0 && sidx[rb] < sidx[ra]);
+            const bool take_b = (eb > ea) || (eb == ea && eb >= 0.0 && sidx[rb] < sidx[ra]);
             if (take_b) {
-                se[r] = b;
+                se[r] = eb;
                 sr[r] = rb;
             }
         }
@@ -120,12 +160,21 @@ __global__ void __launch_bounds__(1024) pick_kernel(const double* __restrict__ m
 
 // One warp per shortlisted candidate r: c = cov(x_r, x_pick) under the posterior before pick t, then the
 // rank-one update of its mean and variance.  C[t][r] keeps c for the later picks.
-__global__ void condition_kernel(const float* __restrict__ Xcand, const int* __restrict__ sidx,
-                                 const float* __restrict__ ell, double sf2, int d, const double* __restrict__ V, int n,
-                                 int npad, double* __restrict__ C, const double* __restrict__ S,
-                                 const double* __restrict__ delta, const int* __restrict__ sel, int t, int R,
-                                 double* __restrict__ mu, double* __restrict__ var)
+__global__ void condition_kernel(const ProposeArrays a, int t)
 {
+    const int g = blockIdx.y;
+    const int n = a.n, d = a.d, npad = a.npad, R = a.R;
+    const float* Xcand = a.Xcand + (size_t)g * a.m * d;
+    const int* sidx = a.sidx + (size_t)g * a.Rk;
+    const float* ell = a.ell + (size_t)g * d;
+    const double sf2 = (double)a.sf2[g];
+    const double* V = a.V + (size_t)g * R * npad;
+    double* C = a.C + (size_t)g * a.q * R;
+    const double* S = a.S + (size_t)g * a.q;
+    const double* delta = a.delta + (size_t)g * a.q;
+    const int* sel = a.sel + (size_t)g * a.q;
+    double* mu = a.mu + (size_t)g * R;
+    double* var = a.var + (size_t)g * R;
     const int r = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
     const int lane = threadIdx.x % 32;
     if (r >= R) return;
@@ -155,51 +204,59 @@ __global__ void condition_kernel(const float* __restrict__ Xcand, const int* __r
 
 }  // namespace
 
-size_t propose_workspace_bytes(int npad, int R, int q)
+size_t propose_workspace_bytes(int batch, int npad, int R, int q)
 {
-    return sizeof(double) * (2 * (size_t)R * npad + (size_t)q * R + 2 * (size_t)R + 2 * (size_t)q) +
-           sizeof(int) * ((size_t)R + q) + 256;
+    return (size_t)batch * (sizeof(double) * (2 * (size_t)R * npad + (size_t)q * R + 2 * (size_t)R + 2 * (size_t)q) +
+                            sizeof(int) * ((size_t)R + q)) + 1024;
 }
 
-// The q picks of GP g.  sidx: device [R] pool indices of the shortlist (by initial EI, descending);
-// idx_out / ei_out: device [q].  ws: propose_workspace_bytes(npad, R, q) bytes.
-r3_status_t propose_shortlist(r3_gp* gp, int g, const float* Xcand_g, const int* sidx, int R, int q, int liar,
+// The q picks of every GP of the handle.  sidx: device [batch][Rk] pool indices of the shortlists (by initial
+// EI, descending; the first R of each row are used); idx_out / ei_out: device [batch][q].
+// ws: propose_workspace_bytes(batch, npad, R, q) bytes.
+r3_status_t propose_shortlist(r3_gp* gp, const float* Xcand, long long m, const int* sidx, int Rk, int R, int q, int liar,
                               int* idx_out, float* ei_out, void* ws, cudaStream_t stream)
 {
-    const int n = gp->n, d = gp->d, npad = gp->npad;
+    const int B = gp->batch, n = gp->n, d = gp->d, npad = gp->npad;
     char* p = (char*)ws;
     auto carve = [&](size_t bytes) {
         char* r = p;
         p += (bytes + 15) / 16 * 16;
         return r;
     };
-    double* Ks = (double*)carve(sizeof(double) * (size_t)R * npad);
-    double* V = (double*)carve(sizeof(double) * (size_t)R * npad);
-    double* C = (double*)carve(sizeof(double) * (size_t)q * R);
-    double* mu = (double*)carve(sizeof(double) * R);
-    double* var = (double*)carve(sizeof(double) * R);
-    double* S = (double*)carve(sizeof(double) * q);
-    double* delta = (double*)carve(sizeof(double) * q);
-    int* picked = (int*)carve(sizeof(int) * R);
-    int* sel = (int*)carve(sizeof(int) * q);
-    const float* Xg = gp->X + (size_t)g * n * d;
-    const float* ellg = gp->ell_d + (size_t)g * d;
-    const double* Wg = gp->W64 + (size_t)g * npad * npad;
-    const double sf2 = (double)gp->sf2[g], sn2 = (double)gp->sn2[g], best = (double)gp->best[g];
+    ProposeArrays a;
+    a.X = gp->X;
+    a.ell = gp->ell_d;
+    a.sf2 = gp->sf2_d;
+    a.sn2 = gp->sn2_d;
+    a.best = gp->best_d;
+    a.alpha = gp->alpha64;
+    a.Xcand = Xcand;
+    a.sidx = sidx;
+    a.m = m;
+    a.n = n;
+    a.d = d;
+    a.npad = npad;
+    a.R = R;
+    a.Rk = Rk;
+    a.q = q;
+    a.Ks = (double*)carve(sizeof(double) * (size_t)B * R * npad);
+    a.V = (double*)carve(sizeof(double) * (size_t)B * R * npad);
+    a.C = (double*)carve(sizeof(double) * (size_t)B * q * R);
+    a.mu = (double*)carve(sizeof(double) * (size_t)B * R);
+    a.var = (double*)carve(sizeof(double) * (size_t)B * R);
+    a.S = (double*)carve(sizeof(double) * (size_t)B * q);
+    a.delta = (double*)carve(sizeof(double) * (size_t)B * q);
+    a.picked = (int*)carve(sizeof(int) * (size_t)B * R);
+    a.sel = (int*)carve(sizeof(int) * (size_t)B * q);
 
-    R3_LAUNCH(shortlist_kstar_kernel, dim3((npad + 127) / 128, R), 128, 0, stream, Xg, ellg, sf2, n, d, npad, Xcand_g,
-              sidx, Ks);
+    R3_LAUNCH(shortlist_kstar_kernel, dim3((npad + 127) / 128, R, B), 128, 0, stream, a);
     // V = Ks W^T (v_r = W k*_r): the same triangular product as the append step of the fit
-    R3_LAUNCH(tri_gemm_kernel<true>, dim3((n + 63) / 64, (R + 31) / 32, 1), 256, 0, stream, Ks, npad, (size_t)0, Wg,
-              npad, (size_t)0, V, npad, (size_t)0, R, n);
-    R3_LAUNCH(shortlist_moments_kernel, (R + 7) / 8, 256, 0, stream, Ks, V, gp->alpha64 + (size_t)g * npad, n, npad, sf2,
-              R, mu, var, picked);
+    R3_LAUNCH(tri_gemm_kernel<true>, dim3((n + 63) / 64, (R + 31) / 32, B), 256, 0, stream, a.Ks, npad,
+              (size_t)R * npad, gp->W64, npad, (size_t)npad * npad, a.V, npad, (size_t)R * npad, R, n);
+    R3_LAUNCH(shortlist_moments_kernel, dim3((R + 7) / 8, B), 256, 0, stream, a);
     for (int t = 0; t < q; ++t) {
-        R3_LAUNCH(pick_kernel, 1, 1024, 0, stream, mu, var, picked, sidx, R, best, sn2, liar, t, sel, S, delta, idx_out,
-                  ei_out, gp->status_d);
-        if (t + 1 < q)
-            R3_LAUNCH(condition_kernel, (R + 7) / 8, 256, 0, stream, Xcand_g, sidx, ellg, sf2, d, V, n, npad, C, S, delta,
-                      sel, t, R, mu, var);
+        R3_LAUNCH(pick_kernel, B, 1024, 0, stream, a, liar, t, idx_out, ei_out, gp->status_d);
+        if (t + 1 < q) R3_LAUNCH(condition_kernel, dim3((R + 7) / 8, B), 256, 0, stream, a, t);
     }
     return R3_OK;
 }
