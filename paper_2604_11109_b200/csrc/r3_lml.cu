@@ -67,9 +67,17 @@ __global__ void __launch_bounds__(256) kinv_kernel(const double* __restrict__ W,
 // partial[block][0 .. d-1] = sum over the tile of w M_ik G_ik u_j^2, partial[block][d] = sum w M_ik Kf_ik,
 // with w = 1 on the diagonal, 2 below it, 0 above.
 __global__ void __launch_bounds__(256) lml_pairs_kernel(const float* __restrict__ X, const float* __restrict__ ell,
-                                                        double sf2, int n, int d, int npad, const double* __restrict__ M,
-                                                        int tiles, double* __restrict__ partial)
+                                                        const float* __restrict__ sf2v, int n, int d, int npad,
+                                                        const double* __restrict__ M, int tiles,
+                                                        double* __restrict__ partial)
 {
+    // blockIdx.y: the GP
+    const int g = blockIdx.y;
+    X += (size_t)g * n * d;
+    ell += (size_t)g * d;
+    M += (size_t)g * npad * npad;
+    partial += (size_t)g * tiles * (d + 1);
+    const double sf2 = (double)sf2v[g];
     // tile index -> (ti, tk) of the lower triangle
     const int b = blockIdx.x;
     int ti = (int)((sqrt(8.0 * b + 1.0) - 1.0) * 0.5);
@@ -148,16 +156,24 @@ __global__ void __launch_bounds__(256) lml_pairs_kernel(const float* __restrict_
             block_sum(v, c0 + c);
         }
     }
-    (void)tiles;
 }
 
 // One block per GP: adds the tiles' partial sums in order, the trace term and the value.
 __global__ void __launch_bounds__(256) lml_finish_kernel(const double* __restrict__ partial, int tiles, int d,
                                                          const double* __restrict__ M, const double* __restrict__ L,
                                                          const double* __restrict__ alpha, const float* __restrict__ y,
-                                                         int n, int npad, double sn2, double* __restrict__ out)
+                                                         int n, int npad, const float* __restrict__ sn2v,
+                                                         double* __restrict__ out)
 {
     __shared__ double red[256];
+    const int g = blockIdx.x;
+    partial += (size_t)g * tiles * (d + 1);
+    M += (size_t)g * npad * npad;
+    L += (size_t)g * npad * npad;
+    alpha += (size_t)g * npad;
+    y += (size_t)g * n;
+    out += (size_t)g * (d + 3);
+    const double sn2 = (double)sn2v[g];
     const int t = threadIdx.x;
     auto block_sum = [&](double v) {
         red[t] = v;
@@ -214,25 +230,18 @@ r3_status_t lml_device(r3_gp* gp, double* out_h, cudaStream_t stream)
         }                                                                                          \
     } while (0)
     TRY_DONE(dev_malloc(&M, sizeof(double) * (size_t)B * npad * npad));
-    TRY_DONE(dev_malloc(&partial, sizeof(double) * (size_t)tiles * (d + 1)));
+    TRY_DONE(dev_malloc(&partial, sizeof(double) * (size_t)B * tiles * (d + 1)));
     TRY_DONE(dev_malloc(&out, sizeof(double) * (size_t)B * (d + 3)));
     const int t64 = (n + 63) / 64;
     kinv_kernel<<<dim3(t64, t64, B), 256, 0, stream>>>(gp->W64, gp->alpha64, n, npad, M);
     ++g_launches;
     TRY_DONE(cudaGetLastError());
-    for (int g = 0; g < B; ++g) {
-        lml_pairs_kernel<<<tiles, 256, 0, stream>>>(gp->X + (size_t)g * n * d, gp->ell_d + (size_t)g * d,
-                                                    (double)gp->sf2[g], n, d, npad, M + (size_t)g * npad * npad, tiles,
-                                                    partial);
-        ++g_launches;
-        TRY_DONE(cudaGetLastError());
-        lml_finish_kernel<<<1, 256, 0, stream>>>(partial, tiles, d, M + (size_t)g * npad * npad,
-                                                 gp->L64 + (size_t)g * npad * npad, gp->alpha64 + (size_t)g * npad,
-                                                 gp->y + (size_t)g * n, n, npad, (double)gp->sn2[g],
-                                                 out + (size_t)g * (d + 3));
-        ++g_launches;
-        TRY_DONE(cudaGetLastError());
-    }
+    lml_pairs_kernel<<<dim3(tiles, B), 256, 0, stream>>>(gp->X, gp->ell_d, gp->sf2_d, n, d, npad, M, tiles, partial);
+    ++g_launches;
+    TRY_DONE(cudaGetLastError());
+    lml_finish_kernel<<<B, 256, 0, stream>>>(partial, tiles, d, M, gp->L64, gp->alpha64, gp->y, n, npad, gp->sn2_d, out);
+    ++g_launches;
+    TRY_DONE(cudaGetLastError());
     TRY_DONE(cudaMemcpyAsync(out_h, out, sizeof(double) * (size_t)B * (d + 3), cudaMemcpyDeviceToHost, stream));
     TRY_DONE(cudaStreamSynchronize(stream));
 #undef TRY_DONE
