@@ -55,3 +55,19 @@ def test_sample_indices_sorted_distinct():
     c = w.get_config(5)
     s = w.sample_indices(c, 8192)
     assert s.shape == (8192,) and np.all(np.diff(s) > 0) and s[-1] < c.m
+
+
+def test_tpe_levels_mark_binary_flags_and_grids():
+    from paper_2604_11109_b200 import workloads as w
+    c2, c5, c4 = w.get_config(2), w.get_config(5), w.get_config(4)
+    lv2 = w.tpe_levels(c2)
+    assert lv2.tolist() == [0, 0, 0, 0, 0, 2] + [2] * 10           # five launch parameters, one bool, ten flags
+    assert w.tpe_levels(c5).tolist() == [0] * 32 + [2] * 32
+    assert w.tpe_levels(c4).tolist() == [0] * 128
+    g2 = w.tpe_levels(c2, grid=True)
+    assert g2[:6].tolist() == [-32, -8, -4, 0, 0, 2]               # equally spaced levels become grids; 224 levels
+    assert w.tpe_levels(c5, grid=True).tolist() == [-16] * 32 + [2] * 32   # and unevenly spaced ones stay ordinal
+    # the declared grids are the generator's own values
+    for l, code in zip(w.feature_levels(c2), g2):
+        if code < 0:
+            assert np.array_equal(np.float32(l), np.float32(np.arange(-code) / (-code - 1)))
