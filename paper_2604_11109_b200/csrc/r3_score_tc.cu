@@ -347,6 +347,19 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                 float zn = 0.f;
                 bool far = false;
                 const float* zrow = prm.xcand + ((size_t)g * prm.m + (valid ? cand : 0)) * prm.d;
+                {
+                    // the row this thread will need for the CTA's next tile: start it on its way to L2 now
+                    const long long nt = tile + tile_step;
+                    if (nt < prm.total_tiles) {
+                        const long long nc = (nt % prm.tiles_per_gp) * TILE_M + row;
+                        if (nc < prm.m) {
+                            const char* pf = reinterpret_cast<const char*>(
+                                prm.xcand + ((size_t)(nt / prm.tiles_per_gp) * prm.m + nc) * prm.d);
+                            for (int off = 0; off < prm.d * 4; off += 128)
+                                asm volatile("prefetch.global.L2 [%0];" ::"l"(pf + off));
+                        }
+                    }
+                }
                 const float* cen = prm.centre + (size_t)g * DP;
                 const float* scl = prm.scale + (size_t)g * DP;
                 const bool vec = (prm.d % 4) == 0;
