@@ -15,8 +15,10 @@ namespace r3 {
 namespace {
 
 constexpr size_t kSlabBytes = 256ull << 20;
-// relative error of one k* entry on this path: FP32 differences, FMA chain, sqrtf, expf
+// relative error of one k* entry on this path: FP32 differences, FMA chain, sqrtf, expf.  The squared
+// distance is an FP32 sum over d features, so its rounding grows like sqrt(d); the figure is for d <= 16.
 constexpr double kEpsSimt = 1.2e-7;
+inline double eps_simt(int d) { return kEpsSimt * (d > 16 ? sqrt((double)d / 16.0) : 1.0); }
 
 struct SimtWorkspace {
     float* ks;         // [slab][npad]
@@ -241,7 +243,7 @@ r3_status_t score_simt(r3_gp* gp, const float* Xcand, long long m, float* mu, fl
             prof_begin(gp, stream);
             R3_LAUNCH(trigemm_sq_kernel, (unsigned)((mc + 127) / 128), 256, 0, stream,
                       gp->W32 + (size_t)g * npad * npad, w.ks, w.mu64, npad, mc, (double)gp->sf2[g],
-                      (double)gp->best[g], kEpsSimt, gp->wnorm[g], mu + off, sigma + off, ei + off,
+                      (double)gp->best[g], eps_simt(d), gp->wnorm[g], mu + off, sigma + off, ei + off,
                       w.guard.err_mu + off, w.guard.err_q + off);
             prof_end(gp, stream);
         }

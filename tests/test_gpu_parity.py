@@ -282,3 +282,34 @@ def test_workload_full_size_sampled_and_full_pool_topk(cfg, engine):
         known.update(zip(pick.tolist(), ei_r.tolist()))
         check_topk(idx[q], lambda i: known[i], ref_idx[:c.k], ref_val[:c.k], ref_val[c.k], float(gold["ei_max"]),
                    what=c.name)
+
+
+# ------------------------------------------------------------------------------------------ the library's size limits
+@pytest.mark.parametrize("engine", ENGINES)
+@pytest.mark.parametrize("d", [256, 128])
+def test_maximum_history_and_feature_count(engine, d):
+    """n = 8192 with d = 256 (the limits of r3_gp_fit; served by the CUDA-core engine) and with d = 128 (the
+    widest the tensor engine takes): factor, weights and scores against the oracle."""
+    rng = np.random.default_rng(8192)
+    n, m = 8192, 200
+    g = {
+        "X": rng.uniform(0, 1, (1, n, d)).astype(np.float32),
+        "y": rng.normal(0, 1, (1, n)).astype(np.float32),
+        "ell": np.full((1, d), 0.25 * np.sqrt(d), np.float32),   # sqrt(d)-sized lengthscales: correlated neighbours
+        "sf2": np.ones(1, np.float32),
+        "sn2": np.full(1, 1e-2, np.float32),
+        "Xcand": rng.uniform(0, 1, (1, m, d)).astype(np.float32),
+    }
+    try:
+        gp = fit_gpu(g, engine)
+    except b.R3Error as e:                                   # pragma: no cover
+        pytest.fail(f"fit at the size limits failed: {e}")
+    f = o.fit(g["X"][0], g["y"][0], g["ell"][0], g["sf2"][0], g["sn2"][0])
+    alpha, L = b.r3_gp_get_factor(gp)
+    assert np.allclose(L[0], f.L, rtol=1e-9, atol=1e-11)
+    assert np.allclose(alpha[0], f.alpha, rtol=1e-6, atol=1e-8 * np.abs(f.alpha).max())
+    mu, sd, ei = (t.cpu().numpy() for t in b.r3_gp_score(gp, dev(g["Xcand"])))
+    b.r3_gp_check(gp)
+    mu_r, sd_r, ei_r = o.score(f, g["Xcand"][0])
+    check_scores(mu[0], sd[0], ei[0], mu_r, sd_r, ei_r, float(np.abs(g["y"]).max()), 1.0, what=f"n=8192 d={d}")
+    gp.close()
