@@ -3,7 +3,9 @@
 mu, sigma: relative 1e-4, with an absolute floor for values that cross zero:
     |d mu|    <= 1e-4 |mu_ref|    + 1e-6 max|y|
     |d sigma| <= 1e-4 sigma_ref   + 1e-6 sqrt(signal_var)
-EI: absolute 1e-5 * max(EI_ref) over the compared set.
+EI: absolute 1e-5 * max(EI_ref) over the compared set -- but never below the smallest normal FP32 number:
+    the library returns EI in FP32, and a pool whose largest EI is 1e-160 (every candidate hopeless) cannot be
+    resolved to 1e-165 in that type; such values come back as 0.
 top-k: with tol = 1e-5 * max(EI_ref): if the oracle's gap between rank k and k+1 exceeds tol the index
 sets must be equal; otherwise every chosen index must have EI_ref >= EI_ref[rank k] - tol.  A position
 may differ from the oracle's only if the two oracle values differ by <= tol.
@@ -13,6 +15,7 @@ import numpy as np
 MU_REL, MU_ABS = 1e-4, 1e-6
 SIGMA_REL, SIGMA_ABS = 1e-4, 1e-6
 EI_REL_OF_MAX = 1e-5
+EI_ABS_FLOOR = float(np.finfo(np.float32).tiny)   # 1.18e-38: EI is an FP32 output
 
 
 def check_scores(mu, sigma, ei, mu_ref, sigma_ref, ei_ref, y_absmax, sf2, ei_max=None, what=""):
@@ -20,7 +23,7 @@ def check_scores(mu, sigma, ei, mu_ref, sigma_ref, ei_ref, y_absmax, sf2, ei_max
     emax = float(np.max(ei_ref)) if ei_max is None else float(ei_max)
     tol_mu = MU_REL * np.abs(mu_ref) + MU_ABS * y_absmax
     tol_sd = SIGMA_REL * sigma_ref + SIGMA_ABS * np.sqrt(sf2)
-    tol_ei = EI_REL_OF_MAX * emax
+    tol_ei = max(EI_REL_OF_MAX * emax, EI_ABS_FLOOR)
     bad_mu = np.abs(mu - mu_ref) > tol_mu
     bad_sd = np.abs(sigma - sigma_ref) > tol_sd
     bad_ei = np.abs(ei - ei_ref) > tol_ei
@@ -44,7 +47,7 @@ def check_topk(idx, ei_ref_of, ref_idx, ref_val, ref_next_val, ei_max, what=""):
     ref_idx/ref_val: the oracle's top-k; ref_next_val: the oracle's value at rank k+1 (or -inf)."""
     idx = np.asarray(idx, dtype=np.int64)
     k = idx.size
-    tol = EI_REL_OF_MAX * float(ei_max)
+    tol = max(EI_REL_OF_MAX * float(ei_max), EI_ABS_FLOOR)
     assert len(set(idx.tolist())) == k, f"{what}: repeated index in top-k"
     kth = float(ref_val[k - 1])
     if kth - float(ref_next_val) > tol:

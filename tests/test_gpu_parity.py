@@ -313,3 +313,34 @@ def test_maximum_history_and_feature_count(engine, d):
     mu_r, sd_r, ei_r = o.score(f, g["Xcand"][0])
     check_scores(mu[0], sd[0], ei[0], mu_r, sd_r, ei_r, float(np.abs(g["y"]).max()), 1.0, what=f"n=8192 d={d}")
     gp.close()
+
+
+# ------------------------------------------------------------------------------------------ seeded random shapes
+@pytest.mark.parametrize("engine", ENGINES)
+def test_random_shapes_and_conditioning(engine):
+    """Thirty seeded problems with random batch, n, d, m, lengthscale spread and noise, a third of them with
+    candidates on or next to observations: every element and the top-k against the oracle."""
+    rng = np.random.default_rng(2604)
+    for it in range(30):
+        batch, n, d, m = int(rng.integers(1, 4)), int(rng.integers(1, 600)), int(rng.integers(1, 129)), int(rng.integers(1, 2500))
+        spread = float(rng.choice([0.3, 1.0, 3.0])) * np.sqrt(d) / 2
+        g = {
+            "X": rng.uniform(0, 1, (batch, n, d)).astype(np.float32),
+            "y": rng.normal(0, 1, (batch, n)).astype(np.float32),
+            "ell": (rng.uniform(0.5, 1.5, (batch, d)) * spread).astype(np.float32),
+            "sf2": rng.uniform(0.5, 2, batch).astype(np.float32),
+            "sn2": np.full(batch, float(rng.choice([1e-2, 1e-3, 1e-5])), np.float32),
+            "Xcand": rng.uniform(-0.1, 1.1, (batch, m, d)).astype(np.float32),
+        }
+        if rng.random() < 0.33 and m > 4 and n > 2:
+            kk = min(n, m // 2)
+            g["Xcand"][:, :kk] = g["X"][:, :kk] + np.float32(rng.choice([0.0, 1e-3]))
+        gp = b.r3_gp_fit(dev(g["X"]), dev(g["y"]), g["ell"], g["sf2"], g["sn2"])
+        try:
+            b.r3_gp_set_engine(gp, engine)
+        except b.R3Error as e:
+            assert e.status == 7
+            gp.close()
+            continue
+        compare_everything(g, gp, min(m, int(rng.integers(1, 65))), f"random #{it} n{n} d{d} m{m}")
+        gp.close()
