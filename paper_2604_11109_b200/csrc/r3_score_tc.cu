@@ -7,11 +7,10 @@
 // the observations in chunks of KC = 32:
 //
 //   distance MMA   D[cand][k] = z~ . x~_k   (A = scaled candidates, kept in TMEM for the whole tile;
-//                  B = scaled observations, depth d), for KD observations at a time.  An MMA whose A
-//                  operand comes from shared memory costs ~130 cycles however narrow it is (the A
-//                  tile is fetched again every time); with A in TMEM a narrow MMA is cheap
+//                  B = scaled observations, depth d), for KD observations at a time
 //   Matern warps   r^2 = |z~|^2 + |x~_k|^2 - 2 D, k* = sf2 M52(r): read D from TMEM, write k* (scaled,
-//                  FP16 hi/lo planes) as the next A operand into shared memory; mu += k* alpha on the way
+//                  FP16 hi/lo planes) as the next A operand into TMEM or shared memory; mu += k* alpha
+//                  on the way
 //   variance MMA   V[cand][i] += k*[cand][k] W[i][k]   (B = pre-tiled chunk of W, scaled FP16 hi/lo planes)
 //   end of pass    q += sum_i V[cand][i]^2 read back from TMEM; after the last pass sigma, EI, outputs
 //
@@ -28,8 +27,9 @@
 // Warp roles: warp 0 streams the operands (lane 0: scaled observations, lane 1: chunks of W), warp 1
 // issues the distance MMAs, warp 2 issues the variance MMAs and owns the TMEM allocation (one thread
 // each), warps 4.. form G Matern/epilogue groups of four warps (one warp per TMEM lane quarter); group
-// g takes every G-th chunk with its own k* buffer, so G chunks are in flight between the two MMA
-// streams.  Stages are handed over through mbarriers; every wait is bounded: when a limit is hit the
+// g takes every G-th chunk; the k* buffers are one per group (shared memory) or a ring of two shared by
+// the groups (TMEM, where columns are scarce; a group that has computed its chunk keeps it in registers
+// until its slot is free).  Stages are handed over through mbarriers; every wait is bounded: when a limit is hit the
 // CTA raises a status bit, all roles leave their loops, in-flight copies and MMAs are drained (bounded
 // again), TMEM is freed and the kernel returns.
 //
