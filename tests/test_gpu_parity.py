@@ -344,3 +344,24 @@ def test_random_shapes_and_conditioning(engine):
             continue
         compare_everything(g, gp, min(m, int(rng.integers(1, 65))), f"random #{it} n{n} d{d} m{m}")
         gp.close()
+
+
+def test_calls_on_a_side_stream_give_the_same_results():
+    """Everything a call enqueues goes to the stream it is given: results computed on a side stream (with the
+    default stream busy with unrelated work) are bit-identical to those of the default stream."""
+    g = rand_problem(91, 2, 150, 20, 5000)
+    gp = fit_gpu(g)
+    xc = dev(g["Xcand"])
+    ref = [t.clone() for t in b.r3_gp_score_topk(gp, xc, 16)]
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    busy = torch.empty(1 << 26, device="cuda")
+    with torch.cuda.stream(side):
+        for _ in range(3):
+            busy.normal_()                      # keeps the default stream's neighbour occupied; no dependency
+        out = b.r3_gp_score_topk(gp, xc, 16)
+        b.r3_gp_check(gp)
+    side.synchronize()
+    for a, c in zip(ref, out):
+        assert torch.equal(a, c)
+    gp.close()
