@@ -320,7 +320,9 @@ typedef struct {
     int max_rounds;      /* stop after this many rounds, >= 1 */
     double max_seconds;  /* stop when this much wall-clock time has passed, <= 0: no limit */
     int patience;        /* stop after this many rounds in a row without a better value, <= 0: no limit */
-    int optimize_every;  /* refit the hyper-parameters by r3_gp_optimize every this many rounds, <= 0: never */
+    int optimize_every;  /* refit the hyper-parameters by r3_gp_optimize every this many rounds, <= 0: never; the noise
+                            is then kept at or above 1e-6 signal_var, and raised tenfold (up to six times) if an
+                            update meets a numerically singular matrix */
     int lie;             /* fantasised value of r3_gp_propose: 0 believer, 1 liar */
     int surrogate;       /* 0: Gaussian process (r3_gp_fit / r3_gp_propose / r3_gp_append);
                             1: Tree-Parzen estimator, the paper's choice (Section VII-C: parallel TPE): every round

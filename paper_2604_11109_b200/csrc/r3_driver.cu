@@ -2,6 +2,8 @@
 // caller replay it, discard incorrect configurations, update the surrogate, until one of the paper's
 // three stopping rules fires.  Host logic around r3_gp_fit / r3_gp_propose / r3_gp_append /
 // r3_gp_optimize; the only kernels of its own move rows of the pool.
+#include <math.h>
+
 #include <chrono>
 #include <vector>
 
@@ -171,6 +173,13 @@ r3_status_t r3_bo_run(const float* X0, const float* y0, int n0, int d, const flo
             if (opt.optimize_every > 0 && round > 0 && round % opt.optimize_every == 0) {
                 st = r3_gp_optimize(gp, 40, 1e-2, nullptr, nullptr, nullptr, nullptr, nullptr, cuda_stream);
                 if (st != R3_OK && st != R3_ERR_NOT_PD) return done(st);   // a failed search keeps the old values
+                if (gp->sn2[0] < 1e-6f * gp->sf2[0]) {
+                    // keep the condition number of K within what the later rank-k updates can take
+                    const std::vector<float> ell = gp->ell;
+                    const float sf2 = gp->sf2[0], sn2 = 1e-6f * sf2;
+                    st = r3_gp_refit(gp, ell.data(), &sf2, &sn2, cuda_stream);
+                    if (st != R3_OK && st != R3_ERR_NOT_PD) return done(st);
+                }
             }
             st = r3_gp_propose(gp, work, left, q, 0, opt.lie, idx_d, nullptr, nullptr, cuda_stream);
             if (st != R3_OK) return done(st);
@@ -218,7 +227,17 @@ r3_status_t r3_bo_run(const float* X0, const float* y0, int n0, int d, const flo
                 TRY_DONE(cudaStreamSynchronize(stream));   // keep_rows / keep_y are reused next round
                 hist_n += k;
             } else {
+                // Hyper-parameters chosen by the optimiser can leave the extended covariance matrix numerically
+                // singular (tiny noise, long lengthscales, a new point next to an old one): raise the noise
+                // by factors of ten and refit until the update goes through.
                 st = r3_gp_append(gp, rows_d, y_d, k, cuda_stream);
+                for (int attempt = 0; st == R3_ERR_NOT_PD && attempt < 6; ++attempt) {
+                    const std::vector<float> ell = gp->ell;
+                    const float sf2 = gp->sf2[0];
+                    const float sn2 = fmaxf(gp->sn2[0] * 10.f, 1e-8f * sf2);
+                    st = r3_gp_refit(gp, ell.data(), &sf2, &sn2, cuda_stream);
+                    if (st == R3_OK) st = r3_gp_append(gp, rows_d, y_d, k, cuda_stream);
+                }
                 if (st != R3_OK) return done(st);
             }
         }

@@ -162,3 +162,13 @@ def test_an_exception_in_the_callback_surfaces():
 
     with pytest.raises(RuntimeError):
         b.r3_bo_run(dev(X0), dev(y0), ell, sf2, sn2, dev(pool), broken, q=2, max_rounds=3)
+
+
+def test_noise_free_replays_with_refitted_hyper_parameters_keep_going():
+    """A noise-free objective drives the fitted noise to its floor and the lengthscales up: the rank-k updates
+    then meet numerically singular matrices.  The loop keeps the noise above 1e-6 signal_var and raises it when
+    an update fails, instead of giving up."""
+    X0, y0, pool, ell, sf2, sn2 = setup(7, 50, 2, 900)
+    res = b.r3_bo_run(dev(X0), dev(y0), ell, sf2, sn2, dev(pool), lambda x: (objective(x), np.ones(len(x), bool)),
+                      q=20, max_rounds=8, optimize_every=1)
+    assert res["rounds"] == 8 and res["evaluated"] == 160 and res["best_y"] <= y0.min()
