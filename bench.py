@@ -160,7 +160,6 @@ def run_tpe(args, c):
     g = w.generate_gp(c, 0)
     levels = w.tpe_levels(c, grid=args.tpe_grid)
     n, d, m, k = c.n, c.d, c.m, c.k
-    evals = float(sum(n + 2 for l in levels if l == 0))      # exponentials per candidate
     base = {"metric": "tpe_candidates_scored_per_sec", "unit": "candidates/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "data": "synthetic",
@@ -208,6 +207,9 @@ def run_tpe(args, c):
     ev[1].record()
     torch.cuda.synchronize()
     fit_ms = ev[0].elapsed_time(ev[1])
+    # exponentials per candidate: the components the fit kept (equal ones merged) of every ordinal dimension
+    counts = b.r3_tpe_get_model(tpe)[3]
+    evals = float(counts[levels == 0].sum())
     score = torch.empty((m,), device="cuda")
     scratch = torch.empty((b.r3_topk_scratch_bytes(1, m, k),), dtype=torch.uint8, device="cuda")
     kernel_ms = []
@@ -292,7 +294,7 @@ def run_tpe(args, c):
         achieved = evals * m / (k_ms * 1e-3) / 1e12
         roofline = {"bound": "alu", "kernel": "tpe_score_kernel", "achieved": achieved, "peak": mufu_peak,
                     "unit": "Texp2/s", "frac": achieved / mufu_peak, "traffic": None,
-                    "note": "one MUFU.EX2 per (candidate, ordinal dimension, component); peak = 148 SMs x 16 MUFU "
+                    "note": "one MUFU.EX2 per (candidate, ordinal dimension, stored component); peak = 148 SMs x 16 MUFU "
                             "results per clock x max SM clock"}
     else:
         achieved = hbm_bytes / (k_ms * 1e-3) / 1e9
@@ -318,7 +320,7 @@ def run_tpe(args, c):
                "sample": f"{done} candidates of {c.name} in {el:.1f} s (numpy FP64, fit excluded)"}
     base.update({
         "value": world * m / (ms_per_step * 1e-3), "n_gpus": world, "ms_per_step": ms_per_step, "dtype": "f32",
-        "fit_ms": fit_ms, "clocks": clocks,
+        "fit_ms": fit_ms, "clocks": clocks, "components_per_candidate": evals,
         "config": dict(base["config"], l2="pool (%.0f MB) exceeds the 126 MB L2" % (xc.numel() * 4 / 1e6)
                        if xc.numel() * 4 > 126e6 else "pool smaller than L2; not flushed"),
         "e2e": {"value": world * m / (e2e_ms * 1e-3), "unit": "candidates/s", "h2d_bytes_per_step": int(xh.numel() * 4),

@@ -420,14 +420,18 @@ r3_status_t r3_tpe_check(r3_tpe_t* tpe, void* cuda_stream);
  *
  *   n_good  host [1]
  *   order   host [n]              history indices by y ascending
- *   comps   host [d][n + 2][4]    per dimension the good set's components then the bad set's
- *                                 (n_good + 1 and n - n_good + 1 of them, each set sorted by mean):
- *                                 {mean, log2(e)/(2 sigma^2), log2(weight/(sigma Z sqrt(2 pi))), sigma};
- *                                 all zero for a categorical dimension
+ *   comps   host [d][n + 2][4]    per dimension the good set's components from entry 0 and the bad set's
+ *                                 from entry n_good + 1, each set sorted by mean:
+ *                                 {mean, log2(e)/(2 sigma^2), log2(weight/(sigma Z sqrt(2 pi))), sigma}.
+ *                                 Components of one set with the same mean and the same sigma (repeated
+ *                                 values of a discrete feature) are stored once, with their weights
+ *                                 summed; entries past a set's count are unspecified
+ *   counts  host [d][2]           components stored for the good and the bad set (at most n_good + 1 and
+ *                                 n - n_good + 1); zero for a categorical dimension
  *   table   host [d][64]          ln P_good(v) - ln P_bad(v) per level v of a categorical dimension,
  *                                 ln l(v/(L-1)) - ln g(v/(L-1)) per grid value of a grid dimension; zero elsewhere
  */
-r3_status_t r3_tpe_get_model(r3_tpe_t* tpe, int* n_good, int* order, float* comps, float* table);
+r3_status_t r3_tpe_get_model(r3_tpe_t* tpe, int* n_good, int* order, float* comps, int* counts, float* table);
 
 /* Frees the handle and its device memory; NULL is allowed. */
 void r3_tpe_free(r3_tpe_t* tpe);

@@ -62,7 +62,7 @@ SIGNATURES = {
                         ctypes.POINTER(_vp)]),
     "r3_tpe_score": (_i, [_vp, _vp, _ll, _vp, _vp]),
     "r3_tpe_check": (_i, [_vp, _vp]),
-    "r3_tpe_get_model": (_i, [_vp, ctypes.POINTER(ctypes.c_int), _vp, _vp, _vp]),
+    "r3_tpe_get_model": (_i, [_vp, ctypes.POINTER(ctypes.c_int), _vp, _vp, _vp, _vp]),
     "r3_tpe_free": (None, [_vp]),
     "r3_topk_noalloc": (_i, [_vp, _i, _ll, _i, _vp, _vp, _vp]),
     "r3_gp_score_topk": (_i, [_vp, _vp, _ll, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -484,14 +484,16 @@ def r3_tpe_check(tpe: TPE):
 
 
 def r3_tpe_get_model(tpe: TPE):
-    """Host copies of the fitted model: (n_good, order [n], comps [d][n+2][4], table [d][64])."""
+    """Host copies of the fitted model: (n_good, order [n], comps [d][n+2][4], counts [d][2], table [d][64])."""
     n_good = ctypes.c_int()
     order = np.empty((tpe.n,), dtype=np.int32)
     comps = np.empty((tpe.d, tpe.n + 2, 4), dtype=np.float32)
+    counts = np.empty((tpe.d, 2), dtype=np.int32)
     table = np.empty((tpe.d, 64), dtype=np.float32)
     _check(load().r3_tpe_get_model(tpe.handle, ctypes.byref(n_good), ctypes.c_void_p(order.ctypes.data),
-                                   ctypes.c_void_p(comps.ctypes.data), ctypes.c_void_p(table.ctypes.data)))
-    return n_good.value, order, comps, table
+                                   ctypes.c_void_p(comps.ctypes.data), ctypes.c_void_p(counts.ctypes.data),
+                                   ctypes.c_void_p(table.ctypes.data)))
+    return n_good.value, order, comps, counts, table
 
 
 def r3_tpe_free(tpe: TPE):

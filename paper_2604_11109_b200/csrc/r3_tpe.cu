@@ -12,6 +12,7 @@
 #include <math.h>
 #include <stdlib.h>
 
+#include <algorithm>
 #include <new>
 #include <vector>
 
@@ -23,7 +24,12 @@ struct r3_tpe {
     std::vector<int> levels;
     int* levels_d = nullptr;   // [d]
     int* order_d = nullptr;    // [n] history indices by y ascending
-    float4* comps_d = nullptr; // [d][n + 2]: good set's components, then the bad set's
+    float4* comps_d = nullptr; // [d][n + 2]: good set's components from 0, the bad set's from n_good + 1
+    int* counts_d = nullptr;   // [d][2]: components of each set after merging equal ones
+    // a model small enough for shared memory is also kept packed: set (j, s) at [offs[2j + s], offs[2j + s + 1])
+    int total = 0;             // components kept over all dimensions and sets
+    float4* packed_d = nullptr;
+    int* offs_d = nullptr;     // [2d + 1]
     float* table_d = nullptr;  // [d][64] ln P_good - ln P_bad per level
     int* status_d = nullptr;   // status bits
     int* status_h = nullptr;   // pinned mirror
@@ -38,6 +44,7 @@ constexpr int kTpeMaxLevels = 64;
 constexpr int kSortThreads = 1024;
 constexpr int kScoreThreads = 256;
 constexpr int kStage = 512;   // components per shared-memory stage
+constexpr size_t kResidentBytes = 72 * 1024;   // largest model a scoring block keeps whole in shared memory
 
 // Unsigned integer with the same order as the float (-0 and +0 equal).
 __device__ __forceinline__ unsigned ordered_bits(float v)
@@ -105,7 +112,8 @@ __global__ void __launch_bounds__(kSortThreads) tpe_mixture_kernel(const float* 
                                                                    const int* __restrict__ order, int n, int d,
                                                                    int n_good, const int* __restrict__ levels,
                                                                    double prior_weight, float4* __restrict__ comps,
-                                                                   float* __restrict__ table, int* __restrict__ status)
+                                                                   int* __restrict__ n_comps, float* __restrict__ table,
+                                                                   int* __restrict__ status)
 {
     extern __shared__ unsigned long long keys[];   // pow2 >= n + 1 keys, then (grid dimensions) 2 (n + 1) doubles
     __shared__ int counts[kTpeMaxLevels];
@@ -139,6 +147,7 @@ __global__ void __launch_bounds__(kSortThreads) tpe_mixture_kernel(const float* 
                 else
                     table[(size_t)j * kTpeMaxLevels + v] = (float)(lnp_good[v] - lnp);
             }
+            if (threadIdx.x == 0) n_comps[2 * j + set] = 0;
             __syncthreads();
             continue;
         }
@@ -172,14 +181,51 @@ __global__ void __launch_bounds__(kSortThreads) tpe_mixture_kernel(const float* 
             const double w = is_prior ? prior_weight : 1.0;
             const double Z = 0.5 * erfc(-(1.0 - mu) / sigma * 0.70710678118654752440) -
                              0.5 * erfc(-(0.0 - mu) / sigma * 0.70710678118654752440);
-            const double a = 1.4426950408889634074 / (2.0 * sigma * sigma);
-            const double b = log2(w / (wsum * sigma * Z * 2.5066282746310005024));
-            out[t] = make_float4((float)mu, (float)a, (float)b, (float)sigma);
-            if (G > 0) {
-                double* par = reinterpret_cast<double*>(keys + count);
-                par[2 * t] = sigma;
-                par[2 * t + 1] = w / (wsum * sigma * Z * 2.5066282746310005024);
+            double* par = reinterpret_cast<double*>(keys + count);
+            par[2 * t] = sigma;
+            par[2 * t + 1] = w / (wsum * sigma * Z * 2.5066282746310005024);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            // Components with the same mean and bandwidth (repeated values of a discrete feature) are one
+            // component with the summed coefficient: the density is the same sum, with far fewer terms.
+            // Equal means are neighbours in the sorted order; among them a run of equal values has one
+            // bandwidth inside and one at each end, so a handful of open slots per mean is enough (a full
+            // set of slots emits its oldest one, which only costs a missed merge).
+            constexpr int kSlots = 4;
+            const double* par = reinterpret_cast<const double*>(keys + count);
+            int c = 0, open = 0;
+            unsigned run_mu = 0;
+            double slot_sigma[kSlots], slot_coef[kSlots];
+            auto emit = [&](int i) {
+                const double a = 1.4426950408889634074 / (2.0 * slot_sigma[i] * slot_sigma[i]);
+                out[c++] = make_float4(from_ordered_bits(run_mu), (float)a, (float)log2(slot_coef[i]), (float)slot_sigma[i]);
+            };
+            for (int t = 0; t <= s; ++t) {
+                const unsigned mu_bits = (unsigned)(keys[t] >> 32);
+                if (mu_bits != run_mu) {
+                    for (int i = 0; i < open; ++i) emit(i);
+                    open = 0;
+                    run_mu = mu_bits;
+                }
+                const double sigma = par[2 * t], coef = par[2 * t + 1];
+                int hit = -1;
+                for (int i = 0; i < open; ++i)
+                    if (slot_sigma[i] == sigma) hit = i;
+                if (hit >= 0) {
+                    slot_coef[hit] += coef;
+                    continue;
+                }
+                if (open == kSlots) {
+                    emit(0);
+                    for (int i = 1; i < kSlots; ++i) slot_sigma[i - 1] = slot_sigma[i], slot_coef[i - 1] = slot_coef[i];
+                    --open;
+                }
+                slot_sigma[open] = sigma;
+                slot_coef[open++] = coef;
             }
+            for (int i = 0; i < open; ++i) emit(i);
+            n_comps[2 * j + set] = c;
         }
         __syncthreads();
         if (G > 0) {
@@ -275,6 +321,7 @@ template <int R>
 __global__ void __launch_bounds__(kScoreThreads) tpe_score_kernel(const float* __restrict__ Xc, long long m, int n,
                                                                   int d, int n_good, const int* __restrict__ levels,
                                                                   const float4* __restrict__ comps,
+                                                                  const int* __restrict__ counts,
                                                                   const float* __restrict__ table,
                                                                   float* __restrict__ score, int* __restrict__ status)
 {
@@ -312,8 +359,116 @@ __global__ void __launch_bounds__(kScoreThreads) tpe_score_kernel(const float* _
             } else {
                 const float4* cj = comps + (size_t)j * (n + 2);
                 float sl[R], sg[R];
-                mixture_sums_staged<R>(cj, n_good + 1, x, sl, stage);
-                mixture_sums_staged<R>(cj + n_good + 1, n - n_good + 1, x, sg, stage);
+                mixture_sums_staged<R>(cj, __ldg(counts + 2 * j), x, sl, stage);
+                mixture_sums_staged<R>(cj + n_good + 1, __ldg(counts + 2 * j + 1), x, sg, stage);
+#pragma unroll
+                for (int r = 0; r < R; ++r) acc[r] += 0.69314718f * (lg2_fast(sl[r]) - lg2_fast(sg[r]));
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+            if (valid[r]) score[base + (long long)r * kScoreThreads] = acc[r];
+    }
+    if (bad) atomicOr(status, DEV_NONFINITE);
+}
+
+// One (dimension, set) per block: copy its kept components to their place in the packed model.
+__global__ void __launch_bounds__(256) tpe_pack_kernel(const float4* __restrict__ comps, int n, int n_good,
+                                                       const int* __restrict__ offs, float4* __restrict__ packed)
+{
+    const int j = blockIdx.x >> 1, set = blockIdx.x & 1;
+    const float4* src = comps + (size_t)j * (n + 2) + (set ? n_good + 1 : 0);
+    const int lo = offs[blockIdx.x], hi = offs[blockIdx.x + 1];
+    for (int i = lo + threadIdx.x; i < hi; i += blockDim.x) packed[i] = src[i - lo];
+}
+
+// sum over components [lo, hi) of a model held in shared memory, for R candidates at once
+template <int R>
+__device__ __forceinline__ void mixture_sums_resident(const float4* __restrict__ model, int lo, int hi,
+                                                      const float (&x)[R], float (&sum)[R])
+{
+    float part[4][R];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int r = 0; r < R; ++r) part[u][r] = 0.f;
+    int c = lo;
+    for (; c + 4 <= hi; c += 4) {
+        float4 q[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) q[u] = model[c + u];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const float t = x[r] - q[u].x;
+                part[u][r] += ex2_fast(fmaf(-t, t * q[u].y, q[u].z));
+            }
+        }
+    }
+    for (; c < hi; ++c) {
+        const float4 q = model[c];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const float t = x[r] - q.x;
+            part[(c - lo) & 3][r] += ex2_fast(fmaf(-t, t * q.y, q.z));
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) sum[r] = (part[0][r] + part[1][r]) + (part[2][r] + part[3][r]);
+}
+
+// (T4) for a model that fits shared memory (discrete features leave a few components per admissible value):
+// every block loads the packed model once and then walks its tiles without a block-wide barrier.  (Reading
+// four or eight features of a row per load, with the feature loop unrolled to match, measured 10-30 % slower:
+// the kernel is bound by instruction issue, not by the row reads.)
+template <int R>
+__global__ void __launch_bounds__(kScoreThreads) tpe_score_resident_kernel(
+    const float* __restrict__ Xc, long long m, int d, const int* __restrict__ levels, const int* __restrict__ offs,
+    const float4* __restrict__ packed, int total, const float* __restrict__ table, float* __restrict__ score,
+    int* __restrict__ status)
+{
+    extern __shared__ float4 model[];   // [total] components, then [2d + 1] offsets, then [d] level codes
+    int* offs_s = reinterpret_cast<int*>(model + total);
+    int* code_s = offs_s + 2 * d + 1;
+    for (int i = threadIdx.x; i < total; i += kScoreThreads) model[i] = __ldg(packed + i);
+    for (int i = threadIdx.x; i <= 2 * d; i += kScoreThreads) offs_s[i] = __ldg(offs + i);
+    for (int i = threadIdx.x; i < d; i += kScoreThreads) code_s[i] = __ldg(levels + i);
+    __syncthreads();
+    const long long tiles = (m + (long long)R * kScoreThreads - 1) / ((long long)R * kScoreThreads);
+    bool bad = false;
+    for (long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+        const long long base = tile * (long long)R * kScoreThreads + threadIdx.x;
+        const float* row[R];
+        bool valid[R];
+        float acc[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const long long cand = base + (long long)r * kScoreThreads;
+            valid[r] = cand < m;
+            row[r] = Xc + (size_t)(valid[r] ? cand : 0) * d;
+            acc[r] = 0.f;
+        }
+        for (int j = 0; j < d; ++j) {
+            float x[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                x[r] = row[r][j];
+                bad |= valid[r] && !isfinite(x[r]);
+            }
+            const int code = code_s[j];
+            const int C = code < 0 ? -code : code;
+            if (C > 0) {
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    const float lv = floorf(__fadd_rn(__fmul_rn(x[r], (float)(C - 1)), 0.5f));
+                    const int v = isfinite(x[r]) ? (int)fminf(fmaxf(lv, 0.f), (float)(C - 1)) : 0;
+                    acc[r] += __ldg(table + (size_t)j * kTpeMaxLevels + v);
+                }
+            } else {
+                float sl[R], sg[R];
+                mixture_sums_resident<R>(model, offs_s[2 * j], offs_s[2 * j + 1], x, sl);
+                mixture_sums_resident<R>(model, offs_s[2 * j + 1], offs_s[2 * j + 2], x, sg);
 #pragma unroll
                 for (int r = 0; r < R; ++r) acc[r] += 0.69314718f * (lg2_fast(sl[r]) - lg2_fast(sg[r]));
             }
@@ -399,12 +554,17 @@ __global__ void __launch_bounds__(256) tpe_table_score_kernel(const float* __res
     if (bad) atomicOr(status, DEV_NONFINITE);
 }
 
+size_t resident_bytes(int total, int d) { return sizeof(float4) * (size_t)total + sizeof(int) * (3 * (size_t)d + 1); }
+
 void tpe_destroy(r3_tpe* t)
 {
     if (!t) return;
     cudaFree(t->levels_d);
     cudaFree(t->order_d);
     cudaFree(t->comps_d);
+    cudaFree(t->counts_d);
+    cudaFree(t->packed_d);
+    cudaFree(t->offs_d);
     cudaFree(t->table_d);
     cudaFree(t->status_d);
     if (t->status_h) cudaFreeHost(t->status_h);
@@ -418,6 +578,7 @@ r3_status_t tpe_fit_impl(r3_tpe* t, const float* X, const float* y, cudaStream_t
     R3_CUDA_TRY(cudaMalloc(&t->levels_d, sizeof(int) * d));
     R3_CUDA_TRY(cudaMalloc(&t->order_d, sizeof(int) * n));
     R3_CUDA_TRY(cudaMalloc(&t->comps_d, sizeof(float4) * (size_t)d * (n + 2)));
+    R3_CUDA_TRY(cudaMalloc(&t->counts_d, sizeof(int) * 2 * (size_t)d));
     R3_CUDA_TRY(cudaMalloc(&t->table_d, sizeof(float) * (size_t)d * kTpeMaxLevels));
     R3_CUDA_TRY(cudaMalloc(&t->status_d, sizeof(int)));
     R3_CUDA_TRY(cudaMallocHost(&t->status_h, sizeof(int)));
@@ -432,12 +593,24 @@ r3_status_t tpe_fit_impl(r3_tpe* t, const float* X, const float* y, cudaStream_t
     if (smem > 48 * 1024)
         R3_CUDA_TRY(cudaFuncSetAttribute(tpe_mixture_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     R3_LAUNCH(tpe_mixture_kernel, d, kSortThreads, smem, stream, X, t->order_d, n, d, t->n_good, t->levels_d,
-              (double)t->prior_weight, t->comps_d, t->table_d, t->status_d);
+              (double)t->prior_weight, t->comps_d, t->counts_d, t->table_d, t->status_d);
     R3_CUDA_TRY(cudaMemcpyAsync(t->status_h, t->status_d, sizeof(int), cudaMemcpyDeviceToHost, stream));
     R3_CUDA_TRY(cudaStreamSynchronize(stream));
     if (*t->status_h & DEV_NONFINITE) {
         set_error("r3_tpe_fit: X or y contains NaN or Inf");
         return R3_ERR_NONFINITE;
+    }
+    // pack a model that a scoring block can hold in shared memory
+    std::vector<int> counts(2 * (size_t)d), offs(2 * (size_t)d + 1, 0);
+    R3_CUDA_TRY(cudaMemcpy(counts.data(), t->counts_d, sizeof(int) * 2 * (size_t)d, cudaMemcpyDeviceToHost));
+    for (int i = 0; i < 2 * d; ++i) offs[i + 1] = offs[i] + counts[i];
+    t->total = offs[2 * d];
+    if (t->total > 0 && resident_bytes(t->total, d) <= kResidentBytes) {
+        R3_CUDA_TRY(cudaMalloc(&t->packed_d, sizeof(float4) * (size_t)t->total));
+        R3_CUDA_TRY(cudaMalloc(&t->offs_d, sizeof(int) * offs.size()));
+        R3_CUDA_TRY(cudaMemcpyAsync(t->offs_d, offs.data(), sizeof(int) * offs.size(), cudaMemcpyHostToDevice, stream));
+        R3_LAUNCH(tpe_pack_kernel, 2 * d, 256, 0, stream, t->comps_d, n, t->n_good, t->offs_d, t->packed_d);
+        R3_CUDA_TRY(cudaStreamSynchronize(stream));   // `offs` leaves scope
     }
     return R3_OK;
 }
@@ -528,6 +701,29 @@ r3_status_t r3_tpe_score(r3_tpe_t* tpe, const float* Xcand, long long m, float* 
 #undef R3_TPE_TABLE
         return R3_OK;
     }
+    if (tpe->packed_d) {
+        // the whole model in shared memory.  Sixteen blocks per SM's worth of grid (several waves of short
+        // blocks) measured up to 8 % faster than one resident wave walking the tiles: the model is a small
+        // read from L2 and the finer grain balances the SMs better.
+        const size_t smem = resident_bytes(tpe->total, tpe->d);
+        const long long tiles2 = (m + 2ll * kScoreThreads - 1) / (2ll * kScoreThreads);
+        const long long tiles1 = (m + kScoreThreads - 1) / kScoreThreads;
+#define R3_TPE_RESIDENT(R, TILES)                                                                              \
+    do {                                                                                                       \
+        if (smem > 48 * 1024)                                                                                  \
+            R3_CUDA_TRY(cudaFuncSetAttribute(tpe_score_resident_kernel<R>,                                     \
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));         \
+        const unsigned grid = (unsigned)std::min<long long>(TILES, 148ll * 16);                                \
+        R3_LAUNCH(tpe_score_resident_kernel<R>, grid, kScoreThreads, smem, stream, Xcand, m, tpe->d,           \
+                  tpe->levels_d, tpe->offs_d, tpe->packed_d, tpe->total, tpe->table_d, score, tpe->status_d);  \
+    } while (0)
+        if (tiles2 >= 148ll * 8)
+            R3_TPE_RESIDENT(2, tiles2);
+        else
+            R3_TPE_RESIDENT(1, tiles1);
+#undef R3_TPE_RESIDENT
+        return R3_OK;
+    }
     // Two candidates per thread (one shared-memory read serves both) when that still gives every SM
     // several blocks; one per thread for small pools.  More per thread measured slower on the full pool
     // (fewer, longer blocks balance worse over the 148 SMs).
@@ -535,11 +731,11 @@ r3_status_t r3_tpe_score(r3_tpe_t* tpe, const float* Xcand, long long m, float* 
     if (tiles2 >= 148ll * 4) {
         const unsigned grid = (unsigned)(tiles2 < 148ll * 64 ? tiles2 : 148ll * 64);
         R3_LAUNCH(tpe_score_kernel<2>, grid, kScoreThreads, 0, stream, Xcand, m, tpe->n, tpe->d, tpe->n_good,
-                  tpe->levels_d, tpe->comps_d, tpe->table_d, score, tpe->status_d);
+                  tpe->levels_d, tpe->comps_d, tpe->counts_d, tpe->table_d, score, tpe->status_d);
     } else {
         const long long tiles1 = (m + kScoreThreads - 1) / kScoreThreads;
         R3_LAUNCH(tpe_score_kernel<1>, (unsigned)tiles1, kScoreThreads, 0, stream, Xcand, m, tpe->n, tpe->d,
-                  tpe->n_good, tpe->levels_d, tpe->comps_d, tpe->table_d, score, tpe->status_d);
+                  tpe->n_good, tpe->levels_d, tpe->comps_d, tpe->counts_d, tpe->table_d, score, tpe->status_d);
     }
     return R3_OK;
 }
@@ -561,7 +757,7 @@ r3_status_t r3_tpe_check(r3_tpe_t* tpe, void* cuda_stream)
     return R3_OK;
 }
 
-r3_status_t r3_tpe_get_model(r3_tpe_t* tpe, int* n_good, int* order, float* comps, float* table)
+r3_status_t r3_tpe_get_model(r3_tpe_t* tpe, int* n_good, int* order, float* comps, int* counts, float* table)
 {
     if (!tpe) {
         set_error("r3_tpe_get_model: NULL handle");
@@ -573,6 +769,7 @@ r3_status_t r3_tpe_get_model(r3_tpe_t* tpe, int* n_good, int* order, float* comp
     if (comps)
         R3_CUDA_TRY(cudaMemcpy(comps, tpe->comps_d, sizeof(float4) * (size_t)tpe->d * (tpe->n + 2),
                                cudaMemcpyDeviceToHost));
+    if (counts) R3_CUDA_TRY(cudaMemcpy(counts, tpe->counts_d, sizeof(int) * 2 * (size_t)tpe->d, cudaMemcpyDeviceToHost));
     if (table)
         R3_CUDA_TRY(cudaMemcpy(table, tpe->table_d, sizeof(float) * (size_t)tpe->d * kTpeMaxLevels,
                                cudaMemcpyDeviceToHost));

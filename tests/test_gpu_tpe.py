@@ -61,8 +61,18 @@ def rand_case(seed, n, d, m, frac_cat=0.4, continuous=True):
     return X.astype(np.float32), y.astype(np.float32), levels, Xc.astype(np.float32)
 
 
+def merged(mu, sigma, coef):
+    """One (mean, sigma, summed coefficient) row per distinct (mean, sigma), sorted."""
+    key = np.lexsort((sigma, mu))
+    mu, sigma, coef = mu[key], sigma[key], coef[key]
+    first = np.ones(mu.shape[0], dtype=bool)
+    first[1:] = (mu[1:] != mu[:-1]) | (np.abs(sigma[1:] - sigma[:-1]) > 1e-6 * sigma[:-1])
+    start = np.flatnonzero(first)
+    return mu[start], sigma[start], np.add.reduceat(coef, start)
+
+
 def check_model(tpe, model, n, d):
-    n_good, order, comps, table = b.r3_tpe_get_model(tpe)
+    n_good, order, comps, counts, table = b.r3_tpe_get_model(tpe)
     assert n_good == model.n_good
     assert order.tolist() == model.order.tolist()
     for j in range(d):
@@ -70,24 +80,27 @@ def check_model(tpe, model, n, d):
             C = int(model.levels[j])
             want = np.log(model.good[j].prob) - np.log(model.bad[j].prob)
             np.testing.assert_allclose(table[j, :C], want, rtol=1e-6, atol=1e-6)
-            assert not comps[j].any()
+            assert counts[j].tolist() == [0, 0]
             continue
-        off = 0
-        for mix in (model.good[j], model.bad[j]):
-            cnt = mix.mu.shape[0]
+        for set_, (mix, off) in enumerate(((model.good[j], 0), (model.bad[j], n_good + 1))):
+            cnt = int(counts[j, set_])
+            assert 1 <= cnt <= mix.mu.shape[0]
             got = comps[j, off:off + cnt].astype(np.float64)
-            off += cnt
-            # the device keeps each set sorted by mean, the prior after equal values
-            srt = np.lexsort((np.arange(cnt), mix.mu))
-            np.testing.assert_array_equal(got[:, 0], mix.mu[srt])
-            # equal means may come in any order; their bandwidths as a multiset must agree
-            key_got = np.lexsort((got[:, 3], got[:, 0]))
-            key_ref = np.lexsort((mix.sigma[srt], mix.mu[srt]))
-            np.testing.assert_allclose(got[key_got, 3], mix.sigma[srt][key_ref], rtol=2e-7)
-            a = np.log2(np.e) / (2 * mix.sigma ** 2)
-            bb = np.log2(mix.weight / (mix.sigma * mix.Z * np.sqrt(2 * np.pi)))
-            np.testing.assert_allclose(np.sort(got[:, 1]), np.sort(a), rtol=3e-7)
-            np.testing.assert_allclose(np.sort(got[:, 2]), np.sort(bb), rtol=3e-7, atol=3e-7)
+            # each set stays sorted by mean
+            assert (np.diff(got[:, 0]) >= 0).all()
+            # the exponent's factor belongs to the stored sigma
+            np.testing.assert_allclose(got[:, 1], np.log2(np.e) / (2 * got[:, 3] ** 2), rtol=3e-7)
+            # equal (mean, sigma) components are one component with the summed coefficient: compare the
+            # two sides after merging both completely (the device merges neighbours in its sorted order)
+            ref_coef = mix.weight / (mix.sigma * mix.Z * np.sqrt(2 * np.pi))
+            rmu, rsig, rcoef = merged(mix.mu.astype(np.float64), mix.sigma, ref_coef)
+            gmu, gsig, gcoef = merged(got[:, 0], got[:, 3], np.exp2(got[:, 2]))
+            np.testing.assert_array_equal(gmu, rmu)
+            np.testing.assert_allclose(gsig, rsig, rtol=2e-7)
+            np.testing.assert_allclose(gcoef, rcoef, rtol=1e-6)
+            # a run of equal values gives at most three neighbour-gap bandwidths (its two ends and its
+            # inside), and the prior can split one run in two
+            assert cnt <= 3 * np.unique(mix.mu).shape[0] + 2
         if model.levels[j] < 0:
             L = int(-model.levels[j])
             xg = (np.arange(L) / (L - 1)).astype(np.float32)
@@ -152,6 +165,57 @@ def test_all_categorical_and_all_ordinal():
         check_model(tpe, model, 150, 6)
         check_score(b.r3_tpe_score(tpe, dev(Xc)).cpu().numpy(), T.tpe_score(model, Xc), atol(150, levels))
         tpe.close()
+
+
+def test_repeated_values_are_merged_and_large_models_are_not_packed():
+    """Unevenly spaced admissible values, one of them the prior's mean, repeated many times: a few components
+    per value remain, and candidates anywhere in [0, 1] score as with the unmerged mixture.  A continuous
+    feature beside them keeps all its components; with the longest history the model exceeds what a block
+    holds in shared memory, so both scoring paths are taken."""
+    rng = np.random.default_rng(77)
+    values = np.array([0.0, 0.1, 0.12, 0.5, 0.55, 0.9, 1.0])
+    for n, m in ((300, 5000), (4096, 3000)):
+        X = values[rng.integers(0, values.shape[0], size=(n, 6))]
+        X[:, 5] = rng.random(n)
+        Xc = rng.random((m, 6))
+        Xc[: m // 2] = values[rng.integers(0, values.shape[0], size=(m // 2, 6))]
+        y = rng.normal(0, 1, n)
+        X, y, Xc = X.astype(np.float32), y.astype(np.float32), Xc.astype(np.float32)
+        levels = np.zeros(6, dtype=np.int32)
+        model = T.tpe_fit(X, y, levels, 0.25, 1.0)
+        tpe = b.r3_tpe_fit(dev(X), dev(y), levels, 0.25, 1.0)
+        check_model(tpe, model, n, 6)
+        counts = b.r3_tpe_get_model(tpe)[3]
+        assert counts[:5].max() <= 3 * values.shape[0] + 2
+        assert counts[5].sum() == n + 2
+        check_score(b.r3_tpe_score(tpe, dev(Xc)).cpu().numpy(), T.tpe_score(model, Xc), atol(n, levels))
+        b.r3_tpe_check(tpe)
+        tpe.close()
+
+
+@pytest.mark.parametrize("d,m", [(8, 40000), (12, 3000), (16, 300001), (10, 5000)])
+def test_packed_model_pool_sizes_and_alignment(d, m):
+    """Discrete ordinal features (a model that a block keeps in shared memory), pools large and small enough
+    for both tile widths, and a pool that does not start on a 16-byte boundary: all give the oracle's
+    scores."""
+    rng = np.random.default_rng(500 + d)
+    n = 400
+    L = rng.integers(3, 20, size=d)
+    X = np.stack([rng.integers(0, L[j], size=n) / (L[j] - 1) for j in range(d)], axis=1).astype(np.float32)
+    Xc = np.stack([rng.integers(0, L[j], size=m) / (L[j] - 1) for j in range(d)], axis=1).astype(np.float32)
+    levels = np.zeros(d, dtype=np.int32)
+    levels[1] = 2
+    X[:, 1], Xc[:, 1] = rng.integers(0, 2, n), rng.integers(0, 2, m)
+    y = rng.normal(size=n).astype(np.float32)
+    model = T.tpe_fit(X, y, levels, 0.25, 1.0)
+    tpe = b.r3_tpe_fit(dev(X), dev(y), levels, 0.25, 1.0)
+    want = T.tpe_score(model, Xc)
+    check_score(b.r3_tpe_score(tpe, dev(Xc)).cpu().numpy(), want, atol(n, levels))
+    shifted = torch.empty(m * d + 1, dtype=torch.float32, device="cuda")[1:].view(m, d)
+    shifted.copy_(dev(Xc))
+    check_score(b.r3_tpe_score(tpe, shifted).cpu().numpy(), want, atol(n, levels))
+    b.r3_tpe_check(tpe)
+    tpe.close()
 
 
 @pytest.mark.parametrize("d,m", [(4, 1000), (8, 5000), (20, 3001), (64, 70000), (132, 2000)])
