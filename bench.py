@@ -160,12 +160,23 @@ def run_tpe(args, c):
     g = w.generate_gp(c, 0)
     levels = w.tpe_levels(c, grid=args.tpe_grid)
     n, d, m, k = c.n, c.d, c.m, c.k
+    if args.tpe_continuous:
+        # continuous parameters in place of the paper's discrete ones: each ordinal value moves by up to half the
+        # smallest level spacing of its feature, so that no two observations share a component
+        rng = np.random.default_rng(20260411)
+        X = g["X"].astype(np.float64)
+        for j in np.flatnonzero(levels == 0):
+            vals = np.unique(X[:, j])
+            half = 0.5 * np.diff(vals).min() if vals.shape[0] > 1 else 0.5
+            X[:, j] = np.clip(X[:, j] + rng.uniform(-half, half, n), 0.0, 1.0)
+        g = dict(g, X=X.astype(np.float32))
     base = {"metric": "tpe_candidates_scored_per_sec", "unit": "candidates/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "data": "synthetic",
             "config": {"workload": c.name + "-tpe", "n": n, "d": d, "m": m, "k": k, "gamma": 0.25,
                        "ordinal_dims": int((levels == 0).sum()), "grid_dims": int((levels < 0).sum()),
-                       "categorical_dims": int((levels > 0).sum())}}
+                       "categorical_dims": int((levels > 0).sum()),
+                       "history": "continuous (jittered)" if args.tpe_continuous else "discrete (the workload's)"}}
     if args.impl == "reference":
         if rank != 0:
             return
@@ -210,6 +221,9 @@ def run_tpe(args, c):
     # exponentials per candidate: the components the fit kept (equal ones merged) of every ordinal dimension
     counts = b.r3_tpe_get_model(tpe)[3]
     evals = float(counts[levels == 0].sum())
+    # the library keeps a model of at most 72 KB (16 B per component, 12 B per dimension) in shared memory
+    score_kernel = ("tpe_table_score_kernel" if evals == 0 and d % 4 == 0 else
+                    "tpe_score_resident_kernel" if 16 * evals + 12 * d + 4 <= 72 * 1024 else "tpe_score_kernel")
     score = torch.empty((m,), device="cuda")
     scratch = torch.empty((b.r3_topk_scratch_bytes(1, m, k),), dtype=torch.uint8, device="cuda")
     kernel_ms = []
@@ -292,13 +306,13 @@ def run_tpe(args, c):
     hbm_bytes = float(m) * (4 * d + 4)
     if evals * m / (mufu_peak * 1e12) >= hbm_bytes / (peaks["hbm_gbs"] * 1e9):
         achieved = evals * m / (k_ms * 1e-3) / 1e12
-        roofline = {"bound": "alu", "kernel": "tpe_score_kernel", "achieved": achieved, "peak": mufu_peak,
+        roofline = {"bound": "alu", "kernel": score_kernel, "achieved": achieved, "peak": mufu_peak,
                     "unit": "Texp2/s", "frac": achieved / mufu_peak, "traffic": None,
                     "note": "one MUFU.EX2 per (candidate, ordinal dimension, stored component); peak = 148 SMs x 16 MUFU "
                             "results per clock x max SM clock"}
     else:
         achieved = hbm_bytes / (k_ms * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "kernel": "tpe_score_kernel", "achieved": achieved, "peak": peaks["hbm_gbs"],
+        roofline = {"bound": "hbm", "kernel": score_kernel, "achieved": achieved, "peak": peaks["hbm_gbs"],
                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
                     "note": f"4d + 4 bytes per candidate (pool read once, one score written); peak = {peak_kind} copy "
                             "bandwidth"}
@@ -347,6 +361,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tpe-grid", action="store_true",
                     help="tpe: declare equally spaced ordinal features as grids (tabulated at fit time)")
+    ap.add_argument("--tpe-continuous", action="store_true",
+                    help="tpe: spread the history's ordinal values uniformly inside their level's cell (a space of "
+                         "continuous parameters: every observation keeps its own component)")
     ap.add_argument("--surrogate", default="gp", choices=["gp", "tpe"],
                     help="gp: the headline GP-EI path; tpe: Parzen-estimator scoring of the same pools")
     args = ap.parse_args()
