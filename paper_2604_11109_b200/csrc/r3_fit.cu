@@ -104,6 +104,14 @@ __global__ void gram_kernel(const float* __restrict__ X, const float* __restrict
 // ------------------------------------------------------------------------------------ Cholesky
 // Factor the 32x32 diagonal block at j0 in shared memory, write it back (upper part zeroed) and
 // store its inverse in Dinv[g][j0/32].
+//
+// One barrier per column.  At step k every thread forms r = 1/sqrt(a_kk) itself and scales what it reads of
+// column k by it, so that nothing has to be written (and waited for) between the pivot and the update; the
+// column stays unscaled in shared memory until the end.  The inverse comes from the same sweep: with
+// L = L_1 ... L_32 (L_k the identity with column k of L), L^-1 = L_32^-1 ... L_1^-1, and applying L_k^-1 to
+// the running product M is the same rank-one update on the columns <= k that the factorisation does on the
+// columns > k -- the threads of the finished columns do it.  Row k of M, like column k of A, is scaled by r
+// only at the end.
 __global__ void __launch_bounds__(1024) potrf_diag_kernel(double* __restrict__ A, int npad, int j0,
                                                           double* __restrict__ Dinv, int* status)
 {
@@ -111,41 +119,37 @@ __global__ void __launch_bounds__(1024) potrf_diag_kernel(double* __restrict__ A
     const int tx = threadIdx.x, ty = threadIdx.y;
     double* Ag = A + (size_t)g * npad * npad + (size_t)j0 * npad + j0;
     __shared__ double a[NB][NB + 1];
-    __shared__ double inv[NB][NB + 1];
+    __shared__ double m[NB][NB + 1];
+    __shared__ double rk[NB], lkk[NB];
     a[ty][tx] = Ag[(size_t)ty * npad + tx];
+    m[ty][tx] = (tx == ty) ? 1.0 : 0.0;
     __syncthreads();
     for (int k = 0; k < NB; ++k) {
-        if (tx == k && ty == k) {
-            double p = a[k][k];
-            if (!(p > 0.0) || !isfinite(p)) {
+        double p = a[k][k];
+        if (!(p > 0.0) || !isfinite(p)) {
+            if (tx == k && ty == k) {
                 atomicOr(&status[0], DEV_NOT_PD);
                 atomicMin(&status[1], j0 + k);
-                p = 1.0;  // keep going without NaNs; the call reports the failure
             }
-            a[k][k] = sqrt(p);
+            p = 1.0;  // keep going without NaNs; the call reports the failure
+        }
+        const double r = rsqrt(p);
+        if (tx == k && ty == k) {
+            rk[k] = r;
+            lkk[k] = sqrt(p);
+        }
+        if (ty > k) {
+            const double lik = a[ty][k] * r;
+            if (tx > k) {
+                if (ty >= tx) a[ty][tx] -= lik * (a[tx][k] * r);
+            } else {
+                m[ty][tx] -= lik * (m[k][tx] * r);
+            }
         }
         __syncthreads();
-        if (tx == k && ty > k) a[ty][k] /= a[k][k];
-        __syncthreads();
-        if (tx > k && ty >= tx) a[ty][tx] -= a[ty][k] * a[tx][k];
-        __syncthreads();
     }
-    // inverse of the lower-triangular block, one column per thread of the first warp row
-    if (ty == 0) {
-        const int c = tx;
-        for (int i = 0; i < NB; ++i) {
-            double s = (i == c) ? 1.0 : 0.0;
-            if (i < c) {
-                inv[i][c] = 0.0;
-                continue;
-            }
-            for (int k = c; k < i; ++k) s -= a[i][k] * inv[k][c];
-            inv[i][c] = s / a[i][i];
-        }
-    }
-    __syncthreads();
-    Ag[(size_t)ty * npad + tx] = (tx <= ty) ? a[ty][tx] : 0.0;
-    Dinv[((size_t)g * (npad / NB) + j0 / NB) * NB * NB + ty * NB + tx] = inv[ty][tx];
+    Ag[(size_t)ty * npad + tx] = (tx < ty) ? a[ty][tx] * rk[tx] : (tx == ty ? lkk[ty] : 0.0);
+    Dinv[((size_t)g * (npad / NB) + j0 / NB) * NB * NB + ty * NB + tx] = m[ty][tx] * rk[ty];
 }
 
 // Panel below the diagonal block: L_panel = A_panel * inv(L_jj)^T, 64 rows per block.
