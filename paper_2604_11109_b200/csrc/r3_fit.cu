@@ -179,45 +179,51 @@ __global__ void __launch_bounds__(256) panel_kernel(double* __restrict__ A, int 
     }
 }
 
-// Trailing update: A[i][j] -= sum_k P[i][k] P[j][k] over the 32 panel columns, 64x64 tiles of the
-// lower triangle of the trailing matrix.
-__global__ void __launch_bounds__(256) syrk_kernel(double* __restrict__ A, int npad, int j0)
+// Trailing update: A[i][j] -= sum_k A[i][k] A[j][k] over the kw finished columns from k0 (kw a multiple of
+// 32), for rows i >= j >= base and columns j < col_end; 64x64 tiles of the lower triangle counted from
+// `base`.  The factorisation calls it twice per 32 columns' worth of work: narrowly (kw = 32) for the
+// columns that remain inside the current 128-column panel, and once per panel (kw = 128) for everything to
+// the right of it, so that the large trailing matrix is read and written once per 128 columns.
+__global__ void __launch_bounds__(256) syrk_kernel(double* __restrict__ A, int npad, int k0, int kw, int base,
+                                                   int col_end)
 {
     const int ti = blockIdx.y, tj = blockIdx.x;
     if (tj > ti) return;
     const int g = blockIdx.z;
-    const int base = j0 + NB;
     double* Ag = A + (size_t)g * npad * npad;
     __shared__ double pi[64][NB + 1], pj[64][NB + 1];
     const int t = threadIdx.x;
-    for (int e = t; e < 64 * NB; e += 256) {
-        int r = e / NB, c = e % NB;
-        int gi = base + ti * 64 + r, gj = base + tj * 64 + r;
-        pi[r][c] = (gi < npad) ? Ag[(size_t)gi * npad + j0 + c] : 0.0;
-        pj[r][c] = (gj < npad) ? Ag[(size_t)gj * npad + j0 + c] : 0.0;
-    }
-    __syncthreads();
     const int ty = t / 16, tx = t % 16;
     double acc[4][4] = {};
-#pragma unroll 8
-    for (int k = 0; k < NB; ++k) {
-        double a[4], b[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            a[u] = pi[ty + 16 * u][k];
-            b[u] = pj[tx + 16 * u][k];
+    for (int kc = 0; kc < kw; kc += NB) {
+        if (kc > 0) __syncthreads();
+        for (int e = t; e < 64 * NB; e += 256) {
+            int r = e / NB, c = e % NB;
+            int gi = base + ti * 64 + r, gj = base + tj * 64 + r;
+            pi[r][c] = (gi < npad) ? Ag[(size_t)gi * npad + k0 + kc + c] : 0.0;
+            pj[r][c] = (gj < npad) ? Ag[(size_t)gj * npad + k0 + kc + c] : 0.0;
         }
+        __syncthreads();
+#pragma unroll 8
+        for (int k = 0; k < NB; ++k) {
+            double a[4], b[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
+            for (int u = 0; u < 4; ++u) {
+                a[u] = pi[ty + 16 * u][k];
+                b[u] = pj[tx + 16 * u][k];
+            }
 #pragma unroll
-            for (int v = 0; v < 4; ++v) acc[u][v] += a[u] * b[v];
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int v = 0; v < 4; ++v) acc[u][v] += a[u] * b[v];
+        }
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u)
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
             int gi = base + ti * 64 + ty + 16 * u, gj = base + tj * 64 + tx + 16 * v;
-            if (gi < npad && gj <= gi) Ag[(size_t)gi * npad + gj] -= acc[u][v];
+            if (gi < npad && gj <= gi && gj < col_end) Ag[(size_t)gi * npad + gj] -= acc[u][v];
         }
 }
 
@@ -466,13 +472,24 @@ r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream)
     LAUNCH_OR_FAIL(gram_kernel, dim3(npad / 16, npad / 16, B), dim3(16, 16), gp->X, gp->ell_d, gp->sf2_d,
                    gp->sn2_d, n, d, npad, gp->L64);
 
-    for (int j0 = 0; j0 < npad; j0 += NB) {
-        LAUNCH_OR_FAIL(potrf_diag_kernel, B, dim3(NB, NB), gp->L64, npad, j0, Dinv, gp->status_d);
-        const int rows = npad - j0 - NB;
-        if (rows > 0) {
+    constexpr int kOuter = 4 * NB;   // columns per panel of the two-level right-looking factorisation
+    for (int J = 0; J < npad; J += kOuter) {
+        const int panel_end = std::min(J + kOuter, npad);
+        for (int j0 = J; j0 < panel_end; j0 += NB) {
+            LAUNCH_OR_FAIL(potrf_diag_kernel, B, dim3(NB, NB), gp->L64, npad, j0, Dinv, gp->status_d);
+            const int rows = npad - j0 - NB;
+            if (rows <= 0) continue;
             const int tiles = (rows + 63) / 64;
             LAUNCH_OR_FAIL(panel_kernel, dim3(tiles, B), 256, gp->L64, npad, j0, Dinv);
-            LAUNCH_OR_FAIL(syrk_kernel, dim3(tiles, tiles, B), 256, gp->L64, npad, j0);
+            const int inner = panel_end - j0 - NB;   // columns of this panel still to be factored
+            if (inner > 0)
+                LAUNCH_OR_FAIL(syrk_kernel, dim3((inner + 63) / 64, tiles, B), 256, gp->L64, npad, j0, NB, j0 + NB,
+                               panel_end);
+        }
+        const int rows = npad - panel_end;
+        if (rows > 0) {
+            const int tiles = (rows + 63) / 64;
+            LAUNCH_OR_FAIL(syrk_kernel, dim3(tiles, tiles, B), 256, gp->L64, npad, J, panel_end - J, panel_end, npad);
         }
     }
 
