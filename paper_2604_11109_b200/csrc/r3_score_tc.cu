@@ -230,6 +230,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                 TICK(0);
                 if (!(ok = mbar_wait(bar(BAR_D_EMPTY + db), d_ph ^ 1u, abort_flag))) break;
                 TICK(1);
+                LOGEV(8, (long long)(tile_iter * (items_per_tile / SL) + u) * SL);
                 tc_fence_after();
                 const uint32_t xH_lo = x_lo0 + ((st * map.x_stage) >> 4), xL_lo = xH_lo + (((uint32_t)DP * KD * 2u) >> 4);
                 const uint32_t dcol = tmem + NV + db * KD;
@@ -245,6 +246,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                 tc_commit(bar(BAR_X_EMPTY + st));
                 tc_commit(bar(BAR_D_FULL + db));
                 TICK(2);
+                LOGEV(7, (long long)(tile_iter * (items_per_tile / SL) + u) * SL);
                 if (++st == XS) { st = 0; ph ^= 1u; }
                 if (++db == 2) { db = 0; d_ph ^= 1u; }
             }
@@ -262,6 +264,10 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
         int w_s = 0, k_s = 0, e_s = 0;   // e_s: chunk number mod 4 (ring mode: which "consumed" barrier)
         uint32_t w_ph = 0, k_ph = 0;
         bool ok = true;
+        // whether the next chunk's k* and W were already seen complete (tested between this chunk's MMAs, while
+        // the pipe has work queued, so that nothing but the commits sits between two chunks' MMAs)
+        bool k_seen = false, w_seen = false;
+        long long tv = 0;
         for (long long tile = first_tile; ok && tile < prm.total_tiles; tile += tile_step) {
             for (int p = 0; ok && p < P; ++p) {
                 const int nchunk = (p + 1) * CPP;
@@ -272,9 +278,11 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                         if (!(ok = mbar_wait(bar(BAR_V_EMPTY), v_ph ^ 1u, abort_flag))) break;
                     }
                     TICK(3);
-                    if (!(ok = mbar_wait(bar(BAR_K_FULL + b), k_ph, abort_flag))) break;
+                    if (!k_seen && !(ok = mbar_wait(bar(BAR_K_FULL + b), k_ph, abort_flag))) break;
                     TICK(4);
-                    if (!(ok = mbar_wait(bar(BAR_W_FULL + s), w_ph, abort_flag))) break;
+                    LOGEV(0, tv);
+                    if (!w_seen && !(ok = mbar_wait(bar(BAR_W_FULL + s), w_ph, abort_flag))) break;
+                    LOGEV(1, tv);
                     if (++k_s == NBK) { k_s = 0; k_ph ^= 1u; }
                     if (++w_s == ws) { w_s = 0; w_ph ^= 1u; }
                     TICK(5);
@@ -294,6 +302,10 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                             for (int jj = 0; jj < KC / 16; ++jj)
                                 tc_mma_f16_ts(vcol, a0 + jj * 8u, pack64(b0 + jj * ((2u * NV * 16u) >> 4), kDescHi), idesc_v,
                                               (c > 0 || combo > 0 || jj > 0) ? 1u : 0u);
+                            if (combo == 1) {
+                                k_seen = mbar_try_wait(bar(BAR_K_FULL + k_s), k_ph);
+                                w_seen = mbar_try_wait(bar(BAR_W_FULL + w_s), w_ph);
+                            }
                         }
                     } else {
                         const uint32_t aH = k_lo0 + ((b * 16384u) >> 4), aL = aH + (8192u >> 4);
@@ -305,6 +317,10 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                                 tc_mma_f16(vcol, pack64(a0 + jj * (4096u >> 4), kDescHi),
                                            pack64(b0 + jj * ((2u * NV * 16u) >> 4), kDescHi), idesc_v,
                                            (c > 0 || combo > 0 || jj > 0) ? 1u : 0u);
+                            if (combo == 1) {
+                                k_seen = mbar_try_wait(bar(BAR_K_FULL + k_s), k_ph);
+                                w_seen = mbar_try_wait(bar(BAR_W_FULL + w_s), w_ph);
+                            }
                         }
                     }
                     tc_commit(bar(BAR_W_EMPTY + s));
@@ -315,6 +331,8 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                         v_ph ^= 1u;
                     }
                     TICK(6);
+                    LOGEV(2, tv);
+                    ++tv;
                 }
             }
         }
@@ -450,6 +468,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     TICK(0);
+                    if (threadIdx.x % 128 == 0) LOGEV(3, t);
                     tc_fence_after();
                     const bool fresh = c >= p * CPP;   // first time this chunk is generated for the tile
                     // k* buffer and the parity of its hand-over: the group's own buffer, or slot t mod NBK of the ring
@@ -523,6 +542,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                         }
                     }
                     TICK(2);
+                    if (threadIdx.x % 128 == 0) LOGEV(4, t);
                     if (NBK == G) {
                         ok = mbar_wait(bar(BAR_K_EMPTY + kbuf), kpar ^ 1u, abort_flag);
                     } else if (t >= NBK) {
@@ -537,6 +557,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     TICK(3);
+                    if (threadIdx.x % 128 == 0) LOGEV(5, t);
 #pragma unroll
                     for (int h = 0; h < KC / 16; ++h) {
                         if (KT) {
@@ -563,6 +584,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     }
                     mbar_arrive(bar(BAR_K_FULL + kbuf));
                     TICK(4);
+                    if (threadIdx.x % 128 == 0) LOGEV(6, t);
                     t += G;
                     own_ph ^= 1u;
                 }
@@ -981,8 +1003,8 @@ r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, floa
     // R3_TC_TRACE=1 prints, for the first CTA, the cycles each role spent per wait / issue category
     prm.trace = nullptr;
     if (getenv("R3_TC_TRACE")) {
-        if (dev_malloc(&prm.trace, sizeof(long long) * grid * 32) != cudaSuccess) prm.trace = nullptr;
-        if (prm.trace) cudaMemset(prm.trace, 0, sizeof(long long) * grid * 32);
+        if (dev_malloc(&prm.trace, sizeof(long long) * (grid * 32 + 16 * 128)) != cudaSuccess) prm.trace = nullptr;
+        if (prm.trace) cudaMemset(prm.trace, 0, sizeof(long long) * (grid * 32 + 16 * 128));
     }
     // The paired kernel (two CTAs of a cluster share a tile and the k* chunks) serves histories with at least
     // two passes; R3_TC_PAIR=0/1 overrides the choice.
@@ -998,8 +1020,13 @@ r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, floa
     }
     prof_end(gp, stream);
     if (prm.trace) {
-        std::vector<long long> h((size_t)grid * 32);
-        cudaMemcpy(h.data(), prm.trace, sizeof(long long) * grid * 32, cudaMemcpyDeviceToHost);
+        std::vector<long long> h((size_t)grid * 32 + 16 * 128);
+        cudaMemcpy(h.data(), prm.trace, sizeof(long long) * h.size(), cudaMemcpyDeviceToHost);
+        for (int i = 0; i < 128; ++i) {
+            fprintf(stderr, "ev %d:", i);
+            for (int e = 0; e < 10; ++e) fprintf(stderr, " %lld", h[(size_t)grid * 32 + e * 128 + i] - h[(size_t)grid * 32]);
+            fprintf(stderr, "\n");
+        }
         dev_free(prm.trace);
         const char* names[4] = {"mmaV", "matern0", "matern1", "mmaD"};
         fprintf(stderr, "trace shape NV=%d G=%d KD=%d kt=%d ws=%d DP=%d P=%d smem=%zu\n", t->NV, t->G, t->KD, (int)t->kt, t->ws,

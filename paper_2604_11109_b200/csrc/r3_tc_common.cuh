@@ -300,7 +300,15 @@ __device__ __noinline__ void refine_close_pairs(float* kv, float v_thresh, float
 // Per-role cycle accounting, compiled in only with -DR3_TC_TRACE (it costs issue slots on the hot path).
 #ifndef R3_TC_TRACE
 #define TICK(cat) do { } while (0)
+#define LOGEV(ev, tt) do { } while (0)
 #else
+// event log of the first CTA: clock of event `ev` for global chunk number tt in [kLogT0, kLogT0 + kLogN)
+constexpr long long kLogT0 = 1088 + 600, kLogN = 128;
+#define LOGEV(ev, tt)                                                                                         \
+    do {                                                                                                      \
+        if (prm.trace && blockIdx.x == 0 && (tt) >= kLogT0 && (tt) < kLogT0 + kLogN)                          \
+            prm.trace[(size_t)gridDim.x * 32 + (ev) * kLogN + ((tt) - kLogT0)] = clock64();                   \
+    } while (0)
 #define TICK(cat)                                                                          \
     do {                                                                                   \
         if (prm.trace) {                                                                   \
