@@ -303,7 +303,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
         mbar_wait(bar(PB_MMA_DONE), 0, abort_flag + 1);
     } else if (warp == 2 && lane == 0) {
         // ------------------------------------------------------------ MMA issuer: variance product (own passes)
-        constexpr uint32_t IDESC_V = instr_desc_f16(NV2);
         const uint32_t k_lo0 = desc_addr(base + map.k) | ((2048u >> 4) << 16);
         const uint32_t w_lo0 = desc_addr(base + map.w) | (((NV2 * 16u) >> 4) << 16);
         const uint32_t k_empty_peer0 = map_to_cta(bar(PB_K_EMPTY), peer);
@@ -332,15 +331,20 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
                         if (++w_s == ws) { w_s = 0; w_ph ^= 1u; }
                         fence_proxy_async();   // the k* buffer was written through the generic proxy, possibly by the peer
                         tc_fence_after();
+                        // In the pass's diagonal block the rows of W above the chunk's columns are zero (W is lower
+                        // triangular): the MMAs start at the first row that can be non-zero and get narrower.
+                        const uint32_t skip = c > p * CPP2 ? (uint32_t)(c - p * CPP2) * KC : 0u;
+                        const uint32_t idesc_v = instr_desc_f16(NV2 - skip);
+                        const uint32_t vcol = tmem + skip;
                         const uint32_t aH = k_lo0 + ((b * 16384u) >> 4), aL = aH + (8192u >> 4);
-                        const uint32_t bH = w_lo0 + ((s * map.w_stage) >> 4), bL = bH + (((uint32_t)KC * NV2 * 2u) >> 4);
+                        const uint32_t bH = w_lo0 + ((s * map.w_stage) >> 4) + skip, bL = bH + (((uint32_t)KC * NV2 * 2u) >> 4);
 #pragma unroll
                         for (int combo = 0; combo < 3; ++combo) {
                             const uint32_t a0 = combo == 2 ? aL : aH, b0 = combo == 1 ? bL : bH;
 #pragma unroll
                             for (int jj = 0; jj < KC / 16; ++jj)
-                                tc_mma_f16(tmem, pack64(a0 + jj * (4096u >> 4), kDescHi),
-                                           pack64(b0 + jj * ((2u * NV2 * 16u) >> 4), kDescHi), IDESC_V,
+                                tc_mma_f16(vcol, pack64(a0 + jj * (4096u >> 4), kDescHi),
+                                           pack64(b0 + jj * ((2u * NV2 * 16u) >> 4), kDescHi), idesc_v,
                                            (c > 0 || combo > 0 || jj > 0) ? 1u : 0u);
                         }
                         tc_commit(bar(PB_W_EMPTY + s));
@@ -581,13 +585,20 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
                     TICK(5);
                     tc_fence_after();
 #pragma unroll 1
-                    for (int c0 = grp * 16; c0 < NV2; c0 += 16 * G2) {
-                        float v[16];
-                        tc_ld16(lane_addr + c0, v);
-                        float part = 0.f;
+                    for (int c0 = grp * 16; c0 < NV2; c0 += 32 * G2) {   // two column blocks per round trip to TMEM
+                        const int c1 = c0 + 16 * G2;
+                        float v[16], w[16];
+                        float part0 = 0.f, part1 = 0.f;
+                        tc_ld16_issue(lane_addr + c0, v);
+                        tc_ld16_issue(lane_addr + c1, w);
+                        tc_wait_ld32(v, w);
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) part = fmaf(v[i], v[i], part);
-                        q_acc += (double)part;
+                        for (int i = 0; i < 16; ++i) {
+                            part0 = fmaf(v[i], v[i], part0);
+                            part1 = fmaf(w[i], w[i], part1);
+                        }
+                        q_acc += (double)part0;
+                        q_acc += (double)part1;
                     }
                     tc_fence_before();
                     mbar_arrive(bar(PB_V_EMPTY));

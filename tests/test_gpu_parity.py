@@ -284,6 +284,31 @@ def test_workload_full_size_sampled_and_full_pool_topk(cfg, engine):
                    what=c.name)
 
 
+# ------------------------------------------------------------------------------------------ the paired tensor kernel
+@pytest.mark.parametrize("batch,n,d,m,k", [
+    (1, 300, 7, 700, 8),        # two passes: one super-pass, both CTAs busy
+    (2, 520, 33, 1000, 16),     # three passes: the last super-pass has a pass for one CTA only
+    (1, 1100, 64, 515, 8),      # five passes, ragged last tile
+    (1, 2050, 20, 260, 4),      # nine passes
+])
+def test_paired_tensor_kernel_every_element(monkeypatch, batch, n, d, m, k):
+    """R3_TC_PAIR=1 sends histories of two or more passes through the kernel that runs a tile on a cluster of
+    two CTAs; its results meet the same tolerances."""
+    monkeypatch.setenv("R3_TC_PAIR", "1")
+    g = rand_problem(900 + n, batch, n, d, m)
+    gp = fit_gpu(g, b.ENGINE_TENSOR)
+    compare_everything(g, gp, k, f"paired n{n} d{d} m{m}")
+    gp.close()
+
+
+def test_paired_tensor_kernel_on_the_largest_workload(monkeypatch):
+    monkeypatch.setenv("R3_TC_PAIR", "1")
+    c = w.get_config(5)
+    g, out = _run_full(c, b.ENGINE_TENSOR)
+    for _ in _sampled_check(c, g, out, 2048):
+        pass
+
+
 # ------------------------------------------------------------------------------------------ the library's size limits
 @pytest.mark.parametrize("engine", ENGINES)
 @pytest.mark.parametrize("d", [256, 128])
