@@ -1003,8 +1003,8 @@ r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, floa
     // R3_TC_TRACE=1 prints, for the first CTA, the cycles each role spent per wait / issue category
     prm.trace = nullptr;
     if (getenv("R3_TC_TRACE")) {
-        if (dev_malloc(&prm.trace, sizeof(long long) * (grid * 32 + 16 * 128)) != cudaSuccess) prm.trace = nullptr;
-        if (prm.trace) cudaMemset(prm.trace, 0, sizeof(long long) * (grid * 32 + 16 * 128));
+        if (dev_malloc(&prm.trace, sizeof(long long) * (grid * 32 + 32 * 128)) != cudaSuccess) prm.trace = nullptr;
+        if (prm.trace) cudaMemset(prm.trace, 0, sizeof(long long) * (grid * 32 + 32 * 128));
     }
     // The paired kernel (two CTAs of a cluster share a tile and the k* chunks) serves histories with at least
     // two passes; R3_TC_PAIR=0/1 overrides the choice.
@@ -1020,11 +1020,11 @@ r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, floa
     }
     prof_end(gp, stream);
     if (prm.trace) {
-        std::vector<long long> h((size_t)grid * 32 + 16 * 128);
+        std::vector<long long> h((size_t)grid * 32 + 32 * 128);
         cudaMemcpy(h.data(), prm.trace, sizeof(long long) * h.size(), cudaMemcpyDeviceToHost);
         for (int i = 0; i < 128; ++i) {
             fprintf(stderr, "ev %d:", i);
-            for (int e = 0; e < 10; ++e) fprintf(stderr, " %lld", h[(size_t)grid * 32 + e * 128 + i] - h[(size_t)grid * 32]);
+            for (int e = 0; e < 24; ++e) fprintf(stderr, " %lld", h[(size_t)grid * 32 + e * 128 + i] - h[(size_t)grid * 32 + 128 * 12]);
             fprintf(stderr, "\n");
         }
         dev_free(prm.trace);

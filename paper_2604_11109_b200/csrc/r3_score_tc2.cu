@@ -31,6 +31,18 @@ namespace r3 {
 
 namespace {
 
+#ifndef R3_TC_TRACE
+#define LOGEV2(ev, tt) do { } while (0)
+#else
+// event log of the first cluster: clock of event `ev` (0..7) of CTA `rank` for stream chunk tt in the window
+constexpr long long kLog2T0 = 576 + 300;
+#define LOGEV2(ev, tt)                                                                                        \
+    do {                                                                                                      \
+        if (prm.trace && blockIdx.x < 2 && (tt) >= kLog2T0 && (tt) < kLog2T0 + kLogN)                         \
+            prm.trace[(size_t)gridDim.x * 32 + (blockIdx.x * 12 + (ev)) * kLogN + ((tt) - kLog2T0)] = clock64(); \
+    } while (0)
+#endif
+
 constexpr int NV2 = 256;      // rows of W per pass
 constexpr int KD2 = 64;       // observations per distance product
 constexpr int SL2 = KD2 / KC; // chunks per distance product == Matern groups per CTA
@@ -310,12 +322,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
         int w_s = 0, k_s = 0;
         uint32_t w_ph = 0, k_ph = 0;
         bool ok = true;
+        long long tv = 0;
         for (long long tile = first_tile; ok && tile < prm.total_tiles; tile += tile_step) {
             for (int j = 0; ok && j < NSP; ++j) {
                 const int p = 2 * j + (int)rank;
                 const int mine = p < P ? (p + 1) * CPP2 : 0;   // chunks of this super-pass that my pass uses
                 const int nchunk = superpass_chunks(j, P);
-                for (int c = 0; ok && c < nchunk; ++c) {
+                for (int c = 0; ok && c < nchunk; ++c, ++tv) {
                     const int b = k_s;
                     TICK(7);
                     if (c < mine) {
@@ -324,13 +337,17 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
                             if (!(ok = mbar_wait(bar(PB_V_EMPTY), v_ph ^ 1u, abort_flag))) break;
                         }
                         TICK(3);
-                        if (!(ok = mbar_wait_cluster(bar(PB_K_FULL + b), k_ph, abort_flag))) break;
+                        if (!(ok = mbar_wait(bar(PB_K_FULL + b), k_ph, abort_flag))) break;
                         TICK(4);
+                        LOGEV2(0, tv);
                         if (!(ok = mbar_wait(bar(PB_W_FULL + s), w_ph, abort_flag))) break;
                         TICK(5);
+                        LOGEV2(1, tv);
                         if (++w_s == ws) { w_s = 0; w_ph ^= 1u; }
-                        fence_proxy_async();   // the k* buffer was written through the generic proxy, possibly by the peer
+                        // (the writers of a k* buffer fence their stores towards the async proxy before they arrive,
+                        // and the peer's copy arrives through the async proxy: no proxy fence on this side)
                         tc_fence_after();
+                        LOGEV2(7, tv);
                         // In the pass's diagonal block the rows of W above the chunk's columns are zero (W is lower
                         // triangular): the MMAs start at the first row that can be non-zero and get narrower.
                         const uint32_t skip = c > p * CPP2 ? (uint32_t)(c - p * CPP2) * KC : 0u;
@@ -347,16 +364,20 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
                                            pack64(b0 + jj * ((2u * NV2 * 16u) >> 4), kDescHi), idesc_v,
                                            (c > 0 || combo > 0 || jj > 0) ? 1u : 0u);
                         }
+                        LOGEV2(8, tv);
                         tc_commit(bar(PB_W_EMPTY + s));
+                        LOGEV2(9, tv);
                         tc_commit_pair(bar(PB_K_EMPTY + b));
+                        LOGEV2(10, tv);
                         if (c == mine - 1) {
                             tc_commit(bar(PB_V_FULL));
                             v_ph ^= 1u;
                         }
                         TICK(6);
+                        LOGEV2(2, tv);
                     } else {
                         // my pass does not use this chunk: release the buffer on both CTAs once it has been filled
-                        if (!(ok = mbar_wait_cluster(bar(PB_K_FULL + b), k_ph, abort_flag))) break;
+                        if (!(ok = mbar_wait(bar(PB_K_FULL + b), k_ph, abort_flag))) break;
                         mbar_arrive(bar(PB_K_EMPTY + b));
                         mbar_arrive_cluster(k_empty_peer0 + (uint32_t)b * 8u);
                         TICK(0);
@@ -369,6 +390,18 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
         mbar_wait(bar(PB_MMA_DONE + 1), 0, abort_flag + 1);
         if (prm.trace)
             for (int i = 0; i < 8; ++i) prm.trace[((size_t)blockIdx.x * 4 + 0) * 8 + i] = tacc[i];
+#ifdef R3_TC_TRACE
+    } else if (warp == 3 && lane == 0) {
+        // observer (trace builds only): when each k* buffer became full in this CTA
+        long long tv = 0;
+        bool ok = true;
+        for (long long tile = first_tile; ok && tile < prm.total_tiles; tile += tile_step)
+            for (int j = 0; ok && j < NSP; ++j)
+                for (int c = 0; ok && c < superpass_chunks(j, P); ++c, ++tv) {
+                    ok = mbar_wait(bar(PB_K_FULL + (int)(tv % NB)), (uint32_t)((tv / NB) & 1), abort_flag);
+                    LOGEV2(11, tv);
+                }
+#endif
     } else if (warp >= 4) {
         // ------------------------------------------------------------ Matern / epilogue warp groups
         const int grp = (warp - 4) >> 2;         // 0..G2-1: which chunk of each own product
@@ -465,6 +498,38 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
             const float* xn_g = prm.xnorm + (size_t)g * prm.NP;
             const float* al_g = prm.alpha + (size_t)g * prm.NP;
             double mu_acc = 0.0, a2_acc = 0.0, s2_acc = 0.0, q_acc = 0.0;
+            // End of a super-pass: q += sum_i V^2 over this group's share of my pass's columns.  It runs only
+            // after the group has generated its first chunk of the NEXT super-pass (the ring has one slot per
+            // group of the pair), so that the variance MMAs find k* waiting when the accumulator is free again.
+            bool epilogue_due = false;
+            auto pass_epilogue = [&]() {
+                TICK(7);
+                ok = mbar_wait(bar(PB_V_FULL), v_ph, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) return;
+                TICK(5);
+                tc_fence_after();
+#pragma unroll 1
+                for (int c0 = grp * 16; c0 < NV2; c0 += 32 * G2) {   // two column blocks per round trip to TMEM
+                    const int c1 = c0 + 16 * G2;
+                    float v[16], w[16];
+                    float part0 = 0.f, part1 = 0.f;
+                    tc_ld16_issue(lane_addr + c0, v);
+                    tc_ld16_issue(lane_addr + c1, w);
+                    tc_wait_ld32(v, w);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        part0 = fmaf(v[i], v[i], part0);
+                        part1 = fmaf(w[i], w[i], part1);
+                    }
+                    q_acc += (double)part0;
+                    q_acc += (double)part1;
+                }
+                tc_fence_before();
+                mbar_arrive(bar(PB_V_EMPTY));
+                v_ph ^= 1u;
+                TICK(6);
+            };
             for (int j = 0; ok && j < NSP; ++j) {
                 const int nchunk = superpass_chunks(j, P);
                 const int nprod = nchunk / SL2;
@@ -480,6 +545,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     TICK(0);
+                    if (q4 == 0 && lane == 0) LOGEV2(3, t);
                     ++own;
                     tc_fence_after();
                     const bool fresh = c >= 2 * j * CPP2;   // first super-pass that generates this chunk
@@ -547,10 +613,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
                     }
                     // both CTAs must have finished with the previous chunk in this ring position
                     TICK(2);
+                    if (q4 == 0 && lane == 0) LOGEV2(4, t);
                     ok = mbar_wait_cluster(bar(PB_K_EMPTY + b), k_par ^ 1u, abort_flag);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     TICK(3);
+                    if (q4 == 0 && lane == 0) LOGEV2(5, t);
+                    // the peer's barrier learns of the 16 KB to come now: the remote arrive takes hundreds of cycles,
+                    // which pass while this group stores the chunk
+                    if (q4 == 1 && lane == 0) mbar_arrive_expect_tx_cluster(k_full_peer0 + (uint32_t)b * 8u, 16384u);
 #pragma unroll
                     for (int h = 0; h < KC / 16; ++h) {
 #pragma unroll
@@ -564,48 +635,30 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
                     if (!ok) break;
                     // The chunk is complete in this CTA's buffer: publish it here, and send a copy to the
                     // same ring position of the peer with one bulk copy that completes the peer's barrier.
+                    if (q4 == 0 && lane == 0) LOGEV2(7, t);
                     fence_proxy_async();
+                    if (q4 == 0 && lane == 0) LOGEV2(8, t);
                     asm volatile("bar.sync %0, 128;" ::"r"(1 + grp) : "memory");
                     if (q4 == 0 && lane == 0) {
+                        LOGEV2(9, t);
                         mbar_arrive(bar(PB_K_FULL + b));
                         const uint32_t peer_bar = k_full_peer0 + (uint32_t)b * 8u;
-                        mbar_arrive_expect_tx_cluster(peer_bar, 16384u);
+                        LOGEV2(10, t);
                         bulk_s2peer(kbuf_peer0 + b * 16384u, base + map.k + b * 16384u, 16384u, peer_bar);
+                        LOGEV2(6, t);
                     }
                     TICK(4);
+                    if (epilogue_due) {   // the previous super-pass's accumulator, now that the next k* is on its way
+                        epilogue_due = false;
+                        pass_epilogue();
+                        if (!ok) break;
+                    }
                 }
                 if (!ok) break;
                 tg += nchunk;
-                // ---- end of the super-pass: q += sum_i V^2 over this group's share of my pass's columns
-                if (2 * j + (int)rank < P) {
-                    TICK(7);
-                    ok = mbar_wait(bar(PB_V_FULL), v_ph, abort_flag);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    TICK(5);
-                    tc_fence_after();
-#pragma unroll 1
-                    for (int c0 = grp * 16; c0 < NV2; c0 += 32 * G2) {   // two column blocks per round trip to TMEM
-                        const int c1 = c0 + 16 * G2;
-                        float v[16], w[16];
-                        float part0 = 0.f, part1 = 0.f;
-                        tc_ld16_issue(lane_addr + c0, v);
-                        tc_ld16_issue(lane_addr + c1, w);
-                        tc_wait_ld32(v, w);
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            part0 = fmaf(v[i], v[i], part0);
-                            part1 = fmaf(w[i], w[i], part1);
-                        }
-                        q_acc += (double)part0;
-                        q_acc += (double)part1;
-                    }
-                    tc_fence_before();
-                    mbar_arrive(bar(PB_V_EMPTY));
-                    v_ph ^= 1u;
-                    TICK(6);
-                }
+                epilogue_due = 2 * j + (int)rank < P;
             }
+            if (ok && epilogue_due) pass_epilogue();
             if (!ok) break;
             // ---- combine: groups within the CTA, then CTA 1 -> CTA 0, which finishes the candidate
             double* mine = red + ((size_t)grp * TILE_M + row) * 4;
