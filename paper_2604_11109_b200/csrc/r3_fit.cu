@@ -152,31 +152,40 @@ __global__ void __launch_bounds__(1024) potrf_diag_kernel(double* __restrict__ A
     Dinv[((size_t)g * (npad / NB) + j0 / NB) * NB * NB + ty * NB + tx] = m[ty][tx] * rk[ty];
 }
 
-// Panel below the diagonal block: L_panel = A_panel * inv(L_jj)^T, 64 rows per block.
-__global__ void __launch_bounds__(256) panel_kernel(double* __restrict__ A, int npad, int j0,
-                                                    const double* __restrict__ Dinv)
+// Panel below the diagonal block: L_panel L_jj^T = A_panel by forward substitution, one row per thread.
+// (Multiplying by the explicit inverse of L_jj instead loses the small entries of an ill-conditioned
+// factor: its error is relative to |A_panel| |L_jj^-1|, not to the result, and the pivots that follow
+// inherit it -- on noise-free smooth data the log-determinant came out wrong in the third digit.)
+constexpr int kPanelRows = 64;
+__global__ void __launch_bounds__(kPanelRows) panel_kernel(double* __restrict__ A, int npad, int j0)
 {
     const int g = blockIdx.y;
-    const int r0 = j0 + NB + blockIdx.x * 64;
+    const int r = j0 + NB + blockIdx.x * kPanelRows + threadIdx.x;
     double* Ag = A + (size_t)g * npad * npad;
-    const double* Dg = Dinv + ((size_t)g * (npad / NB) + j0 / NB) * NB * NB;
-    __shared__ double sd[NB][NB + 1];
-    __shared__ double sa[64][NB + 1];
-    const int t = threadIdx.x;
-    for (int e = t; e < NB * NB; e += 256) sd[e / NB][e % NB] = Dg[e];
-    for (int e = t; e < 64 * NB; e += 256) {
-        int r = e / NB, c = e % NB;
-        sa[r][c] = (r0 + r < npad) ? Ag[(size_t)(r0 + r) * npad + j0 + c] : 0.0;
-    }
+    __shared__ double l[NB][NB + 1];    // L_jj
+    __shared__ double rdiag[NB];
+    for (int e = threadIdx.x; e < NB * NB; e += kPanelRows) l[e / NB][e % NB] = Ag[(size_t)(j0 + e / NB) * npad + j0 + e % NB];
     __syncthreads();
-    const int r = t / 4, cb = (t % 4) * 8;
-    if (r0 + r < npad) {
-        for (int c = cb; c < cb + 8; ++c) {
-            double s = 0.0;
-            for (int k = 0; k <= c; ++k) s += sa[r][k] * sd[c][k];
-            Ag[(size_t)(r0 + r) * npad + j0 + c] = s;
+    if (threadIdx.x < NB) rdiag[threadIdx.x] = 1.0 / l[threadIdx.x][threadIdx.x];
+    __syncthreads();
+    if (r >= npad) return;
+    double* row = Ag + (size_t)r * npad + j0;
+    double x[NB];
+#pragma unroll
+    for (int c = 0; c < NB; ++c) x[c] = row[c];
+#pragma unroll
+    for (int c = 0; c < NB; ++c) {
+        double s0 = 0.0, s1 = 0.0;
+#pragma unroll
+        for (int k = 0; k + 1 < c; k += 2) {
+            s0 = fma(x[k], l[c][k], s0);
+            s1 = fma(x[k + 1], l[c][k + 1], s1);
         }
+        if (c & 1) s0 = fma(x[c - 1], l[c][c - 1], s0);
+        x[c] = (x[c] - (s0 + s1)) * rdiag[c];
     }
+#pragma unroll
+    for (int c = 0; c < NB; ++c) row[c] = x[c];
 }
 
 // Trailing update: A[i][j] -= sum_k A[i][k] A[j][k] over the kw finished columns from k0 (kw a multiple of
@@ -480,7 +489,7 @@ r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream)
             const int rows = npad - j0 - NB;
             if (rows <= 0) continue;
             const int tiles = (rows + 63) / 64;
-            LAUNCH_OR_FAIL(panel_kernel, dim3(tiles, B), 256, gp->L64, npad, j0, Dinv);
+            LAUNCH_OR_FAIL(panel_kernel, dim3((rows + kPanelRows - 1) / kPanelRows, B), kPanelRows, gp->L64, npad, j0);
             const int inner = panel_end - j0 - NB;   // columns of this panel still to be factored
             if (inner > 0)
                 LAUNCH_OR_FAIL(syrk_kernel, dim3((inner + 63) / 64, tiles, B), 256, gp->L64, npad, j0, NB, j0 + NB,
