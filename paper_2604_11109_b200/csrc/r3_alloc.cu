@@ -126,6 +126,34 @@ void trim_cache()
     for (void* b : blocks) cudaFree(b);
 }
 
+// Pinned host words for status read-backs: cudaMallocHost costs far more than the kernels of a small fit,
+// so released words are kept for the life of the process.
+namespace {
+std::vector<int*> g_pinned_words;
+}
+
+int* pinned_word_acquire()
+{
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (!g_pinned_words.empty()) {
+            int* w = g_pinned_words.back();
+            g_pinned_words.pop_back();
+            return w;
+        }
+    }
+    int* w = nullptr;
+    if (cudaMallocHost(&w, sizeof(int)) != cudaSuccess) return nullptr;
+    return w;
+}
+
+void pinned_word_release(int* w)
+{
+    if (!w) return;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    g_pinned_words.push_back(w);
+}
+
 size_t cached_bytes()
 {
     int dev = 0;

@@ -62,6 +62,8 @@ inline cudaError_t dev_malloc(T** p, size_t bytes)
 }
 void dev_free(void* p);
 void trim_cache();
+int* pinned_word_acquire();          // a pinned host int from a process-wide pool (nullptr on failure)
+void pinned_word_release(int* w);
 size_t cached_bytes();
 
 inline int round_up(int a, int b) { return (a + b - 1) / b * b; }

@@ -28,8 +28,10 @@ struct r3_tpe {
     int* counts_d = nullptr;   // [d][2]: components of each set after merging equal ones
     // a model small enough for shared memory is also kept packed: set (j, s) at [offs[2j + s], offs[2j + s + 1])
     int total = 0;             // components kept over all dimensions and sets
+    bool resident = false;     // the packed model is in use
     float4* packed_d = nullptr;
     int* offs_d = nullptr;     // [2d + 1]
+    char* arena_d = nullptr;   // the one allocation all device pointers of the handle point into
     float* table_d = nullptr;  // [d][64] ln P_good - ln P_bad per level
     int* status_d = nullptr;   // status bits
     int* status_h = nullptr;   // pinned mirror
@@ -559,15 +561,8 @@ size_t resident_bytes(int total, int d) { return sizeof(float4) * (size_t)total 
 void tpe_destroy(r3_tpe* t)
 {
     if (!t) return;
-    cudaFree(t->levels_d);
-    cudaFree(t->order_d);
-    cudaFree(t->comps_d);
-    cudaFree(t->counts_d);
-    cudaFree(t->packed_d);
-    cudaFree(t->offs_d);
-    cudaFree(t->table_d);
-    cudaFree(t->status_d);
-    if (t->status_h) cudaFreeHost(t->status_h);
+    dev_free(t->arena_d);
+    pinned_word_release(t->status_h);
     delete t;
 }
 
@@ -575,15 +570,33 @@ r3_status_t tpe_fit_impl(r3_tpe* t, const float* X, const float* y, cudaStream_t
 {
     const int n = t->n, d = t->d;
     R3_CUDA_TRY(cudaGetDevice(&t->device));
-    R3_CUDA_TRY(cudaMalloc(&t->levels_d, sizeof(int) * d));
-    R3_CUDA_TRY(cudaMalloc(&t->order_d, sizeof(int) * n));
-    R3_CUDA_TRY(cudaMalloc(&t->comps_d, sizeof(float4) * (size_t)d * (n + 2)));
-    R3_CUDA_TRY(cudaMalloc(&t->counts_d, sizeof(int) * 2 * (size_t)d));
-    R3_CUDA_TRY(cudaMalloc(&t->table_d, sizeof(float) * (size_t)d * kTpeMaxLevels));
-    R3_CUDA_TRY(cudaMalloc(&t->status_d, sizeof(int)));
-    R3_CUDA_TRY(cudaMallocHost(&t->status_h, sizeof(int)));
+    // one block of device memory for the whole model (the library's cache hands it back to the next fit)
+    auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
+    const size_t b_comps = up(sizeof(float4) * (size_t)d * (n + 2)), b_packed = up(kResidentBytes),
+                 b_table = up(sizeof(float) * (size_t)d * kTpeMaxLevels), b_order = up(sizeof(int) * n),
+                 b_levels = up(sizeof(int) * d), b_counts = up(sizeof(int) * 2 * (size_t)d),
+                 b_offs = up(sizeof(int) * (2 * (size_t)d + 1)), b_status = 256;
+    char* base = nullptr;
+    if (dev_malloc(&base, b_comps + b_packed + b_table + b_order + b_levels + b_counts + b_offs + b_status) != cudaSuccess) {
+        cudaGetLastError();
+        set_error("r3_tpe_fit: out of device memory");
+        return R3_ERR_ALLOC;
+    }
+    t->arena_d = base;
+    t->comps_d = reinterpret_cast<float4*>(base); base += b_comps;
+    t->packed_d = reinterpret_cast<float4*>(base); base += b_packed;
+    t->table_d = reinterpret_cast<float*>(base); base += b_table;
+    t->order_d = reinterpret_cast<int*>(base); base += b_order;
+    t->levels_d = reinterpret_cast<int*>(base); base += b_levels;
+    t->counts_d = reinterpret_cast<int*>(base); base += b_counts;
+    t->offs_d = reinterpret_cast<int*>(base); base += b_offs;
+    t->status_d = reinterpret_cast<int*>(base);
+    t->status_h = pinned_word_acquire();
+    if (!t->status_h) {
+        set_error("r3_tpe_fit: no pinned host memory");
+        return R3_ERR_ALLOC;
+    }
     R3_CUDA_TRY(cudaMemcpyAsync(t->levels_d, t->levels.data(), sizeof(int) * d, cudaMemcpyHostToDevice, stream));
-    R3_CUDA_TRY(cudaMemsetAsync(t->comps_d, 0, sizeof(float4) * (size_t)d * (n + 2), stream));
     R3_CUDA_TRY(cudaMemsetAsync(t->table_d, 0, sizeof(float) * (size_t)d * kTpeMaxLevels, stream));
     R3_CUDA_TRY(cudaMemsetAsync(t->status_d, 0, sizeof(int), stream));
     R3_LAUNCH(tpe_order_kernel, 1, kSortThreads, 0, stream, y, n, t->order_d, t->status_d);
@@ -605,9 +618,8 @@ r3_status_t tpe_fit_impl(r3_tpe* t, const float* X, const float* y, cudaStream_t
     R3_CUDA_TRY(cudaMemcpy(counts.data(), t->counts_d, sizeof(int) * 2 * (size_t)d, cudaMemcpyDeviceToHost));
     for (int i = 0; i < 2 * d; ++i) offs[i + 1] = offs[i] + counts[i];
     t->total = offs[2 * d];
-    if (t->total > 0 && resident_bytes(t->total, d) <= kResidentBytes) {
-        R3_CUDA_TRY(cudaMalloc(&t->packed_d, sizeof(float4) * (size_t)t->total));
-        R3_CUDA_TRY(cudaMalloc(&t->offs_d, sizeof(int) * offs.size()));
+    t->resident = t->total > 0 && resident_bytes(t->total, d) <= kResidentBytes;
+    if (t->resident) {
         R3_CUDA_TRY(cudaMemcpyAsync(t->offs_d, offs.data(), sizeof(int) * offs.size(), cudaMemcpyHostToDevice, stream));
         R3_LAUNCH(tpe_pack_kernel, 2 * d, 256, 0, stream, t->comps_d, n, t->n_good, t->offs_d, t->packed_d);
         R3_CUDA_TRY(cudaStreamSynchronize(stream));   // `offs` leaves scope
@@ -701,7 +713,7 @@ r3_status_t r3_tpe_score(r3_tpe_t* tpe, const float* Xcand, long long m, float* 
 #undef R3_TPE_TABLE
         return R3_OK;
     }
-    if (tpe->packed_d) {
+    if (tpe->resident) {
         // the whole model in shared memory.  Sixteen blocks per SM's worth of grid (several waves of short
         // blocks) measured up to 8 % faster than one resident wave walking the tiles: the model is a small
         // read from L2 and the finer grain balances the SMs better.
