@@ -109,24 +109,25 @@ __global__ void __launch_bounds__(kSortThreads) tpe_order_kernel(const float* __
     for (int i = threadIdx.x; i < n; i += blockDim.x) order[i] = (int)(keys[i] & 0xFFFFFFFFull);
 }
 
-// (T2), (T3): one block per dimension, both sets in turn.
+// (T2), (T3): one block per (dimension, set).  The log-probabilities (categorical) or log-densities (grid) of a
+// set go to lnp[j][set][v]; tpe_table_kernel subtracts the two sets afterwards.
 __global__ void __launch_bounds__(kSortThreads) tpe_mixture_kernel(const float* __restrict__ X,
                                                                    const int* __restrict__ order, int n, int d,
                                                                    int n_good, const int* __restrict__ levels,
                                                                    double prior_weight, float4* __restrict__ comps,
-                                                                   int* __restrict__ n_comps, float* __restrict__ table,
+                                                                   int* __restrict__ n_comps, double* __restrict__ lnp_out,
                                                                    int* __restrict__ status)
 {
     extern __shared__ unsigned long long keys[];   // pow2 >= n + 1 keys, then (grid dimensions) 2 (n + 1) doubles
     __shared__ int counts[kTpeMaxLevels];
-    __shared__ double lnp_good[kTpeMaxLevels];
     __shared__ double wsum_s[32];
-    const int j = blockIdx.x;
+    const int j = blockIdx.x >> 1;
     const int code = levels[j];
     const int C = code > 0 ? code : 0;      // categorical levels
     const int G = code < 0 ? -code : 0;     // grid values of an ordinal dimension
     bool bad = false;
-    for (int set = 0; set < 2; ++set) {
+    double* lnp_set = lnp_out + ((size_t)j * 2 + (blockIdx.x & 1)) * kTpeMaxLevels;
+    for (int set = blockIdx.x & 1; set == (int)(blockIdx.x & 1); set += 2) {
         const int s = set == 0 ? n_good : n - n_good;
         const int first = set == 0 ? 0 : n_good;            // position in `order`
         float4* out = comps + (size_t)j * (n + 2) + (set == 0 ? 0 : n_good + 1);
@@ -143,11 +144,7 @@ __global__ void __launch_bounds__(kSortThreads) tpe_mixture_kernel(const float* 
             }
             __syncthreads();
             for (int v = threadIdx.x; v < C; v += blockDim.x) {
-                const double lnp = log(((double)counts[v] + prior_weight / C) / ((double)s + prior_weight));
-                if (set == 0)
-                    lnp_good[v] = lnp;
-                else
-                    table[(size_t)j * kTpeMaxLevels + v] = (float)(lnp_good[v] - lnp);
+                lnp_set[v] = log(((double)counts[v] + prior_weight / C) / ((double)s + prior_weight));
             }
             if (threadIdx.x == 0) n_comps[2 * j + set] = 0;
             __syncthreads();
@@ -246,17 +243,24 @@ __global__ void __launch_bounds__(kSortThreads) tpe_mixture_kernel(const float* 
                 if (threadIdx.x == 0) {
                     double tot = 0.0;
                     for (int w = 0; w < (int)blockDim.x / 32; ++w) tot += wsum_s[w];
-                    const double lnd = log(tot);
-                    if (set == 0)
-                        lnp_good[v] = lnd;
-                    else
-                        table[(size_t)j * kTpeMaxLevels + v] = (float)(lnp_good[v] - lnd);
+                    lnp_set[v] = log(tot);
                 }
                 __syncthreads();
             }
         }
     }
     if (bad) atomicOr(status, DEV_NONFINITE);
+}
+
+// (T3), (T3g): table[j][v] = ln l_j(v) - ln g_j(v) for the tabulated dimensions, zero elsewhere
+__global__ void tpe_table_kernel(const int* __restrict__ levels, const double* __restrict__ lnp, int d,
+                                 float* __restrict__ table)
+{
+    const int j = blockIdx.x, v = threadIdx.x;
+    const int code = levels[j];
+    const int cnt = code < 0 ? -code : code;
+    const double* l = lnp + (size_t)j * 2 * kTpeMaxLevels;
+    table[(size_t)j * kTpeMaxLevels + v] = v < cnt ? (float)(l[v] - l[kTpeMaxLevels + v]) : 0.f;
 }
 
 __device__ __forceinline__ float ex2_fast(float x)
@@ -575,9 +579,11 @@ r3_status_t tpe_fit_impl(r3_tpe* t, const float* X, const float* y, cudaStream_t
     const size_t b_comps = up(sizeof(float4) * (size_t)d * (n + 2)), b_packed = up(kResidentBytes),
                  b_table = up(sizeof(float) * (size_t)d * kTpeMaxLevels), b_order = up(sizeof(int) * n),
                  b_levels = up(sizeof(int) * d), b_counts = up(sizeof(int) * 2 * (size_t)d),
-                 b_offs = up(sizeof(int) * (2 * (size_t)d + 1)), b_status = 256;
+                 b_offs = up(sizeof(int) * (2 * (size_t)d + 1)), b_status = 256,
+                 b_lnp = up(sizeof(double) * 2 * (size_t)d * kTpeMaxLevels);
     char* base = nullptr;
-    if (dev_malloc(&base, b_comps + b_packed + b_table + b_order + b_levels + b_counts + b_offs + b_status) != cudaSuccess) {
+    if (dev_malloc(&base, b_comps + b_packed + b_table + b_order + b_levels + b_counts + b_offs + b_status + b_lnp) !=
+        cudaSuccess) {
         cudaGetLastError();
         set_error("r3_tpe_fit: out of device memory");
         return R3_ERR_ALLOC;
@@ -590,14 +596,14 @@ r3_status_t tpe_fit_impl(r3_tpe* t, const float* X, const float* y, cudaStream_t
     t->levels_d = reinterpret_cast<int*>(base); base += b_levels;
     t->counts_d = reinterpret_cast<int*>(base); base += b_counts;
     t->offs_d = reinterpret_cast<int*>(base); base += b_offs;
-    t->status_d = reinterpret_cast<int*>(base);
+    t->status_d = reinterpret_cast<int*>(base); base += b_status;
+    double* lnp_d = reinterpret_cast<double*>(base);   // scratch of the fit
     t->status_h = pinned_word_acquire();
     if (!t->status_h) {
         set_error("r3_tpe_fit: no pinned host memory");
         return R3_ERR_ALLOC;
     }
     R3_CUDA_TRY(cudaMemcpyAsync(t->levels_d, t->levels.data(), sizeof(int) * d, cudaMemcpyHostToDevice, stream));
-    R3_CUDA_TRY(cudaMemsetAsync(t->table_d, 0, sizeof(float) * (size_t)d * kTpeMaxLevels, stream));
     R3_CUDA_TRY(cudaMemsetAsync(t->status_d, 0, sizeof(int), stream));
     R3_LAUNCH(tpe_order_kernel, 1, kSortThreads, 0, stream, y, n, t->order_d, t->status_d);
     int count = 1;
@@ -605,8 +611,9 @@ r3_status_t tpe_fit_impl(r3_tpe* t, const float* X, const float* y, cudaStream_t
     const size_t smem = sizeof(unsigned long long) * (size_t)count + sizeof(double) * 2 * ((size_t)n + 2);
     if (smem > 48 * 1024)
         R3_CUDA_TRY(cudaFuncSetAttribute(tpe_mixture_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    R3_LAUNCH(tpe_mixture_kernel, d, kSortThreads, smem, stream, X, t->order_d, n, d, t->n_good, t->levels_d,
-              (double)t->prior_weight, t->comps_d, t->counts_d, t->table_d, t->status_d);
+    R3_LAUNCH(tpe_mixture_kernel, 2 * d, kSortThreads, smem, stream, X, t->order_d, n, d, t->n_good, t->levels_d,
+              (double)t->prior_weight, t->comps_d, t->counts_d, lnp_d, t->status_d);
+    R3_LAUNCH(tpe_table_kernel, d, kTpeMaxLevels, 0, stream, t->levels_d, lnp_d, d, t->table_d);
     R3_CUDA_TRY(cudaMemcpyAsync(t->status_h, t->status_d, sizeof(int), cudaMemcpyDeviceToHost, stream));
     R3_CUDA_TRY(cudaStreamSynchronize(stream));
     if (*t->status_h & DEV_NONFINITE) {
