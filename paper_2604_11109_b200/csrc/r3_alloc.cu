@@ -126,8 +126,8 @@ void trim_cache()
     for (void* b : blocks) cudaFree(b);
 }
 
-// Pinned host words for status read-backs: cudaMallocHost costs far more than the kernels of a small fit,
-// so released words are kept for the life of the process.
+// Pinned host blocks of kPinnedInts ints for status read-backs: cudaMallocHost costs far more than the kernels
+// of a small fit, so released blocks are kept for the life of the process.
 namespace {
 std::vector<int*> g_pinned_words;
 }
@@ -143,7 +143,7 @@ int* pinned_word_acquire()
         }
     }
     int* w = nullptr;
-    if (cudaMallocHost(&w, sizeof(int)) != cudaSuccess) return nullptr;
+    if (cudaMallocHost(&w, sizeof(int) * kPinnedInts) != cudaSuccess) return nullptr;
     return w;
 }
 

@@ -146,8 +146,7 @@ void r3_gp_free(r3_gp_t* gp)
     dev_free(gp->alpha64);
     dev_free(gp->alpha32);
     dev_free(gp->status_d);
-    if (gp->status_h) cudaFreeHost(gp->status_h);
-    if (gp->rescued_h) cudaFreeHost(gp->rescued_h);
+    pinned_word_release(gp->status_h);   // rescued_h lives in the same block
     for (cudaEvent_t e : gp->events) cudaEventDestroy(e);
     dev_free(gp->ws);
     delete gp;
@@ -226,8 +225,12 @@ r3_status_t r3_gp_fit(const float* X, const float* y, const float* lengthscales,
     TRY_BAIL(dev_malloc(&gp->alpha64, sizeof(double) * batch * gp->npad));
     TRY_BAIL(dev_malloc(&gp->alpha32, sizeof(float) * batch * gp->npad));
     TRY_BAIL(dev_malloc(&gp->status_d, 2 * sizeof(int)));
-    TRY_BAIL(cudaMallocHost(&gp->status_h, 2 * sizeof(int)));
-    TRY_BAIL(cudaMallocHost(&gp->rescued_h, 64 * sizeof(int)));
+    gp->status_h = pinned_word_acquire();   // [2] status words, then [64] rescue counters
+    if (!gp->status_h) {
+        set_error("r3_gp_fit: no pinned host memory");
+        return bail(R3_ERR_ALLOC);
+    }
+    gp->rescued_h = gp->status_h + 2;
     for (int i = 0; i < 64; ++i) gp->rescued_h[i] = 0;
     gp->status_h[0] = 0;
     gp->status_h[1] = INT_MAX;

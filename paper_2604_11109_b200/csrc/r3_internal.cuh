@@ -62,7 +62,8 @@ inline cudaError_t dev_malloc(T** p, size_t bytes)
 }
 void dev_free(void* p);
 void trim_cache();
-int* pinned_word_acquire();          // a pinned host int from a process-wide pool (nullptr on failure)
+constexpr int kPinnedInts = 128;
+int* pinned_word_acquire();          // kPinnedInts pinned host ints from a process-wide pool (nullptr on failure)
 void pinned_word_release(int* w);
 size_t cached_bytes();
 
