@@ -102,74 +102,95 @@ __global__ void gram_kernel(const float* __restrict__ X, const float* __restrict
 }
 
 // ------------------------------------------------------------------------------------ Cholesky
-// Factor the 32x32 diagonal block at j0 in shared memory, write it back (upper part zeroed) and
-// store its inverse in Dinv[g][j0/32].
+// One step of the factorisation for the 32 columns at j0, in ONE launch: every block factors the 32x32
+// diagonal block itself (redundantly -- it is the latency of 32 dependent columns either way, and a second
+// launch waiting for a first costs as much again) and then solves its share of the panel below it, one row
+// per thread.  Block 0 also stores the factored diagonal block (to Ldiag, copied into place after the
+// factorisation: the other blocks of this launch may still be reading the unfactored block) and its inverse
+// (to Dinv[g][j0/32], for the inverse factor).
 //
-// One barrier per column.  At step k every thread forms r = 1/sqrt(a_kk) itself and scales what it reads of
-// column k by it, so that nothing has to be written (and waited for) between the pivot and the update; the
-// column stays unscaled in shared memory until the end.  The inverse comes from the same sweep: with
-// L = L_1 ... L_32 (L_k the identity with column k of L), L^-1 = L_32^-1 ... L_1^-1, and applying L_k^-1 to
-// the running product M is the same rank-one update on the columns <= k that the factorisation does on the
-// columns > k -- the threads of the finished columns do it.  Row k of M, like column k of A, is scaled by r
-// only at the end.
-__global__ void __launch_bounds__(1024) potrf_diag_kernel(double* __restrict__ A, int npad, int j0,
-                                                          double* __restrict__ Dinv, int* status)
+// Diagonal block: one barrier per column.  At step k every thread forms r = 1/sqrt(a_kk) itself and scales
+// what it reads of column k by it, so that nothing has to be written (and waited for) between the pivot and
+// the update; the column stays unscaled in shared memory until the end.  The inverse comes from the same
+// sweep: with L = L_1 ... L_32 (L_k the identity with column k of L), L^-1 = L_32^-1 ... L_1^-1, and
+// applying L_k^-1 to the running product M is the same rank-one update on the columns <= k that the
+// factorisation does on the columns > k -- the threads of the finished columns do it.  Row k of M, like
+// column k of A, is scaled by r only at the end.
+//
+// Panel: L_panel L_jj^T = A_panel by forward substitution.  (Multiplying by the explicit inverse of L_jj
+// instead loses the small entries of an ill-conditioned factor: its error is relative to
+// |A_panel| |L_jj^-1|, not to the result, and the pivots that follow inherit it -- on noise-free smooth data
+// the log-determinant came out wrong in the third digit.)
+constexpr int kPanelThreads = 256;   // 32 x 8: four rows of the diagonal block per thread, one panel row per thread
+__global__ void __launch_bounds__(kPanelThreads) potrf_panel_kernel(double* __restrict__ A, int npad, int j0,
+                                                                    double* __restrict__ Dinv,
+                                                                    double* __restrict__ Ldiag, int* status)
 {
-    const int g = blockIdx.x;
-    const int tx = threadIdx.x, ty = threadIdx.y;
-    double* Ag = A + (size_t)g * npad * npad + (size_t)j0 * npad + j0;
+    const int g = blockIdx.y;
+    const int tx = threadIdx.x, tq = threadIdx.y;   // rows tq, tq + 8, tq + 16, tq + 24 of the diagonal block
+    double* Agp = A + (size_t)g * npad * npad;
+    const double* Ag = Agp + (size_t)j0 * npad + j0;
     __shared__ double a[NB][NB + 1];
     __shared__ double m[NB][NB + 1];
     __shared__ double rk[NB], lkk[NB];
-    a[ty][tx] = Ag[(size_t)ty * npad + tx];
-    m[ty][tx] = (tx == ty) ? 1.0 : 0.0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int ty = tq + 8 * i;
+        a[ty][tx] = Ag[(size_t)ty * npad + tx];
+        m[ty][tx] = (tx == ty) ? 1.0 : 0.0;
+    }
     __syncthreads();
     for (int k = 0; k < NB; ++k) {
         double p = a[k][k];
         if (!(p > 0.0) || !isfinite(p)) {
-            if (tx == k && ty == k) {
+            if (tx == 0 && tq == 0 && blockIdx.x == 0) {
                 atomicOr(&status[0], DEV_NOT_PD);
                 atomicMin(&status[1], j0 + k);
             }
             p = 1.0;  // keep going without NaNs; the call reports the failure
         }
         const double r = rsqrt(p);
-        if (tx == k && ty == k) {
+        if (tx == 0 && tq == 0) {
             rk[k] = r;
             lkk[k] = sqrt(p);
         }
-        if (ty > k) {
-            const double lik = a[ty][k] * r;
-            if (tx > k) {
-                if (ty >= tx) a[ty][tx] -= lik * (a[tx][k] * r);
-            } else {
-                m[ty][tx] -= lik * (m[k][tx] * r);
+        const double ck = tx > k ? a[tx][k] * r : m[k][tx] * r;   // what this thread's column contributes
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int ty = tq + 8 * i;
+            if (ty > k) {
+                const double lik = a[ty][k] * r;
+                if (tx > k) {
+                    if (ty >= tx) a[ty][tx] -= lik * ck;
+                } else {
+                    m[ty][tx] -= lik * ck;
+                }
             }
         }
         __syncthreads();
     }
-    Ag[(size_t)ty * npad + tx] = (tx < ty) ? a[ty][tx] * rk[tx] : (tx == ty ? lkk[ty] : 0.0);
-    Dinv[((size_t)g * (npad / NB) + j0 / NB) * NB * NB + ty * NB + tx] = m[ty][tx] * rk[ty];
-}
-
-// Panel below the diagonal block: L_panel L_jj^T = A_panel by forward substitution, one row per thread.
-// (Multiplying by the explicit inverse of L_jj instead loses the small entries of an ill-conditioned
-// factor: its error is relative to |A_panel| |L_jj^-1|, not to the result, and the pivots that follow
-// inherit it -- on noise-free smooth data the log-determinant came out wrong in the third digit.)
-constexpr int kPanelRows = 64;
-__global__ void __launch_bounds__(kPanelRows) panel_kernel(double* __restrict__ A, int npad, int j0)
-{
-    const int g = blockIdx.y;
-    const int r = j0 + NB + blockIdx.x * kPanelRows + threadIdx.x;
-    double* Ag = A + (size_t)g * npad * npad;
-    __shared__ double l[NB][NB + 1];    // L_jj
-    __shared__ double rdiag[NB];
-    for (int e = threadIdx.x; e < NB * NB; e += kPanelRows) l[e / NB][e % NB] = Ag[(size_t)(j0 + e / NB) * npad + j0 + e % NB];
+    // the factor in place of the block (upper part zero), for the substitution below and for block 0's stores
+    double lij[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int ty = tq + 8 * i;
+        lij[i] = (tx < ty) ? a[ty][tx] * rk[tx] : (tx == ty ? lkk[ty] : 0.0);
+    }
     __syncthreads();
-    if (threadIdx.x < NB) rdiag[threadIdx.x] = 1.0 / l[threadIdx.x][threadIdx.x];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int ty = tq + 8 * i;
+        a[ty][tx] = lij[i];
+        if (blockIdx.x == 0) {
+            const size_t blk = ((size_t)g * (npad / NB) + j0 / NB) * NB * NB + ty * NB + tx;
+            Ldiag[blk] = lij[i];
+            Dinv[blk] = m[ty][tx] * rk[ty];
+        }
+    }
     __syncthreads();
+    const int r = j0 + NB + blockIdx.x * kPanelThreads + tq * NB + tx;
     if (r >= npad) return;
-    double* row = Ag + (size_t)r * npad + j0;
+    double* row = Agp + (size_t)r * npad + j0;
     double x[NB];
 #pragma unroll
     for (int c = 0; c < NB; ++c) x[c] = row[c];
@@ -178,14 +199,23 @@ __global__ void __launch_bounds__(kPanelRows) panel_kernel(double* __restrict__ 
         double s0 = 0.0, s1 = 0.0;
 #pragma unroll
         for (int k = 0; k + 1 < c; k += 2) {
-            s0 = fma(x[k], l[c][k], s0);
-            s1 = fma(x[k + 1], l[c][k + 1], s1);
+            s0 = fma(x[k], a[c][k], s0);
+            s1 = fma(x[k + 1], a[c][k + 1], s1);
         }
-        if (c & 1) s0 = fma(x[c - 1], l[c][c - 1], s0);
-        x[c] = (x[c] - (s0 + s1)) * rdiag[c];
+        if (c & 1) s0 = fma(x[c - 1], a[c][c - 1], s0);
+        x[c] = (x[c] - (s0 + s1)) * rk[c];
     }
 #pragma unroll
     for (int c = 0; c < NB; ++c) row[c] = x[c];
+}
+
+// After the factorisation: the factored diagonal blocks into their places.
+__global__ void scatter_ldiag_kernel(const double* __restrict__ Ldiag, int npad, double* __restrict__ L)
+{
+    const int g = blockIdx.y, b = blockIdx.x;
+    const double* Dg = Ldiag + ((size_t)g * (npad / NB) + b) * NB * NB;
+    double* Lg = L + (size_t)g * npad * npad + (size_t)(b * NB) * npad + b * NB;
+    Lg[(size_t)threadIdx.y * npad + threadIdx.x] = Dg[threadIdx.y * NB + threadIdx.x];
 }
 
 // Trailing update: A[i][j] -= sum_k A[i][k] A[j][k] over the kw finished columns from k0 (kw a multiple of
@@ -442,10 +472,11 @@ r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream)
 {
     const int B = gp->batch, n = gp->n, d = gp->d, npad = gp->npad;
     const size_t mat = (size_t)npad * npad;
-    double *Dinv = nullptr, *T = nullptr, *u = nullptr, *slabs = nullptr;
+    double *Dinv = nullptr, *Ldiag = nullptr, *T = nullptr, *u = nullptr, *slabs = nullptr;
     R3_CUDA_TRY(dev_malloc(&Dinv, sizeof(double) * B * (size_t)(npad / NB) * NB * NB));
     auto fail = [&](r3_status_t st) {
         dev_free(Dinv);
+        dev_free(Ldiag);
         dev_free(T);
         dev_free(u);
         dev_free(slabs);
@@ -470,6 +501,7 @@ r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream)
         }                                                                                          \
     } while (0)
 
+    TRY_OR_FAIL(dev_malloc(&Ldiag, sizeof(double) * B * (size_t)(npad / NB) * NB * NB));
     TRY_OR_FAIL(dev_malloc(&T, sizeof(double) * B * mat));
     TRY_OR_FAIL(dev_malloc(&u, sizeof(double) * B * npad));
     TRY_OR_FAIL(dev_malloc(&slabs, sizeof(double) * ((size_t)B + (size_t)B * kRowSlabs * npad)));
@@ -485,11 +517,12 @@ r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream)
     for (int J = 0; J < npad; J += kOuter) {
         const int panel_end = std::min(J + kOuter, npad);
         for (int j0 = J; j0 < panel_end; j0 += NB) {
-            LAUNCH_OR_FAIL(potrf_diag_kernel, B, dim3(NB, NB), gp->L64, npad, j0, Dinv, gp->status_d);
             const int rows = npad - j0 - NB;
+            LAUNCH_OR_FAIL(potrf_panel_kernel, dim3(rows > 0 ? (rows + kPanelThreads - 1) / kPanelThreads : 1, B),
+                           dim3(NB, kPanelThreads / NB), gp->L64, npad,
+                           j0, Dinv, Ldiag, gp->status_d);
             if (rows <= 0) continue;
             const int tiles = (rows + 63) / 64;
-            LAUNCH_OR_FAIL(panel_kernel, dim3((rows + kPanelRows - 1) / kPanelRows, B), kPanelRows, gp->L64, npad, j0);
             const int inner = panel_end - j0 - NB;   // columns of this panel still to be factored
             if (inner > 0)
                 LAUNCH_OR_FAIL(syrk_kernel, dim3((inner + 63) / 64, tiles, B), 256, gp->L64, npad, j0, NB, j0 + NB,
@@ -502,6 +535,7 @@ r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream)
         }
     }
 
+    LAUNCH_OR_FAIL(scatter_ldiag_kernel, dim3(npad / NB, B), dim3(NB, NB), Ldiag, npad, gp->L64);
     TRY_OR_FAIL(cudaMemsetAsync(gp->W64, 0, sizeof(double) * B * mat, stream));
     LAUNCH_OR_FAIL(scatter_dinv_kernel, dim3(npad / NB, B), dim3(NB, NB), Dinv, npad, gp->W64);
     for (int s = NB; s < npad; s *= 2) {
