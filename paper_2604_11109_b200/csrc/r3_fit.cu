@@ -122,6 +122,7 @@ __global__ void gram_kernel(const float* __restrict__ X, const float* __restrict
 // |A_panel| |L_jj^-1|, not to the result, and the pivots that follow inherit it -- on noise-free smooth data
 // the log-determinant came out wrong in the third digit.)
 constexpr int kPanelThreads = 256;   // 32 x 8: four rows of the diagonal block per thread, one panel row per thread
+constexpr size_t kPanelSmem = sizeof(double) * (kPanelThreads / NB) * NB * (NB + 1);   // the warps' row tiles
 __global__ void __launch_bounds__(kPanelThreads) potrf_panel_kernel(double* __restrict__ A, int npad, int j0,
                                                                     double* __restrict__ Dinv,
                                                                     double* __restrict__ Ldiag, int* status)
@@ -152,7 +153,10 @@ __global__ void __launch_bounds__(kPanelThreads) potrf_panel_kernel(double* __re
         const double r = rsqrt(p);
         if (tx == 0 && tq == 0) {
             rk[k] = r;
-            lkk[k] = sqrt(p);
+            // sqrt(p) from r with one correction step (a second long-latency operation here would be on every
+            // column's critical path): s = p r, s += r (p - s^2) / 2
+            const double sq = p * r;
+            lkk[k] = fma(0.5 * r, fma(-sq, sq, p), sq);
         }
         const double ck = tx > k ? a[tx][k] * r : m[k][tx] * r;   // what this thread's column contributes
 #pragma unroll
@@ -188,25 +192,36 @@ __global__ void __launch_bounds__(kPanelThreads) potrf_panel_kernel(double* __re
         }
     }
     __syncthreads();
-    const int r = j0 + NB + blockIdx.x * kPanelThreads + tq * NB + tx;
-    if (r >= npad) return;
-    double* row = Agp + (size_t)r * npad + j0;
-    double x[NB];
+    // Panel rows: warp tq owns rows r0 .. r0 + 31.  The rows go through shared memory so that global memory is
+    // read and written a row at a time by the whole warp (256 contiguous bytes) while each thread works on its
+    // own row.
+    extern __shared__ double tile_all[];                  // [8 warps][32][33]
+    double* tile = tile_all + (size_t)tq * NB * (NB + 1);
+    const int r0 = j0 + NB + blockIdx.x * kPanelThreads + tq * NB;
+    if (r0 >= npad) return;                               // whole warps only: the tile needs no block barrier
+    const int nrows = min(NB, npad - r0);
+    for (int i = 0; i < nrows; ++i) tile[i * (NB + 1) + tx] = Agp[(size_t)(r0 + i) * npad + j0 + tx];
+    __syncwarp();
+    if (tx < nrows) {
+        double x[NB];
 #pragma unroll
-    for (int c = 0; c < NB; ++c) x[c] = row[c];
+        for (int c = 0; c < NB; ++c) x[c] = tile[tx * (NB + 1) + c];
 #pragma unroll
-    for (int c = 0; c < NB; ++c) {
-        double s0 = 0.0, s1 = 0.0;
+        for (int c = 0; c < NB; ++c) {
+            double s0 = 0.0, s1 = 0.0;
 #pragma unroll
-        for (int k = 0; k + 1 < c; k += 2) {
-            s0 = fma(x[k], a[c][k], s0);
-            s1 = fma(x[k + 1], a[c][k + 1], s1);
+            for (int k = 0; k + 1 < c; k += 2) {
+                s0 = fma(x[k], a[c][k], s0);
+                s1 = fma(x[k + 1], a[c][k + 1], s1);
+            }
+            if (c & 1) s0 = fma(x[c - 1], a[c][c - 1], s0);
+            x[c] = (x[c] - (s0 + s1)) * rk[c];
         }
-        if (c & 1) s0 = fma(x[c - 1], a[c][c - 1], s0);
-        x[c] = (x[c] - (s0 + s1)) * rk[c];
-    }
 #pragma unroll
-    for (int c = 0; c < NB; ++c) row[c] = x[c];
+        for (int c = 0; c < NB; ++c) tile[tx * (NB + 1) + c] = x[c];
+    }
+    __syncwarp();
+    for (int i = 0; i < nrows; ++i) Agp[(size_t)(r0 + i) * npad + j0 + tx] = tile[i * (NB + 1) + tx];
 }
 
 // After the factorisation: the factored diagonal blocks into their places.
@@ -513,14 +528,20 @@ r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream)
     LAUNCH_OR_FAIL(gram_kernel, dim3(npad / 16, npad / 16, B), dim3(16, 16), gp->X, gp->ell_d, gp->sf2_d,
                    gp->sn2_d, n, d, npad, gp->L64);
 
+    TRY_OR_FAIL(cudaFuncSetAttribute(potrf_panel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPanelSmem));
     constexpr int kOuter = 4 * NB;   // columns per panel of the two-level right-looking factorisation
     for (int J = 0; J < npad; J += kOuter) {
         const int panel_end = std::min(J + kOuter, npad);
         for (int j0 = J; j0 < panel_end; j0 += NB) {
             const int rows = npad - j0 - NB;
-            LAUNCH_OR_FAIL(potrf_panel_kernel, dim3(rows > 0 ? (rows + kPanelThreads - 1) / kPanelThreads : 1, B),
-                           dim3(NB, kPanelThreads / NB), gp->L64, npad,
-                           j0, Dinv, Ldiag, gp->status_d);
+            potrf_panel_kernel<<<dim3(rows > 0 ? (rows + kPanelThreads - 1) / kPanelThreads : 1, B),
+                                 dim3(NB, kPanelThreads / NB), kPanelSmem, stream>>>(gp->L64, npad, j0, Dinv, Ldiag,
+                                                                                    gp->status_d);
+            ++g_launches;
+            if (cudaError_t e__ = cudaGetLastError(); e__ != cudaSuccess) {
+                set_error("launch of potrf_panel_kernel failed: %s", cudaGetErrorString(e__));
+                return fail(R3_ERR_CUDA);
+            }
             if (rows <= 0) continue;
             const int tiles = (rows + 63) / 64;
             const int inner = panel_end - j0 - NB;   // columns of this panel still to be factored
