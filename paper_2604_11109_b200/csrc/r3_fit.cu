@@ -707,14 +707,30 @@ __global__ void w21_kernel(const double* __restrict__ T2, int n0, int k, double*
     Wnew[(size_t)g * np1 * np1 + (size_t)(n0 + i) * np1 + c] = -s;
 }
 
+// T = Bt - T for the k new rows (Bt: rows n0.. of the extended matrix, leading dimension np1; T: [k][n0])
+__global__ void l21_residual_kernel(const double* __restrict__ Kext, int np1, int n0, int k, double* __restrict__ T)
+{
+    const int g = blockIdx.z, i = blockIdx.y;
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= n0) return;
+    const size_t e = ((size_t)g * k + i) * n0 + c;
+    T[e] = Kext[(size_t)g * np1 * np1 + (size_t)(n0 + i) * np1 + c] - T[e];
+}
+
+__global__ void add_rows_kernel(const double* __restrict__ D, size_t total, double* __restrict__ T)
+{
+    const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e < total) T[e] += D[e];
+}
+
 struct AppendBuffers {
     float *X = nullptr, *y = nullptr, *W32 = nullptr, *alpha32 = nullptr, *best = nullptr;   // best: [2][B]
-    double *L64 = nullptr, *W64 = nullptr, *alpha64 = nullptr, *T1 = nullptr, *T2 = nullptr, *u = nullptr,
+    double *L64 = nullptr, *W64 = nullptr, *alpha64 = nullptr, *T1 = nullptr, *T2 = nullptr, *T3 = nullptr, *u = nullptr,
            *slabs = nullptr, *wnorm = nullptr;
     void release()
     {
         dev_free(X); dev_free(y); dev_free(W32); dev_free(alpha32); dev_free(L64); dev_free(W64); dev_free(alpha64);
-        dev_free(T1); dev_free(T2); dev_free(u); dev_free(slabs); dev_free(best); dev_free(wnorm);
+        dev_free(T1); dev_free(T2); dev_free(T3); dev_free(u); dev_free(slabs); dev_free(best); dev_free(wnorm);
         *this = AppendBuffers();
     }
 };
@@ -787,6 +803,24 @@ r3_status_t append_device(r3_gp* gp, const float* Xnew, const float* ynew, int k
     const dim3 ggrid((n0 + 63) / 64, (k + 31) / 32, B);
     LAUNCH_OR_FAIL(tri_gemm_kernel<true>, ggrid, 256, nb.L64 + (size_t)n0 * np1, np1, mat1, nb.W64, np1, mat1, nb.T1,
                    n0, (size_t)k * n0, k, n0);
+    // The product with the explicit inverse is as accurate as a triangular solve only while K is well
+    // conditioned (its error is relative to |B| |W|, not to L21).  Beyond cond(K) of about 1e8 -- estimated by
+    // |W|_2^2 (sigma_f^2 + sigma_n^2) -- one step of iterative refinement with the factor itself follows:
+    // R = B^T - L21 L^T, L21 += R W^T.  Without it the Schur complement of a noise-free smooth history came out
+    // indefinite where a fit of the whole history succeeds.
+    bool refine = false;
+    for (int g = 0; g < B; ++g)
+        refine |= gp->wnorm[g] * gp->wnorm[g] * ((double)gp->sf2[g] + (double)gp->sn2[g]) > 1e8;
+    if (refine) {
+        TRY_OR_FAIL(dev_malloc(&nb.T3, sizeof(double) * B * (size_t)k * n0));
+        LAUNCH_OR_FAIL(tri_gemm_kernel<true>, ggrid, 256, nb.T1, n0, (size_t)k * n0, nb.L64, np1, mat1, nb.T2, n0,
+                       (size_t)k * n0, k, n0);
+        LAUNCH_OR_FAIL(l21_residual_kernel, dim3((n0 + 127) / 128, k, B), 128, nb.L64, np1, n0, k, nb.T2);
+        LAUNCH_OR_FAIL(tri_gemm_kernel<true>, ggrid, 256, nb.T2, n0, (size_t)k * n0, nb.W64, np1, mat1, nb.T3, n0,
+                       (size_t)k * n0, k, n0);
+        const size_t total = (size_t)B * k * n0;
+        LAUNCH_OR_FAIL(add_rows_kernel, (unsigned)((total + 255) / 256), 256, nb.T3, total, nb.T1);
+    }
     LAUNCH_OR_FAIL(place_l21_kernel, dim3((n0 + 127) / 128, k, B), 128, nb.T1, n0, k, nb.L64, np1);
     LAUNCH_OR_FAIL(schur_kernel, dim3((k + 7) / 8, k, B), 256, nb.T1, n0, k, nb.L64, np1);
     LAUNCH_OR_FAIL(small_chol_inv_kernel, B, 256, nb.L64, nb.W64, np1, n0, k, gp->status_d);
