@@ -249,15 +249,29 @@ __global__ void __launch_bounds__(256) syrk_kernel(double* __restrict__ A, int n
     const int t = threadIdx.x;
     const int ty = t / 16, tx = t % 16;
     double acc[4][4] = {};
+    // the next 32 columns of the two operands travel to registers while the current ones are multiplied
+    double ri[8], rj[8];
+    auto fetch = [&](int kc) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int e = t + 256 * i;
+            const int r = e / NB, c = e % NB;
+            const int gi = base + ti * 64 + r, gj = base + tj * 64 + r;
+            ri[i] = (gi < npad) ? Ag[(size_t)gi * npad + k0 + kc + c] : 0.0;
+            rj[i] = (gj < npad) ? Ag[(size_t)gj * npad + k0 + kc + c] : 0.0;
+        }
+    };
+    fetch(0);
     for (int kc = 0; kc < kw; kc += NB) {
         if (kc > 0) __syncthreads();
-        for (int e = t; e < 64 * NB; e += 256) {
-            int r = e / NB, c = e % NB;
-            int gi = base + ti * 64 + r, gj = base + tj * 64 + r;
-            pi[r][c] = (gi < npad) ? Ag[(size_t)gi * npad + k0 + kc + c] : 0.0;
-            pj[r][c] = (gj < npad) ? Ag[(size_t)gj * npad + k0 + kc + c] : 0.0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int e = t + 256 * i;
+            pi[e / NB][e % NB] = ri[i];
+            pj[e / NB][e % NB] = rj[i];
         }
         __syncthreads();
+        if (kc + NB < kw) fetch(kc + NB);
 #pragma unroll 8
         for (int k = 0; k < NB; ++k) {
             double a[4], b[4];
@@ -328,16 +342,30 @@ __global__ void __launch_bounds__(256) trtri_gemm_kernel(const double* __restric
     __shared__ double sa[64][17], sb[16][65];
     const int t = threadIdx.x, ty = t / 16, tx = t % 16;
     double acc[4][4] = {};
-    for (int k0 = kbeg; k0 < kend; k0 += 16) {
-        for (int e = t; e < 64 * 16; e += 256) {
-            int r = e / 16, c = e % 16;
-            sa[r][c] = (i0 + r < M && k0 + c < K) ? A[(size_t)(i0 + r) * npad + k0 + c] : 0.0;
+    // the next 16 columns of A and rows of B travel from global memory to registers while the current ones are
+    // multiplied out of shared memory
+    double ra[4], rb[4];
+    auto fetch = [&](int k0) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int e = t + 256 * i;
+            const int r = e / 16, c = e % 16;
+            ra[i] = (i0 + r < M && k0 + c < K) ? A[(size_t)(i0 + r) * npad + k0 + c] : 0.0;
+            const int rr = e / 64, cc = e % 64;
+            rb[i] = (k0 + rr < K && j0 + cc < N) ? B[(size_t)(k0 + rr) * npad + j0 + cc] : 0.0;
         }
-        for (int e = t; e < 16 * 64; e += 256) {
-            int r = e / 64, c = e % 64;
-            sb[r][c] = (k0 + r < K && j0 + c < N) ? B[(size_t)(k0 + r) * npad + j0 + c] : 0.0;
+    };
+    if (kbeg < kend) fetch(kbeg);
+    for (int k0 = kbeg; k0 < kend; k0 += 16) {
+        if (k0 > kbeg) __syncthreads();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int e = t + 256 * i;
+            sa[e / 16][e % 16] = ra[i];
+            sb[e / 64][e % 64] = rb[i];
         }
         __syncthreads();
+        if (k0 + 16 < kend) fetch(k0 + 16);
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
             double a[4], b[4];
@@ -351,7 +379,6 @@ __global__ void __launch_bounds__(256) trtri_gemm_kernel(const double* __restric
 #pragma unroll
                 for (int v = 0; v < 4; ++v) acc[u][v] += a[u] * b[v];
         }
-        __syncthreads();
     }
     const double sign = mode == 0 ? 1.0 : -1.0;
 #pragma unroll
