@@ -53,8 +53,9 @@ __global__ void min_y_kernel(const float* __restrict__ y, int n, float* best, fl
 }
 
 // ------------------------------------------------------------------------------------ Gram
-// One 16x16 tile of the lower triangle per block; r^2 by direct differences in FP64 with a true
-// division by the lengthscale, the Matern-5/2 profile, noise on the diagonal.
+// One 16x16 tile of the lower triangle per block; r^2 by direct differences in FP64, scaled by the FP64
+// reciprocal of the lengthscale (one rounding more than a division, a relative 1e-16 in K, for a third of
+// the kernel's time), the Matern-5/2 profile, noise on the diagonal.
 __global__ void gram_kernel(const float* __restrict__ X, const float* __restrict__ ell,
                             const float* __restrict__ sf2, const float* __restrict__ sn2, int n, int d,
                             int npad, double* __restrict__ K)
@@ -69,7 +70,7 @@ __global__ void gram_kernel(const float* __restrict__ X, const float* __restrict
         return;
     }
     __shared__ float sxi[16][33], sxj[16][33];
-    __shared__ float sl[32];
+    __shared__ double sl[32];   // 1 / lengthscale
     const float* Xg = X + (size_t)g * n * d;
     double r2 = 0.0;
     for (int c0 = 0; c0 < d; c0 += 32) {
@@ -80,11 +81,11 @@ __global__ void gram_kernel(const float* __restrict__ X, const float* __restrict
             sxi[r][c] = (gi < n && c0 + c < d) ? Xg[(size_t)gi * d + c0 + c] : 0.f;
             sxj[r][c] = (gj < n && c0 + c < d) ? Xg[(size_t)gj * d + c0 + c] : 0.f;
         }
-        if (t < 32) sl[t] = (c0 + t < d) ? ell[(size_t)g * d + c0 + t] : 1.f;
+        if (t < 32) sl[t] = (c0 + t < d) ? 1.0 / (double)ell[(size_t)g * d + c0 + t] : 1.0;
         __syncthreads();
         const int cmax = min(32, d - c0);
         for (int c = 0; c < cmax; ++c) {
-            double diff = ((double)sxi[ty][c] - (double)sxj[tx][c]) / (double)sl[c];
+            double diff = ((double)sxi[ty][c] - (double)sxj[tx][c]) * sl[c];
             r2 += diff * diff;
         }
         __syncthreads();
@@ -648,7 +649,7 @@ __global__ void cross_gram_kernel(const float* __restrict__ X, const float* __re
     const float* lg = ell + (size_t)g * d;
     double r2 = 0.0;
     for (int j = 0; j < d; ++j) {
-        const double diff = ((double)xi[j] - (double)xc[j]) / (double)lg[j];
+        const double diff = ((double)xi[j] - (double)xc[j]) * (1.0 / (double)lg[j]);   // as gram_kernel does
         r2 += diff * diff;
     }
     const double s = sqrt(5.0) * sqrt(r2);
