@@ -85,8 +85,9 @@ __global__ void __launch_bounds__(256) lml_pairs_kernel(const float* __restrict_
     while (ti * (ti + 1) / 2 > b) --ti;
     const int tk = b - ti * (ti + 1) / 2;
     __shared__ float xi[32][33], xk[32][33];
-    __shared__ float sl[32];
+    __shared__ double sl[32];        // 1 / lengthscale (FP64 reciprocal, as in the fit's Gram kernel)
     __shared__ double red[8];
+    __shared__ double redc[8][32];   // the warps' sums of 32 features' terms
     const int t = threadIdx.x, li = t % 32, lk0 = (t / 32) * 4;
     const int i = ti * 32 + li;
     double r2[4] = {0, 0, 0, 0};
@@ -98,13 +99,13 @@ __global__ void __launch_bounds__(256) lml_pairs_kernel(const float* __restrict_
             xi[r][c] = (gi < n && c0 + c < d) ? X[(size_t)gi * d + c0 + c] : 0.f;
             xk[r][c] = (gk < n && c0 + c < d) ? X[(size_t)gk * d + c0 + c] : 0.f;
         }
-        if (t < 32) sl[t] = (c0 + t < d) ? ell[c0 + t] : 1.f;
+        if (t < 32) sl[t] = (c0 + t < d) ? 1.0 / (double)ell[c0 + t] : 1.0;
         __syncthreads();
         const int cmax = min(32, d - c0);
         for (int c = 0; c < cmax; ++c) {
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                const double u = ((double)xi[li][c] - (double)xk[lk0 + q][c]) / (double)sl[c];
+                const double u = ((double)xi[li][c] - (double)xk[lk0 + q][c]) * sl[c];
                 r2[q] = fma(u, u, r2[q]);
             }
         }
@@ -143,17 +144,25 @@ __global__ void __launch_bounds__(256) lml_pairs_kernel(const float* __restrict_
             xi[r][c] = (gi < n && c0 + c < d) ? X[(size_t)gi * d + c0 + c] : 0.f;
             xk[r][c] = (gk_ < n && c0 + c < d) ? X[(size_t)gk_ * d + c0 + c] : 0.f;
         }
-        if (t < 32) sl[t] = (c0 + t < d) ? ell[c0 + t] : 1.f;
+        if (t < 32) sl[t] = (c0 + t < d) ? 1.0 / (double)ell[c0 + t] : 1.0;
         __syncthreads();
         const int cmax = min(32, d - c0);
         for (int c = 0; c < cmax; ++c) {
             double v = 0.0;
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                const double u = ((double)xi[li][c] - (double)xk[lk0 + q][c]) / (double)sl[c];
+                const double u = ((double)xi[li][c] - (double)xk[lk0 + q][c]) * sl[c];
                 v = fma(gk[q], u * u, v);
             }
-            block_sum(v, c0 + c);
+            // warp sum now, the eight warps in a fixed order once per 32 features
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            if ((t & 31) == 0) redc[t / 32][c] = v;
+        }
+        __syncthreads();
+        if (t < cmax) {
+            double s = 0.0;
+            for (int w = 0; w < 8; ++w) s += redc[w][t];
+            out[c0 + t] = s;
         }
     }
 }
