@@ -280,7 +280,10 @@ r3_status_t r3_gp_propose(r3_gp_t* gp, const float* Xcand, long long m, int q, i
  * With K' = [[K, B], [B^T, C]]:  L21 = (L^-1 B)^T,  L22 L22^T = C - L21 L21^T,  W' = L'^-1 by blocks,
  * alpha' = K'^-1 y'.  The handle afterwards equals, up to FP64 rounding, the one r3_gp_fit returns for
  * the concatenated history with the same hyper-parameters; best becomes min(y') (an incumbent set
- * with r3_gp_set_best is replaced) and the scoring engine is chosen again for the new size.
+ * with r3_gp_set_best is replaced) and the scoring engine is chosen again for the new size.  L21 is
+ * formed with the stored inverse factor; when K is ill-conditioned (|L^-1|_2^2 (signal_var + noise_var)
+ * above 1e8) one step of iterative refinement with L itself follows, so that the extension stays as
+ * accurate as a fit there.
  *
  *   Xnew  device [batch][k][d]     ynew  device [batch][k]      1 <= k <= 128,  n + k <= 8192
  *
