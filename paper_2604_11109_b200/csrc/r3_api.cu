@@ -148,6 +148,8 @@ void r3_gp_free(r3_gp_t* gp)
     dev_free(gp->status_d);
     pinned_word_release(gp->status_h);   // rescued_h lives in the same block
     for (cudaEvent_t e : gp->events) cudaEventDestroy(e);
+    for (cudaEvent_t e : gp->copy_events) cudaEventDestroy(e);
+    if (gp->copy_stream) cudaStreamDestroy(gp->copy_stream);
     dev_free(gp->ws);
     delete gp;
 }
@@ -538,9 +540,43 @@ r3_status_t r3_gp_score_topk_host(r3_gp_t* gp, const float* Xcand_host, long lon
     int* idx = (int*)p;
     p += kb;
     float* val = (float*)p;
-    R3_CUDA_TRY(cudaMemcpyAsync(xc, Xcand_host, sizeof(float) * B * m * gp->d, cudaMemcpyHostToDevice, stream));
-    st = run_score(gp, xc, m, mu, sg, e, gp->ws, sb, stream);
-    if (st != R3_OK) return st;
+    // One GP on the tensor engine with a pool of several pieces: the pieces travel on a second stream while the
+    // earlier ones are scored (a piece is seven full waves of tiles on 148 SMs, so that no launch ends on a
+    // partly filled wave); the accuracy guard runs once over the whole pool, as in the device-buffer call, and
+    // the results are identical.  Everything else: one copy, then the scoring.
+    const long long piece_tiles = 148 * 7;
+    const bool split = B == 1 && pick_engine(gp) == R3_ENGINE_TENSOR && score_tc_can_split(gp) &&
+                       score_tc_tiles(gp, m) > piece_tiles;
+    if (split) {
+        const long long tiles = score_tc_tiles(gp, m);
+        const int pieces = (int)((tiles + piece_tiles - 1) / piece_tiles);
+        if (!gp->copy_stream) R3_CUDA_TRY(cudaStreamCreateWithFlags(&gp->copy_stream, cudaStreamNonBlocking));
+        while ((int)gp->copy_events.size() < pieces + 1) {
+            cudaEvent_t ev;
+            R3_CUDA_TRY(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+            gp->copy_events.push_back(ev);
+        }
+        // the copies start once the caller's stream has reached this call (the staging buffer may still be read)
+        R3_CUDA_TRY(cudaEventRecord(gp->copy_events[pieces], stream));
+        R3_CUDA_TRY(cudaStreamWaitEvent(gp->copy_stream, gp->copy_events[pieces], 0));
+        for (int c = 0; c < pieces; ++c) {
+            const long long lo = c * piece_tiles * 128, hi = std::min<long long>(m, (c + 1) * piece_tiles * 128);
+            R3_CUDA_TRY(cudaMemcpyAsync(xc + lo * gp->d, Xcand_host + lo * gp->d, sizeof(float) * (hi - lo) * gp->d,
+                                        cudaMemcpyHostToDevice, gp->copy_stream));
+            R3_CUDA_TRY(cudaEventRecord(gp->copy_events[c], gp->copy_stream));
+        }
+        for (int c = 0; c < pieces; ++c) {
+            R3_CUDA_TRY(cudaStreamWaitEvent(stream, gp->copy_events[c], 0));
+            st = score_tc_part(gp, xc, m, mu, sg, e, gp->ws, sb, c * piece_tiles, (c + 1) * piece_tiles, false, stream);
+            if (st != R3_OK) return st;
+        }
+        st = score_tc_guard(gp, xc, m, mu, sg, e, gp->ws, stream);
+        if (st != R3_OK) return st;
+    } else {
+        R3_CUDA_TRY(cudaMemcpyAsync(xc, Xcand_host, sizeof(float) * B * m * gp->d, cudaMemcpyHostToDevice, stream));
+        st = run_score(gp, xc, m, mu, sg, e, gp->ws, sb, stream);
+        if (st != R3_OK) return st;
+    }
     st = topk_device(e, gp->batch, m, k, idx, val, (char*)gp->ws + sb, tb, stream);
     if (st != R3_OK) return st;
     if (mu_host) R3_CUDA_TRY(cudaMemcpyAsync(mu_host, mu, sizeof(float) * B * m, cudaMemcpyDeviceToHost, stream));

@@ -112,6 +112,10 @@ struct r3_gp {
     bool profile = false;
     std::vector<cudaEvent_t> events;   // pairs (start, stop)
     size_t events_used = 0;
+
+    // the host-buffer entry point copies the pool in pieces on a stream of its own while earlier pieces are scored
+    cudaStream_t copy_stream = nullptr;
+    std::vector<cudaEvent_t> copy_events;
 };
 
 namespace r3 {
@@ -149,6 +153,15 @@ void tc_release(r3_gp* gp);
 size_t score_tc_workspace_bytes(const r3_gp* gp, long long m);
 r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, float* sigma, float* ei,
                      void* ws, size_t ws_bytes, cudaStream_t stream);
+// The same in pieces, for a caller that overlaps the pool's copy with the scoring: tiles [tile_begin, tile_end) of
+// the score_tc_tiles(gp, m) tiles of 128 candidates (tile_end < 0: all of them), the guard optionally left to
+// one score_tc_guard call after the last piece.
+long long score_tc_tiles(const r3_gp* gp, long long m);
+bool score_tc_can_split(const r3_gp* gp);
+r3_status_t score_tc_part(r3_gp* gp, const float* Xcand, long long m, float* mu, float* sigma, float* ei, void* ws,
+                          size_t ws_bytes, long long tile_begin, long long tile_end, bool guard, cudaStream_t stream);
+r3_status_t score_tc_guard(r3_gp* gp, const float* Xcand, long long m, float* mu, float* sigma, float* ei, void* ws,
+                           cudaStream_t stream);
 
 // top-k (r3_topk.cu)
 size_t topk_workspace_bytes(int batch, long long m, int k);

@@ -151,7 +151,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
     const uint32_t tmem = *tmem_slot;
 
     // tiles of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ...
-    const long long first_tile = blockIdx.x, tile_step = gridDim.x;
+    const long long first_tile = prm.tile_begin + blockIdx.x, tile_step = gridDim.x;
     const int items_per_tile = CPP * P * (P + 1) / 2;
     long long tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     long long tlast = prm.trace ? clock64() : 0;
@@ -956,6 +956,22 @@ size_t score_tc_workspace_bytes(const r3_gp* gp, long long m) { return guard_wor
 r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, float* sigma, float* ei, void* ws,
                      size_t ws_bytes, cudaStream_t stream)
 {
+    return score_tc_part(gp, Xcand, m, mu, sigma, ei, ws, ws_bytes, 0, -1, true, stream);
+}
+
+long long score_tc_tiles(const r3_gp* gp, long long m) { return (m + TILE_M - 1) / TILE_M * gp->batch; }
+
+bool score_tc_can_split(const r3_gp* gp) { return ops_of(gp) != nullptr && env_int("R3_TC_PAIR", 0) == 0; }
+
+r3_status_t score_tc_guard(r3_gp* gp, const float* Xcand, long long m, float* mu, float* sigma, float* ei, void* ws,
+                           cudaStream_t stream)
+{
+    return guard_and_rescue(gp, Xcand, m, guard_carve(gp, m, ws), mu, sigma, ei, stream);
+}
+
+r3_status_t score_tc_part(r3_gp* gp, const float* Xcand, long long m, float* mu, float* sigma, float* ei, void* ws,
+                          size_t ws_bytes, long long tile_begin, long long tile_end, bool guard, cudaStream_t stream)
+{
     TensorOperands* t = ops_of(gp);
     if (!t) {
         set_error("the tensor-core engine does not serve this handle");
@@ -997,9 +1013,16 @@ r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, floa
     prm.status = gp->status_d;
     prm.tiles_per_gp = (m + TILE_M - 1) / TILE_M;
     prm.total_tiles = prm.tiles_per_gp * gp->batch;
+    prm.tile_begin = 0;
+    if (tile_end >= 0) {   // a range of the pool's tiles (the caller runs the guard once, after the last range)
+        prm.tile_begin = tile_begin;
+        prm.total_tiles = tile_end < prm.total_tiles ? tile_end : prm.total_tiles;
+    }
+    const long long launch_tiles = prm.total_tiles - prm.tile_begin;
+    if (launch_tiles <= 0) return R3_OK;
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, gp->device);
-    const unsigned grid = (unsigned)(prm.total_tiles < sms ? prm.total_tiles : sms);
+    const unsigned grid = (unsigned)(launch_tiles < sms ? launch_tiles : sms);
     // R3_TC_TRACE=1 prints, for the first CTA, the cycles each role spent per wait / issue category
     prm.trace = nullptr;
     if (getenv("R3_TC_TRACE")) {
@@ -1009,7 +1032,7 @@ r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, floa
     // The paired kernel (two CTAs of a cluster share a tile and the k* chunks) serves histories with at least
     // two passes; R3_TC_PAIR=0/1 overrides the choice.
     int pair_ws = 0;
-    const bool pair = env_int("R3_TC_PAIR", 0) != 0 && tc_pair_fits(t, &pair_ws);
+    const bool pair = tile_end < 0 && env_int("R3_TC_PAIR", 0) != 0 && tc_pair_fits(t, &pair_ws);
     prof_begin(gp, stream);
     if (pair) {
         const r3_status_t st = launch_tc_pair(t, prm, sms, stream);
@@ -1038,6 +1061,7 @@ r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, floa
                 fprintf(stderr, "\n");
             }
     }
+    if (!guard) return R3_OK;
     return guard_and_rescue(gp, Xcand, m, gb, mu, sigma, ei, stream);
 }
 

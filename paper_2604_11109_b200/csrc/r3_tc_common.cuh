@@ -43,7 +43,8 @@ struct TcParams {
     const double* wnorm;
     int DP, NP, P, ws;
     int* status;
-    long long tiles_per_gp, total_tiles;
+    long long tiles_per_gp, total_tiles;   // total_tiles: one past the last tile of this launch
+    long long tile_begin;                  // first tile of this launch (the single-CTA kernel; 0 for a whole pool)
     long long* trace;   // optional [grid][4 roles][8] cycle counters (diagnostics)
 };
 

@@ -179,6 +179,29 @@ def test_host_buffer_form_equals_device_form():
     gp.close()
 
 
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_buffer_form_in_pieces_equals_device_form(pinned):
+    """A pool of more than seven waves of tiles for one GP on the tensor engine is copied in pieces while earlier
+    pieces are scored; the outputs are bit-identical to the device-buffer call (several pieces, the last one
+    ragged, some candidates on observations so that the guard has work)."""
+    m, k = 148 * 7 * 128 * 2 + 777, 50
+    g = rand_problem(81, 1, 300, 8, m)
+    g["Xcand"][0, 5:25] = g["X"][0, :20]
+    gp = fit_gpu(g, b.ENGINE_TENSOR)
+    mu, sd, ei, idx, val = (t.cpu() for t in b.r3_gp_score_topk(gp, dev(g["Xcand"]), k))
+    xh = torch.from_numpy(g["Xcand"])
+    out = [torch.empty(1, m), torch.empty(1, m), torch.empty(1, m), torch.empty(1, k, dtype=torch.int32),
+           torch.empty(1, k)]
+    if pinned:
+        xh, out = xh.pin_memory(), [t.pin_memory() for t in out]
+    for _ in range(2):   # the second call reuses the staging buffer that the first one's kernels read
+        b.r3_gp_score_topk_host(gp, xh, k, tuple(out))
+        for a, c in zip((mu, sd, ei, idx, val), out):
+            assert torch.equal(a, c)
+    b.r3_gp_check(gp)
+    gp.close()
+
+
 # ------------------------------------------------------------------------------------------ top-k alone (bit-exact)
 @pytest.mark.parametrize("batch,m,k", [(1, 1, 1), (1, 100, 100), (2, 4096, 7), (1, 4097, 1024), (3, 70001, 33),
                                        (1, 1 << 20, 128), (64, 65536, 16)])
