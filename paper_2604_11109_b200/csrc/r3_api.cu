@@ -540,15 +540,17 @@ r3_status_t r3_gp_score_topk_host(r3_gp_t* gp, const float* Xcand_host, long lon
     int* idx = (int*)p;
     p += kb;
     float* val = (float*)p;
-    // One GP on the tensor engine with a pool of several pieces: the pieces travel on a second stream while the
-    // earlier ones are scored (a piece is seven full waves of tiles on 148 SMs, so that no launch ends on a
-    // partly filled wave); the accuracy guard runs once over the whole pool, as in the device-buffer call, and
-    // the results are identical.  Everything else: one copy, then the scoring.
-    const long long piece_tiles = 148 * 7;
-    const bool split = B == 1 && pick_engine(gp) == R3_ENGINE_TENSOR && score_tc_can_split(gp) &&
-                       score_tc_tiles(gp, m) > piece_tiles;
+    // On the tensor engine a pool of several pieces travels on a second stream while the earlier pieces are
+    // scored (a piece is about seven full waves of tiles on 148 SMs, so that no launch ends on a nearly empty
+    // wave); the accuracy guard runs once over the whole pool, as in the device-buffer call, and the results are
+    // identical.  Everything else: one copy, then the scoring.
+    const long long tiles = pick_engine(gp) == R3_ENGINE_TENSOR ? score_tc_tiles(gp, m) : 0;
+    const long long tiles_per_gp = B ? tiles / (long long)B : 0;
+    // pieces are ranges of tiles that are contiguous in memory: any range for one GP, whole GPs for several
+    long long piece_tiles = 148 * 7;
+    if (B > 1) piece_tiles = std::max<long long>(1, (piece_tiles + tiles_per_gp / 2) / std::max<long long>(tiles_per_gp, 1)) * tiles_per_gp;
+    const bool split = pick_engine(gp) == R3_ENGINE_TENSOR && score_tc_can_split(gp) && tiles > piece_tiles;
     if (split) {
-        const long long tiles = score_tc_tiles(gp, m);
         const int pieces = (int)((tiles + piece_tiles - 1) / piece_tiles);
         if (!gp->copy_stream) R3_CUDA_TRY(cudaStreamCreateWithFlags(&gp->copy_stream, cudaStreamNonBlocking));
         while ((int)gp->copy_events.size() < pieces + 1) {
@@ -559,8 +561,13 @@ r3_status_t r3_gp_score_topk_host(r3_gp_t* gp, const float* Xcand_host, long lon
         // the copies start once the caller's stream has reached this call (the staging buffer may still be read)
         R3_CUDA_TRY(cudaEventRecord(gp->copy_events[pieces], stream));
         R3_CUDA_TRY(cudaStreamWaitEvent(gp->copy_stream, gp->copy_events[pieces], 0));
+        const long long rows = (long long)B * m;   // candidate rows of the whole call, GP after GP
+        auto first_row = [&](long long tile) {      // the row at which a tile starts
+            if (B == 1) return std::min<long long>(m, tile * 128);
+            return std::min<long long>(rows, tile / tiles_per_gp * m);
+        };
         for (int c = 0; c < pieces; ++c) {
-            const long long lo = c * piece_tiles * 128, hi = std::min<long long>(m, (c + 1) * piece_tiles * 128);
+            const long long lo = first_row(c * piece_tiles), hi = first_row(std::min(tiles, (c + 1) * piece_tiles));
             R3_CUDA_TRY(cudaMemcpyAsync(xc + lo * gp->d, Xcand_host + lo * gp->d, sizeof(float) * (hi - lo) * gp->d,
                                         cudaMemcpyHostToDevice, gp->copy_stream));
             R3_CUDA_TRY(cudaEventRecord(gp->copy_events[c], gp->copy_stream));

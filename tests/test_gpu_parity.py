@@ -179,19 +179,20 @@ def test_host_buffer_form_equals_device_form():
     gp.close()
 
 
-@pytest.mark.parametrize("pinned", [True, False])
-def test_host_buffer_form_in_pieces_equals_device_form(pinned):
-    """A pool of more than seven waves of tiles for one GP on the tensor engine is copied in pieces while earlier
-    pieces are scored; the outputs are bit-identical to the device-buffer call (several pieces, the last one
-    ragged, some candidates on observations so that the guard has work)."""
-    m, k = 148 * 7 * 128 * 2 + 777, 50
-    g = rand_problem(81, 1, 300, 8, m)
-    g["Xcand"][0, 5:25] = g["X"][0, :20]
+@pytest.mark.parametrize("batch,m,pinned", [(1, 148 * 7 * 128 * 2 + 777, True), (1, 148 * 7 * 128 + 5, False),
+                                            (3, 70000, True), (5, 3000 * 128, False)])
+def test_host_buffer_form_in_pieces_equals_device_form(batch, m, pinned):
+    """On the tensor engine a pool of more than about seven waves of tiles is copied in pieces (ranges of one GP's
+    tiles, or whole GPs of a batched handle) while earlier pieces are scored; the outputs are bit-identical to the
+    device-buffer call.  Some candidates sit on observations so that the guard has work."""
+    k = 50
+    g = rand_problem(81 + batch, batch, 300, 8, m)
+    g["Xcand"][:, 5:25] = g["X"][:, :20]
     gp = fit_gpu(g, b.ENGINE_TENSOR)
     mu, sd, ei, idx, val = (t.cpu() for t in b.r3_gp_score_topk(gp, dev(g["Xcand"]), k))
     xh = torch.from_numpy(g["Xcand"])
-    out = [torch.empty(1, m), torch.empty(1, m), torch.empty(1, m), torch.empty(1, k, dtype=torch.int32),
-           torch.empty(1, k)]
+    out = [torch.empty(batch, m), torch.empty(batch, m), torch.empty(batch, m),
+           torch.empty(batch, k, dtype=torch.int32), torch.empty(batch, k)]
     if pinned:
         xh, out = xh.pin_memory(), [t.pin_memory() for t in out]
     for _ in range(2):   # the second call reuses the staging buffer that the first one's kernels read
