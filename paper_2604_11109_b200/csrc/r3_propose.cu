@@ -53,6 +53,9 @@ __global__ void shortlist_kstar_kernel(const ProposeArrays a)
     double* Ks = a.Ks + (size_t)g * a.R * npad;
     const double sf2 = (double)a.sf2[g];
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    __shared__ double inv[kMaxD];   // FP64 reciprocals of the lengthscales, as the fit's Gram kernel uses them
+    for (int j = threadIdx.x; j < d; j += blockDim.x) inv[j] = 1.0 / (double)ell[j];
+    __syncthreads();
     if (i >= npad) return;
     double v = 0.0;
     if (i < n) {
@@ -60,7 +63,7 @@ __global__ void shortlist_kstar_kernel(const ProposeArrays a)
         const float* x = X + (size_t)i * d;
         double r2 = 0.0;
         for (int j = 0; j < d; ++j) {
-            const double diff = ((double)x[j] - (double)z[j]) / (double)ell[j];
+            const double diff = ((double)x[j] - (double)z[j]) * inv[j];
             r2 += diff * diff;
         }
         const double s = sqrt(5.0) * sqrt(r2);
@@ -251,7 +254,7 @@ r3_status_t propose_shortlist(r3_gp* gp, const float* Xcand, long long m, const 
 
     R3_LAUNCH(shortlist_kstar_kernel, dim3((npad + 127) / 128, R, B), 128, 0, stream, a);
     // V = Ks W^T (v_r = W k*_r): the same triangular product as the append step of the fit
-    R3_LAUNCH(tri_gemm_kernel<true>, dim3((n + 63) / 64, (R + 31) / 32, B), 256, 0, stream, a.Ks, npad,
+    R3_LAUNCH((tri_gemm_kernel<true, 64>), dim3((n + 63) / 64, (R + 63) / 64, B), 256, 0, stream, a.Ks, npad,
               (size_t)R * npad, gp->W64, npad, (size_t)npad * npad, a.V, npad, (size_t)R * npad, R, n);
     R3_LAUNCH(shortlist_moments_kernel, dim3((R + 7) / 8, B), 256, 0, stream, a);
     for (int t = 0; t < q; ++t) {
