@@ -673,45 +673,80 @@ __global__ void schur_kernel(const double* __restrict__ L21, int n0, int k, doub
     if (lane == 0) Lnew[(size_t)g * np1 * np1 + (size_t)(n0 + i) * np1 + n0 + j] -= s;
 }
 
-// In-place Cholesky of the k x k block at (n0, n0) of L' and its inverse into W' (one block per GP, k <= 128).
+// Cholesky of the k x k block at (n0, n0) of L' (in place) and its inverse into W' (one block per GP, k <= 128).
+// Both triangles live in shared memory, packed by rows (entry (i, c), c <= i, at i (i + 1) / 2 + c).
+// Factor: one barrier per column -- every thread forms r = 1 / sqrt(s_jj) itself and scales what it reads of
+// column j by it, the column itself stays unscaled until the end (as in the fit's diagonal blocks).  Inverse:
+// forward substitution L22 v = e_c, one column per thread, out of shared memory.
 __global__ void __launch_bounds__(256) small_chol_inv_kernel(double* __restrict__ Lnew, double* __restrict__ Wnew,
                                                               int np1, int n0, int k, int* __restrict__ status)
 {
     const int g = blockIdx.x;
     double* S = Lnew + (size_t)g * np1 * np1 + (size_t)n0 * np1 + n0;   // S[i][j] at S[i * np1 + j]
     double* V = Wnew + (size_t)g * np1 * np1 + (size_t)n0 * np1 + n0;
-    __shared__ double piv_s;
+    extern __shared__ double tri[];            // packed S, then packed V, then r_j
+    const int nt = k * (k + 1) / 2;
+    double* s = tri;
+    double* v = tri + nt;
+    double* rj = v + nt;
+    auto at = [](int i, int c) { return i * (i + 1) / 2 + c; };
+    for (int e = threadIdx.x; e < k * k; e += blockDim.x) {
+        const int i = e / k, c = e % k;
+        if (c <= i) s[at(i, c)] = S[(size_t)i * np1 + c];
+    }
+    __syncthreads();
     for (int j = 0; j < k; ++j) {
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            double piv = S[(size_t)j * np1 + j];
-            if (!(piv > 0.0)) {
+        double piv = s[at(j, j)];
+        if (!(piv > 0.0)) {
+            if (threadIdx.x == 0) {
                 atomicOr(&status[0], DEV_NOT_PD);
                 atomicMin(&status[1], n0 + j);
-                piv = 1.0;
             }
-            piv_s = sqrt(piv);
+            piv = 1.0;
         }
-        __syncthreads();
-        const double l = piv_s;
-        for (int i = j + threadIdx.x; i < k; i += blockDim.x)
-            S[(size_t)i * np1 + j] = (i == j) ? l : S[(size_t)i * np1 + j] / l;
-        __syncthreads();
+        const double r = rsqrt(piv);
+        if (threadIdx.x == 0) rj[j] = r;
+        // trailing update of the lower triangle: rows i > j, columns j < c <= i
         const int w = k - j - 1;
         for (int e = threadIdx.x; e < w * w; e += blockDim.x) {
             const int i = j + 1 + e / w, c = j + 1 + e % w;
-            if (c <= i) S[(size_t)i * np1 + c] -= S[(size_t)i * np1 + j] * S[(size_t)c * np1 + j];
+            if (c <= i) s[at(i, c)] -= (s[at(i, j)] * r) * (s[at(c, j)] * r);
+        }
+        __syncthreads();
+    }
+    // scale the columns, diagonal = sqrt(pivot) from its reciprocal root with one correction step
+    for (int e = threadIdx.x; e < k * k; e += blockDim.x) {
+        const int i = e / k, c = e % k;
+        if (c > i) continue;
+        double val;
+        if (c == i) {
+            double p = s[at(i, i)];
+            if (!(p > 0.0)) p = 1.0;
+            const double sq = p * rj[i];
+            val = fma(0.5 * rj[i], fma(-sq, sq, p), sq);
+        } else {
+            val = s[at(i, c)] * rj[c];
+        }
+        S[(size_t)i * np1 + c] = val;
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < k * k; e += blockDim.x) {   // the factor itself into shared memory
+        const int i = e / k, c = e % k;
+        if (c <= i) s[at(i, c)] = S[(size_t)i * np1 + c];
+    }
+    __syncthreads();
+    for (int c = threadIdx.x; c < k; c += blockDim.x) {
+        v[at(c, c)] = 1.0 / s[at(c, c)];
+        for (int i = c + 1; i < k; ++i) {
+            double acc = 0.0;
+            for (int j = c; j < i; ++j) acc = fma(s[at(i, j)], v[at(j, c)], acc);
+            v[at(i, c)] = -acc / s[at(i, i)];
         }
     }
     __syncthreads();
-    // inverse by forward substitution, one column per thread: L22 v = e_c
-    for (int c = threadIdx.x; c < k; c += blockDim.x) {
-        V[(size_t)c * np1 + c] = 1.0 / S[(size_t)c * np1 + c];
-        for (int i = c + 1; i < k; ++i) {
-            double s = 0.0;
-            for (int j = c; j < i; ++j) s = fma(S[(size_t)i * np1 + j], V[(size_t)j * np1 + c], s);
-            V[(size_t)i * np1 + c] = -s / S[(size_t)i * np1 + i];
-        }
+    for (int e = threadIdx.x; e < k * k; e += blockDim.x) {
+        const int i = e / k, c = e % k;
+        if (c <= i) V[(size_t)i * np1 + c] = v[at(i, c)];
     }
 }
 
@@ -851,7 +886,13 @@ r3_status_t append_device(r3_gp* gp, const float* Xnew, const float* ynew, int k
     }
     LAUNCH_OR_FAIL(place_l21_kernel, dim3((n0 + 127) / 128, k, B), 128, nb.T1, n0, k, nb.L64, np1);
     LAUNCH_OR_FAIL(schur_kernel, dim3((k + 7) / 8, k, B), 256, nb.T1, n0, k, nb.L64, np1);
-    LAUNCH_OR_FAIL(small_chol_inv_kernel, B, 256, nb.L64, nb.W64, np1, n0, k, gp->status_d);
+    {
+        const size_t smem = sizeof(double) * ((size_t)k * (k + 1) + k);
+        TRY_OR_FAIL(cudaFuncSetAttribute(small_chol_inv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        small_chol_inv_kernel<<<B, 256, smem, stream>>>(nb.L64, nb.W64, np1, n0, k, gp->status_d);
+        ++g_launches;
+        TRY_OR_FAIL(cudaGetLastError());
+    }
     // W21 = -W22 (L21 W)
     LAUNCH_OR_FAIL(tri_gemm_kernel<false>, ggrid, 256, nb.T1, n0, (size_t)k * n0, nb.W64, np1, mat1, nb.T2, n0,
                    (size_t)k * n0, k, n0);
