@@ -835,8 +835,13 @@ r3_status_t append_device(r3_gp* gp, const float* Xnew, const float* ynew, int k
     TRY_OR_FAIL(dev_malloc(&nb.W32, sizeof(float) * B * mat1));
     TRY_OR_FAIL(dev_malloc(&nb.alpha64, sizeof(double) * B * np1));
     TRY_OR_FAIL(dev_malloc(&nb.alpha32, sizeof(float) * B * np1));
-    TRY_OR_FAIL(dev_malloc(&nb.T1, sizeof(double) * B * (size_t)k * n0));
-    TRY_OR_FAIL(dev_malloc(&nb.T2, sizeof(double) * B * (size_t)k * n0));
+    // the triangular products of few rows are cut along their reductions so that they fill the GPU
+    const dim3 ggrid0((n0 + 63) / 64, (k + 31) / 32, B);
+    const size_t blocks0 = (size_t)ggrid0.x * ggrid0.y * ggrid0.z;
+    const int splits = blocks0 >= 2 * 148 ? 1 : (int)std::min<size_t>(8, (6 * 148 + blocks0 - 1) / blocks0);
+    const size_t part = (size_t)B * k * n0;   // doubles of one [B][k][n0] array: the parts of a product lie this far apart
+    TRY_OR_FAIL(dev_malloc(&nb.T1, sizeof(double) * part * splits));
+    TRY_OR_FAIL(dev_malloc(&nb.T2, sizeof(double) * part * splits));
     TRY_OR_FAIL(dev_malloc(&nb.u, sizeof(double) * B * np1));
     TRY_OR_FAIL(dev_malloc(&nb.slabs, sizeof(double) * ((size_t)B + (size_t)B * kRowSlabs * np1)));
     TRY_OR_FAIL(dev_malloc(&nb.best, sizeof(float) * 2 * B));
@@ -863,9 +868,11 @@ r3_status_t append_device(r3_gp* gp, const float* Xnew, const float* ynew, int k
     // new rows of K', then L21 = B^T W^T
     LAUNCH_OR_FAIL(cross_gram_kernel, dim3((n1 + 127) / 128, k, B), 128, nb.X, gp->ell_d, gp->sf2_d, gp->sn2_d, n0, n1,
                    d, np1, nb.L64);
-    const dim3 ggrid((n0 + 63) / 64, (k + 31) / 32, B);
+    const dim3 ggrid((n0 + 63) / 64, (k + 31) / 32, B * splits);
+    const dim3 sgrid((unsigned)(((size_t)k * n0 + 255) / 256), B);
     LAUNCH_OR_FAIL(tri_gemm_kernel<true>, ggrid, 256, nb.L64 + (size_t)n0 * np1, np1, mat1, nb.W64, np1, mat1, nb.T1,
-                   n0, (size_t)k * n0, k, n0);
+                   n0, (size_t)k * n0, k, n0, splits, part);
+    if (splits > 1) LAUNCH_OR_FAIL(tri_gemm_sum_kernel, sgrid, 256, nb.T1, (size_t)k * n0, (size_t)k * n0, splits, part);
     // The product with the explicit inverse is as accurate as a triangular solve only while K is well
     // conditioned (its error is relative to |B| |W|, not to L21).  Beyond cond(K) of about 1e8 -- estimated by
     // |W|_2^2 (sigma_f^2 + sigma_n^2) -- one step of iterative refinement with the factor itself follows:
@@ -875,12 +882,16 @@ r3_status_t append_device(r3_gp* gp, const float* Xnew, const float* ynew, int k
     for (int g = 0; g < B; ++g)
         refine |= gp->wnorm[g] * gp->wnorm[g] * ((double)gp->sf2[g] + (double)gp->sn2[g]) > 1e8;
     if (refine) {
-        TRY_OR_FAIL(dev_malloc(&nb.T3, sizeof(double) * B * (size_t)k * n0));
+        TRY_OR_FAIL(dev_malloc(&nb.T3, sizeof(double) * part * splits));
         LAUNCH_OR_FAIL(tri_gemm_kernel<true>, ggrid, 256, nb.T1, n0, (size_t)k * n0, nb.L64, np1, mat1, nb.T2, n0,
-                       (size_t)k * n0, k, n0);
+                       (size_t)k * n0, k, n0, splits, part);
+        if (splits > 1)
+            LAUNCH_OR_FAIL(tri_gemm_sum_kernel, sgrid, 256, nb.T2, (size_t)k * n0, (size_t)k * n0, splits, part);
         LAUNCH_OR_FAIL(l21_residual_kernel, dim3((n0 + 127) / 128, k, B), 128, nb.L64, np1, n0, k, nb.T2);
         LAUNCH_OR_FAIL(tri_gemm_kernel<true>, ggrid, 256, nb.T2, n0, (size_t)k * n0, nb.W64, np1, mat1, nb.T3, n0,
-                       (size_t)k * n0, k, n0);
+                       (size_t)k * n0, k, n0, splits, part);
+        if (splits > 1)
+            LAUNCH_OR_FAIL(tri_gemm_sum_kernel, sgrid, 256, nb.T3, (size_t)k * n0, (size_t)k * n0, splits, part);
         const size_t total = (size_t)B * k * n0;
         LAUNCH_OR_FAIL(add_rows_kernel, (unsigned)((total + 255) / 256), 256, nb.T3, total, nb.T1);
     }
@@ -895,7 +906,8 @@ r3_status_t append_device(r3_gp* gp, const float* Xnew, const float* ynew, int k
     }
     // W21 = -W22 (L21 W)
     LAUNCH_OR_FAIL(tri_gemm_kernel<false>, ggrid, 256, nb.T1, n0, (size_t)k * n0, nb.W64, np1, mat1, nb.T2, n0,
-                   (size_t)k * n0, k, n0);
+                   (size_t)k * n0, k, n0, splits, part);
+    if (splits > 1) LAUNCH_OR_FAIL(tri_gemm_sum_kernel, sgrid, 256, nb.T2, (size_t)k * n0, (size_t)k * n0, splits, part);
     LAUNCH_OR_FAIL(w21_kernel, dim3((n0 + 127) / 128, k, B), 128, nb.T2, n0, k, nb.W64, np1);
     {
         const r3_status_t st = finish_weights(B, n1, np1, nb.W64, nb.y, nb.alpha64, nb.alpha32, nb.W32, nb.wnorm,

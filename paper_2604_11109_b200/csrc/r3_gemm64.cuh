@@ -12,22 +12,32 @@ namespace r3 {
 // FP64, TM x 64 tile per block of 256 threads (TM / 16 x 4 results per thread; TM = 32 for the few rows of an
 // append, 64 for the many of a proposal's shortlist), reduction in steps of 16 over the part of r that can be
 // non-zero for the tile's columns; the next step's operands are fetched into registers during the current one.
+// With few rows (an append's k <= 128) the tiles are too few to fill the GPU and the long reductions of the
+// right-hand columns dominate: `splits` > 1 cuts every tile's reduction into that many parts (blockIdx.z = GP *
+// splits + part), part p writing its partial product to C + p * strideSplit; tri_gemm_sum_kernel adds the parts
+// in a fixed order.
 template <bool NT, int TM = 32>
 __global__ void __launch_bounds__(256) tri_gemm_kernel(const double* __restrict__ A, int lda, size_t strideA,
                                                        const double* __restrict__ Wm, int ldw, size_t strideW,
-                                                       double* __restrict__ C, int ldc, size_t strideC, int M, int N)
+                                                       double* __restrict__ C, int ldc, size_t strideC, int M, int N,
+                                                       int splits = 1, size_t strideSplit = 0)
 {
     constexpr int RU = TM / 16;   // rows per thread
     __shared__ double As[TM][17], Bs[16][65];
-    const int g = blockIdx.z;
+    const int g = blockIdx.z / splits, part = blockIdx.z % splits;
     A += (size_t)g * strideA;
     Wm += (size_t)g * strideW;
-    C += (size_t)g * strideC;
+    C += (size_t)g * strideC + (size_t)part * strideSplit;
     const int i0 = blockIdx.y * TM, c0 = blockIdx.x * 64;
     const int t = threadIdx.x, ty = t / 16, tx = t % 16;
     double acc[RU][4] = {};
-    const int r_begin = NT ? 0 : (c0 / 16) * 16;
-    const int r_end = NT ? min(c0 + 64, N) : N;
+    int r_begin = NT ? 0 : (c0 / 16) * 16;
+    int r_end = NT ? min(c0 + 64, N) : N;
+    if (splits > 1) {
+        const int steps = (r_end - r_begin + 15) / 16, per = (steps + splits - 1) / splits;
+        r_begin += part * per * 16;
+        r_end = min(r_end, r_begin + per * 16);
+    }
     double ra[RU], rb[4];
     auto fetch = [&](int r0) {
 #pragma unroll
@@ -86,6 +96,17 @@ __global__ void __launch_bounds__(256) tri_gemm_kernel(const double* __restrict_
             const int i = i0 + ty * RU + u, c = c0 + tx * 4 + v;
             if (i < M && c < N) C[(size_t)i * ldc + c] = acc[u][v];
         }
+}
+
+// C[g][e] = sum over the parts, in order (C's parts lie strideSplit apart; the sum goes to part 0)
+static __global__ void tri_gemm_sum_kernel(double* __restrict__ C, size_t count, size_t strideC, int splits, size_t strideSplit)
+{
+    const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= count) return;
+    double* c = C + (size_t)blockIdx.y * strideC + e;
+    double s = c[0];
+    for (int p = 1; p < splits; ++p) s += c[(size_t)p * strideSplit];
+    c[0] = s;
 }
 
 }  // namespace r3
