@@ -166,6 +166,23 @@ r3_status_t r3_gp_score_topk_host(r3_gp_t* gp, const float* Xcand_host, long lon
 /* Synchronise `cuda_stream` and return (then clear) the handle's latched device status. */
 r3_status_t r3_gp_check(r3_gp_t* gp, void* cuda_stream);
 
+/*
+ * Failure handling of the device-side waits (Section IV discards configurations that fail; the paper says
+ * nothing about a surrogate step that fails, so this is the library's own).  Inside the tensor-core
+ * scoring kernel the warp roles hand stages to one another through barriers, and every such wait gives
+ * up after a limit: the kernel then raises a status bit, lets the copies in flight land, frees its
+ * tensor memory and returns, r3_gp_check reports R3_ERR_DEVICE_TIMEOUT, the results of that call are
+ * invalid and the handle stays usable.  r3_gp_set_wait_limit sets the limit in SM clock cycles
+ * (default 4e9, about two seconds; at least 1e5).
+ *
+ * r3_gp_test_withhold is a testing aid for that path: on the next tensor-engine scoring call of this
+ * handle (one call only) every thread block stops streaming the inverse factor before chunk `chunk`
+ * (>= 0) of its own sequence, so that the consumer of that stage waits for data that never comes and
+ * its wait runs out.  Nothing faults and nothing waits longer than the limit; use a short limit with it.
+ */
+r3_status_t r3_gp_set_wait_limit(r3_gp_t* gp, long long cycles);
+r3_status_t r3_gp_test_withhold(r3_gp_t* gp, long long chunk);
+
 /* Incumbent used by EI: defaults to min(y); may be overridden per GP.  host [batch]. */
 r3_status_t r3_gp_get_best(const r3_gp_t* gp, float* best);
 r3_status_t r3_gp_set_best(r3_gp_t* gp, const float* best);
@@ -447,6 +464,15 @@ void r3_tpe_free(r3_tpe_t* tpe);
  */
 void r3_trim_cache(void);
 unsigned long long r3_cached_bytes(void);
+
+/*
+ * Testing aid for the allocation-failure paths (host side; no device is touched): the device
+ * allocation number `after` from now on (0 = the very next one) made by the calling process through
+ * this library fails once as if the device were out of memory, so that a caller can check that
+ * r3_gp_fit returns R3_ERR_ALLOC without leaking and that r3_gp_append leaves its handle unchanged.
+ * A negative value disarms it.  Returns how many allocations were counted since it was last armed.
+ */
+long long r3_test_fail_allocation(long long after);
 
 const char* r3_status_string(r3_status_t status);
 const char* r3_last_error(void);

@@ -17,8 +17,7 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-# R3_LIB_PATH points the binding at another build of the same library (kernel experiments)
-LIB_PATH = os.environ.get("R3_LIB_PATH") or os.path.join(_HERE, "libr3gp.so")
+LIB_PATH = os.path.join(_HERE, "libr3gp.so")
 
 R3_OK = 0
 STATUS_NAMES = {
@@ -68,6 +67,9 @@ SIGNATURES = {
     "r3_gp_score_topk": (_i, [_vp, _vp, _ll, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "r3_gp_score_topk_host": (_i, [_vp, _vp, _ll, _i, _vp, _vp, _vp, _vp, _vp, _vp]),
     "r3_gp_check": (_i, [_vp, _vp]),
+    "r3_gp_set_wait_limit": (_i, [_vp, _ll]),
+    "r3_gp_test_withhold": (_i, [_vp, _ll]),
+    "r3_test_fail_allocation": (_ll, [_ll]),
     "r3_gp_get_best": (_i, [_vp, _fp]),
     "r3_gp_set_best": (_i, [_vp, _fp]),
     "r3_gp_set_engine": (_i, [_vp, _i]),
@@ -369,6 +371,18 @@ def r3_gp_size(gp: GP) -> int:
 
 def r3_gp_check(gp: GP):
     _check(load().r3_gp_check(gp.handle, _stream()))
+
+
+def r3_gp_set_wait_limit(gp: GP, cycles: int):
+    _check(load().r3_gp_set_wait_limit(gp.handle, int(cycles)))
+
+
+def r3_gp_test_withhold(gp: GP, chunk: int):
+    _check(load().r3_gp_test_withhold(gp.handle, int(chunk)))
+
+
+def r3_test_fail_allocation(after: int) -> int:
+    return int(load().r3_test_fail_allocation(int(after)))
 
 
 def r3_gp_get_best(gp: GP) -> np.ndarray:

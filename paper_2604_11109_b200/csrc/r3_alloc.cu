@@ -29,6 +29,9 @@ struct DeviceCache {
 std::mutex g_mutex;
 std::map<int, DeviceCache> g_cache;
 
+// r3_test_fail_allocation: allocations counted since arming, and the one that is to fail (-1: none)
+long long g_alloc_seen = 0, g_alloc_fail_at = -1;
+
 size_t bin_of(size_t bytes)
 {
     if (bytes < kSmall) return bytes;
@@ -55,6 +58,10 @@ cudaError_t dev_malloc_bytes(void** p, size_t bytes)
     const size_t bin = bin_of(bytes);
     {
         std::lock_guard<std::mutex> lock(g_mutex);
+        if (g_alloc_seen++ == g_alloc_fail_at) {   // test aid: this allocation is refused
+            g_alloc_fail_at = -1;
+            return cudaErrorMemoryAllocation;
+        }
         DeviceCache& c = g_cache[dev];
         auto it = c.free_blocks.find(bin);
         if (it != c.free_blocks.end()) {
@@ -167,6 +174,15 @@ size_t cached_bytes()
 extern "C" {
 
 void r3_trim_cache(void) { r3::trim_cache(); }
+
+long long r3_test_fail_allocation(long long after)
+{
+    std::lock_guard<std::mutex> lock(r3::g_mutex);
+    const long long seen = r3::g_alloc_seen;
+    r3::g_alloc_seen = 0;
+    r3::g_alloc_fail_at = after < 0 ? -1 : after;
+    return seen;
+}
 unsigned long long r3_cached_bytes(void) { return r3::cached_bytes(); }
 
 }  // extern "C"

@@ -393,12 +393,26 @@ r3_status_t r3_gp_append(r3_gp_t* gp, const float* Xnew, const float* ynew, int 
         return R3_ERR_INVALID_ARG;
     }
     cudaStream_t stream = (cudaStream_t)cuda_stream;
+    // Bits that an earlier scoring call latched (a non-finite candidate, a wait that ran out) are not this
+    // call's: they are taken out of the status word while the append's own checks use it, and put back after.
+    R3_CUDA_TRY(cudaMemcpyAsync(gp->status_h, gp->status_d, 2 * sizeof(int), cudaMemcpyDeviceToHost, stream));
+    R3_CUDA_TRY(cudaStreamSynchronize(stream));
+    const int latched = gp->status_h[0] & (DEV_NONFINITE | DEV_TIMEOUT);
+    if (latched) R3_CUDA_TRY(cudaMemsetAsync(gp->status_d, 0, sizeof(int), stream));
     r3_status_t st = append_device(gp, Xnew, ynew, k, stream);
     const int bits = gp->status_h ? gp->status_h[0] : 0;
     const int pivot = gp->status_h ? gp->status_h[1] : 0;
+    if (latched) {
+        gp->status_h[0] = latched;
+        if (cudaMemcpyAsync(gp->status_d, gp->status_h, sizeof(int), cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+            cudaStreamSynchronize(stream) != cudaSuccess) {
+            set_error("r3_gp_append: restoring the latched status failed");
+            return R3_ERR_CUDA;
+        }
+    }
     if (st == R3_OK && (bits & (DEV_NONFINITE | DEV_NOT_PD))) {
-        // the handle was not touched; clear the latch so that it stays usable
-        gp->status_h[0] = 0;
+        // the handle was not touched; clear this call's bits so that it stays usable
+        gp->status_h[0] = latched;
         gp->status_h[1] = INT_MAX;
         R3_CUDA_TRY(cudaMemcpyAsync(gp->status_d, gp->status_h, 2 * sizeof(int), cudaMemcpyHostToDevice, stream));
         R3_CUDA_TRY(cudaStreamSynchronize(stream));
@@ -417,7 +431,9 @@ r3_status_t r3_gp_append(r3_gp_t* gp, const float* Xnew, const float* ynew, int 
     tc_release(gp);
     if (tc_supported(gp->n, gp->d)) {
         st = tc_prepare(gp, stream);
-        if (st != R3_OK) return st;
+        // The history is extended at this point.  If only the tensor engine's operands could not be allocated,
+        // the append stands and the CUDA-core engine serves the handle (r3_gp_engine tells).
+        if (st != R3_OK && st != R3_ERR_ALLOC) return st;
     }
     return R3_OK;
 }
@@ -614,6 +630,30 @@ r3_status_t r3_gp_check(r3_gp_t* gp, void* cuda_stream)
         set_error("a candidate contains a non-finite value");
         return R3_ERR_NONFINITE;
     }
+    return R3_OK;
+}
+
+r3_status_t r3_gp_set_wait_limit(r3_gp_t* gp, long long cycles)
+{
+    if (!gp || cycles < 100000) {
+        set_error("r3_gp_set_wait_limit: need a handle and at least 100000 cycles");
+        return R3_ERR_INVALID_ARG;
+    }
+    gp->wait_limit_cycles = cycles;
+    return R3_OK;
+}
+
+r3_status_t r3_gp_test_withhold(r3_gp_t* gp, long long chunk)
+{
+    if (!gp || chunk < 0) {
+        set_error("r3_gp_test_withhold: need a handle and chunk >= 0");
+        return R3_ERR_INVALID_ARG;
+    }
+    if (!gp->tc) {
+        set_error("r3_gp_test_withhold: the tensor-core engine does not serve this handle");
+        return R3_ERR_UNSUPPORTED;
+    }
+    gp->withhold_w = chunk;
     return R3_OK;
 }
 

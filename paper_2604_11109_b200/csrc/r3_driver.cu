@@ -64,6 +64,10 @@ r3_status_t r3_bo_run(const float* X0, const float* y0, int n0, int d, const flo
         set_error("r3_bo_run: NULL argument");
         return R3_ERR_INVALID_ARG;
     }
+    if (n0 < 1 || n0 > kMaxN || d < 1 || d > kMaxD) {
+        set_error("r3_bo_run: need 1 <= n0 <= %d and 1 <= d <= %d (n0=%d, d=%d)", kMaxN, kMaxD, n0, d);
+        return R3_ERR_INVALID_ARG;
+    }
     const r3_bo_options_t opt = *options;
     if (opt.q < 1 || opt.q > kAppendMax || opt.max_rounds < 1 || m < 1 || m >= (1ll << 31) || (opt.lie != 0 && opt.lie != 1)) {
         set_error("r3_bo_run: need 1 <= q <= %d, max_rounds >= 1, 1 <= m < 2^31, lie in {0, 1}", kAppendMax);

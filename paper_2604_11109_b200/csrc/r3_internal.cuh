@@ -108,6 +108,10 @@ struct r3_gp {
 
     r3_engine_t engine_req = R3_ENGINE_AUTO;
 
+    // bounded device-side waits of the tensor engine: the limit in cycles, and the test aid that makes one run out
+    long long wait_limit_cycles = 4000000000ll;   // about 2 s
+    long long withhold_w = -1;
+
     // optional timing of the dominant scoring kernel: event pairs recorded around its launches
     bool profile = false;
     std::vector<cudaEvent_t> events;   // pairs (start, stop)

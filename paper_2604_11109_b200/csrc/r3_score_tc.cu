@@ -111,6 +111,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
     constexpr uint32_t ZCOL = NV + 2 * KD;
     const uint32_t KCOL = ZCOL + (uint32_t)prm.DP;
     const int DP = prm.DP, P = prm.P, ws = prm.ws;
+    const long long wl = prm.wait_limit;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < XS; ++i) {
@@ -168,7 +169,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
             const __half* src = prm.xt + (size_t)g * (prm.NP / KD) * (bytes / 2);
             for (int p = 0; ok && p < P; ++p)
                 for (int c = 0; c < (p + 1) * (NV / KD); ++c, ++issued) {
-                    if (!(ok = mbar_wait(bar(BAR_X_EMPTY + st), ph ^ 1u, abort_flag))) break;
+                    if (!(ok = mbar_wait(bar(BAR_X_EMPTY + st), ph ^ 1u, abort_flag, wl))) break;
                     mbar_arrive_expect_tx(bar(BAR_X_FULL + st), bytes);
                     bulk_g2s(base + map.x + st * bytes, src + (size_t)c * (bytes / 2), bytes, bar(BAR_X_FULL + st));
                     if (++st == XS) { st = 0; ph ^= 1u; }
@@ -178,7 +179,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
             const int pending = (int)(issued < XS ? issued : XS);
             for (int u = 0; u < pending; ++u) {
                 if (--st < 0) { st = XS - 1; ph ^= 1u; }
-                mbar_wait(bar(BAR_X_FULL + st), ph, abort_flag + 1);
+                mbar_wait(bar(BAR_X_FULL + st), ph, abort_flag + 1, wl);
             }
         }
     } else if (warp == 0 && lane == 1) {
@@ -194,7 +195,8 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
             for (int p = 0; ok && p < P; ++p) {
                 const __half* psrc = src + (size_t)(CPP * p * (p + 1) / 2) * (bytes / 2);
                 for (int c = 0; c < (p + 1) * CPP; ++c, ++issued) {
-                    if (!(ok = mbar_wait(bar(BAR_W_EMPTY + st), ph ^ 1u, abort_flag))) break;
+                    if (issued == prm.withhold_w) { ok = false; break; }   // test aid: the stream of W stops here
+                    if (!(ok = mbar_wait(bar(BAR_W_EMPTY + st), ph ^ 1u, abort_flag, wl))) break;
                     mbar_arrive_expect_tx(bar(BAR_W_FULL + st), bytes);
                     bulk_g2s(base + map.w + st * bytes, psrc + (size_t)c * (bytes / 2), bytes, bar(BAR_W_FULL + st));
                     if (++st == ws) { st = 0; ph ^= 1u; }
@@ -205,7 +207,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
             const int pending = (int)(issued < ws ? issued : ws);
             for (int u = 0; u < pending; ++u) {
                 if (--st < 0) { st = ws - 1; ph ^= 1u; }
-                mbar_wait(bar(BAR_W_FULL + st), ph, abort_flag + 1);
+                mbar_wait(bar(BAR_W_FULL + st), ph, abort_flag + 1, wl);
             }
         }
     } else if (warp == 1 && lane == 0) {
@@ -221,14 +223,14 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
         bool ok = true;
         for (long long tile = first_tile; ok && tile < prm.total_tiles; tile += tile_step, ++tile_iter) {
             TICK(7);
-            if (!(ok = mbar_wait(bar(BAR_Z_READY), (uint32_t)(tile_iter & 1), abort_flag))) break;
+            if (!(ok = mbar_wait(bar(BAR_Z_READY), (uint32_t)(tile_iter & 1), abort_flag, wl))) break;
             TICK(3);
             tc_fence_after();
             for (int u = 0; u < items_per_tile / SL; ++u) {
                 TICK(7);
-                if (!(ok = mbar_wait(bar(BAR_X_FULL + st), ph, abort_flag))) break;
+                if (!(ok = mbar_wait(bar(BAR_X_FULL + st), ph, abort_flag, wl))) break;
                 TICK(0);
-                if (!(ok = mbar_wait(bar(BAR_D_EMPTY + db), d_ph ^ 1u, abort_flag))) break;
+                if (!(ok = mbar_wait(bar(BAR_D_EMPTY + db), d_ph ^ 1u, abort_flag, wl))) break;
                 TICK(1);
                 LOGEV(8, (long long)(tile_iter * (items_per_tile / SL) + u) * SL);
                 tc_fence_after();
@@ -253,7 +255,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
         }
         // every MMA issued by this thread must have completed before TMEM is freed
         tc_commit(bar(BAR_MMA_DONE));
-        mbar_wait(bar(BAR_MMA_DONE), 0, abort_flag + 1);
+        mbar_wait(bar(BAR_MMA_DONE), 0, abort_flag + 1, wl);
         if (prm.trace)
             for (int i = 0; i < 8; ++i) prm.trace[((size_t)blockIdx.x * 4 + 3) * 8 + i] = tacc[i];
     } else if (warp == 2 && lane == 0) {
@@ -275,13 +277,13 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     const int b = k_s, s = w_s;
                     TICK(7);
                     if (c == 0) {
-                        if (!(ok = mbar_wait(bar(BAR_V_EMPTY), v_ph ^ 1u, abort_flag))) break;
+                        if (!(ok = mbar_wait(bar(BAR_V_EMPTY), v_ph ^ 1u, abort_flag, wl))) break;
                     }
                     TICK(3);
-                    if (!k_seen && !(ok = mbar_wait(bar(BAR_K_FULL + b), k_ph, abort_flag))) break;
+                    if (!k_seen && !(ok = mbar_wait(bar(BAR_K_FULL + b), k_ph, abort_flag, wl))) break;
                     TICK(4);
                     LOGEV(0, tv);
-                    if (!w_seen && !(ok = mbar_wait(bar(BAR_W_FULL + s), w_ph, abort_flag))) break;
+                    if (!w_seen && !(ok = mbar_wait(bar(BAR_W_FULL + s), w_ph, abort_flag, wl))) break;
                     LOGEV(1, tv);
                     if (++k_s == NBK) { k_s = 0; k_ph ^= 1u; }
                     if (++w_s == ws) { w_s = 0; w_ph ^= 1u; }
@@ -337,7 +339,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
             }
         }
         tc_commit(bar(BAR_MMA_DONE + 1));
-        mbar_wait(bar(BAR_MMA_DONE + 1), 0, abort_flag + 1);
+        mbar_wait(bar(BAR_MMA_DONE + 1), 0, abort_flag + 1, wl);
         if (prm.trace)
             for (int i = 0; i < 8; ++i) prm.trace[((size_t)blockIdx.x * 4 + 0) * 8 + i] = tacc[i];
     } else if (warp >= 4) {
@@ -436,7 +438,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                 tc_fence_before();
                 mbar_arrive(bar(BAR_Z_READY));
             }
-            ok = mbar_wait(bar(BAR_Z_READY), (uint32_t)(tile_iter & 1), abort_flag);
+            ok = mbar_wait(bar(BAR_Z_READY), (uint32_t)(tile_iter & 1), abort_flag, wl);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             const bool far_cand = zn_s[row] < 0.f;
@@ -464,7 +466,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                         asm volatile("prefetch.global.L1 [%0];" ::"l"(pf));
                     }
                     TICK(7);
-                    ok = mbar_wait(bar(BAR_D_FULL + db), (uint32_t)((U >> 1) & 1), abort_flag);
+                    ok = mbar_wait(bar(BAR_D_FULL + db), (uint32_t)((U >> 1) & 1), abort_flag, wl);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     TICK(0);
@@ -544,7 +546,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     TICK(2);
                     if (threadIdx.x % 128 == 0) LOGEV(4, t);
                     if (NBK == G) {
-                        ok = mbar_wait(bar(BAR_K_EMPTY + kbuf), kpar ^ 1u, abort_flag);
+                        ok = mbar_wait(bar(BAR_K_EMPTY + kbuf), kpar ^ 1u, abort_flag, wl);
                     } else if (t >= NBK) {
                         // Ring shorter than the number of groups: slot t mod NBK is free once chunk t - NBK has
                         // been consumed.  A parity wait is only valid at most one phase behind, and with one
@@ -552,7 +554,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                         // issuer two ahead of the group.  The "consumed" barriers are therefore indexed by the
                         // chunk number mod 4: the chunks 4 apart that share a barrier are never both pending.
                         const long long te = t - NBK;
-                        ok = mbar_wait(bar(BAR_K_EMPTY + (int)(te & 3)), (uint32_t)((te >> 2) & 1), abort_flag);
+                        ok = mbar_wait(bar(BAR_K_EMPTY + (int)(te & 3)), (uint32_t)((te >> 2) & 1), abort_flag, wl);
                     }
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
@@ -592,7 +594,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                 pass_base += nchunk;
                 // ---- end of pass: q += sum_i V^2 over this group's share of the columns
                 TICK(7);
-                ok = mbar_wait(bar(BAR_V_FULL), v_ph, abort_flag);
+                ok = mbar_wait(bar(BAR_V_FULL), v_ph, abort_flag, wl);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 TICK(5);
@@ -628,7 +630,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
             mine[0] = mu_acc; mine[1] = a2_acc; mine[2] = s2_acc; mine[3] = q_acc;
             mbar_arrive(bar(BAR_RED_READY));
             if (grp == 0) {   // only the finishing group waits; the others move on to the next tile
-                ok = mbar_wait(bar(BAR_RED_READY), (uint32_t)(tile_iter & 1), abort_flag);
+                ok = mbar_wait(bar(BAR_RED_READY), (uint32_t)(tile_iter & 1), abort_flag, wl);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 if (valid) {
@@ -945,8 +947,15 @@ r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream)
     dev_free(wscale_d);
     wmax_bits = nullptr;
     wscale_d = nullptr;
+    // The cap on dynamic shared memory belongs to the kernel, not to the handle, and handles with different
+    // feature counts share an instantiation with different sizes: raise it to the device's limit (the kernel
+    // has no static shared memory), so that no handle's preparation lowers it for another.
+    int smem_optin = 0;
+    if ((e = cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, gp->device)) != cudaSuccess)
+        return fail("cudaDeviceGetAttribute", e);
+    if ((size_t)smem_optin < t->smem_bytes) return decline();
     e = cudaFuncSetAttribute(kernel_for(t->NV, t->G, t->kt, t->nbk), cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)t->smem_bytes);
+                             smem_optin);
     if (e != cudaSuccess) return fail("cudaFuncSetAttribute", e);
     return R3_OK;
 }
@@ -1014,6 +1023,9 @@ r3_status_t score_tc_part(r3_gp* gp, const float* Xcand, long long m, float* mu,
     prm.tiles_per_gp = (m + TILE_M - 1) / TILE_M;
     prm.total_tiles = prm.tiles_per_gp * gp->batch;
     prm.tile_begin = 0;
+    prm.wait_limit = gp->wait_limit_cycles;
+    prm.withhold_w = gp->withhold_w;
+    gp->withhold_w = -1;   // one call only
     if (tile_end >= 0) {   // a range of the pool's tiles (the caller runs the guard once, after the last range)
         prm.tile_begin = tile_begin;
         prm.total_tiles = tile_end < prm.total_tiles ? tile_end : prm.total_tiles;

@@ -104,14 +104,14 @@ __device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t
         : "memory");
     return ok;
 }
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit)
 {
     if (mbar_try_wait_cluster(bar, parity)) return true;
     const long long t0 = clock64();
     while (true) {
         if (mbar_try_wait_cluster(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+        if (clock64() - t0 > limit) {
             *abort_flag = 1;
             return false;
         }
@@ -167,6 +167,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank(), peer = rank ^ 1u;
     const int DP = prm.DP, P = prm.P, ws = prm.ws;
+    const long long wl = prm.wait_limit;
     const int NSP = (P + 1) / 2;                       // super-passes per tile
     constexpr uint32_t TMEM_COLS = 512u;
     constexpr uint32_t ZCOL = NV2 + 2 * KD2;
@@ -229,7 +230,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
                 const int nprod = superpass_chunks(j, P) / SL2;
                 for (int u = 0; u < nprod; ++u, ++Ug) {
                     if ((uint32_t)(Ug & 1) != rank) continue;
-                    if (!(ok = mbar_wait(bar(PB_X_EMPTY + st), ph ^ 1u, abort_flag))) break;
+                    if (!(ok = mbar_wait(bar(PB_X_EMPTY + st), ph ^ 1u, abort_flag, wl))) break;
                     mbar_arrive_expect_tx(bar(PB_X_FULL + st), bytes);
                     bulk_g2s(base + map.x + st * bytes, src + (size_t)u * (bytes / 2), bytes, bar(PB_X_FULL + st));
                     ++issued;
@@ -241,7 +242,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
             const int pending = (int)(issued < XS ? issued : XS);
             for (int u = 0; u < pending; ++u) {
                 if (--st < 0) { st = XS - 1; ph ^= 1u; }
-                mbar_wait(bar(PB_X_FULL + st), ph, abort_flag + 1);
+                mbar_wait(bar(PB_X_FULL + st), ph, abort_flag + 1, wl);
             }
         }
     } else if (warp == 0 && lane == 1) {
@@ -259,7 +260,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
                 if (p >= P) continue;
                 const __half* psrc = src + (size_t)(CPP2 * p * (p + 1) / 2) * (bytes / 2);
                 for (int c = 0; c < (p + 1) * CPP2; ++c, ++issued) {
-                    if (!(ok = mbar_wait(bar(PB_W_EMPTY + st), ph ^ 1u, abort_flag))) break;
+                    if (issued == prm.withhold_w) { ok = false; break; }   // test aid: the stream of W stops here
+                    if (!(ok = mbar_wait(bar(PB_W_EMPTY + st), ph ^ 1u, abort_flag, wl))) break;
                     mbar_arrive_expect_tx(bar(PB_W_FULL + st), bytes);
                     bulk_g2s(base + map.w + st * bytes, psrc + (size_t)c * (bytes / 2), bytes, bar(PB_W_FULL + st));
                     if (++st == ws) { st = 0; ph ^= 1u; }
@@ -270,7 +272,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
             const int pending = (int)(issued < ws ? issued : ws);
             for (int u = 0; u < pending; ++u) {
                 if (--st < 0) { st = ws - 1; ph ^= 1u; }
-                mbar_wait(bar(PB_W_FULL + st), ph, abort_flag + 1);
+                mbar_wait(bar(PB_W_FULL + st), ph, abort_flag + 1, wl);
             }
         }
     } else if (warp == 1 && lane == 0) {
@@ -284,14 +286,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
         uint32_t ph = 0, d_ph = 0;
         bool ok = true;
         for (long long tile = first_tile; ok && tile < prm.total_tiles; tile += tile_step, ++tile_iter) {
-            if (!(ok = mbar_wait(bar(PB_Z_READY), (uint32_t)(tile_iter & 1), abort_flag))) break;
+            if (!(ok = mbar_wait(bar(PB_Z_READY), (uint32_t)(tile_iter & 1), abort_flag, wl))) break;
             tc_fence_after();
             for (int j = 0; ok && j < NSP; ++j) {
                 const int nprod = superpass_chunks(j, P) / SL2;
                 for (int u = 0; u < nprod; ++u, ++Ug) {
                     if ((uint32_t)(Ug & 1) != rank) continue;
-                    if (!(ok = mbar_wait(bar(PB_X_FULL + st), ph, abort_flag))) break;
-                    if (!(ok = mbar_wait(bar(PB_D_EMPTY + db), d_ph ^ 1u, abort_flag))) break;
+                    if (!(ok = mbar_wait(bar(PB_X_FULL + st), ph, abort_flag, wl))) break;
+                    if (!(ok = mbar_wait(bar(PB_D_EMPTY + db), d_ph ^ 1u, abort_flag, wl))) break;
                     tc_fence_after();
                     const uint32_t xH_lo = x_lo0 + ((st * map.x_stage) >> 4), xL_lo = xH_lo + (((uint32_t)DP * KD2 * 2u) >> 4);
                     const uint32_t dcol = tmem + NV2 + db * KD2;
@@ -312,7 +314,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
             }
         }
         tc_commit(bar(PB_MMA_DONE));
-        mbar_wait(bar(PB_MMA_DONE), 0, abort_flag + 1);
+        mbar_wait(bar(PB_MMA_DONE), 0, abort_flag + 1, wl);
     } else if (warp == 2 && lane == 0) {
         // ------------------------------------------------------------ MMA issuer: variance product (own passes)
         const uint32_t k_lo0 = desc_addr(base + map.k) | ((2048u >> 4) << 16);
@@ -334,13 +336,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
                     if (c < mine) {
                         const int s = w_s;
                         if (c == 0) {
-                            if (!(ok = mbar_wait(bar(PB_V_EMPTY), v_ph ^ 1u, abort_flag))) break;
+                            if (!(ok = mbar_wait(bar(PB_V_EMPTY), v_ph ^ 1u, abort_flag, wl))) break;
                         }
                         TICK(3);
-                        if (!(ok = mbar_wait(bar(PB_K_FULL + b), k_ph, abort_flag))) break;
+                        if (!(ok = mbar_wait(bar(PB_K_FULL + b), k_ph, abort_flag, wl))) break;
                         TICK(4);
                         LOGEV2(0, tv);
-                        if (!(ok = mbar_wait(bar(PB_W_FULL + s), w_ph, abort_flag))) break;
+                        if (!(ok = mbar_wait(bar(PB_W_FULL + s), w_ph, abort_flag, wl))) break;
                         TICK(5);
                         LOGEV2(1, tv);
                         if (++w_s == ws) { w_s = 0; w_ph ^= 1u; }
@@ -377,7 +379,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
                         LOGEV2(2, tv);
                     } else {
                         // my pass does not use this chunk: release the buffer on both CTAs once it has been filled
-                        if (!(ok = mbar_wait(bar(PB_K_FULL + b), k_ph, abort_flag))) break;
+                        if (!(ok = mbar_wait(bar(PB_K_FULL + b), k_ph, abort_flag, wl))) break;
                         mbar_arrive(bar(PB_K_EMPTY + b));
                         mbar_arrive_cluster(k_empty_peer0 + (uint32_t)b * 8u);
                         TICK(0);
@@ -387,7 +389,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
             }
         }
         tc_commit(bar(PB_MMA_DONE + 1));
-        mbar_wait(bar(PB_MMA_DONE + 1), 0, abort_flag + 1);
+        mbar_wait(bar(PB_MMA_DONE + 1), 0, abort_flag + 1, wl);
         if (prm.trace)
             for (int i = 0; i < 8; ++i) prm.trace[((size_t)blockIdx.x * 4 + 0) * 8 + i] = tacc[i];
 #ifdef R3_TC_TRACE
@@ -398,7 +400,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
         for (long long tile = first_tile; ok && tile < prm.total_tiles; tile += tile_step)
             for (int j = 0; ok && j < NSP; ++j)
                 for (int c = 0; ok && c < superpass_chunks(j, P); ++c, ++tv) {
-                    ok = mbar_wait(bar(PB_K_FULL + (int)(tv % NB)), (uint32_t)((tv / NB) & 1), abort_flag);
+                    ok = mbar_wait(bar(PB_K_FULL + (int)(tv % NB)), (uint32_t)((tv / NB) & 1), abort_flag, wl);
                     LOGEV2(11, tv);
                 }
 #endif
@@ -427,7 +429,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
                 // The candidate planes and norms of the previous tile may still be read by the other group's
                 // close-pair refinement until that group has handed in its partial sums.
                 if (tile_iter > 0) {
-                    ok = mbar_wait(bar(PB_RED_READY), (uint32_t)((tile_iter - 1) & 1), abort_flag);
+                    ok = mbar_wait(bar(PB_RED_READY), (uint32_t)((tile_iter - 1) & 1), abort_flag, wl);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                 }
@@ -486,7 +488,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
                 tc_fence_before();
                 mbar_arrive(bar(PB_Z_READY));
             }
-            ok = mbar_wait(bar(PB_Z_READY), (uint32_t)(tile_iter & 1), abort_flag);
+            ok = mbar_wait(bar(PB_Z_READY), (uint32_t)(tile_iter & 1), abort_flag, wl);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             const bool far_cand = zn_s[row] < 0.f;
@@ -504,7 +506,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
             bool epilogue_due = false;
             auto pass_epilogue = [&]() {
                 TICK(7);
-                ok = mbar_wait(bar(PB_V_FULL), v_ph, abort_flag);
+                ok = mbar_wait(bar(PB_V_FULL), v_ph, abort_flag, wl);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) return;
                 TICK(5);
@@ -541,7 +543,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
                     const uint32_t k_par = (uint32_t)((t / NB) & 1);
                     const int db = (int)(own & 1);
                     TICK(7);
-                    ok = mbar_wait(bar(PB_D_FULL + db), (uint32_t)((own >> 1) & 1), abort_flag);
+                    ok = mbar_wait(bar(PB_D_FULL + db), (uint32_t)((own >> 1) & 1), abort_flag, wl);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     TICK(0);
@@ -614,7 +616,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
                     // both CTAs must have finished with the previous chunk in this ring position
                     TICK(2);
                     if (q4 == 0 && lane == 0) LOGEV2(4, t);
-                    ok = mbar_wait_cluster(bar(PB_K_EMPTY + b), k_par ^ 1u, abort_flag);
+                    ok = mbar_wait_cluster(bar(PB_K_EMPTY + b), k_par ^ 1u, abort_flag, wl);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     TICK(3);
@@ -665,7 +667,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
             mine[0] = mu_acc; mine[1] = a2_acc; mine[2] = s2_acc; mine[3] = q_acc;
             mbar_arrive(bar(PB_RED_READY));
             if (grp == 0) {
-                ok = mbar_wait(bar(PB_RED_READY), (uint32_t)(tile_iter & 1), abort_flag);
+                ok = mbar_wait(bar(PB_RED_READY), (uint32_t)(tile_iter & 1), abort_flag, wl);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 mu_acc = a2_acc = s2_acc = q_acc = 0.0;
@@ -682,7 +684,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
                     st_cluster_f64(slot + 24, q_acc);
                     mbar_arrive_cluster(map_to_cta(bar(PB_RED_PEER), 0));
                 } else {
-                    ok = mbar_wait_cluster(bar(PB_RED_PEER), (uint32_t)(tile_iter & 1), abort_flag);
+                    ok = mbar_wait_cluster(bar(PB_RED_PEER), (uint32_t)(tile_iter & 1), abort_flag, wl);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
                     if (valid) {

@@ -46,6 +46,9 @@ struct TcParams {
     long long tiles_per_gp, total_tiles;   // total_tiles: one past the last tile of this launch
     long long tile_begin;                  // first tile of this launch (the single-CTA kernel; 0 for a whole pool)
     long long* trace;   // optional [grid][4 roles][8] cycle counters (diagnostics)
+    long long wait_limit;   // cycles after which a device-side wait gives up (r3_gp_set_wait_limit)
+    long long withhold_w;   // >= 0: every CTA's stream of W stops before that chunk of its own sequence, so that the
+                            // consumer's wait runs out (r3_gp_test_withhold, one call); -1 otherwise
 };
 
 // paired (two-CTA cluster) form of the tensor kernel, r3_score_tc2.cu
@@ -58,7 +61,6 @@ constexpr int KC = 32;        // observations per chunk of the variance product
 constexpr int TILE_M = 128;   // candidates per CTA tile
 constexpr int XS = 2;         // stages of scaled observations
 constexpr int MAX_STAGES = 6; // stages of W
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;  // ~2 s
 
 // Scaled coordinates are x^ = (x - centre) * sqrt(5) log2(e) / lengthscale, so that u = |z^ - x^| is the
 // Matern argument in base-2 units: s = sqrt(5) r = u ln 2, exp(-s) = 2^-u, 1 + s + s^2/3 = 1 + c1 u + c2 u^2.
@@ -106,14 +108,14 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok;
 }
 // Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+        if (clock64() - t0 > limit) {
             *abort_flag = 1;
             return false;
         }

@@ -280,12 +280,35 @@ def _sampled_check(c, g, out, per_gp):
         yield q, f, pick, ei_r
 
 
+_CFG3_ORACLE = {}
+
+
+def _cfg3_oracle(c, g):
+    """The oracle's mu, sigma, EI of every candidate of all 64 pools (scored once, shared by both engines)."""
+    if not _CFG3_ORACLE:
+        _CFG3_ORACLE["scores"] = oracle_all(g)[1:]
+    return _CFG3_ORACLE["scores"]
+
+
 @pytest.mark.parametrize("engine", ENGINES)
-def test_workload_cfg3_batched_full_size_sampled(engine):
+def test_workload_cfg3_batched_full_size_every_candidate(engine):
+    """All 64 GPs at full size: every candidate of every pool against the oracle, and each GP's top-k under the
+    top-k rule, against the oracle's EI of the whole pool and against the stored top list."""
     c = w.get_config(3)
-    g, out = _run_full(c, engine)
-    for _ in _sampled_check(c, g, out, 256):
-        pass
+    g, (mu, sd, ei, idx, val) = _run_full(c, engine)
+    mu_r, sd_r, ei_r = _cfg3_oracle(c, g)
+    gold = json.load(open(os.path.join(GOLDEN, f"topk_{c.name}.json")))
+    assert gold["m"] == c.m and gold["n"] == c.n and gold["seed"] == c.seed and gold["batch"] == c.batch
+    for q in range(c.batch):
+        check_scores(mu[q], sd[q], ei[q], mu_r[q], sd_r[q], ei_r[q], float(np.abs(g["y"][q]).max()),
+                     float(g["sf2"][q]), what=f"{c.name} gp{q}")
+        ridx, rval = o.topk(ei_r[q], c.k + 1)
+        check_topk(idx[q], lambda i, q=q: ei_r[q][i], ridx[:c.k], rval[:c.k], rval[c.k], ei_r[q].max(),
+                   what=f"{c.name} gp{q}")
+        # the stored list is this oracle's
+        gq = gold["gps"][q]
+        assert gq["idx"][:c.k + 1] == ridx.tolist() and float(gq["ei_max"]) == float(ei_r[q].max())
+        assert np.array_equal(val[q], ei[q][idx[q]])
 
 
 @pytest.mark.parametrize("engine", ENGINES)

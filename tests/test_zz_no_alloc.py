@@ -10,6 +10,7 @@ import ctypes
 import numpy as np
 import pytest
 
+from oracle import gp_oracle as o
 from paper_2604_11109_b200 import binding as b
 
 torch = pytest.importorskip("torch")
@@ -34,6 +35,12 @@ def test_noalloc_equals_topk_on_two_calls_in_a_row(batch, m, k):
         torch.cuda.synchronize()
         assert torch.equal(idx, ref_idx)     # integer work: bit-exact
         assert torch.equal(val, ref_val)
+        # and against the oracle's definition of the selection itself
+        e_h, idx_h = e.cpu().numpy(), idx.cpu().numpy()
+        for q in range(batch):
+            oidx, oval = o.topk(e_h[q], k)
+            assert np.array_equal(idx_h[q], oidx)
+            assert np.array_equal(val.cpu().numpy()[q], oval.astype(np.float32))
 
 
 def test_noalloc_rejects_requests_beyond_its_fixed_capacity():
