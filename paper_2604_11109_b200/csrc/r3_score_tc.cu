@@ -86,7 +86,9 @@ constexpr uint32_t kZnOffset = 512;                   // float[128] squared norm
 // NBK: number of k* buffers.  NBK == G: group g owns buffer g.  NBK < G (k* in TMEM, where columns are
 // scarce): the buffers form a ring shared by the groups, chunk t uses buffer t mod NBK; a group that has
 // computed its chunk keeps it in registers until the ring slot is free, so the groups still run ahead.
-template <int NV, int G, int KD, bool KT, int NBK = G>
+// F8: the two cross terms of the variance product (W_hi k_lo, W_lo k_hi) are single E4M3 MMAs of depth 32
+// instead of two FP16 MMAs of depth 16 each: four MMAs per chunk instead of six.
+template <int NV, int G, int KD, bool KT, int NBK = G, bool F8 = false>
 __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcParams prm)
 {
     static_assert(NBK == G || (KT && NBK >= 2 && NBK < G), "ring of k* buffers: TMEM only");
@@ -295,7 +297,30 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     const uint32_t idesc_v = instr_desc_f16(NV - skip);
                     const uint32_t vcol = tmem + skip;
                     const uint32_t bH = w_lo0 + ((s * map.w_stage) >> 4) + skip, bL = bH + (((uint32_t)KC * NV * 2u) >> 4);
-                    if (KT) {
+                    if (F8) {
+                        // main term: FP16 hi x hi, two MMAs of depth 16; cross terms: one E4M3 MMA of depth 32 each
+                        // (planes after the FP16 hi plane: scaled hi parts, then scaled lo parts)
+                        const uint32_t first = c > 0 ? 1u : 0u;
+                        const uint32_t b8H = bH + (((uint32_t)KC * NV * 2u) >> 4), b8L = b8H + (((uint32_t)KC * NV) >> 4);
+                        if (KT) {
+                            const uint32_t aH = tmem + KCOL + (uint32_t)b * KC;
+                            tc_mma_f16_ts(vcol, aH, pack64(bH, kDescHi), idesc_v, first);
+                            tc_mma_f16_ts(vcol, aH + 8u, pack64(bH + ((2u * NV * 16u) >> 4), kDescHi), idesc_v, 1u);
+                            tc_mma_f8_ts(vcol, aH + KC / 2, pack64(b8L, kDescHi), idesc_v, 1u);
+                            k_seen = mbar_try_wait(bar(BAR_K_FULL + k_s), k_ph);
+                            w_seen = mbar_try_wait(bar(BAR_W_FULL + w_s), w_ph);
+                            tc_mma_f8_ts(vcol, aH + KC / 2 + KC / 4, pack64(b8H, kDescHi), idesc_v, 1u);
+                        } else {
+                            const uint32_t aH = k_lo0 + ((b * 16384u) >> 4), a8H = aH + (8192u >> 4), a8L = a8H + (4096u >> 4);
+                            tc_mma_f16(vcol, pack64(aH, kDescHi), pack64(bH, kDescHi), idesc_v, first);
+                            tc_mma_f16(vcol, pack64(aH + (4096u >> 4), kDescHi), pack64(bH + ((2u * NV * 16u) >> 4), kDescHi),
+                                       idesc_v, 1u);
+                            tc_mma_f8(vcol, pack64(a8H, kDescHi), pack64(b8L, kDescHi), idesc_v, 1u);
+                            k_seen = mbar_try_wait(bar(BAR_K_FULL + k_s), k_ph);
+                            w_seen = mbar_try_wait(bar(BAR_W_FULL + w_s), w_ph);
+                            tc_mma_f8(vcol, pack64(a8L, kDescHi), pack64(b8H, kDescHi), idesc_v, 1u);
+                        }
+                    } else if (KT) {
                         const uint32_t aH = tmem + KCOL + (uint32_t)b * KC, aL = aH + KC / 2;
 #pragma unroll
                         for (int combo = 0; combo < 3; ++combo) {
@@ -535,12 +560,19 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                         }
                         // split into the two FP16 planes; the stores wait until the whole chunk is computed
                         // so that the arithmetic does not sit between the buffer's release and its refill
+                        if (F8) {
+                            // kl[h][0..3]: the 16 scaled hi parts as E4M3, kl[h][4..7]: the 16 scaled lo parts
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            __half2 hi, lo;
-                            split2(kv[2 * e], kv[2 * e + 1], hi, lo);
-                            kh[h][e] = *reinterpret_cast<const uint32_t*>(&hi);
-                            kl[h][e] = *reinterpret_cast<const uint32_t*>(&lo);
+                            for (int e = 0; e < 4; ++e)
+                                split4_f8(kv + 4 * e, kh[h][2 * e], kh[h][2 * e + 1], kl[h][e], kl[h][4 + e]);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) {
+                                __half2 hi, lo;
+                                split2(kv[2 * e], kv[2 * e + 1], hi, lo);
+                                kh[h][e] = *reinterpret_cast<const uint32_t*>(&hi);
+                                kl[h][e] = *reinterpret_cast<const uint32_t*>(&lo);
+                            }
                         }
                     }
                     TICK(2);
@@ -560,6 +592,31 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     if (!ok) break;
                     TICK(3);
                     if (threadIdx.x % 128 == 0) LOGEV(5, t);
+                    if (F8) {
+                        if (KT) {
+                            // FP16 hi plane: 16 columns; then the chunk's 32 E4M3 hi parts (8 columns) and lo parts (8)
+                            uint32_t p8[8];
+                            tc_st8(lane_addr + KCOL + (uint32_t)kbuf * KC, kh[0]);
+                            tc_st8(lane_addr + KCOL + (uint32_t)kbuf * KC + 8, kh[1]);
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) { p8[e] = kl[0][e]; p8[4 + e] = kl[1][e]; }
+                            tc_st8(lane_addr + KCOL + (uint32_t)kbuf * KC + KC / 2, p8);
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) { p8[e] = kl[0][4 + e]; p8[4 + e] = kl[1][4 + e]; }
+                            tc_st8(lane_addr + KCOL + (uint32_t)kbuf * KC + KC / 2 + KC / 4, p8);
+                        } else {
+#pragma unroll
+                            for (int h = 0; h < KC / 16; ++h) {
+#pragma unroll
+                                for (int sl = 0; sl < 2; ++sl)
+                                    *reinterpret_cast<uint4*>(kb + (2 * h + sl) * 2048u) =
+                                        make_uint4(kh[h][4 * sl], kh[h][4 * sl + 1], kh[h][4 * sl + 2], kh[h][4 * sl + 3]);
+                                // one 16-byte k-slice of each E4M3 plane per 16 observations
+                                *reinterpret_cast<uint4*>(kb + 8192u + h * 2048u) = make_uint4(kl[h][0], kl[h][1], kl[h][2], kl[h][3]);
+                                *reinterpret_cast<uint4*>(kb + 12288u + h * 2048u) = make_uint4(kl[h][4], kl[h][5], kl[h][6], kl[h][7]);
+                            }
+                        }
+                    } else
 #pragma unroll
                     for (int h = 0; h < KC / 16; ++h) {
                         if (KT) {
@@ -649,7 +706,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     const double eps =
                         far_cand ? 1.0 : kEpsTc0 + kEpsTc1 * (double)(zn + prm.xnmax[g]) * rsqrt((double)DP);
                     prm.err_mu[f] = mu_error_estimate(eps, a2_acc);
-                    prm.err_q[f] = q_error_estimate(eps, prm.wnorm[g], q_acc, s2_acc);
+                    prm.err_q[f] = q_error_estimate(F8 && !far_cand ? eps + kEpsF8 : eps, prm.wnorm[g], q_acc, s2_acc);
                 }
             }
         }
@@ -761,8 +818,10 @@ __global__ void wmax_kernel(const double* __restrict__ W64, int n, int npad_fit,
 
 // One block per (chunk c, pass p, GP): the KC x NV block of 2^eW W (rows p NV.., columns c KC..) as
 // FP16 hi/lo planes in the B-operand layout; zero outside the lower triangle and outside n.
+// With f8 the second plane holds, instead of the FP16 lo parts, two E4M3 planes in the 8-bit form of the same
+// layout (16 k-elements per 16-byte slice): the hi parts times 2^-6, then the lo parts times 2^6.
 __global__ void wt_build_kernel(const double* __restrict__ W64, int n, int npad_fit, int NV, size_t gp_stride,
-                                const float* __restrict__ wscale, __half* __restrict__ wt)
+                                const float* __restrict__ wscale, __half* __restrict__ wt, bool f8)
 {
     const int c = blockIdx.x, p = blockIdx.y, g = blockIdx.z;
     const int CPP = NV / KC;
@@ -779,14 +838,27 @@ __global__ void wt_build_kernel(const double* __restrict__ W64, int n, int npad_
         const __half h = __float2half_rn(w);
         const size_t off = ((size_t)(kk / 8) * NV + r) * 8 + (kk % 8);
         dst[off] = h;
-        dst[(size_t)KC * NV + off] = __float2half_rn(w - __half2float(h));
+        if (f8) {
+            uint8_t* d8 = reinterpret_cast<uint8_t*>(dst + (size_t)KC * NV);
+            const size_t off8 = ((size_t)(kk / 16) * NV + r) * 16 + (kk % 16);
+            const float hf = __half2float(h);
+            d8[off8] = (uint8_t)(e4m3x4(hf * kF8HiScale, 0.f, 0.f, 0.f) & 0xffu);
+            d8[(size_t)KC * NV + off8] = (uint8_t)(e4m3x4((w - hf) * kF8LoScale, 0.f, 0.f, 0.f) & 0xffu);
+        } else {
+            dst[(size_t)KC * NV + off] = __float2half_rn(w - __half2float(h));
+        }
     }
 }
 
 TensorOperands* ops_of(const r3_gp* gp) { return static_cast<TensorOperands*>(gp->tc); }
 
-void (*kernel_for(int NV, int G, bool kt, int nbk))(const TcParams)
+void (*kernel_for(int NV, int G, bool kt, int nbk, bool f8))(const TcParams)
 {
+    if (f8) {   // offered for the shapes of long histories only (tc_prepare)
+        if (kt && nbk == 2 && G == 3) return score_tc_kernel<256, 3, 64, true, 2, true>;
+        if (kt) return G == 3 ? score_tc_kernel<256, 3, 64, true, 3, true> : score_tc_kernel<256, 2, 64, true, 2, true>;
+        return G == 3 ? score_tc_kernel<256, 3, 64, false, 3, true> : score_tc_kernel<256, 2, 64, false, 2, true>;
+    }
     if (kt && nbk == 2 && G == 3)
         return NV == 256 ? score_tc_kernel<256, 3, 64, true, 2> : score_tc_kernel<128, 3, 64, true, 2>;
     if (kt) {
@@ -796,6 +868,8 @@ void (*kernel_for(int NV, int G, bool kt, int nbk))(const TcParams)
     if (NV == 256) return G == 3 ? score_tc_kernel<256, 3, 64, false> : score_tc_kernel<256, 2, 64, false>;
     return G == 3 ? score_tc_kernel<128, 3, 64, false> : score_tc_kernel<128, 2, 64, false>;
 }
+
+constexpr int kF8MinPasses = 4;
 
 int env_int(const char* name, int fallback)
 {
@@ -868,6 +942,9 @@ r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream)
         return R3_OK;
     }
     t->smem_bytes = smem_map(t->DP, t->NV, t->G, t->KD, t->ws, t->kt).bar + kBarBytes + 1024;
+    // FP8 cross terms: R3_TC_F8 = 0/1 decides; by default histories of at least kF8MinPasses passes take them
+    const int want_f8 = env_int("R3_TC_F8", -1);
+    t->f8 = t->NV == 256 && (want_f8 >= 0 ? want_f8 != 0 : t->P >= kF8MinPasses);
     const int CPP = t->NV / KC;
     const size_t tiles = (size_t)CPP * t->P * (t->P + 1) / 2;
     t->wt_gp_stride = tiles * (2 * (size_t)KC * t->NV);
@@ -939,7 +1016,7 @@ r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream)
         return fail("cudaMemcpyAsync", e);
     xnmax_kernel<<<B, 256, 0, stream>>>(t->xnorm, t->NP, t->xnmax);
     wt_build_kernel<<<dim3(t->P * CPP, t->P, B), 256, 0, stream>>>(gp->W64, n, gp->npad, t->NV, t->wt_gp_stride,
-                                                                   wscale_d, t->wt);
+                                                                   wscale_d, t->wt, t->f8);
     g_launches += 2;
     if ((e = cudaGetLastError()) != cudaSuccess) return fail("operand preparation launch", e);
     if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return fail("operand preparation", e);
@@ -954,7 +1031,7 @@ r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream)
     if ((e = cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, gp->device)) != cudaSuccess)
         return fail("cudaDeviceGetAttribute", e);
     if ((size_t)smem_optin < t->smem_bytes) return decline();
-    e = cudaFuncSetAttribute(kernel_for(t->NV, t->G, t->kt, t->nbk), cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(kernel_for(t->NV, t->G, t->kt, t->nbk, t->f8), cudaFuncAttributeMaxDynamicSharedMemorySize,
                              smem_optin);
     if (e != cudaSuccess) return fail("cudaFuncSetAttribute", e);
     return R3_OK;
@@ -1044,13 +1121,13 @@ r3_status_t score_tc_part(r3_gp* gp, const float* Xcand, long long m, float* mu,
     // The paired kernel (two CTAs of a cluster share a tile and the k* chunks) serves histories with at least
     // two passes; R3_TC_PAIR=0/1 overrides the choice.
     int pair_ws = 0;
-    const bool pair = tile_end < 0 && env_int("R3_TC_PAIR", 0) != 0 && tc_pair_fits(t, &pair_ws);
+    const bool pair = tile_end < 0 && !t->f8 && env_int("R3_TC_PAIR", 0) != 0 && tc_pair_fits(t, &pair_ws);
     prof_begin(gp, stream);
     if (pair) {
         const r3_status_t st = launch_tc_pair(t, prm, sms, stream);
         if (st != R3_OK) return st;
     } else {
-        void (*kernel)(const TcParams) = kernel_for(t->NV, t->G, t->kt, t->nbk);
+        void (*kernel)(const TcParams) = kernel_for(t->NV, t->G, t->kt, t->nbk, t->f8);
         R3_LAUNCH(kernel, grid, 128 + 128 * t->G, t->smem_bytes, stream, prm);
     }
     prof_end(gp, stream);
