@@ -407,7 +407,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                 }
                 const float* cen = prm.centre + (size_t)g * DP;
                 const float* scl = prm.scale + (size_t)g * DP;
-                const bool vec = (prm.d % 4) == 0;
+                const bool vec = (prm.d % 4) == 0 && (reinterpret_cast<uintptr_t>(prm.xcand) & 15) == 0;
                 uint32_t zh[8], zl[8];
                 for (int j8 = 0; j8 < DP / 8; ++j8) {
                     __half2 hi2[4], lo2[4];
@@ -869,7 +869,7 @@ void (*kernel_for(int NV, int G, bool kt, int nbk, bool f8))(const TcParams)
     return G == 3 ? score_tc_kernel<128, 3, 64, false> : score_tc_kernel<128, 2, 64, false>;
 }
 
-constexpr int kF8MinPasses = 4;
+constexpr int kF8MinPasses = 8;   // n > 1792: below that the guard hands more candidates to the FP64 pass than the cheaper MMAs save
 
 int env_int(const char* name, int fallback)
 {

@@ -439,7 +439,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
                 const float* zrow = prm.xcand + ((size_t)g * prm.m + (valid ? cand : 0)) * prm.d;
                 const float* cen = prm.centre + (size_t)g * DP;
                 const float* scl = prm.scale + (size_t)g * DP;
-                const bool vec = (prm.d % 4) == 0;
+                const bool vec = (prm.d % 4) == 0 && (reinterpret_cast<uintptr_t>(prm.xcand) & 15) == 0;
                 uint32_t zh[8], zl[8];
                 for (int j8 = 0; j8 < DP / 8; ++j8) {
                     __half2 hi2[4], lo2[4];
