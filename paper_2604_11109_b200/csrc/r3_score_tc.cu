@@ -66,7 +66,9 @@ __host__ __device__ inline SmemMap smem_map(int DP, int NV, int G, int KD, int w
     s.bar = s.w + (uint32_t)ws * s.w_stage;
     return s;
 }
-constexpr uint32_t kBarBytes = 1024;   // barriers, flags, TMEM slot, candidate norms
+// barriers, flags, TMEM slot, candidate norms; then the tile's cache of refined close pairs
+constexpr uint32_t kCacheOffset = 1024;
+constexpr uint32_t kBarBytes = kCacheOffset + TILE_M * kCacheSlots * 8;
 
 // barrier slots (8 bytes each) inside the barrier block
 enum : uint32_t {
@@ -101,6 +103,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + map.bar + kFlagOffset);
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + map.bar + kFlagOffset + 8);
     float* zn_s = reinterpret_cast<float*>(sm + map.bar + kZnOffset);
+    unsigned long long* pair_cache = reinterpret_cast<unsigned long long*>(sm + map.bar + kCacheOffset);
     auto bar = [&](uint32_t slot) { return bars + slot * 8u; };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -138,6 +141,11 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
         mbar_init(bar(BAR_MMA_DONE + 1), 1);
         abort_flag[0] = 0;
         abort_flag[1] = 0;   // private flag of the bounded drain waits
+    }
+    if (threadIdx.x < TILE_M * kCacheSlots / 4) {   // no entry yet: a key that no (tile, observation) forms
+        for (int i = 0; i < 4; ++i) pair_cache[threadIdx.x * 4 + i] = ~0ull;
+    }
+    if (threadIdx.x == 0) {
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 2) {
@@ -531,14 +539,42 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                         for (int i = 4; i < 16; i += 4)
                             vmax = fmaxf(vmax, fmaxf(fmaxf(kv[i], kv[i + 1]), fmaxf(kv[i + 2], kv[i + 3])));
                         if (__any_sync(0xffffffffu, vmax > v_thresh)) {
-                            // rare: hand the 16 values to the out-of-line refinement through a local array so
-                            // that the hot path keeps kv in registers
-                            float tmp[16];
+                            // rare: close pairs.  Values refined in an earlier pass of this tile come back from the
+                            // cache without a call; what is left goes to the out-of-line refinement through a local
+                            // array, so that the hot path keeps kv in registers.
+                            const uint32_t key0 = (((uint32_t)tile_iter & 0x3ffffu) << 13) | (uint32_t)(c * KC + h * 16);
+                            unsigned long long* slots = P > 1 ? pair_cache + row * kCacheSlots : nullptr;
+                            bool need = vmax > v_thresh;
+                            if (need && slots && !fresh) {
+                                uint32_t marked = 0;
 #pragma unroll
-                            for (int i = 0; i < 16; ++i) tmp[i] = kv[i];
-                            refine_close_pairs(tmp, v_thresh, kvscale, lane_addr + ZCOL, DP, xs_g + (size_t)(c * KC + h * 16) * DP);
+                                for (int i = 0; i < 16; ++i) marked |= (kv[i] > v_thresh) ? (1u << i) : 0u;
+                                need = false;
+                                for (; marked; marked &= marked - 1) {
+                                    const uint32_t i = (uint32_t)__ffs(marked) - 1u;
+                                    const unsigned long long e = slots[cache_slot(key0 + i)];
+                                    if ((uint32_t)(e >> 32) != key0 + i) {
+                                        need = true;
+                                        break;
+                                    }
+                                    const float val = __uint_as_float((uint32_t)e);
 #pragma unroll
-                            for (int i = 0; i < 16; ++i) kv[i] = tmp[i];
+                                    for (int e2 = 0; e2 < 16; ++e2) kv[e2] = (uint32_t)e2 == i ? val : kv[e2];
+                                }
+                            }
+                            if (__any_sync(0xffffffffu, need)) {
+                                float tmp[16];
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) tmp[i] = kv[i];
+                                if (slots)
+                                    refine_close_pairs<true>(tmp, v_thresh, kvscale, lane_addr + ZCOL, DP,
+                                                             xs_g + (size_t)(c * KC + h * 16) * DP, slots, key0, !fresh);
+                                else
+                                    refine_close_pairs<false>(tmp, v_thresh, kvscale, lane_addr + ZCOL, DP,
+                                                              xs_g + (size_t)(c * KC + h * 16) * DP, nullptr, 0u, false);
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) kv[i] = tmp[i];
+                            }
                         }
                         if (fresh) {   // warp-uniform: the mean and the error scales see every observation once
                             float mpart = 0.f, apart = 0.f, spart = 0.f;

@@ -583,7 +583,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(128 + 128 * G2, 1) s
                             float tmp[16];
 #pragma unroll
                             for (int i = 0; i < 16; ++i) tmp[i] = kv[i];
-                            refine_close_pairs(tmp, v_thresh, kvscale, lane_addr + ZCOL, DP, xs_g + (size_t)(c * KC + h * 16) * DP);
+                            refine_close_pairs<false>(tmp, v_thresh, kvscale, lane_addr + ZCOL, DP, xs_g + (size_t)(c * KC + h * 16) * DP, nullptr, 0u, false);
 #pragma unroll
                             for (int i = 0; i < 16; ++i) kv[i] = tmp[i];
                         }

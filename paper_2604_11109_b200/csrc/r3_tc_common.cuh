@@ -306,12 +306,34 @@ __device__ __forceinline__ constexpr uint32_t instr_desc_f16(uint32_t n)
 // computed from r^2 = sum_j (z~_j - x~_j)^2, with z~ = hi + lo read back from the TMEM planes at z_taddr
 // and x~ in FP32 from global memory.  Called by all 32 lanes of a warp together (TMEM loads are
 // warp-wide); a lane without marked pairs only takes part in the loads.
+// Refined values are kept for the later passes of the same tile (k* chunks are regenerated for every pass, and this
+// path is what a regeneration costs most: the warp that takes it holds up its group and then the MMA issuer).
+// `slots`: the candidate row's kCacheSlots direct-mapped entries (key << 32 | value bits) in shared memory, or
+// nullptr; key0 + i identifies (tile, observation) of kv[i]; `lookup`: earlier passes may have left the values.
+// An overwritten slot is a miss, and a miss is recomputed.
+constexpr uint32_t kCacheSlots = 4;
+__device__ __forceinline__ uint32_t cache_slot(uint32_t key) { return (key + (key >> 4)) & (kCacheSlots - 1); }
+template <bool CACHE>
 __device__ __noinline__ void refine_close_pairs(float* kv, float v_thresh, float kvscale, uint32_t z_taddr, int DP,
-                                                const float* __restrict__ xrow0)
+                                                const float* __restrict__ xrow0, unsigned long long* slots,
+                                                uint32_t key0, bool lookup)
 {
     uint32_t close = 0;
 #pragma unroll
     for (int i = 0; i < 16; ++i) close |= (kv[i] > v_thresh) ? (1u << i) : 0u;
+    if (CACHE && lookup) {
+        uint32_t missing = 0;
+        for (uint32_t rest = close; rest; rest &= rest - 1) {
+            const int i = __ffs(rest) - 1;
+            const unsigned long long e = slots[cache_slot(key0 + i)];
+            if ((uint32_t)(e >> 32) == key0 + i)
+                kv[i] = __uint_as_float((uint32_t)e);
+            else
+                missing |= 1u << i;
+        }
+        if (!__any_sync(0xffffffffu, missing != 0)) return;
+        close = missing;
+    }
     float r2x[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) r2x[i] = 0.f;
@@ -351,6 +373,7 @@ __device__ __noinline__ void refine_close_pairs(float* kv, float v_thresh, float
         const int i = __ffs(rest) - 1;
         const float u = sqrtf(r2x[i]);
         kv[i] = kvscale * fmaf(u, fmaf(u, kPolyC2, kPolyC1), 1.f) * exp2f(-u);
+        if (CACHE) slots[cache_slot(key0 + i)] = ((unsigned long long)(key0 + i) << 32) | __float_as_uint(kv[i]);
     }
 }
 
@@ -366,6 +389,9 @@ constexpr long long kLogT0 = 1088 + 600, kLogN = 128;
         if (prm.trace && blockIdx.x == 0 && (tt) >= kLogT0 && (tt) < kLogT0 + kLogN)                          \
             prm.trace[(size_t)gridDim.x * 32 + (ev) * kLogN + ((tt) - kLogT0)] = clock64();                   \
     } while (0)
+#ifdef R3_TC_TRACE_EVENTS_ONLY
+#define TICK(cat) do { } while (0)
+#else
 #define TICK(cat)                                                                          \
     do {                                                                                   \
         if (prm.trace) {                                                                   \
@@ -374,6 +400,7 @@ constexpr long long kLogT0 = 1088 + 600, kLogN = 128;
             tlast = now__;                                                                 \
         }                                                                                  \
     } while (0)
+#endif
 #endif
 
 }  // namespace
