@@ -59,6 +59,8 @@ void prof_end(r3_gp* gp, cudaStream_t stream)
     gp->events_used += 2;
 }
 
+constexpr int kAutoSimtMaxD = 8, kAutoSimtMaxN = 128;
+
 static r3_engine_t pick_engine(const r3_gp* gp)
 {
     const bool tc_ok = gp->tc != nullptr;
@@ -66,6 +68,10 @@ static r3_engine_t pick_engine(const r3_gp* gp)
         case R3_ENGINE_SIMT: return R3_ENGINE_SIMT;
         case R3_ENGINE_TENSOR: return tc_ok ? R3_ENGINE_TENSOR : R3_ENGINE_SIMT;
         default:
+            // Few features and a short history: the squared distance by direct differences costs next to nothing
+            // and keeps full FP32 accuracy for the near pairs such pools are full of, whereas the norm expansion
+            // of the tensor path sends a third of a pool like that to the FP64 pass.
+            if (gp->d <= kAutoSimtMaxD && gp->n <= kAutoSimtMaxN) return R3_ENGINE_SIMT;
             return tc_ok ? R3_ENGINE_TENSOR : R3_ENGINE_SIMT;
     }
 }
@@ -514,13 +520,19 @@ r3_status_t r3_gp_score_topk(r3_gp_t* gp, const float* Xcand, long long m, int k
     st = check_topk_args(ei, gp->batch, m, k, idx);
     if (st != R3_OK) return st;
     const size_t sb = align256(score_workspace_bytes(gp, m));
-    const size_t tb = topk_workspace_bytes(gp->batch, m, k);
+    const size_t tb = guard_topk_workspace_bytes(gp->batch, m, k);
     st = ensure_workspace(gp, sb + tb);
     if (st != R3_OK) return st;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
+    // the selection rides on the scoring call: its first level is taken by the guard's kernel
+    gp->topk_req.k = k;
+    gp->topk_req.idx = idx;
+    gp->topk_req.val = val;
+    gp->topk_req.ws = (char*)gp->ws + sb;
+    gp->topk_req.ws_bytes = tb;
     st = run_score(gp, Xcand, m, mu, sigma, ei, gp->ws, sb, stream);
-    if (st != R3_OK) return st;
-    return topk_device(ei, gp->batch, m, k, idx, val, (char*)gp->ws + sb, tb, stream);
+    gp->topk_req = TopkRequest();
+    return st;
 }
 
 r3_status_t r3_gp_score_topk_host(r3_gp_t* gp, const float* Xcand_host, long long m, int k, float* mu_host,
@@ -537,7 +549,7 @@ r3_status_t r3_gp_score_topk_host(r3_gp_t* gp, const float* Xcand_host, long lon
     }
     const size_t B = gp->batch;
     const size_t sb = align256(score_workspace_bytes(gp, m));
-    const size_t tb = align256(topk_workspace_bytes(gp->batch, m, k));
+    const size_t tb = align256(guard_topk_workspace_bytes(gp->batch, m, k));
     const size_t xb = align256(sizeof(float) * B * m * gp->d);
     const size_t ob = align256(sizeof(float) * B * m);
     const size_t kb = align256(sizeof(float) * B * k);
@@ -556,6 +568,15 @@ r3_status_t r3_gp_score_topk_host(r3_gp_t* gp, const float* Xcand_host, long lon
     int* idx = (int*)p;
     p += kb;
     float* val = (float*)p;
+    gp->topk_req.k = k;
+    gp->topk_req.idx = idx;
+    gp->topk_req.val = val;
+    gp->topk_req.ws = (char*)gp->ws + sb;
+    gp->topk_req.ws_bytes = tb;
+    struct ClearRequest {
+        r3_gp* gp;
+        ~ClearRequest() { gp->topk_req = TopkRequest(); }
+    } clear_request{gp};
     // On the tensor engine a pool of several pieces travels on a second stream while the earlier pieces are
     // scored (a piece is about seven full waves of tiles on 148 SMs, so that no launch ends on a nearly empty
     // wave); the accuracy guard runs once over the whole pool, as in the device-buffer call, and the results are
@@ -600,8 +621,6 @@ r3_status_t r3_gp_score_topk_host(r3_gp_t* gp, const float* Xcand_host, long lon
         st = run_score(gp, xc, m, mu, sg, e, gp->ws, sb, stream);
         if (st != R3_OK) return st;
     }
-    st = topk_device(e, gp->batch, m, k, idx, val, (char*)gp->ws + sb, tb, stream);
-    if (st != R3_OK) return st;
     if (mu_host) R3_CUDA_TRY(cudaMemcpyAsync(mu_host, mu, sizeof(float) * B * m, cudaMemcpyDeviceToHost, stream));
     if (sigma_host) R3_CUDA_TRY(cudaMemcpyAsync(sigma_host, sg, sizeof(float) * B * m, cudaMemcpyDeviceToHost, stream));
     if (ei_host) R3_CUDA_TRY(cudaMemcpyAsync(ei_host, e, sizeof(float) * B * m, cudaMemcpyDeviceToHost, stream));

@@ -72,6 +72,16 @@ inline long long round_up_ll(long long a, long long b) { return (a + b - 1) / b 
 
 }  // namespace r3
 
+// A top-k that rides on the next scoring call of a handle: the guard kernel, which runs over the final EI
+// anyway, leaves the k largest of each of its slices, and the selection's later levels follow at once.
+struct TopkRequest {
+    int k = 0;                 // 0: none
+    int* idx = nullptr;        // device [batch][k]
+    float* val = nullptr;      // device [batch][k] or nullptr
+    void* ws = nullptr;        // at least guard_topk_workspace_bytes(batch, m, k)
+    size_t ws_bytes = 0;
+};
+
 // The handle.  Device arrays are allocated at fit time and freed by r3_gp_free.
 struct r3_gp {
     int batch = 0, n = 0, d = 0;
@@ -107,6 +117,7 @@ struct r3_gp {
     size_t ws_bytes = 0;
 
     r3_engine_t engine_req = R3_ENGINE_AUTO;
+    TopkRequest topk_req;      // set by r3_gp_score_topk for the scoring call it makes, consumed by the guard
 
     // bounded device-side waits of the tensor engine: the limit in cycles, and the test aid that makes one run out
     long long wait_limit_cycles = 4000000000ll;   // about 2 s
@@ -141,14 +152,18 @@ r3_status_t score_simt(r3_gp* gp, const float* Xcand, long long m, float* mu, fl
 struct GuardBuffers {
     float* err_mu;      // [batch][m]
     float* err_q;       // [batch][m]
-    int* list;          // [batch][m] candidate indices to recompute
     int* count;         // [batch]
     unsigned* maxbits;  // [batch] bit pattern of the largest EI
 };
 size_t guard_workspace_bytes(const r3_gp* gp, long long m);
+// Zeroes the pool's maximum EI and the rescue counters; the engines call it before their first scoring kernel.
+r3_status_t guard_begin(r3_gp* gp, const GuardBuffers& b, cudaStream_t stream);
+// Key storage the guard kernel needs to leave the first level of a top-k of k (see TopkRequest).
+size_t guard_topk_workspace_bytes(int batch, long long m, int k);
 GuardBuffers guard_carve(const r3_gp* gp, long long m, void* ws);
+// have_max: the engine's kernels have already raised maxbits to the pool's largest EI
 r3_status_t guard_and_rescue(r3_gp* gp, const float* Xcand, long long m, const GuardBuffers& b, float* mu,
-                             float* sigma, float* ei, cudaStream_t stream);
+                             float* sigma, float* ei, bool have_max, cudaStream_t stream);
 
 // tensor-core scoring (r3_score_tc.cu)
 bool tc_supported(int n, int d);
@@ -169,6 +184,8 @@ r3_status_t score_tc_guard(r3_gp* gp, const float* Xcand, long long m, float* mu
 
 // top-k (r3_topk.cu)
 size_t topk_workspace_bytes(int batch, long long m, int k);
+r3_status_t topk_finish_from_keys(unsigned long long* keys_in, unsigned long long* keys_tmp, int batch, long long count,
+                                  int k, const float* ei, long long m, int* idx, float* val, cudaStream_t stream);
 r3_status_t topk_device(const float* ei, int batch, long long m, int k, int* idx, float* val, void* ws,
                         size_t ws_bytes, cudaStream_t stream);
 

@@ -147,7 +147,7 @@ __global__ void __launch_bounds__(256) trigemm_sq_kernel(const float* __restrict
                                                          long long mc, double sf2, double best, double eps_k, double wnorm,
                                                          float* __restrict__ mu, float* __restrict__ sigma,
                                                          float* __restrict__ ei, float* __restrict__ err_mu,
-                                                         float* __restrict__ err_q)
+                                                         float* __restrict__ err_q, unsigned* __restrict__ maxbits)
 {
     __shared__ __align__(16) float sw[16][132];
     __shared__ __align__(16) float sk[16][132];
@@ -199,6 +199,7 @@ __global__ void __launch_bounds__(256) trigemm_sq_kernel(const float* __restrict
     __syncthreads();
     if (t < 128) {
         const long long c = c0 + t;
+        float ei_mine = 0.f;
         if (c < mc) {
             double q = 0.0;
 #pragma unroll
@@ -209,7 +210,11 @@ __global__ void __launch_bounds__(256) trigemm_sq_kernel(const float* __restrict
             ei[c] = res.ei;
             err_mu[c] = mu_error_estimate(eps_k, mu64[3 * c + 1]);
             err_q[c] = q_error_estimate(eps_k, wnorm, q, mu64[3 * c + 2]);
+            if (res.ei == res.ei) ei_mine = res.ei;
         }
+        // the pool's largest EI, for the guard's EI tolerance: one atomic per warp
+        const unsigned ei_top = __reduce_max_sync(0xffffffffu, __float_as_uint(ei_mine));
+        if ((t & 31) == 0 && ei_top) atomicMax(maxbits, ei_top);
     }
 }
 
@@ -231,6 +236,10 @@ r3_status_t score_simt(r3_gp* gp, const float* Xcand, long long m, float* mu, fl
     }
     SimtWorkspace w = carve(gp, m, ws);
     const int n = gp->n, d = gp->d, npad = gp->npad;
+    {
+        const r3_status_t st0 = guard_begin(gp, w.guard, stream);
+        if (st0 != R3_OK) return st0;
+    }
     for (int g = 0; g < gp->batch; ++g) {
         for (long long s0 = 0; s0 < m; s0 += w.slab) {
             const long long mc = (m - s0) < w.slab ? (m - s0) : w.slab;
@@ -244,11 +253,11 @@ r3_status_t score_simt(r3_gp* gp, const float* Xcand, long long m, float* mu, fl
             R3_LAUNCH(trigemm_sq_kernel, (unsigned)((mc + 127) / 128), 256, 0, stream,
                       gp->W32 + (size_t)g * npad * npad, w.ks, w.mu64, npad, mc, (double)gp->sf2[g],
                       (double)gp->best[g], eps_simt(d), gp->wnorm[g], mu + off, sigma + off, ei + off,
-                      w.guard.err_mu + off, w.guard.err_q + off);
+                      w.guard.err_mu + off, w.guard.err_q + off, w.guard.maxbits + g);
             prof_end(gp, stream);
         }
     }
-    return guard_and_rescue(gp, Xcand, m, w.guard, mu, sigma, ei, stream);
+    return guard_and_rescue(gp, Xcand, m, w.guard, mu, sigma, ei, true, stream);
 }
 
 }  // namespace r3

@@ -1088,7 +1088,7 @@ bool score_tc_can_split(const r3_gp* gp) { return ops_of(gp) != nullptr && env_i
 r3_status_t score_tc_guard(r3_gp* gp, const float* Xcand, long long m, float* mu, float* sigma, float* ei, void* ws,
                            cudaStream_t stream)
 {
-    return guard_and_rescue(gp, Xcand, m, guard_carve(gp, m, ws), mu, sigma, ei, stream);
+    return guard_and_rescue(gp, Xcand, m, guard_carve(gp, m, ws), mu, sigma, ei, false, stream);
 }
 
 r3_status_t score_tc_part(r3_gp* gp, const float* Xcand, long long m, float* mu, float* sigma, float* ei, void* ws,
@@ -1145,6 +1145,10 @@ r3_status_t score_tc_part(r3_gp* gp, const float* Xcand, long long m, float* mu,
     }
     const long long launch_tiles = prm.total_tiles - prm.tile_begin;
     if (launch_tiles <= 0) return R3_OK;
+    if (prm.tile_begin == 0) {   // the pool's first (or only) piece: the rescue counters start at zero
+        const r3_status_t st0 = guard_begin(gp, gb, stream);
+        if (st0 != R3_OK) return st0;
+    }
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, gp->device);
     const unsigned grid = (unsigned)(launch_tiles < sms ? launch_tiles : sms);
@@ -1187,7 +1191,7 @@ r3_status_t score_tc_part(r3_gp* gp, const float* Xcand, long long m, float* mu,
             }
     }
     if (!guard) return R3_OK;
-    return guard_and_rescue(gp, Xcand, m, gb, mu, sigma, ei, stream);
+    return guard_and_rescue(gp, Xcand, m, gb, mu, sigma, ei, false, stream);
 }
 
 }  // namespace r3

@@ -1,61 +1,46 @@
 // Top-k selection: the k largest EI of each GP's pool, ties to the lower index.
 //
-// A value and its index are packed in one 64-bit key whose unsigned order is exactly
-// (value descending-friendly, index ascending): the float is mapped to an order-preserving unsigned
-// integer in the high word and the low word holds ~index, so "larger key" means "larger value, or
-// equal value and smaller index".  A block sorts a chunk of keys in shared memory (bitonic network)
-// and emits its k largest; levels repeat until one chunk is left, whose k largest are the answer.
-// The first level reads the EI array once (4 bytes per candidate); later levels touch k keys per
-// chunk of the level before.
+// A value and its index are packed in one 64-bit key (r3_topk.cuh) whose unsigned order is exactly "larger
+// value, or equal value and smaller index".  A block takes a chunk of 4096 keys into shared memory and keeps
+// its k largest (block_topk_desc: blocks of k sorted by a bitonic network, then halving merges); levels repeat
+// until one chunk is left, and the block that handles it writes the indices and values.  The first level
+// reads the EI array once (4 bytes per candidate); later levels touch k keys per chunk of the level before.
+// When the scoring call asked for a top-k, the accuracy guard's kernel has already left the first level's keys
+// (r3_rescue.cu), and only the later levels run here.
 #include <mutex>
 
 #include "r3_internal.cuh"
+#include "r3_topk.cuh"
 
 namespace r3 {
 
 namespace {
 
-constexpr int CHUNK = 4096;      // keys sorted per block
+constexpr int CHUNK = 4096;      // keys per block
 constexpr int THREADS = 1024;
 
-__device__ __forceinline__ unsigned long long make_key(float v, unsigned idx)
+// The last level writes the answer instead of keys: idx (and val, read back from the EI array) are non-null.
+__device__ __forceinline__ void emit(const unsigned long long* s, int k, unsigned long long* out_keys,
+                                     const float* __restrict__ ei, long long m, int* __restrict__ idx,
+                                     float* __restrict__ val)
 {
-    unsigned u;
-    if (v != v) {
-        u = 0u;  // NaN ranks below every number
-    } else {
-        if (v == 0.0f) v = 0.0f;  // -0 and +0 tie
-        u = __float_as_uint(v);
-        u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-        if (u == 0u) u = 1u;  // keep 0 for NaN / padding (only -NaN patterns map here)
-    }
-    return ((unsigned long long)u << 32) | (unsigned long long)(0xFFFFFFFFu - idx);
-}
-
-// Sort CHUNK keys descending in shared memory.
-__device__ __forceinline__ void bitonic_sort_desc(unsigned long long* s)
-{
-    for (int size = 2; size <= CHUNK; size <<= 1) {
-        for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            __syncthreads();
-            for (int t = threadIdx.x; t < CHUNK / 2; t += THREADS) {
-                const int lo = 2 * t - (t & (stride - 1));
-                const int hi = lo + stride;
-                const bool desc = ((lo & size) == 0);
-                const unsigned long long a = s[lo], b = s[hi];
-                if ((a < b) == desc) {
-                    s[lo] = b;
-                    s[hi] = a;
-                }
-            }
+    const int g = blockIdx.y;
+    if (idx) {
+        for (int t = threadIdx.x; t < k; t += blockDim.x) {
+            const unsigned i = topk_key_index(s[t]);
+            idx[(size_t)g * k + t] = (int)i;
+            if (val) val[(size_t)g * k + t] = ((long long)i < m) ? ei[(size_t)g * m + i] : __int_as_float(0x7fc00000);
         }
+    } else {
+        unsigned long long* o = out_keys + ((size_t)g * gridDim.x + blockIdx.x) * k;
+        for (int t = threadIdx.x; t < k; t += blockDim.x) o[t] = s[t];
     }
-    __syncthreads();
 }
 
 // Level 0: keys from the EI array.  grid = (chunks, batch).
 __global__ void __launch_bounds__(THREADS) topk_from_values_kernel(const float* __restrict__ ei, long long m,
-                                                                   int k, unsigned long long* __restrict__ out)
+                                                                   int k, int K2, unsigned long long* __restrict__ out,
+                                                                   int* __restrict__ idx, float* __restrict__ val)
 {
     __shared__ unsigned long long s[CHUNK];
     const int g = blockIdx.y;
@@ -63,17 +48,18 @@ __global__ void __launch_bounds__(THREADS) topk_from_values_kernel(const float* 
     const float* e = ei + (size_t)g * m;
     for (int t = threadIdx.x; t < CHUNK; t += THREADS) {
         const long long i = base + t;
-        s[t] = (i < m) ? make_key(e[i], (unsigned)i) : 0ull;
+        s[t] = (i < m) ? topk_make_key(e[i], (unsigned)i) : 0ull;
     }
-    bitonic_sort_desc(s);
-    unsigned long long* o = out + ((size_t)g * gridDim.x + blockIdx.x) * k;
-    for (int t = threadIdx.x; t < k; t += THREADS) o[t] = s[t];
+    block_topk_desc(s, CHUNK, K2);
+    emit(s, k, out, ei, m, idx, val);
 }
 
 // Later levels: keys from the level before.  count = keys per GP in `in`.
 __global__ void __launch_bounds__(THREADS) topk_from_keys_kernel(const unsigned long long* __restrict__ in,
-                                                                 long long count, int k,
-                                                                 unsigned long long* __restrict__ out)
+                                                                 long long count, int k, int K2,
+                                                                 unsigned long long* __restrict__ out,
+                                                                 const float* __restrict__ ei, long long m,
+                                                                 int* __restrict__ idx, float* __restrict__ val)
 {
     __shared__ unsigned long long s[CHUNK];
     const int g = blockIdx.y;
@@ -83,20 +69,8 @@ __global__ void __launch_bounds__(THREADS) topk_from_keys_kernel(const unsigned 
         const long long i = base + t;
         s[t] = (i < count) ? src[i] : 0ull;
     }
-    bitonic_sort_desc(s);
-    unsigned long long* o = out + ((size_t)g * gridDim.x + blockIdx.x) * k;
-    for (int t = threadIdx.x; t < k; t += THREADS) o[t] = s[t];
-}
-
-__global__ void topk_write_kernel(const unsigned long long* __restrict__ keys, const float* __restrict__ ei,
-                                  long long m, int k, int* __restrict__ idx, float* __restrict__ val)
-{
-    const int g = blockIdx.y;
-    const int t = blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= k) return;
-    const unsigned i = 0xFFFFFFFFu - (unsigned)(keys[(size_t)g * k + t] & 0xFFFFFFFFull);
-    idx[(size_t)g * k + t] = (int)i;
-    if (val) val[(size_t)g * k + t] = ((long long)i < m) ? ei[(size_t)g * m + i] : __int_as_float(0x7fc00000);
+    block_topk_desc(s, CHUNK, K2);
+    emit(s, k, out, ei, m, idx, val);
 }
 
 long long chunks_of(long long count) { return (count + CHUNK - 1) / CHUNK; }
@@ -143,6 +117,27 @@ size_t topk_workspace_bytes(int batch, long long m, int k)
     return 2 * level0 * sizeof(unsigned long long) + 64;
 }
 
+// The levels after the first: `count` keys per GP in keys_in (k per block of the level before), ping-pong
+// through keys_tmp, indices and values out.  count == k means a single block produced them, sorted: only the
+// write is left, and the last level's kernel does it all the same (one chunk).
+r3_status_t topk_finish_from_keys(unsigned long long* keys_in, unsigned long long* keys_tmp, int batch, long long count,
+                                  int k, const float* ei, long long m, int* idx, float* val, cudaStream_t stream)
+{
+    const int K2 = topk_pow2_at_least(k);
+    unsigned long long* buf[2] = {keys_in, keys_tmp};
+    int cur = 0;
+    while (true) {
+        const long long chunks = chunks_of(count);
+        const bool last = chunks == 1;
+        R3_LAUNCH(topk_from_keys_kernel, dim3((unsigned)chunks, batch), THREADS, 0, stream, buf[cur], count, k, K2,
+                  buf[cur ^ 1], ei, m, last ? idx : nullptr, last ? val : nullptr);
+        if (last) break;
+        cur ^= 1;
+        count = chunks * k;
+    }
+    return R3_OK;
+}
+
 r3_status_t topk_device(const float* ei, int batch, long long m, int k, int* idx, float* val, void* ws,
                         size_t ws_bytes, cudaStream_t stream)
 {
@@ -152,19 +147,13 @@ r3_status_t topk_device(const float* ei, int batch, long long m, int k, int* idx
     }
     const size_t level0 = (size_t)batch * chunks_of(m) * k;
     unsigned long long* buf[2] = {(unsigned long long*)ws, (unsigned long long*)ws + level0};
-    long long chunks = chunks_of(m);
-    R3_LAUNCH(topk_from_values_kernel, dim3((unsigned)chunks, batch), THREADS, 0, stream, ei, m, k, buf[0]);
-    int cur = 0;
-    long long count = chunks * k;
-    while (chunks > 1) {
-        chunks = chunks_of(count);
-        R3_LAUNCH(topk_from_keys_kernel, dim3((unsigned)chunks, batch), THREADS, 0, stream, buf[cur], count, k,
-                  buf[cur ^ 1]);
-        cur ^= 1;
-        count = chunks * k;
-    }
-    R3_LAUNCH(topk_write_kernel, dim3((k + 255) / 256, batch), 256, 0, stream, buf[cur], ei, m, k, idx, val);
-    return R3_OK;
+    const long long chunks = chunks_of(m);
+    const int K2 = topk_pow2_at_least(k);
+    const bool last = chunks == 1;
+    R3_LAUNCH(topk_from_values_kernel, dim3((unsigned)chunks, batch), THREADS, 0, stream, ei, m, k, K2, buf[0],
+              last ? idx : nullptr, last ? val : nullptr);
+    if (last) return R3_OK;
+    return topk_finish_from_keys(buf[0], buf[1], batch, chunks * k, k, ei, m, idx, val, stream);
 }
 
 }  // namespace r3
