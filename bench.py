@@ -9,7 +9,9 @@ candidates scored per second, whole job.  The fit (once per BO round) is timed s
 reported in ``fit_ms``.  Prints ONE JSON line.
 
 N > 1 (launched with torch.distributed.run): every rank scores its own pool of m candidates of the
-same GP (weak scaling) and the ranks' top-k lists are merged with one all-gather per step.
+same GP (weak scaling) and the ranks' top-k lists are merged with one all-gather per step.  With
+``--scaling strong`` the ranks split ONE pool of m candidates into contiguous shards instead, and rank 0
+checks the merged selection against the selection of the whole pool.
 ``--impl reference`` times the FP64 CPU oracle on a bounded sample of the same workload.
 """
 from __future__ import annotations
@@ -364,6 +366,8 @@ def main():
     ap.add_argument("--tpe-continuous", action="store_true",
                     help="tpe: spread the history's ordinal values uniformly inside their level's cell (a space of "
                          "continuous parameters: every observation keeps its own component)")
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="N > 1: weak = one pool of m candidates per rank; strong = one pool of m candidates split over the ranks")
     ap.add_argument("--surrogate", default="gp", choices=["gp", "tpe"],
                     help="gp: the headline GP-EI path; tpe: Parzen-estimator scoring of the same pools")
     args = ap.parse_args()
@@ -381,7 +385,7 @@ def main():
     import torch
     import torch.distributed as dist
     from paper_2604_11109_b200 import binding as b
-    from paper_2604_11109_b200.sharding import merge_topk
+    from paper_2604_11109_b200.sharding import merge_topk, shard_bounds
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -391,14 +395,22 @@ def main():
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    strong = args.scaling == "strong" and world > 1 and c.batch == 1
 
-    # every rank: the same GP history, its own pool (weak scaling): pool r is drawn with seed offset r
+    # every rank: the same GP history.  Weak scaling: its own pool (pool r is drawn with seed offset r); strong
+    # scaling: its contiguous shard of the one pool.
     g = w.generate(c)
-    if rank > 0 and c.batch == 1:
+    pool_full = g["Xcand"]
+    shard_lo = 0
+    if strong:
+        shard_lo, shard_hi = shard_bounds(c.m, world, rank)
+        g["Xcand"] = np.ascontiguousarray(pool_full[:, shard_lo:shard_hi])
+    elif rank > 0 and c.batch == 1:
         g["Xcand"] = w.generate_gp(c, rank)["Xcand"][None]   # another seeded pool from the same grid
     X, y = torch.from_numpy(g["X"]).cuda(), torch.from_numpy(g["y"]).cuda()
     xc = torch.from_numpy(g["Xcand"]).cuda()
-    B, m, k, n, d = c.batch, c.m, c.k, c.n, c.d
+    B, m, k, n, d = c.batch, int(g["Xcand"].shape[1]), c.k, c.n, c.d
+    k = min(k, m)
 
     b.r3_gp_fit(X, y, g["ell"], g["sf2"], g["sn2"]).close()   # warm-up fit: module load and first-use costs
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
@@ -454,10 +466,13 @@ def main():
     out = (torch.empty((B, m), device="cuda"), torch.empty((B, m), device="cuda"), torch.empty((B, m), device="cuda"),
            torch.empty((B, k), dtype=torch.int32, device="cuda"), torch.empty((B, k), device="cuda"))
 
+    merged = [None]
+
     def step():
         b.r3_gp_score_topk(gp, xc, k, out)
         if world > 1 and B == 1:
-            merge_topk(out[4][0], out[3][0], k, rank * m, topk_fn=lambda v, kk: b.r3_topk(v, kk)[0])
+            offset = shard_lo if strong else rank * m
+            merged[0] = merge_topk(out[4][0], out[3][0], k, offset, topk_fn=lambda v, kk: b.r3_topk(v, kk)[0])
 
     def barrier():
         if world > 1:
@@ -493,7 +508,17 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms_total = float(t.item())
     ms_per_step = ms_total / args.steps
-    value = world * B * m / (ms_per_step * 1e-3)
+    total_candidates = B * c.m if strong else world * B * m   # the units all ranks processed per step
+    value = total_candidates / (ms_per_step * 1e-3)
+    strong_ok = None
+    if strong and rank == 0:
+        # the merged selection against the selection of the whole pool scored on this rank alone
+        whole = b.r3_gp_score_topk(gp, torch.from_numpy(pool_full).cuda(), k)
+        a_idx, w_idx = merged[0][1].cpu().to(torch.int64), whole[3][0].cpu().to(torch.int64)
+        # (a shard's accuracy guard works against the shard's own largest EI, so a candidate recomputed in FP64 in
+        # one run and not in the other can move by less than the tolerance: positions may swap between near ties)
+        strong_ok = {"same_set": bool(set(a_idx.tolist()) == set(w_idx.tolist())),
+                     "positions_that_differ": int((a_idx != w_idx).sum())}
 
     # ---- end to end through the host-buffer entry point ------------------------------------------
     xh = torch.from_numpy(g["Xcand"]).pin_memory()
@@ -525,24 +550,44 @@ def main():
     per_launch_ms = kernel_ms / max(kernel_launches, 1)
     cands_per_launch = B * m * args.steps / max(kernel_launches, 1)
     npad = (n + 31) // 32 * 32
+    split = "f16x3"
     if engine == "tensor":
-        # Variance contraction S4: algorithmic n^2 flops per candidate (n^2/2 MACs over the lower triangle); the
-        # kernel issues three FP16 MMAs per product (hi*hi + hi*lo + lo*hi), so issued = 3x that, at the FP16/BF16
-        # tensor rate.  The distance products and the diagonal blocks' zero halves are not counted.
+        # Variance contraction S4: algorithmic n^2 flops per candidate (n^2/2 MACs over the lower triangle).  The
+        # 22-bit product needs three FP16 MMAs per product (hi*hi + hi*lo + lo*hi), so the work counted is 3x that,
+        # at the FP16/BF16 tensor rate -- the count stays the same when the two cross terms run as E4M3 MMAs at
+        # twice the rate (then the tensor time actually issued is that of two FP16 MMAs: `issued_f16_equivalent`).
+        # The distance products and the diagonal blocks' zero halves are not in the count; `issued_total_tflops`
+        # is everything the pipe was given, in FP16-rate equivalents: per chunk of 32 observations of a tile,
+        # 128 x NV x 32 MACs of the variance product three (two with E4M3 cross terms) times over, and
+        # 128 x 32 x DP MACs of the distance product three times, for every (re)generation of the chunk.
+        info = b.r3_gp_tensor_info(gp)
+        f8 = bool(info["f8_cross_terms"])
+        split = "f16 + 2 x e4m3 cross terms" if f8 else "f16x3"
         alg_flops = float(n) * n
         issued = 3.0 * alg_flops
         achieved = issued * cands_per_launch / (per_launch_ms * 1e-3) / 1e12
         peak = peaks["bf16_tflops"]
+        NV, P, DP = info["NV"], info["P"], info["DP"]
+        chunks_per_tile = (NV // 32) * P * (P + 1) // 2
+        tiles_per_launch = B * ((m + 127) // 128) * args.steps / max(kernel_launches, 1)
+        per_chunk = (2.0 if f8 else 3.0) * 2 * 128 * NV * 32 + 3.0 * 2 * 128 * 32 * DP
+        issued_total = per_chunk * chunks_per_tile * tiles_per_launch / (per_launch_ms * 1e-3) / 1e12
         roofline = {"bound": "tensor", "kernel": "score_tc_kernel", "achieved": achieved, "peak": peak,
                     "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
-                    "note": f"issued FP16 flops of the variance contraction (3 MMAs per product); peak = {peak_kind} "
-                            "bf16 burst (same tensor rate as fp16)",
+                    "note": "3 n^2 flops per candidate: the three FP16-rate MMAs per product that a 22-bit variance "
+                            f"contraction needs (split: {split}); peak = {peak_kind} bf16 burst (same tensor rate as fp16)",
                     "algorithmic_tflops": achieved / 3.0,
-                    "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"]}
-        if c.cfg == 5 and args.m is None:
-            # dram bytes per launch from the ncu capture of this kernel on m = 32768 (profiles/score_tc_kernel_cfg5.md):
-            # 37.7 MB of pre-tiled operands read once + 263 B per candidate (244 read, 18.6 written)
-            roofline["traffic"] = 37.7e6 + 263.0 * cands_per_launch
+                    "issued_f16_equivalent_tflops": achieved * (2.0 / 3.0 if f8 else 1.0),
+                    "issued_total_tflops": issued_total,
+                    "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
+                    "shape": info}
+        # DRAM bytes per launch, modelled: the pre-tiled operands are read once per launch (their sizes follow
+        # from the shape: chunks of W as 2 x 32 x NV x 2 bytes each, observation planes, FP32 observations), and
+        # an ncu capture of this kernel on 32,768 candidates of the largest workload measured 244 B read and
+        # 18.6 B written per candidate beside them (algorithmic: 4 d read, 20 written).
+        operands = B * ((NV // 32) * P * (P + 1) // 2 * 2 * 32 * NV * 2 + info["NP"] * DP * (4 + 4) + info["NP"] * 8)
+        roofline["traffic"] = float(operands + (4 * d * 244.0 / 256.0 + 18.6) * cands_per_launch)
+        roofline["traffic_kind"] = "modelled from operand sizes and a small-case ncu capture"
     else:
         alg_flops = float(npad) * npad
         achieved = alg_flops * cands_per_launch / (per_launch_ms * 1e-3) / 1e12
@@ -566,15 +611,17 @@ def main():
     print(json.dumps({
         "metric": "gp_ei_candidates_scored_per_sec", "value": value, "unit": "candidates/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32" if engine == "simt" else "f16x3", "data": "synthetic",
+        "scaling": "strong" if strong else "weak", "vs_baseline": None, "dtype": "f32" if engine == "simt" else split,
+        "data": "synthetic",
         "config": {"workload": c.name, "batch": B, "n": n, "d": d, "m": m, "k": k, "engine": engine,
                    "l2": "pool (%.0f MB) and outputs exceed the 126 MB L2" % (xc.numel() * 4 / 1e6)
                    if xc.numel() * 4 > 126e6 else "pool smaller than L2; not flushed"},
         "fit_ms": fit_ms, "append_ms": append_ms, "append_k": ka, "propose_ms": propose_ms,
         "propose_q": qp, "propose_certified": propose_cert, "lml_ms": lml_ms, "clocks": clocks,
-        "e2e": {"value": world * B * m / (e2e_ms * 1e-3), "unit": "candidates/s", "h2d_bytes_per_step": h2d,
+        "e2e": {"value": total_candidates / (e2e_ms * 1e-3), "unit": "candidates/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "matches_device_run": bool(same)},
         "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu, "peaks": peak_kind,
+        **({"strong_scaling_selection_matches_whole_pool": strong_ok} if strong else {}),
     }))
     gp.close()
     if world > 1:

@@ -194,6 +194,17 @@ r3_status_t r3_gp_set_engine(r3_gp_t* gp, r3_engine_t engine);
 r3_engine_t r3_gp_engine(const r3_gp_t* gp);
 
 /*
+ * Diagnostics: the shape the tensor-core engine runs this handle in (all zero when it does not serve it).
+ * info[0] NV   rows of the inverse factor per pass (columns of the accumulator in tensor memory)
+ * info[1] P    passes per tile of 128 candidates (the chunks of k* are generated (P + 1) / 2 times on average)
+ * info[2] DP   feature count padded to a multiple of 16 (depth of the distance product)
+ * info[3] NP   history length padded to a multiple of NV
+ * info[4] G    Matern warp groups;  info[5] W stages in shared memory;  info[6] 1: k* operand in tensor memory
+ * info[7] 1: the cross terms of the variance product are E4M3 MMAs (histories of eight passes and more)
+ */
+r3_status_t r3_gp_tensor_info(const r3_gp_t* gp, int* info /* host [8] */);
+
+/*
  * Diagnostics: synchronises `cuda_stream` and returns how many candidates the last scoring call on
  * this handle recomputed in FP64 (summed over the first 64 GPs of the batch).  The scoring engines
  * work at FP32 level and hand to an FP64 pass every candidate whose estimated rounding error could

@@ -76,6 +76,7 @@ SIGNATURES = {
     "r3_gp_engine": (_i, [_vp]),
     "r3_gp_get_factor": (_i, [_vp, _vp, _vp]),
     "r3_gp_last_rescued": (_i, [_vp, _vp, ctypes.POINTER(_ll)]),
+    "r3_gp_tensor_info": (_i, [_vp, ctypes.POINTER(ctypes.c_int)]),
     "r3_gp_profile": (_i, [_vp, _i]),
     "r3_gp_profile_read": (_i, [_vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_ll)]),
     "r3_launch_count": (_ull, []),
@@ -383,6 +384,14 @@ def r3_gp_test_withhold(gp: GP, chunk: int):
 
 def r3_test_fail_allocation(after: int) -> int:
     return int(load().r3_test_fail_allocation(int(after)))
+
+
+def r3_gp_tensor_info(gp: GP) -> dict:
+    """Shape of the tensor-core engine for this handle (zeros when it does not serve it)."""
+    info = (ctypes.c_int * 8)()
+    _check(load().r3_gp_tensor_info(gp.handle, info))
+    names = ("NV", "P", "DP", "NP", "G", "w_stages", "kstar_in_tmem", "f8_cross_terms")
+    return dict(zip(names, (int(v) for v in info)))
 
 
 def r3_gp_get_best(gp: GP) -> np.ndarray:

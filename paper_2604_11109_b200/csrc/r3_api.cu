@@ -730,6 +730,16 @@ r3_status_t r3_gp_last_rescued(r3_gp_t* gp, void* cuda_stream, long long* total)
     return R3_OK;
 }
 
+r3_status_t r3_gp_tensor_info(const r3_gp_t* gp, int* info)
+{
+    if (!gp || !info) {
+        set_error("r3_gp_tensor_info: NULL argument");
+        return R3_ERR_INVALID_ARG;
+    }
+    tc_info(gp, info);
+    return R3_OK;
+}
+
 r3_status_t r3_gp_profile(r3_gp_t* gp, int enable)
 {
     if (!gp) {

@@ -169,6 +169,7 @@ r3_status_t guard_and_rescue(r3_gp* gp, const float* Xcand, long long m, const G
 bool tc_supported(int n, int d);
 r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream);
 void tc_release(r3_gp* gp);
+void tc_info(const r3_gp* gp, int* info);   // r3_gp_tensor_info
 size_t score_tc_workspace_bytes(const r3_gp* gp, long long m);
 r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, float* sigma, float* ei,
                      void* ws, size_t ws_bytes, cudaStream_t stream);

@@ -1073,6 +1073,15 @@ r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream)
     return R3_OK;
 }
 
+void tc_info(const r3_gp* gp, int* info)
+{
+    const TensorOperands* t = ops_of(gp);
+    for (int i = 0; i < 8; ++i) info[i] = 0;
+    if (!t) return;
+    info[0] = t->NV; info[1] = t->P; info[2] = t->DP; info[3] = t->NP;
+    info[4] = t->G; info[5] = t->ws; info[6] = t->kt ? 1 : 0; info[7] = t->f8 ? 1 : 0;
+}
+
 size_t score_tc_workspace_bytes(const r3_gp* gp, long long m) { return guard_workspace_bytes(gp, m); }
 
 r3_status_t score_tc(r3_gp* gp, const float* Xcand, long long m, float* mu, float* sigma, float* ei, void* ws,
