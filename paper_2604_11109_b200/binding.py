@@ -17,7 +17,8 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libr3gp.so")
+# R3_LIB_VARIANT=check loads the bounds-checking build of the same library (build.py --check)
+LIB_PATH = os.path.join(_HERE, "libr3gp_check.so" if os.environ.get("R3_LIB_VARIANT") == "check" else "libr3gp.so")
 
 R3_OK = 0
 STATUS_NAMES = {

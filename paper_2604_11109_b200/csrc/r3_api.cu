@@ -232,13 +232,14 @@ r3_status_t r3_gp_fit(const float* X, const float* y, const float* lengthscales,
     TRY_BAIL(dev_malloc(&gp->W32, sizeof(float) * batch * mat));
     TRY_BAIL(dev_malloc(&gp->alpha64, sizeof(double) * batch * gp->npad));
     TRY_BAIL(dev_malloc(&gp->alpha32, sizeof(float) * batch * gp->npad));
-    TRY_BAIL(dev_malloc(&gp->status_d, 2 * sizeof(int)));
-    gp->status_h = pinned_word_acquire();   // [2] status words, then [64] rescue counters
+    TRY_BAIL(dev_malloc(&gp->status_d, 4 * sizeof(int)));
+    TRY_BAIL(cudaMemsetAsync(gp->status_d, 0, 4 * sizeof(int), stream));
+    gp->status_h = pinned_word_acquire();   // [4] status words, then [64] rescue counters
     if (!gp->status_h) {
         set_error("r3_gp_fit: no pinned host memory");
         return bail(R3_ERR_ALLOC);
     }
-    gp->rescued_h = gp->status_h + 2;
+    gp->rescued_h = gp->status_h + 4;
     for (int i = 0; i < 64; ++i) gp->rescued_h[i] = 0;
     gp->status_h[0] = 0;
     gp->status_h[1] = INT_MAX;
@@ -637,10 +638,16 @@ r3_status_t r3_gp_check(r3_gp_t* gp, void* cuda_stream)
         return R3_ERR_INVALID_ARG;
     }
     cudaStream_t stream = (cudaStream_t)cuda_stream;
-    R3_CUDA_TRY(cudaMemcpyAsync(gp->status_h, gp->status_d, 2 * sizeof(int), cudaMemcpyDeviceToHost, stream));
+    R3_CUDA_TRY(cudaMemcpyAsync(gp->status_h, gp->status_d, 3 * sizeof(int), cudaMemcpyDeviceToHost, stream));
     R3_CUDA_TRY(cudaMemsetAsync(gp->status_d, 0, sizeof(int), stream));
+    R3_CUDA_TRY(cudaMemsetAsync(gp->status_d + 2, 0, sizeof(int), stream));
     R3_CUDA_TRY(cudaStreamSynchronize(stream));
     const int bits = gp->status_h[0];
+    if (bits & DEV_BOUNDS) {
+        set_error("bounds-checking build: an index check failed (source line %d of its kernel's file); results are invalid",
+                  gp->status_h[2]);
+        return R3_ERR_CUDA;
+    }
     if (bits & DEV_TIMEOUT) {
         set_error("a bounded device-side wait ran out; results are invalid");
         return R3_ERR_DEVICE_TIMEOUT;

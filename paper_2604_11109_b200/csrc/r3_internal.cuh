@@ -45,7 +45,27 @@ enum : int {
     DEV_NONFINITE = 1,   // NaN/Inf met in an input
     DEV_NOT_PD = 2,      // non-positive Cholesky pivot
     DEV_TIMEOUT = 4,     // a bounded wait gave up
+    DEV_BOUNDS = 8,      // an index check of the bounds-checking build failed (R3_BOUNDS_CHECK)
 };
+
+// Index checks of the bounds-checking build (python -m paper_2604_11109_b200.build --check; compute-sanitizer is
+// not available where this library is developed).  R3_IDX(i, n, status) is i in the normal build.  In the
+// checking build an index outside [0, n) raises DEV_BOUNDS in the handle's status word, leaves the source line
+// of the check in the word after the pivot index, and is replaced by 0: the access goes to a valid element
+// instead of faulting, control flow stays as it was (warp-wide instructions keep all their lanes), and
+// r3_gp_check reports the line.
+#ifdef R3_BOUNDS_CHECK
+__device__ __forceinline__ long long checked_index(long long i, long long n, int* status, int line)
+{
+    if (i >= 0 && i < n) return i;
+    atomicOr(status, DEV_BOUNDS);
+    atomicMax(status + 2, line);
+    return 0;
+}
+#define R3_IDX(i, n, status) r3::checked_index((long long)(i), (long long)(n), (status), __LINE__)
+#else
+#define R3_IDX(i, n, status) (i)
+#endif
 
 constexpr int kFitBlock = 32;   // Cholesky / inverse block size; n is padded to a multiple of it
 constexpr int kMaxN = 8192;
@@ -105,7 +125,7 @@ struct r3_gp {
     float* W32 = nullptr;      // [batch][npad][npad] W rounded to FP32
     double* alpha64 = nullptr; // [batch][npad]  (zero in the padding)
     float* alpha32 = nullptr;  // [batch][npad]
-    int* status_d = nullptr;   // [2]: status bits, first bad pivot index
+    int* status_d = nullptr;   // [4]: status bits, first bad pivot index, line of a failed index check, unused
     int* status_h = nullptr;   // pinned mirror of status_d
     int* rescued_h = nullptr;  // pinned [64]: candidates recomputed in FP64 by the last scoring call, per GP
 

@@ -34,6 +34,7 @@ struct GuardArgs {
     const float *err_mu, *err_q;
     const unsigned* maxbits;      // [batch] bit pattern of the pool's largest EI
     int* count;                   // [batch] candidates recomputed (diagnostics)
+    int* status;                  // the handle's status words (index checks of the bounds-checking build)
     int k, K2;                    // top-k request (k = 0: none); K2 = min(2^ceil(log2 k), slice)
     unsigned long long* keys;     // [batch][blocks][k]
 };
@@ -92,7 +93,7 @@ __global__ void __launch_bounds__(256) guard_kernel(const GuardArgs a)
             const float phi = expf(-0.5f * z * z) * 0.39894228f;
             if (isfinite(dsd)) flag |= !(Phi * dmu + phi * dsd <= 0.5f * tol_ei);
             flag |= !(sd * sd >= 1e-3f * sf2);   // deep cancellation: do not trust the estimates either
-            if (flag) list[atomicAdd(&nflag_s, 1)] = (int)i;
+            if (flag) list[R3_IDX(atomicAdd(&nflag_s, 1), a.slice, a.status)] = (int)i;
         }
     }
     __syncthreads();
@@ -112,8 +113,8 @@ __global__ void __launch_bounds__(256) guard_kernel(const GuardArgs a)
             __syncthreads();
             for (int e = t; e < R * d; e += 256) {
                 const int r = e / d, j = e % d;
-                const int c = list[e0 + min(r, nr - 1)];
-                zs[e] = (double)a.Xcand[((size_t)g * m + c) * d + j];
+                const int c = list[R3_IDX(e0 + min(r, nr - 1), a.slice, a.status)];
+                zs[e] = (double)a.Xcand[(size_t)R3_IDX((long long)g * m + c, (long long)gridDim.y * m, a.status) * d + j];
             }
             __syncthreads();
             double mu_part[R];
@@ -136,7 +137,7 @@ __global__ void __launch_bounds__(256) guard_kernel(const GuardArgs a)
                 for (int r = 0; r < R; ++r) {
                     const double sq = sqrt(5.0) * sqrt(r2[r]);
                     const double kv = sf2 * (1.0 + sq + sq * sq / 3.0) * exp(-sq);
-                    ks[(size_t)r * npad + i] = kv;
+                    ks[(size_t)R3_IDX((long long)r * npad + i, (long long)R * npad, a.status)] = kv;
                     mu_part[r] += kv * al;
                 }
             }
@@ -175,7 +176,7 @@ __global__ void __launch_bounds__(256) guard_kernel(const GuardArgs a)
                     mu_s += red[0][t][w];
                     q += red[1][t][w];
                 }
-                const size_t f = (size_t)g * m + list[e0 + t];
+                const size_t f = (size_t)R3_IDX((long long)g * m + list[e0 + t], (long long)gridDim.y * m, a.status);
                 const CandidateResult res = finalize_candidate(mu_s, q, sf2, (double)a.bestv[g]);
                 a.mu[f] = res.mu;
                 a.sigma[f] = res.sigma;
@@ -195,7 +196,7 @@ __global__ void __launch_bounds__(256) guard_kernel(const GuardArgs a)
     }
     block_topk_desc(keys_s, a.slice, a.K2);
     unsigned long long* out = a.keys + ((size_t)g * gridDim.x + blockIdx.x) * a.k;
-    for (int i = t; i < a.k; i += 256) out[i] = i < a.slice ? keys_s[i] : 0ull;
+    for (int i = t; i < a.k; i += 256) out[i] = i < a.slice ? keys_s[R3_IDX(i, a.slice, a.status)] : 0ull;
 }
 
 }  // namespace
@@ -262,6 +263,7 @@ r3_status_t guard_and_rescue(r3_gp* gp, const float* Xcand, long long m, const G
     a.err_mu = b.err_mu; a.err_q = b.err_q;
     a.maxbits = b.maxbits;
     a.count = b.count;
+    a.status = gp->status_d;
     a.k = req.k;
     a.K2 = req.k > 0 ? std::min(topk_pow2_at_least(req.k), a.slice) : 1;
     a.keys = (unsigned long long*)req.ws;

@@ -181,7 +181,8 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                 for (int c = 0; c < (p + 1) * (NV / KD); ++c, ++issued) {
                     if (!(ok = mbar_wait(bar(BAR_X_EMPTY + st), ph ^ 1u, abort_flag, wl))) break;
                     mbar_arrive_expect_tx(bar(BAR_X_FULL + st), bytes);
-                    bulk_g2s(base + map.x + st * bytes, src + (size_t)c * (bytes / 2), bytes, bar(BAR_X_FULL + st));
+                    bulk_g2s(base + map.x + (uint32_t)R3_IDX(st, XS, prm.status) * bytes,
+                             src + (size_t)R3_IDX(c, prm.NP / KD, prm.status) * (bytes / 2), bytes, bar(BAR_X_FULL + st));
                     if (++st == XS) { st = 0; ph ^= 1u; }
                 }
         }
@@ -208,7 +209,9 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     if (issued == prm.withhold_w) { ok = false; break; }   // test aid: the stream of W stops here
                     if (!(ok = mbar_wait(bar(BAR_W_EMPTY + st), ph ^ 1u, abort_flag, wl))) break;
                     mbar_arrive_expect_tx(bar(BAR_W_FULL + st), bytes);
-                    bulk_g2s(base + map.w + st * bytes, psrc + (size_t)c * (bytes / 2), bytes, bar(BAR_W_FULL + st));
+                    (void)R3_IDX(CPP * p * (p + 1) / 2 + c, CPP * P * (P + 1) / 2, prm.status);   // chunk of W within the GP's tiles
+                    bulk_g2s(base + map.w + (uint32_t)R3_IDX(st, ws, prm.status) * bytes, psrc + (size_t)c * (bytes / 2), bytes,
+                             bar(BAR_W_FULL + st));
                     if (++st == ws) { st = 0; ph ^= 1u; }
                 }
             }
@@ -301,7 +304,9 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     tc_fence_after();
                     // In the pass's diagonal block the rows of W above the chunk's columns are zero (W is lower
                     // triangular): the MMAs start at the first row that can be non-zero and get narrower.
-                    const uint32_t skip = c > p * CPP ? (uint32_t)(c - p * CPP) * KC : 0u;
+                    (void)R3_IDX(s, ws, prm.status);
+                    (void)R3_IDX(b, NBK, prm.status);
+                    const uint32_t skip = c > p * CPP ? (uint32_t)R3_IDX((c - p * CPP) * KC, NV, prm.status) : 0u;
                     const uint32_t idesc_v = instr_desc_f16(NV - skip);
                     const uint32_t vcol = tmem + skip;
                     const uint32_t bH = w_lo0 + ((s * map.w_stage) >> 4) + skip, bL = bH + (((uint32_t)KC * NV * 2u) >> 4);
@@ -399,7 +404,8 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                 // ---- scale the candidate, split it, store it as the A operand of the distance MMA
                 float zn = 0.f;
                 bool far = false;
-                const float* zrow = prm.xcand + ((size_t)g * prm.m + (valid ? cand : 0)) * prm.d;
+                const float* zrow =
+                    prm.xcand + (size_t)R3_IDX((long long)g * prm.m + (valid ? cand : 0), (long long)prm.batch * prm.m, prm.status) * prm.d;
                 {
                     // the row this thread will need for the CTA's next tile: start it on its way to L2 now
                     const long long nt = tile + tile_step;
@@ -431,8 +437,8 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
 #pragma unroll
                             for (int e = 0; e < 4; ++e) z[e] = (4 * j4 + e < prm.d) ? __ldcs(zrow + 4 * j4 + e) : 0.f;
                         }
-                        const float4 c4 = __ldg(reinterpret_cast<const float4*>(cen + 4 * j4));
-                        const float4 s4 = __ldg(reinterpret_cast<const float4*>(scl + 4 * j4));
+                        const float4 c4 = __ldg(reinterpret_cast<const float4*>(cen + R3_IDX(4 * j4, DP - 3, prm.status)));
+                        const float4 s4 = __ldg(reinterpret_cast<const float4*>(scl + R3_IDX(4 * j4, DP - 3, prm.status)));
                         const float cc[4] = {c4.x, c4.y, c4.z, c4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
                         float zt[4];
 #pragma unroll
@@ -456,6 +462,8 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                             zh[4 + e] = *reinterpret_cast<const uint32_t*>(&hi2[e]);
                             zl[4 + e] = *reinterpret_cast<const uint32_t*>(&lo2[e]);
                         }
+                        // candidate planes: columns [ZCOL, ZCOL + DP) of the 512
+                        (void)R3_IDX(ZCOL + DP / 2 + (j8 >> 1) * 8 + 7, min((int)TMEM_COLS, (int)ZCOL + DP), prm.status);
                         tc_st8(lane_addr + ZCOL + (uint32_t)(j8 >> 1) * 8u, zh);
                         tc_st8(lane_addr + ZCOL + (uint32_t)DP / 2 + (uint32_t)(j8 >> 1) * 8u, zl);
                     } else {
@@ -467,7 +475,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     }
                 }
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-                zn_s[row] = far ? -zn : zn;   // the sign carries the out-of-range mark
+                zn_s[R3_IDX(row, TILE_M, prm.status)] = far ? -zn : zn;   // the sign carries the out-of-range mark
                 tc_fence_before();
                 mbar_arrive(bar(BAR_Z_READY));
             }
@@ -509,12 +517,14 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     // k* buffer and the parity of its hand-over: the group's own buffer, or slot t mod NBK of the ring
                     const int kbuf = NBK == G ? grp : (int)(t % NBK);
                     const uint32_t kpar = NBK == G ? own_ph : (uint32_t)((t / NBK) & 1);
-                    uint8_t* kb = sm + map.k + kbuf * 16384u + row * 16;
+                    uint8_t* kb = sm + map.k + (uint32_t)R3_IDX(kbuf, NBK, prm.status) * 16384u + row * 16;
+                    if (KT) (void)R3_IDX(KCOL + kbuf * KC + KC - 1, TMEM_COLS, prm.status);   // the slot's columns in tensor memory
                     uint32_t kh[KC / 16][8], kl[KC / 16][8];
                     // both halves of the chunk's dot products in one round trip to TMEM, then the buffer is free
                     float dots[KC / 16][16];
 #pragma unroll
-                    for (int h = 0; h < KC / 16; ++h) tc_ld16_issue(lane_addr + NV + db * KD + slice * KC + h * 16, dots[h]);
+                    for (int h = 0; h < KC / 16; ++h)
+                        tc_ld16_issue(lane_addr + NV + (uint32_t)R3_IDX(db * KD + slice * KC + h * 16, 2 * KD - 15, prm.status), dots[h]);
                     tc_wait_ld32(dots[0], dots[1]);
                     tc_fence_before();
                     mbar_arrive(bar(BAR_D_EMPTY + db));
@@ -525,7 +535,8 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                         float kv[16];   // k* times kvscale (the power of two of its FP16 split)
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
-                            const float4 xn4 = __ldg(reinterpret_cast<const float4*>(xn_g + c * KC + h * 16 + 4 * q));
+                            const float4 xn4 =
+                                __ldg(reinterpret_cast<const float4*>(xn_g + R3_IDX(c * KC + h * 16 + 4 * q, prm.NP - 3, prm.status)));
                             const float xn[4] = {xn4.x, xn4.y, xn4.z, xn4.w};
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
@@ -543,7 +554,8 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                             // cache without a call; what is left goes to the out-of-line refinement through a local
                             // array, so that the hot path keeps kv in registers.
                             const uint32_t key0 = (((uint32_t)tile_iter & 0x3ffffu) << 13) | (uint32_t)(c * KC + h * 16);
-                            unsigned long long* slots = P > 1 ? pair_cache + row * kCacheSlots : nullptr;
+                            unsigned long long* slots = P > 1 ? pair_cache + R3_IDX(row, TILE_M, prm.status) * kCacheSlots : nullptr;
+                            (void)R3_IDX(c * KC + h * 16 + 15, prm.NP, prm.status);   // rows of the FP32 observations the refinement reads
                             bool need = vmax > v_thresh;
                             if (need && slots && !fresh) {
                                 uint32_t marked = 0;
@@ -580,7 +592,8 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                             float mpart = 0.f, apart = 0.f, spart = 0.f;
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {
-                                const float4 al4 = __ldg(reinterpret_cast<const float4*>(al_g + c * KC + h * 16 + 4 * q));
+                                const float4 al4 =
+                                    __ldg(reinterpret_cast<const float4*>(al_g + R3_IDX(c * KC + h * 16 + 4 * q, prm.NP - 3, prm.status)));
                                 const float al[4] = {al4.x, al4.y, al4.z, al4.w};
 #pragma unroll
                                 for (int e = 0; e < 4; ++e) {
@@ -695,6 +708,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
 #pragma unroll 1
                 for (int c0 = grp * 16; c0 < NV; c0 += 32 * G) {   // two column blocks per round trip to TMEM
                     const int c1 = c0 + 16 * G;
+                    (void)R3_IDX(c0 + 15, NV, prm.status);
                     float v[16], w[16];
                     float part0 = 0.f, part1 = 0.f;
                     if (c1 < NV) {
@@ -719,7 +733,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
             if (!ok) break;
             t_tile0 += items_per_tile;
             // ---- combine the groups' partial sums; group 0 finishes the candidate
-            double* mine = red + ((size_t)grp * TILE_M + row) * 4;
+            double* mine = red + (size_t)R3_IDX(grp * TILE_M + row, G * TILE_M, prm.status) * 4;
             mine[0] = mu_acc; mine[1] = a2_acc; mine[2] = s2_acc; mine[3] = q_acc;
             mbar_arrive(bar(BAR_RED_READY));
             if (grp == 0) {   // only the finishing group waits; the others move on to the next tile
@@ -734,8 +748,8 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                         mu_acc += o[0]; a2_acc += o[1]; s2_acc += o[2]; q_acc += o[3];
                     }
                     q_acc *= prm.vinv2[g];   // undo the power-of-two scaling of k* and W
-                    const size_t f = (size_t)g * prm.m + cand;
-                    const CandidateResult res = finalize_candidate(mu_acc, q_acc, (double)sf2, (double)prm.best[g]);
+                    const size_t f = (size_t)R3_IDX((long long)g * prm.m + cand, (long long)prm.batch * prm.m, prm.status);
+                    const CandidateResult res = finalize_candidate(mu_acc, q_acc, (double)sf2, (double)prm.best[R3_IDX(g, prm.batch, prm.status)]);
                     __stcs(prm.mu + f, res.mu);
                     __stcs(prm.sigma + f, res.sigma);
                     __stcs(prm.ei + f, res.ei);
