@@ -277,11 +277,11 @@ r3_status_t guard_and_rescue(r3_gp* gp, const float* Xcand, long long m, const G
     region = std::max(region, sizeof(unsigned long long) * (size_t)a.slice);
     const size_t smem = region + sizeof(int) * (size_t)a.slice;
     if (R == RESCUE_GROUP) {
-        if (smem > 48 * 1024)
+        if (smem + 1024 > 48 * 1024)   // the kernel's static shared memory counts against the same limit
             R3_CUDA_TRY(cudaFuncSetAttribute(guard_kernel<RESCUE_GROUP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         R3_LAUNCH(guard_kernel<RESCUE_GROUP>, dim3((unsigned)blocks, B), 256, smem, stream, a);
     } else {
-        if (smem > 48 * 1024)
+        if (smem + 1024 > 48 * 1024)   // the kernel's static shared memory counts against the same limit
             R3_CUDA_TRY(cudaFuncSetAttribute(guard_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         R3_LAUNCH(guard_kernel<1>, dim3((unsigned)blocks, B), 256, smem, stream, a);
     }
