@@ -90,7 +90,13 @@ constexpr uint32_t kZnOffset = 512;                   // float[128] squared norm
 // computed its chunk keeps it in registers until the ring slot is free, so the groups still run ahead.
 // F8: the two cross terms of the variance product (W_hi k_lo, W_lo k_hi) are single E4M3 MMAs of depth 32
 // instead of two FP16 MMAs of depth 16 each: four MMAs per chunk instead of six.
-template <int NV, int G, int KD, bool KT, int NBK = G, bool F8 = false>
+// PUTOFF: a pass's epilogue (read the accumulator back, hand it over) is put off until the group's first chunk of
+// the next pass is on its way, when that chunk can be handed over without the accumulator's release (its k* slot is
+// freed by chunks of the old pass): the MMA issuer then finds the new pass's first chunks waiting when the
+// accumulator is released, instead of waiting for them to be computed after it.  With few passes per tile the
+// refill after a hand-over is a visible part of a tile (4-6 % on histories of two to four passes); with many it is
+// not, and the loop structure it needs costs the long histories more than it saves, hence a kernel variant.
+template <int NV, int G, int KD, bool KT, int NBK = G, bool F8 = false, bool PUTOFF = false>
 __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcParams prm)
 {
     static_assert(NBK == G || (KT && NBK >= 2 && NBK < G), "ring of k* buffers: TMEM only");
@@ -493,11 +499,9 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
             const float* al_g = prm.alpha + (size_t)g * prm.NP;
             double mu_acc = 0.0, a2_acc = 0.0, s2_acc = 0.0, q_acc = 0.0;
             int pass_base = 0;   // chunks of this tile before pass p
-            for (int p = 0; ok && p < P; ++p) {
-                const int nchunk = (p + 1) * CPP;
-                // own chunks of this pass: global t with t - t_tile0 - pass_base in [0, nchunk)
-                while (t - t_tile0 - pass_base < nchunk) {
-                    const int c = (int)(t - t_tile0 - pass_base);
+            // one chunk of this group: chunk c of pass p (which has nchunk chunks); clears ok when the CTA aborts
+            auto do_chunk = [&](const int c, const int p, const int nchunk) {
+                {
                     const long long U = t / SL;       // distance product and the slice of its buffer
                     const int db = (int)(U & 1), slice = (int)(t % SL);
                     // the next own chunk's norms and weights: pull them towards L1 while this one is worked on
@@ -509,7 +513,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     TICK(7);
                     ok = mbar_wait(bar(BAR_D_FULL + db), (uint32_t)((U >> 1) & 1), abort_flag, wl);
                     ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
+                    if (!ok) return;
                     TICK(0);
                     if (threadIdx.x % 128 == 0) LOGEV(3, t);
                     tc_fence_after();
@@ -638,7 +642,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                         ok = mbar_wait(bar(BAR_K_EMPTY + (int)(te & 3)), (uint32_t)((te >> 2) & 1), abort_flag, wl);
                     }
                     ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
+                    if (!ok) return;
                     TICK(3);
                     if (threadIdx.x % 128 == 0) LOGEV(5, t);
                     if (F8) {
@@ -683,7 +687,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                             }
                         }
                     }
-                    if (!ok) break;
+                    if (!ok) return;
                     if (KT) {
                         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                         tc_fence_before();
@@ -696,13 +700,13 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     t += G;
                     own_ph ^= 1u;
                 }
-                if (!ok) break;
-                pass_base += nchunk;
-                // ---- end of pass: q += sum_i V^2 over this group's share of the columns
+            };
+            // end of a pass: q += sum_i V^2 over this group's share of the columns, then the accumulator is free
+            auto do_epilogue = [&]() {
                 TICK(7);
                 ok = mbar_wait(bar(BAR_V_FULL), v_ph, abort_flag, wl);
                 ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
+                if (!ok) return;
                 TICK(5);
                 tc_fence_after();
 #pragma unroll 1
@@ -729,6 +733,37 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                 mbar_arrive(bar(BAR_V_EMPTY));
                 TICK(6);
                 v_ph ^= 1u;
+            };
+            if constexpr (!PUTOFF) {
+                for (int p = 0; ok && p < P; ++p) {
+                    const int nchunk = (p + 1) * CPP;
+                    // own chunks of this pass: global t with t - t_tile0 - pass_base in [0, nchunk)
+                    while (ok && t - t_tile0 - pass_base < nchunk) do_chunk((int)(t - t_tile0 - pass_base), p, nchunk);
+                    if (!ok) break;
+                    pass_base += nchunk;
+                    do_epilogue();
+                }
+            } else {
+                // one loop over the group's chunks of the tile, pass after pass, the epilogues in between
+                int p = 0, nchunk = CPP, epilogues_due = 0;
+                while (ok) {
+                    bool first_of_pass = false;
+                    if (t - t_tile0 - pass_base >= nchunk) {   // this group's chunks of pass p are done
+                        pass_base += nchunk;
+                        ++p;
+                        nchunk += CPP;
+                        ++epilogues_due;
+                        first_of_pass = true;
+                    }
+                    const int c = (int)(t - t_tile0 - pass_base);
+                    const bool put_off = first_of_pass && p < P && (NBK == G || c < NBK);
+                    for (int run = epilogues_due - (put_off ? 1 : 0); ok && run > 0; --run) {
+                        --epilogues_due;
+                        do_epilogue();
+                    }
+                    if (!ok || p >= P) break;
+                    do_chunk(c, p, nchunk);
+                }
             }
             if (!ok) break;
             t_tile0 += items_per_tile;
@@ -902,8 +937,12 @@ __global__ void wt_build_kernel(const double* __restrict__ W64, int n, int npad_
 
 TensorOperands* ops_of(const r3_gp* gp) { return static_cast<TensorOperands*>(gp->tc); }
 
-void (*kernel_for(int NV, int G, bool kt, int nbk, bool f8))(const TcParams)
+void (*kernel_for(int NV, int G, bool kt, int nbk, bool f8, bool putoff))(const TcParams)
 {
+    if (putoff && !f8 && NV == 256 && G == 3) {   // histories of two to seven passes in the two preferred shapes
+        if (kt && nbk == 2) return score_tc_kernel<256, 3, 64, true, 2, false, true>;
+        if (!kt && nbk == 3) return score_tc_kernel<256, 3, 64, false, 3, false, true>;
+    }
     if (f8) {   // offered for the shapes of long histories only (tc_prepare)
         if (kt && nbk == 2 && G == 3) return score_tc_kernel<256, 3, 64, true, 2, true>;
         if (kt) return G == 3 ? score_tc_kernel<256, 3, 64, true, 3, true> : score_tc_kernel<256, 2, 64, true, 2, true>;
@@ -1081,7 +1120,7 @@ r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream)
     if ((e = cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, gp->device)) != cudaSuccess)
         return fail("cudaDeviceGetAttribute", e);
     if ((size_t)smem_optin < t->smem_bytes) return decline();
-    e = cudaFuncSetAttribute(kernel_for(t->NV, t->G, t->kt, t->nbk, t->f8), cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(kernel_for(t->NV, t->G, t->kt, t->nbk, t->f8, t->P >= 2 && t->P < kF8MinPasses), cudaFuncAttributeMaxDynamicSharedMemorySize,
                              smem_optin);
     if (e != cudaSuccess) return fail("cudaFuncSetAttribute", e);
     return R3_OK;
@@ -1190,7 +1229,7 @@ r3_status_t score_tc_part(r3_gp* gp, const float* Xcand, long long m, float* mu,
         const r3_status_t st = launch_tc_pair(t, prm, sms, stream);
         if (st != R3_OK) return st;
     } else {
-        void (*kernel)(const TcParams) = kernel_for(t->NV, t->G, t->kt, t->nbk, t->f8);
+        void (*kernel)(const TcParams) = kernel_for(t->NV, t->G, t->kt, t->nbk, t->f8, t->P >= 2 && t->P < kF8MinPasses);
         R3_LAUNCH(kernel, grid, 128 + 128 * t->G, t->smem_bytes, stream, prm);
     }
     prof_end(gp, stream);
