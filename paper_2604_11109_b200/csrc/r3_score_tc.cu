@@ -51,9 +51,14 @@ namespace {
 
 // shared-memory map (byte offsets from a 1024-aligned base)
 struct SmemMap {
-    uint32_t z, k, x, w, bar;   // z: reduction scratch; k: k* buffers (absent when k* lives in TMEM)
+    uint32_t z, k, x, w, zs, bar;   // z: reduction scratch; k: k* buffers (absent when k* lives in TMEM); zs: see kZsStride
     uint32_t x_stage, w_stage;
 };
+// With at most 16 (padded) features the scaled candidates of the tile are also kept in FP32 in shared memory,
+// 128 rows of kZsStride floats (the odd stride keeps a warp's 32 rows on 32 banks): close pairs then get their
+// squared distance from direct differences inline, without the out-of-line refinement and its round trips.
+constexpr uint32_t kZsStride = 17;
+constexpr int kZsMaxDP = 16;
 __host__ __device__ inline SmemMap smem_map(int DP, int NV, int G, int KD, int ws, bool kt)
 {
     SmemMap s;
@@ -63,7 +68,8 @@ __host__ __device__ inline SmemMap smem_map(int DP, int NV, int G, int KD, int w
     s.x_stage = 2u * DP * KD * 2u;
     s.w = s.x + (uint32_t)XS * s.x_stage;          // ws stages x 2 planes x [KC/8][NV][8] halves
     s.w_stage = 2u * KC * NV * 2u;
-    s.bar = s.w + (uint32_t)ws * s.w_stage;
+    s.zs = s.w + (uint32_t)ws * s.w_stage;
+    s.bar = s.zs + (DP <= kZsMaxDP ? TILE_M * kZsStride * 4u : 0u);
     return s;
 }
 // barriers, flags, TMEM slot, candidate norms; then the tile's cache of refined close pairs
@@ -96,7 +102,10 @@ constexpr uint32_t kZnOffset = 512;                   // float[128] squared norm
 // accumulator is released, instead of waiting for them to be computed after it.  With few passes per tile the
 // refill after a hand-over is a visible part of a tile (4-6 % on histories of two to four passes); with many it is
 // not, and the loop structure it needs costs the long histories more than it saves, hence a kernel variant.
-template <int NV, int G, int KD, bool KT, int NBK = G, bool F8 = false, bool PUTOFF = false>
+// ZS: the feature count is at most 16: close pairs are refined inline from the FP32 copy of the scaled tile in
+// shared memory (pools of few features are full of close pairs: on the 16-feature workload 98 % of a warp's
+// 16-entry blocks hold one, and the out-of-line refinement was most of the kernel's time).
+template <int NV, int G, int KD, bool KT, int NBK = G, bool F8 = false, bool PUTOFF = false, bool ZS = false>
 __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcParams prm)
 {
     static_assert(NBK == G || (KT && NBK >= 2 && NBK < G), "ring of k* buffers: TMEM only");
@@ -110,6 +119,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + map.bar + kFlagOffset + 8);
     float* zn_s = reinterpret_cast<float*>(sm + map.bar + kZnOffset);
     unsigned long long* pair_cache = reinterpret_cast<unsigned long long*>(sm + map.bar + kCacheOffset);
+    float* zs_s = reinterpret_cast<float*>(sm + map.zs);
     auto bar = [&](uint32_t slot) { return bars + slot * 8u; };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -460,6 +470,10 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                         }
                         split2(zt[0], zt[1], hi2[2 * h], lo2[2 * h]);
                         split2(zt[2], zt[3], hi2[2 * h + 1], lo2[2 * h + 1]);
+                        if (ZS) {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) zs_s[row * kZsStride + 4 * j4 + e] = zt[e];
+                        }
                     }
                     // 8 features = 4 columns of each plane; two such groups make one 8-column store
                     if (j8 & 1) {
@@ -553,6 +567,36 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
 #pragma unroll
                         for (int i = 4; i < 16; i += 4)
                             vmax = fmaxf(vmax, fmaxf(fmaxf(kv[i], kv[i + 1]), fmaxf(kv[i + 2], kv[i + 3])));
+                        if (ZS) {
+                            if (vmax > v_thresh) {   // close pairs of this candidate: direct differences, inline
+                                uint32_t marked = 0;
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) marked |= (kv[i] > v_thresh) ? (1u << i) : 0u;
+                                const float* zr = zs_s + row * kZsStride;
+                                for (; marked; marked &= marked - 1) {
+                                    const uint32_t i = (uint32_t)__ffs(marked) - 1u;
+                                    const float4* xp = reinterpret_cast<const float4*>(
+                                        xs_g + (size_t)R3_IDX(c * KC + h * 16 + (int)i, prm.NP, prm.status) * kZsMaxDP);
+                                    float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+                                    for (int e = 0; e < 4; ++e) {
+                                        const float4 x4 = __ldg(xp + e);
+                                        float df = zr[4 * e] - x4.x;
+                                        acc0 = fmaf(df, df, acc0);
+                                        df = zr[4 * e + 1] - x4.y;
+                                        acc1 = fmaf(df, df, acc1);
+                                        df = zr[4 * e + 2] - x4.z;
+                                        acc0 = fmaf(df, df, acc0);
+                                        df = zr[4 * e + 3] - x4.w;
+                                        acc1 = fmaf(df, df, acc1);
+                                    }
+                                    const float u = sqrtf(acc0 + acc1);
+                                    const float val = kvscale * fmaf(u, fmaf(u, kPolyC2, kPolyC1), 1.f) * exp2f(-u);
+#pragma unroll
+                                    for (int e2 = 0; e2 < 16; ++e2) kv[e2] = (uint32_t)e2 == i ? val : kv[e2];
+                                }
+                            }
+                        } else
                         if (__any_sync(0xffffffffu, vmax > v_thresh)) {
                             // rare: close pairs.  Values refined in an earlier pass of this tile come back from the
                             // cache without a call; what is left goes to the out-of-line refinement through a local
@@ -937,8 +981,12 @@ __global__ void wt_build_kernel(const double* __restrict__ W64, int n, int npad_
 
 TensorOperands* ops_of(const r3_gp* gp) { return static_cast<TensorOperands*>(gp->tc); }
 
-void (*kernel_for(int NV, int G, bool kt, int nbk, bool f8, bool putoff))(const TcParams)
+void (*kernel_for(int NV, int G, bool kt, int nbk, bool f8, bool putoff, bool zs))(const TcParams)
 {
+    if (zs && kt && nbk == 2 && G == 3 && !f8) {   // at most 16 features, in the preferred shape
+        if (NV == 128) return score_tc_kernel<128, 3, 64, true, 2, false, false, true>;
+        return putoff ? score_tc_kernel<256, 3, 64, true, 2, false, true, true> : score_tc_kernel<256, 3, 64, true, 2, false, false, true>;
+    }
     if (putoff && !f8 && NV == 256 && G == 3) {   // histories of two to seven passes in the two preferred shapes
         if (kt && nbk == 2) return score_tc_kernel<256, 3, 64, true, 2, false, true>;
         if (!kt && nbk == 3) return score_tc_kernel<256, 3, 64, false, 3, false, true>;
@@ -1120,7 +1168,7 @@ r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream)
     if ((e = cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, gp->device)) != cudaSuccess)
         return fail("cudaDeviceGetAttribute", e);
     if ((size_t)smem_optin < t->smem_bytes) return decline();
-    e = cudaFuncSetAttribute(kernel_for(t->NV, t->G, t->kt, t->nbk, t->f8, t->P >= 2 && t->P < kF8MinPasses), cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(kernel_for(t->NV, t->G, t->kt, t->nbk, t->f8, t->P >= 2 && t->P < kF8MinPasses, t->DP <= kZsMaxDP), cudaFuncAttributeMaxDynamicSharedMemorySize,
                              smem_optin);
     if (e != cudaSuccess) return fail("cudaFuncSetAttribute", e);
     return R3_OK;
@@ -1229,7 +1277,7 @@ r3_status_t score_tc_part(r3_gp* gp, const float* Xcand, long long m, float* mu,
         const r3_status_t st = launch_tc_pair(t, prm, sms, stream);
         if (st != R3_OK) return st;
     } else {
-        void (*kernel)(const TcParams) = kernel_for(t->NV, t->G, t->kt, t->nbk, t->f8, t->P >= 2 && t->P < kF8MinPasses);
+        void (*kernel)(const TcParams) = kernel_for(t->NV, t->G, t->kt, t->nbk, t->f8, t->P >= 2 && t->P < kF8MinPasses, t->DP <= kZsMaxDP);
         R3_LAUNCH(kernel, grid, 128 + 128 * t->G, t->smem_bytes, stream, prm);
     }
     prof_end(gp, stream);
