@@ -136,6 +136,17 @@ def test_candidates_on_and_near_observations_are_rescued(engine):
     gp.close()
 
 
+@pytest.mark.parametrize("engine", ENGINES)
+@pytest.mark.parametrize("batch,m,k", [(1, 33, 1), (2, 40, 40), (1, 1500, 1024), (3, 5000, 300), (1, 70000, 1000)])
+def test_selection_sizes_through_the_scoring_call(engine, batch, m, k):
+    """The first level of the selection is taken by the guard's kernel, a block per slice of candidates: k larger
+    than a slice, k equal to the pool, slices with a ragged tail, several GPs."""
+    g = rand_problem(300 + m, batch, 90, 5, m)
+    gp = fit_gpu(g, engine)
+    compare_everything(g, gp, k, f"selection m{m} k{k}")
+    gp.close()
+
+
 def test_incumbent_override_and_engine_query():
     g = rand_problem(77, 2, 40, 4, 300)
     gp = fit_gpu(g)
