@@ -147,6 +147,22 @@ def test_selection_sizes_through_the_scoring_call(engine, batch, m, k):
     gp.close()
 
 
+@pytest.mark.parametrize("spread,sn2", [(1.0, 1e-3), (3.0, 1e-4)])
+def test_long_history_with_fp8_cross_terms_near_observations(spread, sn2):
+    """From eight passes on (n > 1792) the variance product's cross terms are E4M3 MMAs; their error estimate has to
+    send the candidates for which that matters -- on and next to observations, long lengthscales -- to the FP64
+    pass.  Every element and the top-k against the oracle."""
+    n, d, m = 2100, 20, 700
+    g = rand_problem(2100 + int(spread), 1, n, d, m, sn2=sn2, spread=spread * np.sqrt(d) / 2)
+    g["Xcand"][0, :200] = g["X"][0, :200]
+    g["Xcand"][0, 200:400] = g["X"][0, 200:400] + np.float32(2e-3)
+    gp = fit_gpu(g, b.ENGINE_TENSOR)
+    assert b.r3_gp_tensor_info(gp)["f8_cross_terms"] == 1
+    compare_everything(g, gp, 32, f"fp8 cross terms, spread {spread}")
+    assert b.r3_gp_last_rescued(gp) >= 200          # the candidates on observations at the least
+    gp.close()
+
+
 def test_incumbent_override_and_engine_query():
     g = rand_problem(77, 2, 40, 4, 300)
     gp = fit_gpu(g)
