@@ -438,60 +438,130 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                 const float* cen = prm.centre + (size_t)g * DP;
                 const float* scl = prm.scale + (size_t)g * DP;
                 const bool vec = (prm.d % 4) == 0 && (reinterpret_cast<uintptr_t>(prm.xcand) & 15) == 0;
-                uint32_t zh[8], zl[8];
-                for (int j8 = 0; j8 < DP / 8; ++j8) {
-                    __half2 hi2[4], lo2[4];
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const int j4 = 2 * j8 + h;
-                        float z[4];
-                        if (vec && 4 * j4 < prm.d) {
-                            // read once: streaming load, so that the pool does not push W out of L2
-                            const float4 v = __ldcs(reinterpret_cast<const float4*>(zrow + 4 * j4));
-                            z[0] = v.x; z[1] = v.y; z[2] = v.z; z[3] = v.w;
-                        } else {
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) z[e] = (4 * j4 + e < prm.d) ? __ldcs(zrow + 4 * j4 + e) : 0.f;
-                        }
-                        const float4 c4 = __ldg(reinterpret_cast<const float4*>(cen + R3_IDX(4 * j4, DP - 3, prm.status)));
-                        const float4 s4 = __ldg(reinterpret_cast<const float4*>(scl + R3_IDX(4 * j4, DP - 3, prm.status)));
-                        const float cc[4] = {c4.x, c4.y, c4.z, c4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
-                        float zt[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            bad |= !isfinite(z[e]);
-                            float v = valid ? (z[e] - cc[e]) * ss[e] : 0.f;
-                            if (fabsf(v) > kMaxScaled) {   // outside the FP16 planes' range: clamp, and have it recomputed
-                                v = copysignf(kMaxScaled, v);
-                                far = true;
+                // Two forms of the same loop over the row's features.  The long-history kernel keeps the plain one: its
+                // chunk loop sits at the register limit, and the pipelined form, although it runs once per tile, costs
+                // that loop registers (config 5: 45.9 ms to 47.9 ms per pool); everywhere else the row's loads overlap
+                // (config 3: 5.74 ms to 5.52 ms).
+                if constexpr (F8) {
+                    uint32_t zh[8], zl[8];
+                    for (int j8 = 0; j8 < DP / 8; ++j8) {
+                        __half2 hi2[4], lo2[4];
+    #pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const int j4 = 2 * j8 + h;
+                            float z[4];
+                            if (vec && 4 * j4 < prm.d) {
+                                // read once: streaming load, so that the pool does not push W out of L2
+                                const float4 v = __ldcs(reinterpret_cast<const float4*>(zrow + 4 * j4));
+                                z[0] = v.x; z[1] = v.y; z[2] = v.z; z[3] = v.w;
+                            } else {
+    #pragma unroll
+                                for (int e = 0; e < 4; ++e) z[e] = (4 * j4 + e < prm.d) ? __ldcs(zrow + 4 * j4 + e) : 0.f;
                             }
-                            zt[e] = v;
-                            zn = fmaf(v, v, zn);
+                            const float4 c4 = __ldg(reinterpret_cast<const float4*>(cen + R3_IDX(4 * j4, DP - 3, prm.status)));
+                            const float4 s4 = __ldg(reinterpret_cast<const float4*>(scl + R3_IDX(4 * j4, DP - 3, prm.status)));
+                            const float cc[4] = {c4.x, c4.y, c4.z, c4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
+                            float zt[4];
+    #pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                bad |= !isfinite(z[e]);
+                                float v = valid ? (z[e] - cc[e]) * ss[e] : 0.f;
+                                if (fabsf(v) > kMaxScaled) {   // outside the FP16 planes' range: clamp, and have it recomputed
+                                    v = copysignf(kMaxScaled, v);
+                                    far = true;
+                                }
+                                zt[e] = v;
+                                zn = fmaf(v, v, zn);
+                            }
+                            split2(zt[0], zt[1], hi2[2 * h], lo2[2 * h]);
+                            split2(zt[2], zt[3], hi2[2 * h + 1], lo2[2 * h + 1]);
+                            if (ZS) {
+    #pragma unroll
+                                for (int e = 0; e < 4; ++e) zs_s[row * kZsStride + 4 * j4 + e] = zt[e];
+                            }
                         }
-                        split2(zt[0], zt[1], hi2[2 * h], lo2[2 * h]);
-                        split2(zt[2], zt[3], hi2[2 * h + 1], lo2[2 * h + 1]);
-                        if (ZS) {
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) zs_s[row * kZsStride + 4 * j4 + e] = zt[e];
+                        // 8 features = 4 columns of each plane; two such groups make one 8-column store
+                        if (j8 & 1) {
+    #pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                zh[4 + e] = *reinterpret_cast<const uint32_t*>(&hi2[e]);
+                                zl[4 + e] = *reinterpret_cast<const uint32_t*>(&lo2[e]);
+                            }
+                            // candidate planes: columns [ZCOL, ZCOL + DP) of the 512
+                            (void)R3_IDX(ZCOL + DP / 2 + (j8 >> 1) * 8 + 7, min((int)TMEM_COLS, (int)ZCOL + DP), prm.status);
+                            tc_st8(lane_addr + ZCOL + (uint32_t)(j8 >> 1) * 8u, zh);
+                            tc_st8(lane_addr + ZCOL + (uint32_t)DP / 2 + (uint32_t)(j8 >> 1) * 8u, zl);
+                        } else {
+    #pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                zh[e] = *reinterpret_cast<const uint32_t*>(&hi2[e]);
+                                zl[e] = *reinterpret_cast<const uint32_t*>(&lo2[e]);
+                            }
                         }
                     }
-                    // 8 features = 4 columns of each plane; two such groups make one 8-column store
-                    if (j8 & 1) {
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            zh[4 + e] = *reinterpret_cast<const uint32_t*>(&hi2[e]);
-                            zl[4 + e] = *reinterpret_cast<const uint32_t*>(&lo2[e]);
+                } else {
+                    // 16 features per step (one 8-column store to each plane); the next step's four loads are under way
+                    // while this one is scaled and split, so that the row costs one trip to L2 or HBM and not DP / 8
+                    auto load4 = [&](int j4) {
+                        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (vec && 4 * j4 < prm.d) {
+                            // read once: streaming load, so that the pool does not push W out of L2
+                            v = __ldcs(reinterpret_cast<const float4*>(zrow + 4 * j4));
+                        } else if (4 * j4 < prm.d) {
+                            v.x = __ldcs(zrow + 4 * j4);
+                            v.y = (4 * j4 + 1 < prm.d) ? __ldcs(zrow + 4 * j4 + 1) : 0.f;
+                            v.z = (4 * j4 + 2 < prm.d) ? __ldcs(zrow + 4 * j4 + 2) : 0.f;
+                            v.w = (4 * j4 + 3 < prm.d) ? __ldcs(zrow + 4 * j4 + 3) : 0.f;
+                        }
+                        return v;
+                    };
+                    float4 nxt[4];
+    #pragma unroll
+                    for (int h = 0; h < 4; ++h) nxt[h] = load4(h);
+                    for (int j16 = 0; j16 < DP / 16; ++j16) {
+                        float4 cur[4];
+    #pragma unroll
+                        for (int h = 0; h < 4; ++h) cur[h] = nxt[h];
+                        if (j16 + 1 < DP / 16) {
+    #pragma unroll
+                            for (int h = 0; h < 4; ++h) nxt[h] = load4(4 * (j16 + 1) + h);
+                        }
+                        uint32_t zh[8], zl[8];
+    #pragma unroll
+                        for (int h = 0; h < 4; ++h) {
+                            const int j4 = 4 * j16 + h;
+                            const float z[4] = {cur[h].x, cur[h].y, cur[h].z, cur[h].w};
+                            const float4 c4 = __ldg(reinterpret_cast<const float4*>(cen + R3_IDX(4 * j4, DP - 3, prm.status)));
+                            const float4 s4 = __ldg(reinterpret_cast<const float4*>(scl + R3_IDX(4 * j4, DP - 3, prm.status)));
+                            const float cc[4] = {c4.x, c4.y, c4.z, c4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
+                            float zt[4];
+    #pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                bad |= !isfinite(z[e]);
+                                float v = valid ? (z[e] - cc[e]) * ss[e] : 0.f;
+                                if (fabsf(v) > kMaxScaled) {   // outside the FP16 planes' range: clamp, and have it recomputed
+                                    v = copysignf(kMaxScaled, v);
+                                    far = true;
+                                }
+                                zt[e] = v;
+                                zn = fmaf(v, v, zn);
+                            }
+                            __half2 hi0, lo0, hi1, lo1;
+                            split2(zt[0], zt[1], hi0, lo0);
+                            split2(zt[2], zt[3], hi1, lo1);
+                            zh[2 * h] = *reinterpret_cast<const uint32_t*>(&hi0);
+                            zh[2 * h + 1] = *reinterpret_cast<const uint32_t*>(&hi1);
+                            zl[2 * h] = *reinterpret_cast<const uint32_t*>(&lo0);
+                            zl[2 * h + 1] = *reinterpret_cast<const uint32_t*>(&lo1);
+                            if (ZS) {
+    #pragma unroll
+                                for (int e = 0; e < 4; ++e) zs_s[row * kZsStride + 4 * j4 + e] = zt[e];
+                            }
                         }
                         // candidate planes: columns [ZCOL, ZCOL + DP) of the 512
-                        (void)R3_IDX(ZCOL + DP / 2 + (j8 >> 1) * 8 + 7, min((int)TMEM_COLS, (int)ZCOL + DP), prm.status);
-                        tc_st8(lane_addr + ZCOL + (uint32_t)(j8 >> 1) * 8u, zh);
-                        tc_st8(lane_addr + ZCOL + (uint32_t)DP / 2 + (uint32_t)(j8 >> 1) * 8u, zl);
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            zh[e] = *reinterpret_cast<const uint32_t*>(&hi2[e]);
-                            zl[e] = *reinterpret_cast<const uint32_t*>(&lo2[e]);
-                        }
+                        (void)R3_IDX(ZCOL + DP / 2 + j16 * 8 + 7, min((int)TMEM_COLS, (int)ZCOL + DP), prm.status);
+                        tc_st8(lane_addr + ZCOL + (uint32_t)j16 * 8u, zh);
+                        tc_st8(lane_addr + ZCOL + (uint32_t)DP / 2 + (uint32_t)j16 * 8u, zl);
                     }
                 }
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
