@@ -10,7 +10,7 @@
 //   flags    the candidates of its slice whose estimated error exceeds half of the accuracy contract
 //            (1e-4 relative on mu and sigma with absolute floors, 1e-5 max(EI) on EI),
 //   rescues  them: recomputes them from the raw inputs entirely in FP64 -- direct-difference distances with
-//            a true division by the lengthscale, FP64 weights and the FP64 inverse factor -- and overwrites
+//            FP64 reciprocal lengthscales, FP64 weights and the FP64 inverse factor -- and overwrites
 //            their mu, sigma and EI,
 //   selects  (when the call asked for a top-k) the k largest final EI of its slice as 64-bit keys: the first
 //            level of the selection, taken while the slice's values are at hand; r3_topk.cu finishes it.
@@ -59,7 +59,7 @@ __global__ void __launch_bounds__(256) guard_kernel(const GuardArgs a)
     // rescue: ks [R][npad], zs [R][d], ls [d]; afterwards the same bytes hold the slice's keys
     double* ks = smem;
     double* zs = smem + (size_t)R * a.npad;
-    double* ls = zs + (size_t)R * a.d;
+    double* ls = zs + (size_t)R * a.d;   // [d] reciprocal lengthscales
     __shared__ double red[2][R][8];
     __shared__ int nflag_s;
     const int g = blockIdx.y;
@@ -107,7 +107,9 @@ __global__ void __launch_bounds__(256) guard_kernel(const GuardArgs a)
         const double* ag = a.alpha64 + (size_t)g * a.npad;
         const double sf2 = (double)a.sf2v[g];
         const int n = a.n, d = a.d, npad = a.npad;
-        for (int j = t; j < d; j += 256) ls[j] = (double)a.ell[(size_t)g * d + j];
+        // reciprocal lengthscales in FP64: one rounding of 2^-53 per difference against an FP64 division per
+        // difference (the divisions were most of a rescue's time at d = 128)
+        for (int j = t; j < d; j += 256) ls[j] = 1.0 / (double)a.ell[(size_t)g * d + j];
         for (int e0 = 0; e0 < total; e0 += R) {
             const int nr = min(R, total - e0);
             __syncthreads();
@@ -125,10 +127,10 @@ __global__ void __launch_bounds__(256) guard_kernel(const GuardArgs a)
 #pragma unroll
                 for (int r = 0; r < R; ++r) r2[r] = 0.0;
                 for (int j = 0; j < d; ++j) {
-                    const double x = (double)Xg[(size_t)i * d + j], l = ls[j];
+                    const double x = (double)Xg[(size_t)i * d + j], il = ls[j];
 #pragma unroll
                     for (int r = 0; r < R; ++r) {
-                        const double df = (x - zs[r * d + j]) / l;
+                        const double df = (x - zs[r * d + j]) * il;
                         r2[r] += df * df;
                     }
                 }
