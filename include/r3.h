@@ -149,6 +149,10 @@ r3_status_t r3_topk_noalloc(const float* ei, int batch, long long m, int k, int*
  * r3_gp_score_topk -- r3_gp_score followed by r3_topk on the EI it produced, with
  * the handle's own workspace; asynchronous on `cuda_stream`.  This is the "one
  * BO proposal round" call: idx [batch][k] are the pool members to replay next.
+ * The first level of the selection is taken by the accuracy guard's kernel, which
+ * runs over the final EI anyway, so a step is four or five kernel launches.  Once
+ * the workspace has its size (a first call with this m and k) the call only
+ * enqueues work on `cuda_stream` and can be captured in a CUDA graph.
  */
 r3_status_t r3_gp_score_topk(r3_gp_t* gp, const float* Xcand, long long m, int k, float* mu,
                              float* sigma, float* ei, int* idx, float* val, void* cuda_stream);
