@@ -36,6 +36,7 @@
 // Operand layouts are the no-swizzle K-major "core matrix" form: 8 rows x 16 bytes contiguous, 8-row
 // groups 128 bytes apart, 16-byte k-slices one full panel apart.  W and the observations are stored
 // in global memory already tiled that way by the fit, so a stage is one contiguous bulk copy.
+#include <algorithm>
 #include <cuda_fp16.h>
 #include <math.h>
 #include <stdio.h>
@@ -1131,6 +1132,11 @@ r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream)
         {true, 3, 3, 2},  {false, 3, 3, 3}, {true, 3, 3, 3}, {true, 2, 3, 2},
         {false, 2, 3, 2}, {false, 3, 2, 3}, {true, 2, 2, 2}, {false, 2, 2, 2}};
     const int want_nbk = env_int("R3_TC_NBK", 0);
+    // Stages of W: four by default although shared memory would hold up to six for few features.  Measured, the
+    // fifth and sixth buy nothing on any workload and cost the short histories 3-5 % (256 observations, 16
+    // features: 0.241 ms to 0.228 ms per pool; 512 and 32: 5.79 ms to 5.63 ms; 1024 and 4096 observations:
+    // unchanged down to three).  R3_TC_MAXWS = 2..6 overrides.
+    const int max_ws = std::min(std::max(env_int("R3_TC_MAXWS", 4), 2), MAX_STAGES);
     for (const auto& pr : prefs) {
         if (found) break;
         t->kt = pr.kt;
@@ -1140,7 +1146,7 @@ r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream)
         if (want_g && t->G != want_g) continue;
         if (want_nbk && t->nbk != want_nbk) continue;
         if (t->NV + 2 * t->KD + t->DP + (t->kt ? t->nbk * KC : 0) > 512) continue;
-        for (t->ws = MAX_STAGES; t->ws >= 2; --t->ws)
+        for (t->ws = max_ws; t->ws >= 2; --t->ws)
             if (smem_map(t->DP, t->NV, t->G, t->KD, t->ws, t->kt).bar <= budget) break;
         found = t->ws >= pr.min_ws;
     }
