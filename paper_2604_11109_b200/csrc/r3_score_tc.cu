@@ -60,6 +60,11 @@ struct SmemMap {
 // squared distance from direct differences inline, without the out-of-line refinement and its round trips.
 constexpr uint32_t kZsStride = 17;
 constexpr int kZsMaxDP = 16;
+// Registers per thread after the roles have parted: the kernel starts with the register file split evenly
+// (128 per thread for 512 threads, 168 for 384); the four control warps, whose loops are short, give theirs back
+// and the Matern groups, whose chunk loop does not fit 128 without spills, take them.
+constexpr int kRegsControl = 80;
+__host__ __device__ constexpr int regs_matern(int G) { return G == 3 ? 144 : 208; }
 __host__ __device__ inline SmemMap smem_map(int DP, int NV, int G, int KD, int ws, bool kt)
 {
     SmemMap s;
@@ -184,6 +189,8 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
     long long tacc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     long long tlast = prm.trace ? clock64() : 0;
 
+    if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsControl));
     if (warp == 0 && lane == 0) {
         // ------------------------------------------------------------ producer: scaled observations
         const uint32_t bytes = map.x_stage;
@@ -397,7 +404,9 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
         mbar_wait(bar(BAR_MMA_DONE + 1), 0, abort_flag + 1, wl);
         if (prm.trace)
             for (int i = 0; i < 8; ++i) prm.trace[((size_t)blockIdx.x * 4 + 0) * 8 + i] = tacc[i];
-    } else if (warp >= 4) {
+    }
+    } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(regs_matern(G)));
         // ------------------------------------------------------------ Matern / epilogue warp groups
         const int grp = (warp - 4) >> 2;         // 0..G-1
         const int q4 = warp & 3;                 // TMEM lane quarter == warp % 4
