@@ -35,7 +35,8 @@ struct GuardArgs {
     const unsigned* maxbits;      // [batch] bit pattern of the pool's largest EI
     int* count;                   // [batch] candidates recomputed (diagnostics)
     int* status;                  // the handle's status words (index checks of the bounds-checking build)
-    int k, K2;                    // top-k request (k = 0: none); K2 = min(2^ceil(log2 k), slice)
+    int k, K2;                    // top-k request (k = 0: none); K2 = min(k, slice): keys a block selects
+    unsigned select_offset;       // byte offset of the selection's scratch in the dynamic shared memory
     unsigned long long* keys;     // [batch][blocks][k]
 };
 
@@ -196,7 +197,7 @@ __global__ void __launch_bounds__(256) guard_kernel(const GuardArgs a)
         const long long c = c_begin + i;
         keys_s[i] = (c < m) ? topk_make_key(e[c], (unsigned)c) : 0ull;
     }
-    block_topk_desc(keys_s, a.slice, a.K2);
+    block_select_desc(keys_s, a.slice, a.K2, reinterpret_cast<char*>(smem) + a.select_offset);
     unsigned long long* out = a.keys + ((size_t)g * gridDim.x + blockIdx.x) * a.k;
     for (int i = t; i < a.k; i += 256) out[i] = i < a.slice ? keys_s[R3_IDX(i, a.slice, a.status)] : 0ull;
 }
@@ -267,7 +268,7 @@ r3_status_t guard_and_rescue(r3_gp* gp, const float* Xcand, long long m, const G
     a.count = b.count;
     a.status = gp->status_d;
     a.k = req.k;
-    a.K2 = req.k > 0 ? std::min(topk_pow2_at_least(req.k), a.slice) : 1;
+    a.K2 = req.k > 0 ? std::min(req.k, a.slice) : 1;   // keys a block selects
     a.keys = (unsigned long long*)req.ws;
     const long long blocks = (m + a.slice - 1) / a.slice;
     if (req.k > 0 && req.ws_bytes < guard_topk_workspace_bytes(B, m, req.k)) {
@@ -277,7 +278,9 @@ r3_status_t guard_and_rescue(r3_gp* gp, const float* Xcand, long long m, const G
     const int R = gp->npad <= 4096 ? RESCUE_GROUP : 1;
     size_t region = sizeof(double) * ((size_t)R * gp->npad + (size_t)R * gp->d + gp->d);
     region = std::max(region, sizeof(unsigned long long) * (size_t)a.slice);
-    const size_t smem = region + sizeof(int) * (size_t)a.slice;
+    // after the flag list (unused by then, but kept apart): the scratch of the slice's top-k selection
+    a.select_offset = (unsigned)((region + sizeof(int) * (size_t)a.slice + 7) & ~(size_t)7);
+    const size_t smem = a.select_offset + (req.k > 0 ? topk_select_scratch_bytes(a.K2) : 0);
     if (R == RESCUE_GROUP) {
         if (smem + 1024 > 48 * 1024)   // the kernel's static shared memory counts against the same limit
             R3_CUDA_TRY(cudaFuncSetAttribute(guard_kernel<RESCUE_GROUP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

@@ -2,8 +2,8 @@
 //
 // A value and its index are packed in one 64-bit key (r3_topk.cuh) whose unsigned order is exactly "larger
 // value, or equal value and smaller index".  A block takes a chunk of 4096 keys into shared memory and keeps
-// its k largest (block_topk_desc: blocks of k sorted by a bitonic network, then halving merges); levels repeat
-// until one chunk is left, and the block that handles it writes the indices and values.  The first level
+// its k largest (block_select_desc: radix selection of the k-th largest, then a rank sort of the k survivors);
+// levels repeat until one chunk is left, and the block that handles it writes the indices and values.  The first level
 // reads the EI array once (4 bytes per candidate); later levels touch k keys per chunk of the level before.
 // When the scoring call asked for a top-k, the accuracy guard's kernel has already left the first level's keys
 // (r3_rescue.cu), and only the later levels run here.
@@ -18,6 +18,8 @@ namespace {
 
 constexpr int CHUNK = 4096;      // keys per block
 constexpr int THREADS = 1024;
+constexpr int kMaxK = 1024;      // the interface's limit on k
+constexpr size_t kSelectBytes = sizeof(unsigned long long) * kMaxK + sizeof(unsigned) * (kMaxK + 256 + 8);
 
 // The last level writes the answer instead of keys: idx (and val, read back from the EI array) are non-null.
 __device__ __forceinline__ void emit(const unsigned long long* s, int k, unsigned long long* out_keys,
@@ -39,10 +41,11 @@ __device__ __forceinline__ void emit(const unsigned long long* s, int k, unsigne
 
 // Level 0: keys from the EI array.  grid = (chunks, batch).
 __global__ void __launch_bounds__(THREADS) topk_from_values_kernel(const float* __restrict__ ei, long long m,
-                                                                   int k, int K2, unsigned long long* __restrict__ out,
+                                                                   int k, unsigned long long* __restrict__ out,
                                                                    int* __restrict__ idx, float* __restrict__ val)
 {
     __shared__ unsigned long long s[CHUNK];
+    __shared__ unsigned long long scratch[kSelectBytes / 8];
     const int g = blockIdx.y;
     const long long base = (long long)blockIdx.x * CHUNK;
     const float* e = ei + (size_t)g * m;
@@ -50,18 +53,19 @@ __global__ void __launch_bounds__(THREADS) topk_from_values_kernel(const float* 
         const long long i = base + t;
         s[t] = (i < m) ? topk_make_key(e[i], (unsigned)i) : 0ull;
     }
-    block_topk_desc(s, CHUNK, K2);
+    block_select_desc(s, CHUNK, k, scratch);
     emit(s, k, out, ei, m, idx, val);
 }
 
 // Later levels: keys from the level before.  count = keys per GP in `in`.
 __global__ void __launch_bounds__(THREADS) topk_from_keys_kernel(const unsigned long long* __restrict__ in,
-                                                                 long long count, int k, int K2,
+                                                                 long long count, int k,
                                                                  unsigned long long* __restrict__ out,
                                                                  const float* __restrict__ ei, long long m,
                                                                  int* __restrict__ idx, float* __restrict__ val)
 {
     __shared__ unsigned long long s[CHUNK];
+    __shared__ unsigned long long scratch[kSelectBytes / 8];
     const int g = blockIdx.y;
     const long long base = (long long)blockIdx.x * CHUNK;
     const unsigned long long* src = in + (size_t)g * count;
@@ -69,7 +73,7 @@ __global__ void __launch_bounds__(THREADS) topk_from_keys_kernel(const unsigned 
         const long long i = base + t;
         s[t] = (i < count) ? src[i] : 0ull;
     }
-    block_topk_desc(s, CHUNK, K2);
+    block_select_desc(s, CHUNK, k, scratch);
     emit(s, k, out, ei, m, idx, val);
 }
 
@@ -123,13 +127,12 @@ size_t topk_workspace_bytes(int batch, long long m, int k)
 r3_status_t topk_finish_from_keys(unsigned long long* keys_in, unsigned long long* keys_tmp, int batch, long long count,
                                   int k, const float* ei, long long m, int* idx, float* val, cudaStream_t stream)
 {
-    const int K2 = topk_pow2_at_least(k);
     unsigned long long* buf[2] = {keys_in, keys_tmp};
     int cur = 0;
     while (true) {
         const long long chunks = chunks_of(count);
         const bool last = chunks == 1;
-        R3_LAUNCH(topk_from_keys_kernel, dim3((unsigned)chunks, batch), THREADS, 0, stream, buf[cur], count, k, K2,
+        R3_LAUNCH(topk_from_keys_kernel, dim3((unsigned)chunks, batch), THREADS, 0, stream, buf[cur], count, k,
                   buf[cur ^ 1], ei, m, last ? idx : nullptr, last ? val : nullptr);
         if (last) break;
         cur ^= 1;
@@ -148,9 +151,8 @@ r3_status_t topk_device(const float* ei, int batch, long long m, int k, int* idx
     const size_t level0 = (size_t)batch * chunks_of(m) * k;
     unsigned long long* buf[2] = {(unsigned long long*)ws, (unsigned long long*)ws + level0};
     const long long chunks = chunks_of(m);
-    const int K2 = topk_pow2_at_least(k);
     const bool last = chunks == 1;
-    R3_LAUNCH(topk_from_values_kernel, dim3((unsigned)chunks, batch), THREADS, 0, stream, ei, m, k, K2, buf[0],
+    R3_LAUNCH(topk_from_values_kernel, dim3((unsigned)chunks, batch), THREADS, 0, stream, ei, m, k, buf[0],
               last ? idx : nullptr, last ? val : nullptr);
     if (last) return R3_OK;
     return topk_finish_from_keys(buf[0], buf[1], batch, chunks * k, k, ei, m, idx, val, stream);
