@@ -249,6 +249,38 @@ def test_topk_matches_oracle_exactly(batch, m, k):
         assert np.array_equal(val[q], rval.astype(np.float32))
 
 
+def test_topk_degenerate_pools():
+    """Pools that defeat a selection by value alone: every value equal (the indices decide), a handful of distinct
+    values, values that differ in their last mantissa bits only, mostly NaN, signed values with an odd k above the
+    size from which the survivors go through the sorting network."""
+    rng = np.random.default_rng(77)
+    for k in (50, 300, 1024):
+        idx, val = b.r3_topk(dev(np.zeros((2, 10000), dtype=np.float32)), k)
+        assert np.array_equal(idx.cpu().numpy(), np.tile(np.arange(k), (2, 1)))
+        assert not val.cpu().numpy().any()
+    cases = [
+        (rng.choice(np.array([0.0, 1e-30, 0.5], dtype=np.float32), size=(1, 70001)), 600),
+        ((1.0 + rng.integers(0, 64, size=(2, 20000)) * 2.0 ** -23).astype(np.float32), 129),
+        (rng.normal(size=(3, 8191)).astype(np.float32), 257),
+        (np.full((1, 4096), 7.0, dtype=np.float32), 4096 // 4),
+    ]
+    for e, k in cases:
+        idx, val = b.r3_topk(dev(e), k)
+        for q in range(e.shape[0]):
+            ridx, rval = o.topk(e[q], k)
+            assert np.array_equal(idx[q].cpu().numpy(), ridx)
+            assert np.array_equal(val[q].cpu().numpy(), rval.astype(np.float32))
+    # NaN ranks below every number, ties among NaN by index
+    e = np.full((1, 5000), np.nan, dtype=np.float32)
+    numbers = rng.choice(5000, size=10, replace=False)
+    e[0, numbers] = rng.normal(size=10).astype(np.float32)
+    idx, _ = b.r3_topk(dev(e), 64)
+    idx = idx.cpu().numpy()[0]
+    assert np.array_equal(idx[:10], o.topk(np.where(np.isnan(e[0]), -np.inf, e[0]), 10)[0])
+    rest = np.setdiff1d(np.arange(5000), numbers)
+    assert np.array_equal(idx[10:], rest[:54])
+
+
 def test_topk_special_values():
     e = np.array([[0.0, -0.0, np.nan, -np.inf, 1.0, np.inf, -1.0, 0.0]], dtype=np.float32)
     idx, val = b.r3_topk(dev(e), 8)
