@@ -4,7 +4,8 @@
 // larger pool): cudaMalloc and cudaFree of 100 MB blocks cost milliseconds each -- more than the
 // kernels of an append -- so freed blocks are kept, per device, and handed out again.  Sizes are
 // rounded up to five significant bits so that neighbouring sizes (a history that grew by a few
-// rows) share a bin.  dev_free waits for the device like cudaFree does, which makes the block safe to
+// rows) share a bin; blocks below 1 MiB -- a small history's fit is two dozen of them, and their cudaMalloc and
+// cudaFree calls were most of its time -- are rounded up to a multiple of 512 bytes and kept as well.  dev_free waits for the device like cudaFree does, which makes the block safe to
 // reuse at once.  The cache holds at most kCacheLimit bytes per device; r3_trim_cache() returns
 // everything to the driver.
 #include <map>
@@ -18,7 +19,8 @@ namespace r3 {
 namespace {
 
 constexpr size_t kCacheLimit = 2ull << 30;
-constexpr size_t kSmall = 1 << 20;   // blocks below 1 MiB are not worth caching
+constexpr size_t kSmall = 1 << 20;   // below 1 MiB: bins of 512 bytes
+constexpr size_t kCacheBlocks = 4096;   // at most this many kept blocks per device
 
 struct DeviceCache {
     std::multimap<size_t, void*> free_blocks;   // bin size -> block
@@ -34,7 +36,7 @@ long long g_alloc_seen = 0, g_alloc_fail_at = -1;
 
 size_t bin_of(size_t bytes)
 {
-    if (bytes < kSmall) return bytes;
+    if (bytes < kSmall) return (bytes + 511) & ~(size_t)511;
     size_t top = bytes;
     int shift = 0;
     while (top >= 32) {   // keep five leading bits: bins are at most 1/16 apart
@@ -103,14 +105,14 @@ void dev_free(void* p)
             c.live.erase(it);
         }
     }
-    if (bin < kSmall) {   // not ours, or small: plain free
+    if (bin == 0) {   // not ours: plain free
         cudaFree(p);
         return;
     }
     cudaDeviceSynchronize();   // as cudaFree would: nothing in flight may still use the block
     std::lock_guard<std::mutex> lock(g_mutex);
     DeviceCache& c = g_cache[dev];
-    if (c.cached_bytes + bin > kCacheLimit) {
+    if (c.cached_bytes + bin > kCacheLimit || c.free_blocks.size() >= kCacheBlocks) {
         cudaFree(p);
         return;
     }
