@@ -516,8 +516,17 @@ r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream)
     const int B = gp->batch, n = gp->n, d = gp->d, npad = gp->npad;
     const size_t mat = (size_t)npad * npad;
     double *Dinv = nullptr, *Ldiag = nullptr, *T = nullptr, *u = nullptr, *slabs = nullptr;
+    // stream and events of the factorisation's look-ahead (see the panel loop)
+    cudaStream_t aux = nullptr;
+    cudaEvent_t panel_done = nullptr, wide_done = nullptr;
     R3_CUDA_TRY(dev_malloc(&Dinv, sizeof(double) * B * (size_t)(npad / NB) * NB * NB));
     auto fail = [&](r3_status_t st) {
+        if (aux) {
+            cudaStreamSynchronize(aux);
+            cudaStreamDestroy(aux);
+        }
+        if (panel_done) cudaEventDestroy(panel_done);
+        if (wide_done) cudaEventDestroy(wide_done);
         dev_free(Dinv);
         dev_free(Ldiag);
         dev_free(T);
@@ -558,30 +567,72 @@ r3_status_t fit_device(r3_gp* gp, const float* y, cudaStream_t stream)
 
     TRY_OR_FAIL(cudaFuncSetAttribute(potrf_panel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPanelSmem));
     constexpr int kOuter = 4 * NB;   // columns per panel of the two-level right-looking factorisation
+    // Look-ahead: a panel's update of everything to its right is split.  The columns of the NEXT panel are updated
+    // first, and that panel's factorisation (a chain of eight short dependent launches) follows at once, both on a
+    // stream of the highest priority so that their few blocks are placed ahead of the queued blocks of the wide
+    // update; the update of the columns beyond -- most of the arithmetic -- runs on the caller's stream meanwhile.
+    // The two touch disjoint columns; the next panel's own update waits for the wide one (same elements).
+    const bool look_ahead = npad > 2 * kOuter;
+    cudaStream_t cs = stream;   // the stream of the chain
+    if (look_ahead) {
+        int least = 0, greatest = 0;
+        TRY_OR_FAIL(cudaDeviceGetStreamPriorityRange(&least, &greatest));
+        TRY_OR_FAIL(cudaStreamCreateWithPriority(&aux, cudaStreamNonBlocking, greatest));
+        TRY_OR_FAIL(cudaEventCreateWithFlags(&panel_done, cudaEventDisableTiming));
+        TRY_OR_FAIL(cudaEventCreateWithFlags(&wide_done, cudaEventDisableTiming));
+        cs = aux;
+        TRY_OR_FAIL(cudaEventRecord(wide_done, stream));   // the Gram matrix is ready
+        TRY_OR_FAIL(cudaStreamWaitEvent(cs, wide_done, 0));
+    }
+#define CHAIN_LAUNCH(kernel, grid, block, smem, ...)                                               \
+    do {                                                                                           \
+        kernel<<<(grid), (block), (smem), cs>>>(__VA_ARGS__);                                      \
+        ++g_launches;                                                                              \
+        cudaError_t e__ = cudaGetLastError();                                                      \
+        if (e__ != cudaSuccess) {                                                                  \
+            set_error("launch of %s failed: %s", #kernel, cudaGetErrorString(e__));                \
+            return fail(R3_ERR_CUDA);                                                              \
+        }                                                                                          \
+    } while (0)
+    bool wide_pending = false;
     for (int J = 0; J < npad; J += kOuter) {
         const int panel_end = std::min(J + kOuter, npad);
         for (int j0 = J; j0 < panel_end; j0 += NB) {
             const int rows = npad - j0 - NB;
-            potrf_panel_kernel<<<dim3(rows > 0 ? (rows + kPanelThreads - 1) / kPanelThreads : 1, B),
-                                 dim3(NB, kPanelThreads / NB), kPanelSmem, stream>>>(gp->L64, npad, j0, Dinv, Ldiag,
-                                                                                    gp->status_d);
-            ++g_launches;
-            if (cudaError_t e__ = cudaGetLastError(); e__ != cudaSuccess) {
-                set_error("launch of potrf_panel_kernel failed: %s", cudaGetErrorString(e__));
-                return fail(R3_ERR_CUDA);
-            }
+            CHAIN_LAUNCH(potrf_panel_kernel, dim3(rows > 0 ? (rows + kPanelThreads - 1) / kPanelThreads : 1, B),
+                         dim3(NB, kPanelThreads / NB), kPanelSmem, gp->L64, npad, j0, Dinv, Ldiag, gp->status_d);
             if (rows <= 0) continue;
             const int tiles = (rows + 63) / 64;
             const int inner = panel_end - j0 - NB;   // columns of this panel still to be factored
             if (inner > 0)
-                LAUNCH_OR_FAIL(syrk_kernel, dim3((inner + 63) / 64, tiles, B), 256, gp->L64, npad, j0, NB, j0 + NB,
-                               panel_end);
+                CHAIN_LAUNCH(syrk_kernel, dim3((inner + 63) / 64, tiles, B), 256, 0, gp->L64, npad, j0, NB, j0 + NB, panel_end);
         }
         const int rows = npad - panel_end;
-        if (rows > 0) {
-            const int tiles = (rows + 63) / 64;
+        if (rows <= 0) continue;
+        const int tiles = (rows + 63) / 64;
+        if (!look_ahead) {
             LAUNCH_OR_FAIL(syrk_kernel, dim3(tiles, tiles, B), 256, gp->L64, npad, J, panel_end - J, panel_end, npad);
+            continue;
         }
+        TRY_OR_FAIL(cudaEventRecord(panel_done, cs));
+        if (wide_pending) TRY_OR_FAIL(cudaStreamWaitEvent(cs, wide_done, 0));
+        const int next_cols = std::min(kOuter, rows);
+        CHAIN_LAUNCH(syrk_kernel, dim3((next_cols + 63) / 64, tiles, B), 256, 0, gp->L64, npad, J, panel_end - J, panel_end,
+                     panel_end + next_cols);
+        const int wide = rows - next_cols;
+        if (wide > 0) {
+            const int wtiles = (wide + 63) / 64;
+            TRY_OR_FAIL(cudaStreamWaitEvent(stream, panel_done, 0));
+            LAUNCH_OR_FAIL(syrk_kernel, dim3(wtiles, wtiles, B), 256, gp->L64, npad, J, panel_end - J, panel_end + next_cols,
+                           npad);
+            TRY_OR_FAIL(cudaEventRecord(wide_done, stream));
+            wide_pending = true;
+        }
+    }
+#undef CHAIN_LAUNCH
+    if (look_ahead) {   // the caller's stream goes on when the chain has ended
+        TRY_OR_FAIL(cudaEventRecord(panel_done, cs));
+        TRY_OR_FAIL(cudaStreamWaitEvent(stream, panel_done, 0));
     }
 
     LAUNCH_OR_FAIL(scatter_ldiag_kernel, dim3(npad / NB, B), dim3(NB, NB), Ldiag, npad, gp->L64);
