@@ -554,15 +554,15 @@ def main():
     if engine == "tensor":
         # Variance contraction S4: algorithmic n^2 flops per candidate (n^2/2 MACs over the lower triangle).  The
         # 22-bit product needs three FP16 MMAs per product (hi*hi + hi*lo + lo*hi), so the work counted is 3x that,
-        # at the FP16/BF16 tensor rate -- the count stays the same when the two cross terms run as E4M3 MMAs at
+        # at the FP16/BF16 tensor rate -- the count stays the same when the two cross terms run as FP8 MMAs at
         # twice the rate (then the tensor time actually issued is that of two FP16 MMAs: `issued_f16_equivalent`).
         # The distance products and the diagonal blocks' zero halves are not in the count; `issued_total_tflops`
         # is everything the pipe was given, in FP16-rate equivalents: per chunk of 32 observations of a tile,
-        # 128 x NV x 32 MACs of the variance product three (two with E4M3 cross terms) times over, and
+        # 128 x NV x 32 MACs of the variance product three (two with FP8 cross terms) times over, and
         # 128 x 32 x DP MACs of the distance product three times, for every (re)generation of the chunk.
         info = b.r3_gp_tensor_info(gp)
         f8 = bool(info["f8_cross_terms"])
-        split = "f16 + 2 x e4m3 cross terms" if f8 else "f16x3"
+        split = "f16 + 2 x fp8 cross terms (k* e5m2; W e4m3/e5m2)" if f8 else "f16x3"
         alg_flops = float(n) * n
         issued = 3.0 * alg_flops
         achieved = issued * cands_per_launch / (per_launch_ms * 1e-3) / 1e12

@@ -204,7 +204,7 @@ r3_engine_t r3_gp_engine(const r3_gp_t* gp);
  * info[2] DP   feature count padded to a multiple of 16 (depth of the distance product)
  * info[3] NP   history length padded to a multiple of NV
  * info[4] G    Matern warp groups;  info[5] W stages in shared memory;  info[6] 1: k* operand in tensor memory
- * info[7] 1: the cross terms of the variance product are E4M3 MMAs (histories of eight passes and more)
+ * info[7] 1: the cross terms of the variance product are FP8 MMAs (histories of eight passes and more)
  */
 r3_status_t r3_gp_tensor_info(const r3_gp_t* gp, int* info /* host [8] */);
 

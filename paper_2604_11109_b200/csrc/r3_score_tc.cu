@@ -100,7 +100,7 @@ constexpr uint32_t kZnOffset = 512;                   // float[128] squared norm
 // NBK: number of k* buffers.  NBK == G: group g owns buffer g.  NBK < G (k* in TMEM, where columns are
 // scarce): the buffers form a ring shared by the groups, chunk t uses buffer t mod NBK; a group that has
 // computed its chunk keeps it in registers until the ring slot is free, so the groups still run ahead.
-// F8: the two cross terms of the variance product (W_hi k_lo, W_lo k_hi) are single E4M3 MMAs of depth 32
+// F8: the two cross terms of the variance product (W_hi k_lo, W_lo k_hi) are single FP8 MMAs of depth 32
 // instead of two FP16 MMAs of depth 16 each: four MMAs per chunk instead of six.
 // PUTOFF: a pass's epilogue (read the accumulator back, hand it over) is put off until the group's first chunk of
 // the next pass is on its way, when that chunk can be handed over without the accumulator's release (its k* slot is
@@ -335,27 +335,30 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     const uint32_t vcol = tmem + skip;
                     const uint32_t bH = w_lo0 + ((s * map.w_stage) >> 4) + skip, bL = bH + (((uint32_t)KC * NV * 2u) >> 4);
                     if (F8) {
-                        // main term: FP16 hi x hi, two MMAs of depth 16; cross terms: one E4M3 MMA of depth 32 each
+                        // main term: FP16 hi x hi, two MMAs of depth 16; cross terms: one FP8 MMA of depth 32 each
                         // (planes after the FP16 hi plane: scaled hi parts, then scaled lo parts)
                         const uint32_t first = c > 0 ? 1u : 0u;
                         const uint32_t b8H = bH + (((uint32_t)KC * NV * 2u) >> 4), b8L = b8H + (((uint32_t)KC * NV) >> 4);
+                        // k* parts are E5M2; W's hi parts E4M3, its lo parts E5M2
+                        const uint32_t idesc_hl = instr_desc_f8(NV - skip, kFmtE5M2, kFmtE5M2);   // k*_hi x W_lo
+                        const uint32_t idesc_lh = instr_desc_f8(NV - skip, kFmtE5M2, kFmtE4M3);   // k*_lo x W_hi
                         if (KT) {
                             const uint32_t aH = tmem + KCOL + (uint32_t)b * KC;
                             tc_mma_f16_ts(vcol, aH, pack64(bH, kDescHi), idesc_v, first);
                             tc_mma_f16_ts(vcol, aH + 8u, pack64(bH + ((2u * NV * 16u) >> 4), kDescHi), idesc_v, 1u);
-                            tc_mma_f8_ts(vcol, aH + KC / 2, pack64(b8L, kDescHi), idesc_v, 1u);
+                            tc_mma_f8_ts(vcol, aH + KC / 2, pack64(b8L, kDescHi), idesc_hl, 1u);
                             k_seen = mbar_try_wait(bar(BAR_K_FULL + k_s), k_ph);
                             w_seen = mbar_try_wait(bar(BAR_W_FULL + w_s), w_ph);
-                            tc_mma_f8_ts(vcol, aH + KC / 2 + KC / 4, pack64(b8H, kDescHi), idesc_v, 1u);
+                            tc_mma_f8_ts(vcol, aH + KC / 2 + KC / 4, pack64(b8H, kDescHi), idesc_lh, 1u);
                         } else {
                             const uint32_t aH = k_lo0 + ((b * 16384u) >> 4), a8H = aH + (8192u >> 4), a8L = a8H + (4096u >> 4);
                             tc_mma_f16(vcol, pack64(aH, kDescHi), pack64(bH, kDescHi), idesc_v, first);
                             tc_mma_f16(vcol, pack64(aH + (4096u >> 4), kDescHi), pack64(bH + ((2u * NV * 16u) >> 4), kDescHi),
                                        idesc_v, 1u);
-                            tc_mma_f8(vcol, pack64(a8H, kDescHi), pack64(b8L, kDescHi), idesc_v, 1u);
+                            tc_mma_f8(vcol, pack64(a8H, kDescHi), pack64(b8L, kDescHi), idesc_hl, 1u);
                             k_seen = mbar_try_wait(bar(BAR_K_FULL + k_s), k_ph);
                             w_seen = mbar_try_wait(bar(BAR_W_FULL + w_s), w_ph);
-                            tc_mma_f8(vcol, pack64(a8L, kDescHi), pack64(b8H, kDescHi), idesc_v, 1u);
+                            tc_mma_f8(vcol, pack64(a8L, kDescHi), pack64(b8H, kDescHi), idesc_lh, 1u);
                         }
                     } else if (KT) {
                         const uint32_t aH = tmem + KCOL + (uint32_t)b * KC, aL = aH + KC / 2;
@@ -738,7 +741,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                         // split into the two FP16 planes; the stores wait until the whole chunk is computed
                         // so that the arithmetic does not sit between the buffer's release and its refill
                         if (F8) {
-                            // kl[h][0..3]: the 16 scaled hi parts as E4M3, kl[h][4..7]: the 16 scaled lo parts
+                            // kl[h][0..3]: the 16 hi parts as E5M2, kl[h][4..7]: the 16 lo parts
 #pragma unroll
                             for (int e = 0; e < 4; ++e)
                                 split4_f8(kv + 4 * e, kh[h][2 * e], kh[h][2 * e + 1], kl[h][e], kl[h][4 + e]);
@@ -771,7 +774,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                     if (threadIdx.x % 128 == 0) LOGEV(5, t);
                     if (F8) {
                         if (KT) {
-                            // FP16 hi plane: 16 columns; then the chunk's 32 E4M3 hi parts (8 columns) and lo parts (8)
+                            // FP16 hi plane: 16 columns; then the chunk's 32 E5M2 hi parts (8 columns) and lo parts (8)
                             uint32_t p8[8];
                             tc_st8(lane_addr + KCOL + (uint32_t)kbuf * KC, kh[0]);
                             tc_st8(lane_addr + KCOL + (uint32_t)kbuf * KC + 8, kh[1]);
@@ -788,7 +791,7 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                                 for (int sl = 0; sl < 2; ++sl)
                                     *reinterpret_cast<uint4*>(kb + (2 * h + sl) * 2048u) =
                                         make_uint4(kh[h][4 * sl], kh[h][4 * sl + 1], kh[h][4 * sl + 2], kh[h][4 * sl + 3]);
-                                // one 16-byte k-slice of each E4M3 plane per 16 observations
+                                // one 16-byte k-slice of each 8-bit plane per 16 observations
                                 *reinterpret_cast<uint4*>(kb + 8192u + h * 2048u) = make_uint4(kl[h][0], kl[h][1], kl[h][2], kl[h][3]);
                                 *reinterpret_cast<uint4*>(kb + 12288u + h * 2048u) = make_uint4(kl[h][4], kl[h][5], kl[h][6], kl[h][7]);
                             }
@@ -1027,8 +1030,9 @@ __global__ void wmax_kernel(const double* __restrict__ W64, int n, int npad_fit,
 
 // One block per (chunk c, pass p, GP): the KC x NV block of 2^eW W (rows p NV.., columns c KC..) as
 // FP16 hi/lo planes in the B-operand layout; zero outside the lower triangle and outside n.
-// With f8 the second plane holds, instead of the FP16 lo parts, two E4M3 planes in the 8-bit form of the same
-// layout (16 k-elements per 16-byte slice): the hi parts times 2^-6, then the lo parts times 2^6.
+// With f8 the second plane holds, instead of the FP16 lo parts, two 8-bit planes in the 8-bit form of the same
+// layout (16 k-elements per 16-byte slice): the hi parts as E4M3 (|2^eW W| < 2^8 for these histories), then the
+// lo parts as E5M2.
 __global__ void wt_build_kernel(const double* __restrict__ W64, int n, int npad_fit, int NV, size_t gp_stride,
                                 const float* __restrict__ wscale, __half* __restrict__ wt, bool f8)
 {
@@ -1051,8 +1055,8 @@ __global__ void wt_build_kernel(const double* __restrict__ W64, int n, int npad_
             uint8_t* d8 = reinterpret_cast<uint8_t*>(dst + (size_t)KC * NV);
             const size_t off8 = ((size_t)(kk / 16) * NV + r) * 16 + (kk % 16);
             const float hf = __half2float(h);
-            d8[off8] = (uint8_t)(e4m3x4(hf * kF8HiScale, 0.f, 0.f, 0.f) & 0xffu);
-            d8[(size_t)KC * NV + off8] = (uint8_t)(e4m3x4((w - hf) * kF8LoScale, 0.f, 0.f, 0.f) & 0xffu);
+            d8[off8] = (uint8_t)(e4m3x4(hf, 0.f, 0.f, 0.f) & 0xffu);
+            d8[(size_t)KC * NV + off8] = (uint8_t)(e5m2x4(w - hf, 0.f, 0.f, 0.f) & 0xffu);
         } else {
             dst[(size_t)KC * NV + off] = __float2half_rn(w - __half2float(h));
         }
@@ -1224,7 +1228,7 @@ r3_status_t tc_prepare(r3_gp* gp, cudaStream_t stream)
         int ew = 0, ek = 0;
         frexp((double)wmax[g], &ew);               // wmax < 2^ew
         frexp((double)gp->sf2[g], &ek);            // sf2  < 2^ek  (k* <= sf2)
-        const int sw = kScaleExp - ew, sk = kScaleExp - ek;
+        const int sw = (t->f8 ? kScaleExpF8 : kScaleExp) - ew, sk = kScaleExp - ek;
         if (!(wmax[g] > 0.f) || sw < -60 || sw > 60 || sk < -60 || sk > 60) return decline();   // degenerate scales
         wscale[g] = (float)ldexp(1.0, sw);
         kscale[g] = (float)ldexp(1.0, sk);

@@ -15,7 +15,7 @@ namespace r3 {
 struct TensorOperands {
     int NV = 0, G = 0, KD = 0, DP = 0, NP = 0, P = 0, ws = 0;
     bool kt = false;           // k* buffers in TMEM
-    bool f8 = false;           // cross terms of the variance product as FP8 (E4M3) MMAs
+    bool f8 = false;           // cross terms of the variance product as FP8 MMAs
     int nbk = 0;               // number of k* buffers (== G: one per group; smaller: a shared ring)
     size_t smem_bytes = 0;
     size_t wt_gp_stride = 0;   // halves per GP in wt
@@ -27,7 +27,7 @@ struct TensorOperands {
     float* xnmax = nullptr;    // [B]      max_k |x~_k|^2
     float* alpha = nullptr;    // [B][NP]  weights, zero padded
     __half* wt = nullptr;      // [B][tile(p,c)][2][KC/8][NV][8]  chunks of 2^eW W, FP16 hi/lo planes; with f8 the
-                               // second plane is two E4M3 planes [2][KC/16][NV][16]: 2^-6 hi, then 2^6 lo
+                               // second plane is two 8-bit planes [2][KC/16][NV][16]: hi parts (E4M3), then lo parts (E5M2)
     float* kscale = nullptr;   // [B]  2^eK, applied to k* before its split
     double* vinv2 = nullptr;   // [B]  2^(-2 (eK + eW)): scales sum V^2 back
 };
@@ -160,7 +160,8 @@ __device__ __forceinline__ void tc_mma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, 
         ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-// kind::f8f6f4 with both operands E4M3 (format code 0, the same instruction descriptor as FP16 x FP16): K = 32
+// kind::f8f6f4, K = 32; the instruction descriptor is the FP16 one plus the operands' format codes
+// (instr_desc_f8)
 __device__ __forceinline__ void tc_mma_f8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                           uint32_t accumulate)
 {
@@ -171,7 +172,7 @@ __device__ __forceinline__ void tc_mma_f8(uint32_t d_tmem, uint64_t adesc, uint6
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-// A operand from TMEM (lane = row, one 32-bit column = four consecutive E4M3 k-elements)
+// A operand from TMEM (lane = row, one 32-bit column = four consecutive 8-bit k-elements)
 __device__ __forceinline__ void tc_mma_f8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
                                              uint32_t accumulate)
 {
@@ -260,12 +261,16 @@ __device__ __forceinline__ void split2(float a, float b, __half2& hi, __half2& l
 }
 
 // Cross terms of the variance product in FP8.  With x = hi + lo (hi = fp16(x)) the product W k* is
-// W_hi k_hi + W_hi k_lo + W_lo k_hi; the two cross terms are 2^-11 of the first, so E4M3 factors (4 significant
-// bits) leave them with a relative error of about 2^-4 and the sum with about 2^-16 -- enough wherever q = |W k*|^2
-// is a modest part of the signal variance, and the accuracy guard recomputes the rest in FP64.  hi parts (below
-// 2^14) are multiplied by 2^-6 and lo parts (below 2^3) by 2^6 before the conversion, so that both sit inside
-// E4M3's range and every cross product keeps the scale of the main term.
-constexpr float kF8HiScale = 0.015625f, kF8LoScale = 64.f;
+// W_hi k_hi + W_hi k_lo + W_lo k_hi; the two cross terms are 2^-11 of the first, so 8-bit factors leave them with a
+// relative error of 2^-3 to 2^-4 and the sum with about 2^-15 -- enough wherever q = |W k*|^2 is a modest part of
+// the signal variance, and the accuracy guard recomputes the rest in FP64.
+// Formats: the parts of k* are E5M2, taken from the FP16 hi part and the FP32 remainder as they are (hi parts
+// below 2^14, lo parts below 2^3: both inside E5M2's range, no scaling -- the conversion is all the Matern warps
+// pay, and with E4M3 the two multiplications per element that brought the parts into its range were a tenth of
+// their instructions); W is scaled to below 2^8 for these histories, so that its hi parts fit E4M3 unscaled
+// (three mantissa bits where it costs nothing: W is converted once per fit) and its lo parts, below 2^-3, go to
+// E5M2 for the range.
+constexpr int kScaleExpF8 = 8;   // |scaled W| < 2^8 when the cross terms are FP8 (E4M3 holds up to 448)
 // (a, b, c, d) -> four E4M3 bytes, a in the lowest
 __device__ __forceinline__ uint32_t e4m3x4(float a, float b, float c, float d)
 {
@@ -274,20 +279,34 @@ __device__ __forceinline__ uint32_t e4m3x4(float a, float b, float c, float d)
     asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi16) : "f"(d), "f"(c));
     return (uint32_t)lo16 | ((uint32_t)hi16 << 16);
 }
-// four values -> FP16 hi parts (two half2), and the E4M3 forms of the scaled hi parts and of the scaled remainders
+// (a, b, c, d) -> four E5M2 bytes, a in the lowest
+__device__ __forceinline__ uint32_t e5m2x4(float a, float b, float c, float d)
+{
+    uint16_t lo16, hi16;
+    asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(lo16) : "f"(b), "f"(a));
+    asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(hi16) : "f"(d), "f"(c));
+    return (uint32_t)lo16 | ((uint32_t)hi16 << 16);
+}
+// two packed halves -> two E5M2 bytes (the lower half in the lower byte)
+__device__ __forceinline__ uint32_t e5m2x2_of_half2(uint32_t h2)
+{
+    uint16_t r;
+    asm("cvt.rn.satfinite.e5m2x2.f16x2 %0, %1;" : "=h"(r) : "r"(h2));
+    return (uint32_t)r;
+}
+// four values -> FP16 hi parts (two half2), and the E5M2 forms of the hi parts and of the remainders
 __device__ __forceinline__ void split4_f8(const float* v, uint32_t& h01, uint32_t& h23, uint32_t& hi8, uint32_t& lo8)
 {
     const __half2 a = __floats2half2_rn(v[0], v[1]), b = __floats2half2_rn(v[2], v[3]);
     const float2 fa = __half22float2(a), fb = __half22float2(b);
     h01 = *reinterpret_cast<const uint32_t*>(&a);
     h23 = *reinterpret_cast<const uint32_t*>(&b);
-    hi8 = e4m3x4(fa.x * kF8HiScale, fa.y * kF8HiScale, fb.x * kF8HiScale, fb.y * kF8HiScale);
-    lo8 = e4m3x4((v[0] - fa.x) * kF8LoScale, (v[1] - fa.y) * kF8LoScale, (v[2] - fb.x) * kF8LoScale,
-                 (v[3] - fb.y) * kF8LoScale);
+    hi8 = e5m2x2_of_half2(h01) | (e5m2x2_of_half2(h23) << 16);
+    lo8 = e5m2x4(v[0] - fa.x, v[1] - fa.y, v[2] - fb.x, v[3] - fb.y);
 }
 // relative error of one cross product in that form (root mean square over rounding positions), added to the
 // per-entry error of k* in the estimate of the error of q
-constexpr double kEpsF8 = 1.2e-5;
+constexpr double kEpsF8 = 2.9e-5;
 
 // Shared-memory matrix descriptors are the no-swizzle K-major form: bits 0-13 start address >> 4,
 // bits 16-29 the byte distance between the two 16-byte k-slices of one MMA >> 4, bits 32-45 the byte
@@ -300,6 +319,12 @@ __device__ __forceinline__ uint32_t desc_addr(uint32_t saddr) { return (saddr & 
 __device__ __forceinline__ constexpr uint32_t instr_desc_f16(uint32_t n)
 {
     return (1u << 4) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+}
+// kind::f8f6f4: format code of A in bits 7-9 and of B in bits 10-12 (0 = E4M3, 1 = E5M2)
+constexpr uint32_t kFmtE4M3 = 0u, kFmtE5M2 = 1u;
+__device__ __forceinline__ constexpr uint32_t instr_desc_f8(uint32_t n, uint32_t a_fmt, uint32_t b_fmt)
+{
+    return instr_desc_f16(n) | (a_fmt << 7) | (b_fmt << 10);
 }
 
 // Out-of-line (cold) path of the Matern warps: for the pairs whose (scaled) k* exceeds v_thresh, replace it by the value

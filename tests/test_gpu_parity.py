@@ -149,7 +149,7 @@ def test_selection_sizes_through_the_scoring_call(engine, batch, m, k):
 
 @pytest.mark.parametrize("spread,sn2", [(1.0, 1e-3), (3.0, 1e-4)])
 def test_long_history_with_fp8_cross_terms_near_observations(spread, sn2):
-    """From eight passes on (n > 1792) the variance product's cross terms are E4M3 MMAs; their error estimate has to
+    """From eight passes on (n > 1792) the variance product's cross terms are FP8 MMAs; their error estimate has to
     send the candidates for which that matters -- on and next to observations, long lengthscales -- to the FP64
     pass.  Every element and the top-k against the oracle."""
     n, d, m = 2100, 20, 700
