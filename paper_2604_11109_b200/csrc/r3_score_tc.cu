@@ -646,10 +646,9 @@ __global__ void __launch_bounds__(128 + 128 * G, 1) score_tc_kernel(const TcPara
                                 kv[4 * q + e] = fmaf(u, fmaf(u, pc2, pc1), pc0) * exp2_approx(-u);
                             }
                         }
-                        float vmax = fmaxf(fmaxf(kv[0], kv[1]), fmaxf(kv[2], kv[3]));
-#pragma unroll
-                        for (int i = 4; i < 16; i += 4)
-                            vmax = fmaxf(vmax, fmaxf(fmaxf(kv[i], kv[i + 1]), fmaxf(kv[i + 2], kv[i + 3])));
+                        // largest of the sixteen in eight three-input maxima
+                        const float vmax = max3(max3(max3(kv[0], kv[1], kv[2]), max3(kv[3], kv[4], kv[5]), max3(kv[6], kv[7], kv[8])),
+                                                max3(max3(kv[9], kv[10], kv[11]), max3(kv[12], kv[13], kv[14]), kv[15]), 0.f);
                         if (ZS) {
                             if (vmax > v_thresh) {   // close pairs of this candidate: direct differences, inline
                                 uint32_t marked = 0;
