@@ -3,7 +3,7 @@
 * a device-side wait that runs out: the tensor-core kernel's bounded waits, provoked by withholding one stage
   of its operand stream under a short limit; the kernel returns by itself, the status is reported, the handle
   keeps working;
-* allocation failures injected on the host;
+* allocation failures injected on the host; the device-memory cache across fits;
 * status bits latched by one call do not leak into the next call's own checks;
 * two live handles of different shapes that share a kernel instantiation.
 """
@@ -127,6 +127,30 @@ def test_append_after_an_unchecked_scoring_call_keeps_that_calls_latched_status(
         b.r3_gp_check(gp)
     assert e.value.status == 2
     compare_everything(g, gp, 8, "after append")
+    gp.close()
+
+
+def test_freed_blocks_of_every_size_are_kept_and_given_back_on_request():
+    """The device-memory cache keeps a closed handle's blocks, the small ones included (a small history's fit is
+    two dozen of them), hands them to the next fit of the same shape, and returns everything on r3_trim_cache."""
+    b.r3_trim_cache()
+    assert b.r3_cached_bytes() == 0
+    g = rand_problem(21, 1, 48, 5, 64)
+    fit_gpu(g).close()
+    kept = b.r3_cached_bytes()
+    assert kept > 0
+    gp = fit_gpu(g)                       # the same shape again: served from the cache
+    assert b.r3_cached_bytes() < kept
+    compare_everything(g, gp, 8, "fit from cached blocks")
+    gp.close()
+    assert b.r3_cached_bytes() >= kept
+    big = rand_problem(22, 1, 700, 9, 64)  # blocks above 1 MiB go through the same cache
+    fit_gpu(big).close()
+    assert b.r3_cached_bytes() > kept + (1 << 20)
+    b.r3_trim_cache()
+    assert b.r3_cached_bytes() == 0
+    gp = fit_gpu(g)
+    compare_everything(g, gp, 8, "fit after the cache was emptied")
     gp.close()
 
 
